@@ -1,0 +1,142 @@
+/*
+ * qalora.h -- C ABI of the QA-LoRA linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer (arXiv 2309.14717, "QA-LoRA"): a weight matrix W [D_in x D_out]
+ * quantized group-wise with min-max quantization (Eq. 1 applied per group of
+ * `group_size` consecutive input channels and per output column, Section 3.3),
+ * plus a low-rank adapter that sees the input summed over each group
+ * (Algorithm 1; Appendix B Eq. 3 and Eq. 4):
+ *
+ *     y = x * W~  +  s * (pool(x) * A) * B
+ *     W~[k, n]   = alpha[k / g, n] * c[k, n] + beta[k / g, n]
+ *     pool(x)[m, q] = sum of x[m, k] over the g channels k of group q
+ *
+ * Notation used below: K = d_in, N = d_out, g = group_size, G = K / g (the
+ * paper's symbol L is this NUMBER of groups), r = rank (the paper's D_int),
+ * b = bits, s = scale, M = number of token rows.
+ *
+ * Conventions that hold for every entry point
+ *   - Every data pointer is DEVICE memory owned by the caller unless the
+ *     comment says "host".  The library allocates no device memory.
+ *   - All matrices are dense row-major.  x, y, dy, dx, A, B are bfloat16
+ *     (passed as void*); alpha/beta (qparams), dA, dB and W are float32.
+ *   - Pointers must be 16-byte aligned.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL
+ *     is the legacy default stream); calls do not synchronize the host.
+ *   - Outputs are overwritten, never accumulated into.
+ *   - Return value: QALORA_OK or a negative qalora_status.  Nothing is
+ *     launched when an argument is rejected.  No call traps or aborts.
+ *
+ * Packed code layout (version QALORA_LAYOUT_VERSION; the paper only says the
+ * codes are stored as b-bit integers, Section 3.1 -- the arrangement is this
+ * library's own).  A pack unit is 32 consecutive input channels (k-block
+ * kb = k / 32) of one output column n; j = k % 32.  `codes` is a little-endian
+ * uint32 array [K/32][N][words]:
+ *   b = 4: 4 words; position j lives in word j/8,  e = j%8,  at bit 16*(e&1) + 4*(e>>1)
+ *   b = 2: 2 words; position j lives in word j/16, e = j%16, at bit 16*(e&1) + 2*(e>>1)
+ *   b = 3: 3 words; words 0..1 hold (c & 3) in the b = 2 arrangement, word 2
+ *          holds (c >> 2) of position j at bit 16*(j&1) + (j>>1)
+ * `qparams` is float32 [G][N][2] = {alpha, beta} per (group, column).
+ */
+#ifndef QALORA_H_
+#define QALORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QALORA_LAYOUT_VERSION 1
+
+typedef enum qalora_status {
+  QALORA_OK = 0,
+  QALORA_ERR_INVALID_ARG = -1,      /* a size or enum outside its domain        */
+  QALORA_ERR_NULL_POINTER = -2,     /* a required pointer is NULL               */
+  QALORA_ERR_UNSUPPORTED_SHAPE = -3,/* see qalora_desc                          */
+  QALORA_ERR_MISALIGNED = -4,       /* a pointer is not 16-byte aligned         */
+  QALORA_ERR_WORKSPACE_TOO_SMALL = -5,
+  QALORA_ERR_CUDA = -6              /* a CUDA call or launch failed             */
+} qalora_status;
+
+/* Shape and hyper-parameters of one layer.  Supported: d_in a multiple of
+ * group_size; group_size a multiple of 32; d_out a multiple of 8; bits in
+ * {2, 3, 4}; 0 <= rank <= 256 and a multiple of 8.  rank == 0 is the plain
+ * (merged, deployed) quantized layer: A and B are then ignored and may be NULL. */
+typedef struct qalora_desc {
+  int32_t d_in;        /* K */
+  int32_t d_out;       /* N */
+  int32_t group_size;  /* g */
+  int32_t bits;        /* b */
+  int32_t rank;        /* r */
+  float   scale;       /* s */
+} qalora_desc;
+
+typedef enum qalora_op { QALORA_OP_FORWARD = 0, QALORA_OP_BACKWARD = 1 } qalora_op;
+
+/* Library version * 100 + QALORA_LAYOUT_VERSION. */
+int qalora_version(void);
+
+/* Static, NUL-terminated description of a status code (host memory, never freed). */
+const char* qalora_status_string(int status);
+
+/* Sizes in bytes of the packed `codes` array and of `qparams` for a layer.
+ * Both outputs are host pointers. */
+int qalora_packed_bytes(const qalora_desc* desc, size_t* code_bytes, size_t* qparam_bytes);
+
+/* Bytes of scratch `workspace` that qalora_forward / qalora_backward need for
+ * `m` token rows (host pointer out; may be 0).  The workspace holds the pooled
+ * input, the rank-r intermediates and split-K partial sums; its content is
+ * undefined on entry and on exit. */
+int qalora_workspace_bytes(const qalora_desc* desc, int64_t m, int op, size_t* bytes);
+
+/* Group-wise min-max quantization, Eq. 1 per (group, column) (Section 3.3):
+ *   lo, hi = min, max of W[q*g .. (q+1)*g - 1, n];  beta = lo;
+ *   alpha = (hi - lo) / (2^b - 1), or 1 when hi == lo;
+ *   c = clamp(round_half_even((W - beta) / alpha), 0, 2^b - 1)
+ * evaluated in IEEE float32, one correctly rounded operation at a time.
+ *   W        in : float32 [K][N]
+ *   codes    out: packed codes, qalora_packed_bytes() bytes
+ *   qparams  out: float32 [G][N][2]
+ *   dev_status out, optional: one int32 in device memory; bit 0 is OR-ed in
+ *            when a non-finite weight is met (the codes of that group are then
+ *            unspecified).  The caller zeroes it.  May be NULL. */
+int qalora_quantize(const qalora_desc* desc, const float* W, void* codes, float* qparams,
+                    int32_t* dev_status, void* cuda_stream);
+
+/* Forward pass, Algorithm 1 / Appendix B Eq. 4:
+ *   y = x * W~ + s * (pool(x) * A) * B.
+ *   x bf16 [m][K];  A bf16 [G][r];  B bf16 [r][N];  y out bf16 [m][N].
+ * Products are bf16 x bf16 accumulated in float32.  Any m >= 0 is accepted; the
+ * kernel is chosen from m (a bandwidth-bound path for a few rows, a
+ * tensor-core path otherwise). */
+int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
+                   const float* qparams, const void* A, const void* B, void* y,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward pass with the base weights frozen (Section 3.1: only A and B are
+ * adjusted).  With l the loss and dy = dl/dy:
+ *   dT = s * dy * B^T;   dx = dy * W~^T + repeat_g(dT * A^T);
+ *   dA = pool(x)^T * dT; dB = s * (pool(x) * A)^T * dy.
+ *   x bf16 [m][K]; dy bf16 [m][N];
+ *   dx out bf16 [m][K]; dA out float32 [G][r]; dB out float32 [r][N].
+ * rank must be > 0.  dx, dA or dB may be NULL to skip that output. */
+int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
+                    const void* codes, const float* qparams, const void* A, const void* B,
+                    void* dx, float* dA, float* dB,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Merge for deployment (Algorithm 1, merge_with_quantization; Appendix B
+ * Eq. 7): folds s*A*B into the zero factors, after which the plain quantized
+ * layer (rank 0) reproduces the adapted one.  For the additive zero of Eq. 1:
+ *   beta'[q, n] = beta[q, n] + s * sum_i A[q, i] * B[i, n]   (alpha unchanged)
+ * which is the paper's zero-point update z' = z - s*A*B/alpha under
+ * z = -beta/alpha.  qparams_out may alias qparams_in. */
+int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A, const void* B,
+                 float* qparams_out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QALORA_H_ */

@@ -1,0 +1,148 @@
+"""Thin ctypes binding of libqalora.so (include/qalora.h).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA
+kernels.  torch supplies device memory and the current stream.  There is no CPU
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_void_p
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqalora.so")
+
+OP_FORWARD, OP_BACKWARD = 0, 1
+
+EXPORTS = (
+    "qalora_version", "qalora_status_string", "qalora_packed_bytes", "qalora_workspace_bytes",
+    "qalora_quantize", "qalora_forward", "qalora_backward", "qalora_merge",
+)
+
+
+class QaloraDesc(Structure):
+    _fields_ = [("d_in", c_int32), ("d_out", c_int32), ("group_size", c_int32), ("bits", c_int32),
+                ("rank", c_int32), ("scale", c_float)]
+
+
+class QaloraError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads libqalora.so (built in-tree by paper_2309_14717_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2309_14717_b200.build` first "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    D = POINTER(QaloraDesc)
+    lib.qalora_version.restype = c_int
+    lib.qalora_version.argtypes = []
+    lib.qalora_status_string.restype = c_char_p
+    lib.qalora_status_string.argtypes = [c_int]
+    lib.qalora_packed_bytes.restype = c_int
+    lib.qalora_packed_bytes.argtypes = [D, POINTER(c_size_t), POINTER(c_size_t)]
+    lib.qalora_workspace_bytes.restype = c_int
+    lib.qalora_workspace_bytes.argtypes = [D, c_int64, c_int, POINTER(c_size_t)]
+    lib.qalora_quantize.restype = c_int
+    lib.qalora_quantize.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.qalora_forward.restype = c_int
+    lib.qalora_forward.argtypes = [D, c_int64] + [c_void_p] * 6 + [c_void_p, c_size_t, c_void_p]
+    lib.qalora_backward.restype = c_int
+    lib.qalora_backward.argtypes = [D, c_int64] + [c_void_p] * 9 + [c_void_p, c_size_t, c_void_p]
+    lib.qalora_merge.restype = c_int
+    lib.qalora_merge.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    _lib = lib
+    return lib
+
+
+def desc(d_in: int, d_out: int, group_size: int, bits: int, rank: int, scale: float) -> QaloraDesc:
+    return QaloraDesc(d_in, d_out, group_size, bits, rank, scale)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("tensors must live on a CUDA device")
+    if not t.is_contiguous():
+        raise ValueError("tensors must be contiguous")
+    return c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return c_void_p(s.cuda_stream)
+
+
+def _check(fn: str, status: int):
+    if status != 0:
+        raise QaloraError(fn, status)
+
+
+def qalora_version() -> int:
+    return int(load().qalora_version())
+
+
+def status_string(status: int) -> str:
+    return load().qalora_status_string(int(status)).decode()
+
+
+def qalora_packed_bytes(d: QaloraDesc):
+    cb, qb = c_size_t(), c_size_t()
+    _check("qalora_packed_bytes", load().qalora_packed_bytes(byref(d), byref(cb), byref(qb)))
+    return cb.value, qb.value
+
+
+def qalora_workspace_bytes(d: QaloraDesc, m: int, op: int) -> int:
+    b = c_size_t()
+    _check("qalora_workspace_bytes", load().qalora_workspace_bytes(byref(d), m, op, byref(b)))
+    return b.value
+
+
+def alloc_packed(d: QaloraDesc, device="cuda"):
+    """Allocates (codes int32 [K/32, N, words], qparams float32 [G, N, 2]) on the device."""
+    cb, qb = qalora_packed_bytes(d)
+    words = cb // 4 // ((d.d_in // 32) * d.d_out)
+    codes = torch.empty((d.d_in // 32, d.d_out, words), dtype=torch.int32, device=device)
+    qparams = torch.empty((d.d_in // d.group_size, d.d_out, 2), dtype=torch.float32, device=device)
+    return codes, qparams
+
+
+def alloc_workspace(d: QaloraDesc, m: int, op: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(qalora_workspace_bytes(d, m, op), 16), dtype=torch.uint8, device=device)
+
+
+def qalora_quantize(d: QaloraDesc, W, codes, qparams, dev_status=None, stream=None):
+    _check("qalora_quantize", load().qalora_quantize(byref(d), _ptr(W), _ptr(codes), _ptr(qparams),
+                                                     _ptr(dev_status), _stream(stream)))
+
+
+def qalora_forward(d: QaloraDesc, m: int, x, codes, qparams, A, B, y, workspace, stream=None):
+    _check("qalora_forward", load().qalora_forward(byref(d), m, _ptr(x), _ptr(codes), _ptr(qparams), _ptr(A),
+                                                   _ptr(B), _ptr(y), _ptr(workspace),
+                                                   workspace.numel() if workspace is not None else 0,
+                                                   _stream(stream)))
+
+
+def qalora_backward(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, dB, workspace, stream=None):
+    _check("qalora_backward", load().qalora_backward(byref(d), m, _ptr(x), _ptr(dy), _ptr(codes), _ptr(qparams),
+                                                     _ptr(A), _ptr(B), _ptr(dx), _ptr(dA), _ptr(dB),
+                                                     _ptr(workspace),
+                                                     workspace.numel() if workspace is not None else 0,
+                                                     _stream(stream)))
+
+
+def qalora_merge(d: QaloraDesc, qparams_in, A, B, qparams_out, stream=None):
+    _check("qalora_merge", load().qalora_merge(byref(d), _ptr(qparams_in), _ptr(A), _ptr(B), _ptr(qparams_out),
+                                               _stream(stream)))

@@ -1,0 +1,191 @@
+// C-ABI entry points: argument checks, scratch layout and kernel dispatch.
+#include "common.cuh"
+
+namespace qalora {
+
+int check_desc(const qalora_desc* d, Shape* sh) {
+  if (d == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (d->d_in <= 0 || d->d_out <= 0 || d->group_size <= 0 || d->rank < 0) return QALORA_ERR_INVALID_ARG;
+  if (d->bits != 2 && d->bits != 3 && d->bits != 4) return QALORA_ERR_INVALID_ARG;
+  if (!(d->scale == d->scale) || d->scale > 3.0e38f || d->scale < -3.0e38f) return QALORA_ERR_INVALID_ARG;
+  if (d->group_size % 32 != 0 || d->d_in % d->group_size != 0) return QALORA_ERR_UNSUPPORTED_SHAPE;
+  if (d->d_out % 8 != 0) return QALORA_ERR_UNSUPPORTED_SHAPE;
+  if (d->rank > 256 || d->rank % 8 != 0) return QALORA_ERR_UNSUPPORTED_SHAPE;
+  sh->K = d->d_in; sh->N = d->d_out; sh->g = d->group_size; sh->G = d->d_in / d->group_size;
+  sh->bits = d->bits; sh->r = d->rank; sh->s = d->scale; sh->words = words_per_unit(d->bits);
+  return QALORA_OK;
+}
+
+Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
+  Workspace w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t at = off; off += round_up(bytes, 256); return at; };
+  const size_t M = (size_t)(m > 0 ? m : 0);
+  const bool bwd = op == QALORA_OP_BACKWARD;
+  w.xp = take(bwd ? M * sh.G * sizeof(float) : 0);
+  w.T = take(M * sh.r * sizeof(float));
+  w.dT = take(bwd ? M * sh.r * sizeof(float) : 0);
+  w.Tb = take(M * sh.r * sizeof(__nv_bfloat16));
+  w.dTb = take(bwd ? M * sh.r * sizeof(__nv_bfloat16) : 0);
+  size_t pb = 0;
+  if (bwd) {
+    const size_t a = atb_partial_bytes(m, sh.G, sh.r), b = atb_partial_bytes(m, sh.r, sh.N);
+    pb = a > b ? a : b;
+  }
+  w.partial_bytes = pb;
+  w.partial = take(pb);
+  w.total = off;
+  return w;
+}
+
+}  // namespace qalora
+
+using namespace qalora;
+
+extern "C" {
+
+int qalora_version(void) { return 100 + QALORA_LAYOUT_VERSION; }
+
+const char* qalora_status_string(int status) {
+  switch (status) {
+    case QALORA_OK: return "ok";
+    case QALORA_ERR_INVALID_ARG: return "invalid argument";
+    case QALORA_ERR_NULL_POINTER: return "null pointer";
+    case QALORA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case QALORA_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+    case QALORA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case QALORA_ERR_CUDA: return "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+int qalora_packed_bytes(const qalora_desc* desc, size_t* code_bytes, size_t* qparam_bytes) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (code_bytes == nullptr || qparam_bytes == nullptr) return QALORA_ERR_NULL_POINTER;
+  *code_bytes = (size_t)(sh.K / 32) * sh.N * sh.words * sizeof(uint32_t);
+  *qparam_bytes = (size_t)sh.G * sh.N * 2 * sizeof(float);
+  return QALORA_OK;
+}
+
+int qalora_workspace_bytes(const qalora_desc* desc, int64_t m, int op, size_t* bytes) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (bytes == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (m < 0 || (op != QALORA_OP_FORWARD && op != QALORA_OP_BACKWARD)) return QALORA_ERR_INVALID_ARG;
+  *bytes = workspace_layout(sh, m, op).total;
+  return QALORA_OK;
+}
+
+int qalora_quantize(const qalora_desc* desc, const float* W, void* codes, float* qparams,
+                    int32_t* dev_status, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (W == nullptr || codes == nullptr || qparams == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(W) || !aligned16(codes) || !aligned16(qparams)) return QALORA_ERR_MISALIGNED;
+  if (dev_status != nullptr && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return QALORA_ERR_MISALIGNED;
+  return launch_quantize(sh, W, static_cast<uint32_t*>(codes), reinterpret_cast<float2*>(qparams), dev_status,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A, const void* B,
+                 float* qparams_out, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (qparams_in == nullptr || qparams_out == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (sh.r > 0 && (A == nullptr || B == nullptr)) return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(qparams_in) || !aligned16(qparams_out) || !aligned16(A) || !aligned16(B)) return QALORA_ERR_MISALIGNED;
+  return launch_merge(sh, reinterpret_cast<const float2*>(qparams_in), static_cast<const __nv_bfloat16*>(A),
+                      static_cast<const __nv_bfloat16*>(B), reinterpret_cast<float2*>(qparams_out),
+                      static_cast<cudaStream_t>(cuda_stream));
+}
+
+int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
+                   const float* qparams, const void* A, const void* B, void* y,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (m < 0) return QALORA_ERR_INVALID_ARG;
+  if (m == 0) return QALORA_OK;
+  if (x == nullptr || codes == nullptr || qparams == nullptr || y == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (sh.r > 0 && (A == nullptr || B == nullptr)) return QALORA_ERR_NULL_POINTER;
+  const Workspace ws = workspace_layout(sh, m, QALORA_OP_FORWARD);
+  if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) || !aligned16(B) ||
+      !aligned16(y) || !aligned16(workspace))
+    return QALORA_ERR_MISALIGNED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* wsp = static_cast<char*>(workspace);
+  float* T = reinterpret_cast<float*>(wsp + ws.T);
+  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
+  if (sh.r > 0) {
+    st = launch_pool_T(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(A),
+                       nullptr, T, Tb, stream);
+    if (st != QALORA_OK) return st;
+  }
+  return launch_simt_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
+                             reinterpret_cast<const float2*>(qparams), T, static_cast<const __nv_bfloat16*>(B),
+                             static_cast<__nv_bfloat16*>(y), stream);
+}
+
+int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
+                    const void* codes, const float* qparams, const void* A, const void* B,
+                    void* dx, float* dA, float* dB,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (m < 0 || sh.r == 0) return QALORA_ERR_INVALID_ARG;
+  if (x == nullptr || dy == nullptr || codes == nullptr || qparams == nullptr || A == nullptr || B == nullptr)
+    return QALORA_ERR_NULL_POINTER;
+  const Workspace ws = workspace_layout(sh, m, QALORA_OP_BACKWARD);
+  if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(x) || !aligned16(dy) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) ||
+      !aligned16(B) || !aligned16(dx) || !aligned16(dA) || !aligned16(dB) || !aligned16(workspace))
+    return QALORA_ERR_MISALIGNED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* wsp = static_cast<char*>(workspace);
+  float* xp = reinterpret_cast<float*>(wsp + ws.xp);
+  float* T = reinterpret_cast<float*>(wsp + ws.T);
+  float* dT = reinterpret_cast<float*>(wsp + ws.dT);
+  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
+  __nv_bfloat16* dTb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.dTb);
+  float* partial = reinterpret_cast<float*>(wsp + ws.partial);
+  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+  const __nv_bfloat16* dyb = static_cast<const __nv_bfloat16*>(dy);
+  const __nv_bfloat16* Ab = static_cast<const __nv_bfloat16*>(A);
+  const __nv_bfloat16* Bb = static_cast<const __nv_bfloat16*>(B);
+
+  if (m == 0) {
+    if (dA != nullptr && (st = cuda_status(cudaMemsetAsync(dA, 0, (size_t)sh.G * sh.r * sizeof(float), stream)))) return st;
+    if (dB != nullptr && (st = cuda_status(cudaMemsetAsync(dB, 0, (size_t)sh.r * sh.N * sizeof(float), stream)))) return st;
+    return QALORA_OK;
+  }
+  if ((st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream)) != QALORA_OK) return st;
+  if (dA != nullptr || dB != nullptr) {
+    if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
+  }
+  if (dx != nullptr) {
+    st = launch_simt_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
+                        dT, Ab, static_cast<__nv_bfloat16*>(dx), stream);
+    if (st != QALORA_OK) return st;
+  }
+  if (dA != nullptr) {
+    st = launch_atb_f32(m, sh.G, sh.r, xp, dT, dA, partial, ws.partial_bytes, stream);
+    if (st != QALORA_OK) return st;
+  }
+  if (dB != nullptr) {
+    st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial, ws.partial_bytes, stream);
+    if (st != QALORA_OK) return st;
+  }
+  return QALORA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+// Shared device/host helpers of the QA-LoRA kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qalora.h"
+
+namespace qalora {
+
+// ---------------------------------------------------------------- host side --
+struct Shape {
+  int K, N, g, G, bits, r, words;   // words = uint32 words per pack unit
+  float s;
+};
+
+__host__ __device__ inline int words_per_unit(int bits) { return bits == 4 ? 4 : (bits == 3 ? 3 : 2); }
+
+// Validates a descriptor and fills `sh`.  Returns a qalora_status.
+int check_desc(const qalora_desc* desc, Shape* sh);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Scratch layout shared by forward and backward (offsets in bytes, 256-aligned).
+struct Workspace {
+  size_t xp;        // float  [M][G]   pooled input                      (backward)
+  size_t T;         // float  [M][r]   s * pool(x) * A                   (both)
+  size_t dT;        // float  [M][r]   s * dy * B^T                      (backward)
+  size_t Tb;        // bf16   [M][r]   T rounded, operand of the tensor-core path
+  size_t dTb;       // bf16   [M][r]   dT rounded
+  size_t partial;   // float  split-K / split-M partial sums
+  size_t partial_bytes;
+  size_t total;
+};
+Workspace workspace_layout(const Shape& sh, int64_t m, int op);
+
+// --------------------------------------------------------------- device side --
+__device__ __forceinline__ float bf16_to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Code of position j (0..31) of a pack unit whose words are u[0..words).
+template <int BITS>
+__device__ __forceinline__ uint32_t unit_code(const uint32_t* u, int j) {
+  if (BITS == 4) {
+    const int e = j & 7;
+    return (u[j >> 3] >> (16 * (e & 1) + 4 * (e >> 1))) & 15u;
+  } else if (BITS == 2) {
+    const int e = j & 15;
+    return (u[j >> 4] >> (16 * (e & 1) + 2 * (e >> 1))) & 3u;
+  } else {
+    const int e = j & 15;
+    const uint32_t lo = (u[j >> 4] >> (16 * (e & 1) + 2 * (e >> 1))) & 3u;
+    const uint32_t hi = (u[2] >> (16 * (j & 1) + (j >> 1))) & 1u;
+    return lo | (hi << 2);
+  }
+}
+
+// ORs code c of position j into the unit's words.
+template <int BITS>
+__device__ __forceinline__ void unit_insert(uint32_t* u, int j, uint32_t c) {
+  if (BITS == 4) {
+    const int e = j & 7;
+    u[j >> 3] |= c << (16 * (e & 1) + 4 * (e >> 1));
+  } else if (BITS == 2) {
+    const int e = j & 15;
+    u[j >> 4] |= c << (16 * (e & 1) + 2 * (e >> 1));
+  } else {
+    const int e = j & 15;
+    u[j >> 4] |= (c & 3u) << (16 * (e & 1) + 2 * (e >> 1));
+    u[2] |= (c >> 2) << (16 * (j & 1) + (j >> 1));
+  }
+}
+
+// Launch helpers implemented in the kernel files (all asynchronous on `st`).
+int launch_quantize(const Shape& sh, const float* W, uint32_t* codes, float2* qparams,
+                    int32_t* dev_status, cudaStream_t st);
+int launch_merge(const Shape& sh, const float2* qin, const __nv_bfloat16* A, const __nv_bfloat16* B,
+                 float2* qout, cudaStream_t st);
+// pool + T = s*pool(x)*A.  xp may be NULL (not stored).  Tb may be NULL.
+int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv_bfloat16* A,
+                  float* xp, float* T, __nv_bfloat16* Tb, cudaStream_t st);
+int launch_simt_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
+                        const float2* qparams, const float* T, const __nv_bfloat16* B,
+                        __nv_bfloat16* y, cudaStream_t st);
+int launch_dT(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const __nv_bfloat16* B,
+              float* dT, __nv_bfloat16* dTb, cudaStream_t st);
+int launch_simt_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint32_t* codes,
+                   const float2* qparams, const float* dT, const __nv_bfloat16* A,
+                   __nv_bfloat16* dx, cudaStream_t st);
+// out[p][q] = sum_m X[m][p] * Y[m][q]   (X float [M][P]; Y bf16 or float [M][Q])
+size_t atb_partial_bytes(int64_t M, int P, int Q);
+int launch_atb_bf16(int64_t M, int P, int Q, const float* X, const __nv_bfloat16* Y, float* out,
+                    float* partial, size_t partial_bytes, cudaStream_t st);
+int launch_atb_f32(int64_t M, int P, int Q, const float* X, const float* Y, float* out,
+                   float* partial, size_t partial_bytes, cudaStream_t st);
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? QALORA_OK : QALORA_ERR_CUDA; }
+
+}  // namespace qalora

@@ -1,0 +1,114 @@
+// Group-wise min-max quantization + bit packing (Eq. 1 per group, Section 3.3)
+// and the merge of the adapter into the zero factors (Appendix B Eq. 7).
+// Both are streaming, HBM-bound kernels: one thread owns one output column of
+// one quantization group, so a warp reads 128 contiguous bytes of each W row.
+#include <float.h>
+
+#include "common.cuh"
+
+namespace qalora {
+
+constexpr int QCOLS = 128;   // columns (threads) per block
+
+// Each thread: two passes over its g weights.  Pass 1 finds min/max, pass 2
+// re-reads (L1/L2 hits), rounds and packs one 32-channel unit at a time.  Every
+// floating-point step is a single IEEE fp32 operation (no FMA contraction, no
+// reciprocal), so the integer decision is reproducible bit for bit on a CPU.
+template <int BITS>
+__global__ void __launch_bounds__(QCOLS)
+quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
+                float2* __restrict__ qparams, int N, int g, int ntiles, int32_t* dev_status) {
+  constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
+  constexpr float QMAX = float((1 << BITS) - 1);
+  const int q = blockIdx.x / ntiles;
+  const int n = (blockIdx.x % ntiles) * QCOLS + threadIdx.x;
+  if (n >= N) return;
+  const float* w = W + (size_t)q * g * N + n;
+
+  float lo = FLT_MAX, hi = -FLT_MAX;
+  bool bad = false;
+  for (int k0 = 0; k0 < g; k0 += 32) {
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __ldg(w + (size_t)(k0 + j) * N);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      bad |= !(fabsf(v[j]) <= FLT_MAX);
+      lo = fminf(lo, v[j]);
+      hi = fmaxf(hi, v[j]);
+    }
+  }
+  const float alpha = (hi == lo) ? 1.0f : __fdiv_rn(__fsub_rn(hi, lo), QMAX);
+  const float beta = lo;
+  qparams[(size_t)q * N + n] = make_float2(alpha, beta);
+  if (bad && dev_status != nullptr) atomicOr(dev_status, 1);
+
+  const int kb0 = q * (g / 32);
+  for (int k0 = 0; k0 < g; k0 += 32) {
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __ldg(w + (size_t)(k0 + j) * N);
+    uint32_t u[WORDS];
+#pragma unroll
+    for (int i = 0; i < WORDS; ++i) u[i] = 0u;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const float t = __fdiv_rn(__fsub_rn(v[j], beta), alpha);
+      float c = rintf(t);                              // round half to even
+      c = fminf(fmaxf(c, 0.0f), QMAX);
+      unit_insert<BITS>(u, j, (uint32_t)(int)c);
+    }
+    uint32_t* dst = codes + ((size_t)(kb0 + k0 / 32) * N + n) * WORDS;
+    if (WORDS == 4) {
+      *reinterpret_cast<uint4*>(dst) = make_uint4(u[0], u[1], u[2], u[3]);
+    } else if (WORDS == 2) {
+      *reinterpret_cast<uint2*>(dst) = make_uint2(u[0], u[1]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < WORDS; ++i) dst[i] = u[i];
+    }
+  }
+}
+
+int launch_quantize(const Shape& sh, const float* W, uint32_t* codes, float2* qparams,
+                    int32_t* dev_status, cudaStream_t st) {
+  const int ntiles = (sh.N + QCOLS - 1) / QCOLS;
+  const long long blocks = (long long)sh.G * ntiles;
+  if (blocks > 0x7fffffffLL) return QALORA_ERR_UNSUPPORTED_SHAPE;
+  dim3 grid((unsigned)blocks), block(QCOLS);
+  if (sh.bits == 4) quantize_kernel<4><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
+  else if (sh.bits == 3) quantize_kernel<3><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
+  else quantize_kernel<2><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
+  return cuda_status(cudaGetLastError());
+}
+
+// beta'[q][n] = beta[q][n] + s * sum_i A[q][i] * B[i][n]; alpha is copied.
+// One thread per (group, column); the row of A sits in shared memory.  In-place
+// use is safe: a thread reads only the element it then writes.
+__global__ void __launch_bounds__(QCOLS)
+merge_kernel(const float2* __restrict__ qin, const __nv_bfloat16* __restrict__ A,
+             const __nv_bfloat16* __restrict__ B, float2* __restrict__ qout,
+             int N, int r, float s, int ntiles) {
+  extern __shared__ float a_row[];
+  const int q = blockIdx.x / ntiles;
+  const int n = (blockIdx.x % ntiles) * QCOLS + threadIdx.x;
+  for (int i = threadIdx.x; i < r; i += QCOLS) a_row[i] = bf16_to_float(A[(size_t)q * r + i]);
+  __syncthreads();
+  if (n >= N) return;
+  float acc = 0.0f;
+  for (int i = 0; i < r; ++i) acc = fmaf(a_row[i], bf16_to_float(B[(size_t)i * N + n]), acc);
+  float2 p = qin[(size_t)q * N + n];
+  p.y = fmaf(s, acc, p.y);
+  qout[(size_t)q * N + n] = p;
+}
+
+int launch_merge(const Shape& sh, const float2* qin, const __nv_bfloat16* A, const __nv_bfloat16* B,
+                 float2* qout, cudaStream_t st) {
+  const int ntiles = (sh.N + QCOLS - 1) / QCOLS;
+  const long long blocks = (long long)sh.G * ntiles;
+  if (blocks > 0x7fffffffLL) return QALORA_ERR_UNSUPPORTED_SHAPE;
+  merge_kernel<<<(unsigned)blocks, QCOLS, sh.r * sizeof(float), st>>>(qin, A, B, qout, sh.N, sh.r, sh.s, ntiles);
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace qalora

@@ -1,0 +1,393 @@
+// General-shape CUDA-core kernels of the QA-LoRA layer.  They accept every
+// supported shape and serve (a) shapes the tensor-core kernels do not tile and
+// (b) the small rank-r side products.  fp32 accumulation throughout.
+#include "common.cuh"
+
+namespace qalora {
+
+// ------------------------------------------------------------ pool and T -----
+// One block per token row: xp[q] = sum of the g channels of group q
+// (Appendix B Eq. 3), then T[i] = s * sum_q xp[q] * A[q][i].
+constexpr int POOL_THREADS = 256;
+
+__global__ void __launch_bounds__(POOL_THREADS)
+pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
+              float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
+              int K, int g, int G, int r, float s) {
+  extern __shared__ float xp[];                       // [G]
+  const size_t m = blockIdx.x;
+  const __nv_bfloat16* xr = x + m * (size_t)K;
+  // four lanes per group, 8 channels (16 bytes) per lane and step; g is a multiple of 32
+  for (int q0 = 0; q0 < G; q0 += POOL_THREADS / 4) {   // uniform trip count: the shuffles see whole warps
+    const int q = q0 + threadIdx.x / 4;
+    const int lane4 = threadIdx.x & 3;
+    float acc = 0.0f;
+    if (q < G) {
+      for (int k = lane4 * 8; k < g; k += 32) {
+        const uint4 v = *reinterpret_cast<const uint4*>(xr + (size_t)q * g + k);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(h[i]);
+          acc += f.x + f.y;
+        }
+      }
+    }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+    if (lane4 == 0 && q < G) {
+      xp[q] = acc;
+      if (xp_out != nullptr) xp_out[m * (size_t)G + q] = acc;
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < r; i += POOL_THREADS) {
+    float acc = 0.0f;
+    for (int q = 0; q < G; ++q) acc = fmaf(xp[q], bf16_to_float(A[(size_t)q * r + i]), acc);
+    acc *= s;
+    T[m * (size_t)r + i] = acc;
+    if (Tb != nullptr) Tb[m * (size_t)r + i] = __float2bfloat16_rn(acc);
+  }
+}
+
+int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv_bfloat16* A,
+                  float* xp, float* T, __nv_bfloat16* Tb, cudaStream_t st) {
+  if (M == 0) return QALORA_OK;
+  pool_T_kernel<<<(unsigned)M, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G,
+                                                                        sh.r, sh.s);
+  return cuda_status(cudaGetLastError());
+}
+
+// ------------------------------------------------------------- dT ------------
+// dT[m][i] = s * sum_n dy[m][n] * B[i][n]; one block per row, one warp per i.
+constexpr int DT_THREADS = 256;
+
+__global__ void __launch_bounds__(DT_THREADS)
+dT_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ B,
+          float* __restrict__ dT, __nv_bfloat16* __restrict__ dTb, int N, int r, float s) {
+  const size_t m = blockIdx.x;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const __nv_bfloat16* dyr = dy + m * (size_t)N;
+  for (int i = warp; i < r; i += DT_THREADS / 32) {
+    const __nv_bfloat16* br = B + (size_t)i * N;
+    float acc = 0.0f;
+    for (int n = lane * 8; n < N; n += 256) {            // N is a multiple of 8
+      const uint4 a = *reinterpret_cast<const uint4*>(dyr + n);
+      const uint4 b = *reinterpret_cast<const uint4*>(br + n);
+      const __nv_bfloat162* ha = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 fa = __bfloat1622float2(ha[j]), fb = __bfloat1622float2(hb[j]);
+        acc = fmaf(fa.x, fb.x, acc);
+        acc = fmaf(fa.y, fb.y, acc);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) {
+      acc *= s;
+      dT[m * (size_t)r + i] = acc;
+      if (dTb != nullptr) dTb[m * (size_t)r + i] = __float2bfloat16_rn(acc);
+    }
+  }
+}
+
+int launch_dT(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const __nv_bfloat16* B,
+              float* dT, __nv_bfloat16* dTb, cudaStream_t st) {
+  if (M == 0) return QALORA_OK;
+  dT_kernel<<<(unsigned)M, DT_THREADS, 0, st>>>(dy, B, dT, dTb, sh.N, sh.r, sh.s);
+  return cuda_status(cudaGetLastError());
+}
+
+// ------------------------------------------------------ tiled main products --
+// 64 x 64 output tile, 256 threads, 4 x 4 outputs per thread, 32-deep steps.
+constexpr int TM = 64, TN = 64, TK = 32, SIMT_THREADS = 256;
+
+// y[m][n] = sum_k x[m][k] * W~[k][n] + sum_i T[m][i] * B[i][n]
+template <int BITS>
+__global__ void __launch_bounds__(SIMT_THREADS)
+simt_forward_kernel(const __nv_bfloat16* __restrict__ x, const uint32_t* __restrict__ codes,
+                    const float2* __restrict__ qparams, const float* __restrict__ T,
+                    const __nv_bfloat16* __restrict__ B, __nv_bfloat16* __restrict__ y,
+                    long long M, int K, int N, int g, int r) {
+  constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
+  __shared__ __align__(16) float xs[TK][TM + 4];
+  __shared__ __align__(16) float ws[TK][TN + 4];
+  const int tid = threadIdx.x;
+  const long long m0 = (long long)blockIdx.y * TM;
+  const int n0 = blockIdx.x * TN;
+  const int ty = tid / 16, tx = tid % 16;
+  float acc[4][4] = {};
+
+  const int lrow = tid / 4, lseg = (tid % 4) * 8;       // x loader: row, 8-channel segment
+  const int un = tid % 64, uj = (tid / 64) * 8;         // W loader: column, first position
+  for (int k0 = 0; k0 < K; k0 += TK) {
+    {
+      float v[8] = {};
+      if (m0 + lrow < M) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(x + (size_t)(m0 + lrow) * K + k0 + lseg);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(h[i]);
+          v[2 * i] = f.x; v[2 * i + 1] = f.y;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) xs[lseg + i][lrow] = v[i];
+    }
+    {
+      const int n = n0 + un;
+      if (n < N) {
+        const uint32_t* u = codes + ((size_t)(k0 / 32) * N + n) * WORDS;
+        uint32_t w[WORDS];
+#pragma unroll
+        for (int i = 0; i < WORDS; ++i) w[i] = __ldg(u + i);
+        const float2 ab = __ldg(qparams + (size_t)(k0 / g) * N + n);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ws[uj + i][un] = fmaf(ab.x, (float)unit_code<BITS>(w, uj + i), ab.y);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ws[uj + i][un] = 0.0f;
+      }
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int kk = 0; kk < TK; ++kk) {
+      const float4 a = *reinterpret_cast<const float4*>(&xs[kk][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&ws[kk][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  // adapter term and store
+  const int nb = n0 + tx * 4;
+  if (nb >= N) return;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long long m = m0 + ty * 4 + i;
+    if (m >= M) continue;
+    for (int t = 0; t < r; ++t) {
+      const float tv = __ldg(T + (size_t)m * r + t);
+      const uint2 raw = *reinterpret_cast<const uint2*>(B + (size_t)t * N + nb);
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      const float2 b0 = __bfloat1622float2(h[0]), b1 = __bfloat1622float2(h[1]);
+      acc[i][0] = fmaf(tv, b0.x, acc[i][0]); acc[i][1] = fmaf(tv, b0.y, acc[i][1]);
+      acc[i][2] = fmaf(tv, b1.x, acc[i][2]); acc[i][3] = fmaf(tv, b1.y, acc[i][3]);
+    }
+    __nv_bfloat162 o[2] = {__floats2bfloat162_rn(acc[i][0], acc[i][1]), __floats2bfloat162_rn(acc[i][2], acc[i][3])};
+    *reinterpret_cast<uint2*>(y + (size_t)m * N + nb) = *reinterpret_cast<uint2*>(o);
+  }
+}
+
+int launch_simt_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
+                        const float2* qparams, const float* T, const __nv_bfloat16* B,
+                        __nv_bfloat16* y, cudaStream_t st) {
+  if (M == 0) return QALORA_OK;
+  const long long mt = (M + TM - 1) / TM;
+  if (mt > 65535) return QALORA_ERR_UNSUPPORTED_SHAPE;
+  dim3 grid((sh.N + TN - 1) / TN, (unsigned)mt), block(SIMT_THREADS);
+#define QALORA_FWD(BITS) simt_forward_kernel<BITS><<<grid, block, 0, st>>>(x, codes, qparams, T, B, y, M, sh.K, sh.N, sh.g, sh.r)
+  if (sh.bits == 4) QALORA_FWD(4); else if (sh.bits == 3) QALORA_FWD(3); else QALORA_FWD(2);
+#undef QALORA_FWD
+  return cuda_status(cudaGetLastError());
+}
+
+// dx[m][k] = sum_n dy[m][n] * W~[k][n] + sum_i dT[m][i] * A[k/g][i]
+template <int BITS>
+__global__ void __launch_bounds__(SIMT_THREADS)
+simt_dx_kernel(const __nv_bfloat16* __restrict__ dy, const uint32_t* __restrict__ codes,
+               const float2* __restrict__ qparams, const float* __restrict__ dT,
+               const __nv_bfloat16* __restrict__ A, __nv_bfloat16* __restrict__ dx,
+               long long M, int K, int N, int g, int r) {
+  constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
+  __shared__ __align__(16) float ds[TK][TM + 4];        // [n][m]
+  __shared__ __align__(16) float ws[TK][TN + 4];        // [n][k]
+  const int tid = threadIdx.x;
+  const long long m0 = (long long)blockIdx.y * TM;
+  const int k0 = blockIdx.x * TN;                       // 64 output channels = 2 k-blocks
+  const int ty = tid / 16, tx = tid % 16;
+  float acc[4][4] = {};
+
+  const int lrow = tid / 4, lseg = (tid % 4) * 8;
+  const int un = tid % 32, ukb = (tid / 32) % 2, uj = (tid / 64) * 8;
+  for (int n0 = 0; n0 < N; n0 += TK) {
+    {
+      float v[8] = {};
+      if (m0 + lrow < M && n0 + lseg < N) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(dy + (size_t)(m0 + lrow) * N + n0 + lseg);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(h[i]);
+          v[2 * i] = f.x; v[2 * i + 1] = f.y;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ds[lseg + i][lrow] = v[i];
+    }
+    {
+      const int n = n0 + un, k = k0 + ukb * 32;
+      if (n < N && k < K) {
+        const uint32_t* u = codes + ((size_t)(k / 32) * N + n) * WORDS;
+        uint32_t w[WORDS];
+#pragma unroll
+        for (int i = 0; i < WORDS; ++i) w[i] = __ldg(u + i);
+        const float2 ab = __ldg(qparams + (size_t)(k / g) * N + n);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          ws[un][ukb * 32 + uj + i] = fmaf(ab.x, (float)unit_code<BITS>(w, uj + i), ab.y);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ws[un][ukb * 32 + uj + i] = 0.0f;
+      }
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int nn = 0; nn < TK; ++nn) {
+      const float4 a = *reinterpret_cast<const float4*>(&ds[nn][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&ws[nn][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  const int kc = k0 + tx * 4;
+  if (kc >= K) return;
+  const int q = kc / g;                                 // 4 consecutive channels share a group
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long long m = m0 + ty * 4 + i;
+    if (m >= M) continue;
+    float lora = 0.0f;
+    for (int t = 0; t < r; ++t)
+      lora = fmaf(__ldg(dT + (size_t)m * r + t), bf16_to_float(A[(size_t)q * r + t]), lora);
+    __nv_bfloat162 o[2] = {__floats2bfloat162_rn(acc[i][0] + lora, acc[i][1] + lora),
+                           __floats2bfloat162_rn(acc[i][2] + lora, acc[i][3] + lora)};
+    *reinterpret_cast<uint2*>(dx + (size_t)m * K + kc) = *reinterpret_cast<uint2*>(o);
+  }
+}
+
+int launch_simt_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint32_t* codes,
+                   const float2* qparams, const float* dT, const __nv_bfloat16* A,
+                   __nv_bfloat16* dx, cudaStream_t st) {
+  if (M == 0) return QALORA_OK;
+  const long long mt = (M + TM - 1) / TM;
+  if (mt > 65535) return QALORA_ERR_UNSUPPORTED_SHAPE;
+  dim3 grid((sh.K + TN - 1) / TN, (unsigned)mt), block(SIMT_THREADS);
+#define QALORA_DX(BITS) simt_dx_kernel<BITS><<<grid, block, 0, st>>>(dy, codes, qparams, dT, A, dx, M, sh.K, sh.N, sh.g, sh.r)
+  if (sh.bits == 4) QALORA_DX(4); else if (sh.bits == 3) QALORA_DX(3); else QALORA_DX(2);
+#undef QALORA_DX
+  return cuda_status(cudaGetLastError());
+}
+
+// ----------------------------------------------- X^T * Y reductions over M ---
+// out[p][q] = sum_m X[m][p] * Y[m][q].  The token range is split over
+// blockIdx.z; each split writes its own partial tile and a second kernel adds
+// the partials in a fixed order, so the result does not depend on scheduling.
+template <typename TY> __device__ __forceinline__ float load_as_float(const TY* p);
+template <> __device__ __forceinline__ float load_as_float<float>(const float* p) { return __ldg(p); }
+template <> __device__ __forceinline__ float load_as_float<__nv_bfloat16>(const __nv_bfloat16* p) { return bf16_to_float(*p); }
+
+template <typename TY>
+__global__ void __launch_bounds__(SIMT_THREADS)
+atb_partial_kernel(const float* __restrict__ X, const TY* __restrict__ Y, float* __restrict__ partial,
+                   long long M, int P, int Q, long long rows_per_split) {
+  __shared__ __align__(16) float xs[TK][TM + 4];
+  __shared__ __align__(16) float ys[TK][TN + 4];
+  const int tid = threadIdx.x;
+  const int p0 = blockIdx.y * TM, q0 = blockIdx.x * TN;
+  const int ty = tid / 16, tx = tid % 16;
+  const long long mbeg = (long long)blockIdx.z * rows_per_split;
+  const long long mend = min(M, mbeg + rows_per_split);
+  float acc[4][4] = {};
+  for (long long m0 = mbeg; m0 < mend; m0 += TK) {
+    for (int e = tid; e < TK * TM; e += SIMT_THREADS) {
+      const int mm = e / TM, c = e % TM;
+      const long long m = m0 + mm;
+      xs[mm][c] = (m < mend && p0 + c < P) ? __ldg(X + (size_t)m * P + p0 + c) : 0.0f;
+      ys[mm][c] = (m < mend && q0 + c < Q) ? load_as_float<TY>(Y + (size_t)m * Q + q0 + c) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int mm = 0; mm < TK; ++mm) {
+      const float4 a = *reinterpret_cast<const float4*>(&xs[mm][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&ys[mm][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* dst = partial + (size_t)blockIdx.z * P * Q;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int p = p0 + ty * 4 + i, q = q0 + tx * 4 + j;
+      if (p < P && q < Q) dst[(size_t)p * Q + q] = acc[i][j];
+    }
+}
+
+__global__ void sum_partials_kernel(const float* __restrict__ partial, float* __restrict__ out,
+                                    size_t count, int splits) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  float acc = 0.0f;
+  for (int z = 0; z < splits; ++z) acc += partial[(size_t)z * count + i];
+  out[i] = acc;
+}
+
+static long long atb_splits(int64_t M, int P, int Q) {
+  const int tiles = ((P + TM - 1) / TM) * ((Q + TN - 1) / TN);
+  long long splits = (2 * 148 + tiles - 1) / tiles;        // about two blocks per SM
+  const long long max_by_rows = (M + 4 * TK - 1) / (4 * TK);
+  if (splits > max_by_rows) splits = max_by_rows;
+  return splits < 1 ? 1 : splits;
+}
+
+size_t atb_partial_bytes(int64_t M, int P, int Q) {
+  const size_t count = (size_t)P * Q;
+  if (count == 0 || M <= 0) return 0;
+  return (size_t)atb_splits(M, P, Q) * count * sizeof(float);
+}
+
+template <typename TY>
+static int launch_atb(int64_t M, int P, int Q, const float* X, const TY* Y, float* out,
+                      float* partial, size_t partial_bytes, cudaStream_t st) {
+  const size_t count = (size_t)P * Q;
+  if (count == 0) return QALORA_OK;
+  if (M == 0) return cuda_status(cudaMemsetAsync(out, 0, count * sizeof(float), st));
+  long long splits = atb_splits(M, P, Q);
+  const long long max_by_space = (long long)(partial_bytes / (count * sizeof(float)));
+  if (splits > max_by_space) splits = max_by_space;
+  if (splits < 1) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  long long rows = (M + splits - 1) / splits;
+  rows = (rows + TK - 1) / TK * TK;
+  splits = (M + rows - 1) / rows;
+  dim3 grid((Q + TN - 1) / TN, (P + TM - 1) / TM, (unsigned)splits);
+  atb_partial_kernel<TY><<<grid, SIMT_THREADS, 0, st>>>(X, Y, partial, M, P, Q, rows);
+  sum_partials_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(partial, out, count, (int)splits);
+  return cuda_status(cudaGetLastError());
+}
+
+int launch_atb_bf16(int64_t M, int P, int Q, const float* X, const __nv_bfloat16* Y, float* out,
+                    float* partial, size_t partial_bytes, cudaStream_t st) {
+  return launch_atb<__nv_bfloat16>(M, P, Q, X, Y, out, partial, partial_bytes, st);
+}
+int launch_atb_f32(int64_t M, int P, int Q, const float* X, const float* Y, float* out,
+                   float* partial, size_t partial_bytes, cudaStream_t st) {
+  return launch_atb<float>(M, P, Q, X, Y, out, partial, partial_bytes, st);
+}
+
+}  // namespace qalora

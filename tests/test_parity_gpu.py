@@ -1,0 +1,182 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle on the
+same seeded inputs.  Integer results (codes, packed words) and the quantization
+parameters must be bit-exact; floating-point results must satisfy
+max|gpu - ref| / max|ref| <= 5e-3 (bf16 inputs/outputs, fp32 accumulation)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import qalora_oracle as O
+from paper_2309_14717_b200 import binding as Q
+from paper_2309_14717_b200.synthetic import CONFIGS, LayerConfig, make_inputs, to_f64
+
+pytestmark = pytest.mark.gpu
+TOL = 5e-3
+
+
+def rel_err(got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape
+    if ref.size == 0:
+        return 0.0
+    denom = np.max(np.abs(ref))
+    return float(np.max(np.abs(got - ref)) / (denom if denom > 0 else 1.0))
+
+
+class GpuLayer:
+    """Quantizes cfg's synthetic weights on the GPU and keeps everything on the device."""
+
+    def __init__(self, cfg: LayerConfig, need=("W", "x", "A", "B", "dy")):
+        self.cfg = cfg
+        self.cpu = make_inputs(cfg, need=need)
+        self.dev = {k: v.cuda() for k, v in self.cpu.items()}
+        self.d = Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, cfg.rank, cfg.scale)
+        self.codes, self.qparams = Q.alloc_packed(self.d)
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        Q.qalora_quantize(self.d, self.dev["W"], self.codes, self.qparams, self.status)
+        torch.cuda.synchronize()
+
+    def forward(self, x=None, qparams=None, rank=None):
+        cfg = self.cfg
+        x = self.dev["x"] if x is None else x
+        d = self.d if rank is None else Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, rank, cfg.scale)
+        m = x.shape[0]
+        y = torch.empty((m, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+        ws = Q.alloc_workspace(d, m, Q.OP_FORWARD)
+        Q.qalora_forward(d, m, x, self.codes, self.qparams if qparams is None else qparams,
+                         self.dev.get("A") if d.rank else None, self.dev.get("B") if d.rank else None, y, ws)
+        torch.cuda.synchronize()
+        return y
+
+    def backward(self):
+        cfg = self.cfg
+        m = self.dev["x"].shape[0]
+        dx = torch.empty((m, cfg.d_in), dtype=torch.bfloat16, device="cuda")
+        dA = torch.full((cfg.groups, cfg.rank), float("nan"), dtype=torch.float32, device="cuda")
+        dB = torch.full((cfg.rank, cfg.d_out), float("nan"), dtype=torch.float32, device="cuda")
+        ws = Q.alloc_workspace(self.d, m, Q.OP_BACKWARD)
+        Q.qalora_backward(self.d, m, self.dev["x"], self.dev["dy"], self.codes, self.qparams, self.dev["A"],
+                          self.dev["B"], dx, dA, dB, ws)
+        torch.cuda.synchronize()
+        return dx, dA, dB
+
+    def oracle_quant(self):
+        cfg = self.cfg
+        return O.quantize(self.cpu["W"].numpy(), cfg.group_size, cfg.bits)
+
+
+def check_quantize(layer: GpuLayer):
+    cfg = layer.cfg
+    codes, alpha, beta = layer.oracle_quant()
+    packed = O.pack(codes, cfg.bits)
+    got_words = layer.codes.cpu().numpy().view(np.uint32)
+    assert np.array_equal(got_words, packed), "packed codes differ"
+    qp = layer.qparams.cpu().numpy()
+    assert np.array_equal(qp[..., 0], alpha) and np.array_equal(qp[..., 1], beta), "alpha/beta differ"
+    assert int(layer.status.item()) == 0
+    return codes, alpha, beta
+
+
+SMALL = [
+    # name, K, N, g, bits, r, s, M
+    ("tiny4", 64, 64, 32, 4, 8, 1.0, 5),
+    ("ragged4", 320, 200, 32, 4, 16, 0.5, 77),
+    ("ragged3", 192, 136, 64, 3, 24, 1.5, 130),
+    ("ragged2", 256, 72, 128, 2, 8, 2.0, 33),
+    ("g64_4", 512, 384, 64, 4, 64, 1.0, 200),
+    ("colwise", 128, 64, 128, 4, 8, 1.0, 16),
+]
+
+
+@pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
+def test_small_shapes_all_ops(case):
+    name, K, N, g, bits, r, s, M = case
+    cfg = LayerConfig(name, K, N, g, bits, r, s, M, dy_std=1.0, outlier_frac=0.01, seed=len(name) + K)
+    layer = GpuLayer(cfg)
+    codes, alpha, beta = check_quantize(layer)
+    x, A, B, dy = (to_f64(layer.cpu[k]) for k in ("x", "A", "B", "dy"))
+    y_ref = O.forward(x, codes, alpha, beta, g, A, B, s)
+    assert rel_err(layer.forward().float().cpu().numpy(), y_ref) <= TOL
+    dx, dA, dB = layer.backward()
+    dx_ref, dA_ref, dB_ref = O.backward(x, dy, codes, alpha, beta, g, A, B, s)
+    assert rel_err(dx.float().cpu().numpy(), dx_ref) <= TOL
+    assert rel_err(dA.cpu().numpy(), dA_ref) <= TOL
+    assert rel_err(dB.cpu().numpy(), dB_ref) <= TOL
+    # merge, then the plain quantized layer must reproduce the adapted one
+    q2 = torch.empty_like(layer.qparams)
+    Q.qalora_merge(layer.d, layer.qparams, layer.dev["A"], layer.dev["B"], q2)
+    torch.cuda.synchronize()
+    q2n = q2.cpu().numpy()
+    assert np.array_equal(q2n[..., 0], alpha)
+    assert rel_err(q2n[..., 1], O.merge(beta, A, B, s)) <= TOL
+    y_merged = layer.forward(qparams=q2, rank=0)
+    assert rel_err(y_merged.float().cpu().numpy(), y_ref) <= TOL
+    # in-place merge gives the same bytes
+    q3 = layer.qparams.clone()
+    Q.qalora_merge(layer.d, q3, layer.dev["A"], layer.dev["B"], q3)
+    torch.cuda.synchronize()
+    assert torch.equal(q3, q2)
+
+
+def test_config1_full():
+    cfg = CONFIGS["cfg1_512"]
+    layer = GpuLayer(cfg)
+    codes, alpha, beta = check_quantize(layer)
+    x, A, B, dy = (to_f64(layer.cpu[k]) for k in ("x", "A", "B", "dy"))
+    g, s = cfg.group_size, cfg.scale
+    assert rel_err(layer.forward().float().cpu().numpy(), O.forward(x, codes, alpha, beta, g, A, B, s)) <= TOL
+    dx, dA, dB = layer.backward()
+    dx_ref, dA_ref, dB_ref = O.backward(x, dy, codes, alpha, beta, g, A, B, s)
+    assert rel_err(dx.float().cpu().numpy(), dx_ref) <= TOL
+    assert rel_err(dA.cpu().numpy(), dA_ref) <= TOL
+    assert rel_err(dB.cpu().numpy(), dB_ref) <= TOL
+
+
+@pytest.mark.parametrize("M", [1, 4, 16])
+def test_config2_small_m_forward_and_merge(M):
+    cfg = CONFIGS["cfg2_7b_attn"].with_(tokens=M)
+    layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
+    codes, alpha, beta = check_quantize(layer)
+    x, A, B = (to_f64(layer.cpu[k]) for k in ("x", "A", "B"))
+    g, s = cfg.group_size, cfg.scale
+    y_ref = O.forward(x, codes, alpha, beta, g, A, B, s)
+    assert rel_err(layer.forward().float().cpu().numpy(), y_ref) <= TOL
+    q2 = torch.empty_like(layer.qparams)
+    Q.qalora_merge(layer.d, layer.qparams, layer.dev["A"], layer.dev["B"], q2)
+    assert rel_err(q2.cpu().numpy()[..., 1], O.merge(beta, A, B, s)) <= TOL
+    assert rel_err(layer.forward(qparams=q2, rank=0).float().cpu().numpy(), y_ref) <= TOL
+
+
+def test_edge_cases():
+    cfg = LayerConfig("edge", 64, 64, 32, 4, 8, 1.0, 3, seed=9)
+    layer = GpuLayer(cfg)
+    # constant groups and an all-zero matrix
+    W = torch.zeros((64, 64), dtype=torch.float32)
+    W[32:, 5] = 0.75
+    W[:32, 7] = torch.linspace(-1, 1, 32)
+    Wd = W.cuda()
+    Q.qalora_quantize(layer.d, Wd, layer.codes, layer.qparams, layer.status)
+    torch.cuda.synchronize()
+    codes, alpha, beta = O.quantize(W.numpy(), 32, 4)
+    assert np.array_equal(layer.codes.cpu().numpy().view(np.uint32), O.pack(codes, 4))
+    qp = layer.qparams.cpu().numpy()
+    assert np.array_equal(qp[..., 0], alpha) and np.array_equal(qp[..., 1], beta)
+    # a non-finite weight raises the device status bit instead of trapping
+    Wd[3, 3] = float("inf")
+    Q.qalora_quantize(layer.d, Wd, layer.codes, layer.qparams, layer.status)
+    torch.cuda.synchronize()
+    assert int(layer.status.item()) & 1
+    # m = 0 is a no-op that still succeeds
+    empty = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
+    assert layer.forward(x=empty).shape == (0, 64)
+
+
+def test_results_do_not_depend_on_scheduling():
+    cfg = LayerConfig("det", 256, 256, 32, 4, 16, 1.0, 300, seed=5)
+    layer = GpuLayer(cfg)
+    y1, b1 = layer.forward(), layer.backward()
+    y2, b2 = layer.forward(), layer.backward()
+    assert torch.equal(y1, y2)
+    for a, b in zip(b1, b2):
+        assert torch.equal(a, b)
