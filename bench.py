@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the QA-LoRA linear layer on B200.
+
+One step = one pass of the whole layer path over one batch, for both LLaMA-7B
+MLP shapes (4096 -> 11008 and 11008 -> 4096, INT4, group size 32, rank 64,
+M = 8192 tokens): quantize + pack, forward, backward (dX, dA, dB), merge, and
+the merged layer's single-token forward.  The reported value is the forward +
+backward TFLOP/s (algorithmic flops of Algorithm 1 and its gradients divided
+by the time of the whole step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
+runs the same step on its own batch (data parallel over tokens) and the
+adapter gradients are all-reduced over NCCL.  `--impl reference` times the CPU
+oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "QA-LoRA W4 linear fwd+bwd TFLOP/s (M=8192) & M=1 GB/s, % of roofline"
+WORKLOAD = "cfg3_7b_mlp_int4_g32_r64_m8192"
+SHAPES = ("cfg3_7b_up", "cfg3_7b_down")
+SMALL_M = "cfg2_7b_attn"
+
+
+# ----------------------------------------------------------- work accounting --
+def fwd_flops(M, K, N, G, r):
+    return 2 * M * K * N + M * K + 2 * M * G * r + 2 * M * r * N
+
+
+def bwd_flops(M, K, N, G, r):
+    return 2 * M * K * N + 2 * M * N * r + 2 * M * r * G + M * K + 2 * M * r * N + 2 * M * G * r
+
+
+def fwd_bytes(M, K, N, G, r, bits):
+    return K * N * bits // 8 + 8 * G * N + 2 * (G * r + r * N) + 2 * M * K + 2 * M * N
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm": p["hbm_gbs"], "tensor": p["bf16_tflops_sustained"], "tensor_burst": p["bf16_tflops"],
+                "source": "measured"}
+    return {"hbm": 6650.0, "tensor": 1400.0, "tensor_burst": 1590.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------- clock sampler --
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_uuid):
+        self.uuid = gpu_uuid
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------- CPU reference --
+def oracle_sample(rows=32):
+    """Times the CPU oracle (as it stands) on `rows` token rows of the first
+    shape: forward + backward.  Returns (TFLOP/s, seconds, description)."""
+    import numpy as np
+    import torch
+
+    from oracle import qalora_oracle as O
+    from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs, to_f64
+
+    cfg = CONFIGS[SHAPES[0]].with_(tokens=rows)
+    t = make_inputs(cfg)
+    codes, alpha, beta = O.quantize(t["W"].numpy(), cfg.group_size, cfg.bits)
+    x, A, B, dy = (to_f64(t[k]) for k in ("x", "A", "B", "dy"))
+    t0 = time.perf_counter()
+    O.forward(x, codes, alpha, beta, cfg.group_size, A, B, cfg.scale)
+    O.backward(x, dy, codes, alpha, beta, cfg.group_size, A, B, cfg.scale)
+    dt = time.perf_counter() - t0
+    fl = fwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank) + bwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank)
+    cores = torch.get_num_threads()
+    desc = (f"fp64 numpy oracle, forward+backward on {rows} of 8192 token rows of {SHAPES[0]} "
+            f"(each call dequantizes the full {cfg.d_in}x{cfg.d_out} weight); quantize excluded")
+    return fl / dt / 1e12, dt, desc, cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times, val, desc, cores = [], 0.0, "", 0
+    for i in range(args.warmup + args.steps):
+        v, dt, desc, cores = oracle_sample(rows=16)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / max(1, len(times))
+    cfg_rows = 16
+    from paper_2309_14717_b200.synthetic import CONFIGS
+    c = CONFIGS[SHAPES[0]]
+    fl = fwd_flops(cfg_rows, c.d_in, c.d_out, c.groups, c.rank) + bwd_flops(cfg_rows, c.d_in, c.d_out, c.groups, c.rank)
+    value = fl / (ms / 1e3) / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": desc},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ GPU arm ---
+class ShapeState:
+    def __init__(self, name, rank, Q, torch):
+        from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
+        cfg = CONFIGS[name]
+        self.cfg = cfg
+        shared = make_inputs(cfg, need=("W", "A", "B"))
+        batch = make_inputs(cfg.with_(seed=cfg.seed + 1000 * (rank + 1)), need=("x", "dy"))
+        self.host = {"x": batch["x"].pin_memory(), "dy": batch["dy"].pin_memory()}
+        self.W = shared["W"].cuda()
+        self.A = shared["A"].cuda()
+        self.B = shared["B"].cuda()
+        self.x = batch["x"].cuda()
+        self.dy = batch["dy"].cuda()
+        M, K, N, G, r = cfg.tokens, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank
+        self.d = Q.desc(K, N, cfg.group_size, cfg.bits, r, cfg.scale)
+        self.d0 = Q.desc(K, N, cfg.group_size, cfg.bits, 0, cfg.scale)
+        self.codes, self.qparams = Q.alloc_packed(self.d)
+        self.qmerged = torch.empty_like(self.qparams)
+        self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        self.dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        self.dA = torch.empty((G, r), dtype=torch.float32, device="cuda")
+        self.dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
+        self.ws_f = Q.alloc_workspace(self.d, M, Q.OP_FORWARD)
+        self.ws_b = Q.alloc_workspace(self.d, M, Q.OP_BACKWARD)
+        self.x1 = self.x[:1].contiguous()
+        self.y1 = torch.empty((1, N), dtype=torch.bfloat16, device="cuda")
+        self.ws1 = Q.alloc_workspace(self.d0, 1, Q.OP_FORWARD)
+        self.host_out = {"y": torch.empty((M, N), dtype=torch.bfloat16).pin_memory(),
+                         "dx": torch.empty((M, K), dtype=torch.bfloat16).pin_memory(),
+                         "dA": torch.empty((G, r), dtype=torch.float32).pin_memory(),
+                         "dB": torch.empty((r, N), dtype=torch.float32).pin_memory()}
+        self.flops = fwd_flops(M, K, N, G, r) + bwd_flops(M, K, N, G, r)
+        self.main_flops = 2 * M * K * N
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2309_14717_b200 import binding as Q
+    from paper_2309_14717_b200 import build as _build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if local == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    Q.load()
+
+    shapes = [ShapeState(n, rank, Q, torch) for n in SHAPES]
+    stream = torch.cuda.current_stream()
+
+    def device_step(s):
+        Q.qalora_quantize(s.d, s.W, s.codes, s.qparams)
+        Q.qalora_forward(s.d, s.cfg.tokens, s.x, s.codes, s.qparams, s.A, s.B, s.y, s.ws_f)
+        Q.qalora_backward(s.d, s.cfg.tokens, s.x, s.dy, s.codes, s.qparams, s.A, s.B, s.dx, s.dA, s.dB, s.ws_b)
+        if world > 1:
+            dist.all_reduce(s.dA)
+            dist.all_reduce(s.dB)
+        Q.qalora_merge(s.d, s.qparams, s.A, s.B, s.qmerged)
+        Q.qalora_forward(s.d0, 1, s.x1, s.codes, s.qmerged, None, None, s.y1, s.ws1)
+
+    def step():
+        for s in shapes:
+            device_step(s)
+
+    def e2e_step():
+        for s in shapes:
+            s.x.copy_(s.host["x"], non_blocking=True)
+            s.dy.copy_(s.host["dy"], non_blocking=True)
+            device_step(s)
+            s.host_out["y"].copy_(s.y, non_blocking=True)
+            s.host_out["dx"].copy_(s.dx, non_blocking=True)
+            s.host_out["dA"].copy_(s.dA, non_blocking=True)
+            s.host_out["dB"].copy_(s.dB, non_blocking=True)
+
+    def timed(fn, steps, sampler=None):
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        clocks = sampler.stop() if sampler else None
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, clocks
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    launches0 = Q.qalora_kernel_launches()
+    ms_total, clocks = timed(step, args.steps, ClockSampler(uuid))
+    launches = (Q.qalora_kernel_launches() - launches0) // max(1, args.steps)
+    ms_step = ms_total / args.steps
+    flops_step = sum(s.flops for s in shapes) * world
+    value = flops_step / (ms_step / 1e3) / 1e12
+
+    # dominant kernel (the forward contraction of the first shape), timed live with
+    # events recorded by the library around that one launch, on the launching stream
+    s0 = shapes[0]
+    ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ka.record(stream); kb.record(stream)            # creates the underlying CUDA events
+    kernel_ms = []
+    for _ in range(max(3, min(args.steps, 10))):
+        Q.qalora_profile_next_main_kernel(ka, kb)
+        Q.qalora_forward(s0.d, s0.cfg.tokens, s0.x, s0.codes, s0.qparams, s0.A, s0.B, s0.y, s0.ws_f)
+        torch.cuda.synchronize()
+        kernel_ms.append(ka.elapsed_time(kb))
+    kms = sum(kernel_ms) / len(kernel_ms)
+    pk = peaks()
+    achieved = s0.main_flops / (kms / 1e3) / 1e12
+    roofline = {"bound": "tensor", "kernel": Q.qalora_main_kernel_name(), "achieved": achieved, "peak": pk["tensor"],
+                "unit": "TFLOP/s", "frac": achieved / pk["tensor"], "peak_source": pk["source"] + " (sustained bf16)",
+                "kernel_ms": kms, "traffic": None}
+
+    # single-token forward of the merged layer: HBM-bound leg of the metric
+    small = small_m_bandwidth(Q, torch, pk)
+
+    e2e_ms, _ = timed(e2e_step, args.steps)
+    e2e_ms /= args.steps
+    h2d = sum(s.host["x"].numel() * 2 + s.host["dy"].numel() * 2 for s in shapes)
+    d2h = sum(sum(t.numel() * t.element_size() for t in s.host_out.values()) for s in shapes)
+
+    if rank == 0:
+        v, dt, desc, cores = oracle_sample(rows=32)
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "shapes": list(SHAPES), "tokens_per_gpu": 8192, "bits": 4,
+                       "group_size": 32, "rank": 64,
+                       "step": "quantize+forward+backward+merge+merged M=1 forward, both shapes",
+                       "l2": "inputs exceed L2 (x+dy+y+dx > 470 MB per shape)",
+                       "parallelism": f"dp{world}" if world > 1 else "single"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "e2e": {"value": flops_step / (e2e_ms / 1e3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "roofline": roofline, "small_m": small,
+            "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc,
+                             "seconds": dt},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def small_m_bandwidth(Q, torch, pk):
+    """M in {1, 4, 16} forward of the LLaMA-7B attention shape, rotating over
+    enough weight copies (> 4 x L2) that the codes come from HBM."""
+    from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
+    cfg = CONFIGS[SMALL_M]
+    t = make_inputs(cfg, need=("W", "x", "A", "B"))
+    d = Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, cfg.rank, cfg.scale)
+    W = t["W"].cuda()
+    A, B = t["A"].cuda(), t["B"].cuda()
+    copies = []
+    codes, qparams = Q.alloc_packed(d)
+    Q.qalora_quantize(d, W, codes, qparams)
+    ncopies = 48                                      # 48 x 12.6 MB = 604 MB > 4 x 126 MB
+    for _ in range(ncopies):
+        copies.append((codes.clone(), qparams.clone()))
+    out = {}
+    stream = torch.cuda.current_stream()
+    for M in (1, 4, 16):
+        x = t["x"][:M].contiguous().cuda()
+        y = torch.empty((M, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+        ws = Q.alloc_workspace(d, M, Q.OP_FORWARD)
+        for c, q in copies[:4]:
+            Q.qalora_forward(d, M, x, c, q, A, B, y, ws)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 2
+        e0.record(stream)
+        for _ in range(reps):
+            for c, q in copies:
+                Q.qalora_forward(d, M, x, c, q, A, B, y, ws)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * ncopies)
+        nbytes = fwd_bytes(M, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank, cfg.bits)
+        gbs = nbytes / (us * 1e-6) / 1e9
+        out[f"M{M}"] = {"us_per_call": us, "GB/s": gbs, "frac_of_hbm": gbs / pk["hbm"], "bytes": nbytes}
+    out["shape"] = SMALL_M
+    out["peak_GB/s"] = pk["hbm"]
+    out["peak_source"] = pk["source"]
+    out["l2"] = f"rotates over {ncopies} weight copies (604 MB) so codes stream from HBM; includes the pool/adapter pre-kernel"
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

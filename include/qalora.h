@@ -136,6 +136,25 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
 int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A, const void* B,
                  float* qparams_out, void* cuda_stream);
 
+/* ---- Instrumentation (no counterpart in the paper) ------------------------ */
+
+/* Number of CUDA kernels this library has launched in this process so far
+ * (all threads; monotonically increasing). */
+uint64_t qalora_kernel_launches(void);
+
+/* Arms a one-shot probe on the calling thread: the next main contraction kernel
+ * (the x * W~ product of qalora_forward or the dy * W~^T product of
+ * qalora_backward) launched from this thread records `start_event` just before
+ * and `stop_event` just after that one launch, on the launch stream.  Both are
+ * cudaEvent_t handles created with timing enabled, passed as void*; NULL
+ * disarms.  Host pointers are not retained after the launch. */
+int qalora_profile_next_main_kernel(void* start_event, void* stop_event);
+
+/* Name of the main contraction kernel chosen by the most recent qalora_forward
+ * or qalora_backward call on this thread ("" before any call).  Static host
+ * string. */
+const char* qalora_main_kernel_name(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -19,6 +19,7 @@ OP_FORWARD, OP_BACKWARD = 0, 1
 EXPORTS = (
     "qalora_version", "qalora_status_string", "qalora_packed_bytes", "qalora_workspace_bytes",
     "qalora_quantize", "qalora_forward", "qalora_backward", "qalora_merge",
+    "qalora_kernel_launches", "qalora_profile_next_main_kernel", "qalora_main_kernel_name",
 )
 
 
@@ -62,6 +63,12 @@ def load() -> ctypes.CDLL:
     lib.qalora_backward.argtypes = [D, c_int64] + [c_void_p] * 9 + [c_void_p, c_size_t, c_void_p]
     lib.qalora_merge.restype = c_int
     lib.qalora_merge.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.qalora_kernel_launches.restype = ctypes.c_uint64
+    lib.qalora_kernel_launches.argtypes = []
+    lib.qalora_profile_next_main_kernel.restype = c_int
+    lib.qalora_profile_next_main_kernel.argtypes = [c_void_p, c_void_p]
+    lib.qalora_main_kernel_name.restype = c_char_p
+    lib.qalora_main_kernel_name.argtypes = []
     _lib = lib
     return lib
 
@@ -146,3 +153,19 @@ def qalora_backward(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, 
 def qalora_merge(d: QaloraDesc, qparams_in, A, B, qparams_out, stream=None):
     _check("qalora_merge", load().qalora_merge(byref(d), _ptr(qparams_in), _ptr(A), _ptr(B), _ptr(qparams_out),
                                                _stream(stream)))
+
+
+def qalora_kernel_launches() -> int:
+    return int(load().qalora_kernel_launches())
+
+
+def qalora_profile_next_main_kernel(start_event, stop_event):
+    """start_event/stop_event: torch.cuda.Event(enable_timing=True) that have been
+    recorded at least once (so that their CUDA handles exist), or None to disarm."""
+    a = c_void_p(start_event.cuda_event) if start_event is not None else None
+    b = c_void_p(stop_event.cuda_event) if stop_event is not None else None
+    _check("qalora_profile_next_main_kernel", load().qalora_profile_next_main_kernel(a, b))
+
+
+def qalora_main_kernel_name() -> str:
+    return load().qalora_main_kernel_name().decode()

@@ -1,7 +1,27 @@
 // C-ABI entry points: argument checks, scratch layout and kernel dispatch.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace qalora {
+
+static std::atomic<uint64_t> g_launches{0};
+static thread_local cudaEvent_t t_probe_start = nullptr, t_probe_stop = nullptr;
+static thread_local const char* t_main_kernel = "";
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+MainKernelProbe::MainKernelProbe(const char* name, cudaStream_t s) : st(s), stop(nullptr) {
+  t_main_kernel = name;
+  if (t_probe_start != nullptr && t_probe_stop != nullptr) {
+    cudaEventRecord(t_probe_start, st);
+    stop = t_probe_stop;
+  }
+  t_probe_start = t_probe_stop = nullptr;
+}
+MainKernelProbe::~MainKernelProbe() {
+  if (stop != nullptr) cudaEventRecord(stop, st);
+}
 
 int check_desc(const qalora_desc* d, Shape* sh) {
   if (d == nullptr) return QALORA_ERR_NULL_POINTER;
@@ -45,6 +65,16 @@ using namespace qalora;
 extern "C" {
 
 int qalora_version(void) { return 100 + QALORA_LAYOUT_VERSION; }
+
+uint64_t qalora_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int qalora_profile_next_main_kernel(void* start_event, void* stop_event) {
+  t_probe_start = static_cast<cudaEvent_t>(start_event);
+  t_probe_stop = static_cast<cudaEvent_t>(stop_event);
+  return QALORA_OK;
+}
+
+const char* qalora_main_kernel_name(void) { return t_main_kernel; }
 
 const char* qalora_status_string(int status) {
   switch (status) {

@@ -97,4 +97,13 @@ int launch_atb_f32(int64_t M, int P, int Q, const float* X, const float* Y, floa
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? QALORA_OK : QALORA_ERR_CUDA; }
 
+// Instrumentation: launch counter and the one-shot event probe around a main kernel.
+void count_launch(int n = 1);
+struct MainKernelProbe {            // records the armed events around one launch
+  MainKernelProbe(const char* name, cudaStream_t st);
+  ~MainKernelProbe();
+  cudaStream_t st;
+  cudaEvent_t stop;
+};
+
 }  // namespace qalora

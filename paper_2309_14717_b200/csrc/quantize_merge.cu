@@ -79,6 +79,7 @@ int launch_quantize(const Shape& sh, const float* W, uint32_t* codes, float2* qp
   if (sh.bits == 4) quantize_kernel<4><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
   else if (sh.bits == 3) quantize_kernel<3><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
   else quantize_kernel<2><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
+  count_launch();
   return cuda_status(cudaGetLastError());
 }
 
@@ -108,6 +109,7 @@ int launch_merge(const Shape& sh, const float2* qin, const __nv_bfloat16* A, con
   const long long blocks = (long long)sh.G * ntiles;
   if (blocks > 0x7fffffffLL) return QALORA_ERR_UNSUPPORTED_SHAPE;
   merge_kernel<<<(unsigned)blocks, QCOLS, sh.r * sizeof(float), st>>>(qin, A, B, qout, sh.N, sh.r, sh.s, ntiles);
+  count_launch();
   return cuda_status(cudaGetLastError());
 }
 

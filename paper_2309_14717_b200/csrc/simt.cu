@@ -55,6 +55,7 @@ int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv
   if (M == 0) return QALORA_OK;
   pool_T_kernel<<<(unsigned)M, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G,
                                                                         sh.r, sh.s);
+  count_launch();
   return cuda_status(cudaGetLastError());
 }
 
@@ -97,6 +98,7 @@ int launch_dT(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const __nv_bf
               float* dT, __nv_bfloat16* dTb, cudaStream_t st) {
   if (M == 0) return QALORA_OK;
   dT_kernel<<<(unsigned)M, DT_THREADS, 0, st>>>(dy, B, dT, dTb, sh.N, sh.r, sh.s);
+  count_launch();
   return cuda_status(cudaGetLastError());
 }
 
@@ -193,7 +195,11 @@ int launch_simt_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, cons
   if (mt > 65535) return QALORA_ERR_UNSUPPORTED_SHAPE;
   dim3 grid((sh.N + TN - 1) / TN, (unsigned)mt), block(SIMT_THREADS);
 #define QALORA_FWD(BITS) simt_forward_kernel<BITS><<<grid, block, 0, st>>>(x, codes, qparams, T, B, y, M, sh.K, sh.N, sh.g, sh.r)
-  if (sh.bits == 4) QALORA_FWD(4); else if (sh.bits == 3) QALORA_FWD(3); else QALORA_FWD(2);
+  {
+    MainKernelProbe probe("simt_forward_kernel", st);
+    if (sh.bits == 4) QALORA_FWD(4); else if (sh.bits == 3) QALORA_FWD(3); else QALORA_FWD(2);
+  }
+  count_launch();
 #undef QALORA_FWD
   return cuda_status(cudaGetLastError());
 }
@@ -284,7 +290,11 @@ int launch_simt_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const ui
   if (mt > 65535) return QALORA_ERR_UNSUPPORTED_SHAPE;
   dim3 grid((sh.K + TN - 1) / TN, (unsigned)mt), block(SIMT_THREADS);
 #define QALORA_DX(BITS) simt_dx_kernel<BITS><<<grid, block, 0, st>>>(dy, codes, qparams, dT, A, dx, M, sh.K, sh.N, sh.g, sh.r)
-  if (sh.bits == 4) QALORA_DX(4); else if (sh.bits == 3) QALORA_DX(3); else QALORA_DX(2);
+  {
+    MainKernelProbe probe("simt_dx_kernel", st);
+    if (sh.bits == 4) QALORA_DX(4); else if (sh.bits == 3) QALORA_DX(3); else QALORA_DX(2);
+  }
+  count_launch();
 #undef QALORA_DX
   return cuda_status(cudaGetLastError());
 }
@@ -378,6 +388,7 @@ static int launch_atb(int64_t M, int P, int Q, const float* X, const TY* Y, floa
   dim3 grid((Q + TN - 1) / TN, (P + TM - 1) / TM, (unsigned)splits);
   atb_partial_kernel<TY><<<grid, SIMT_THREADS, 0, st>>>(X, Y, partial, M, P, Q, rows);
   sum_partials_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(partial, out, count, (int)splits);
+  count_launch(2);
   return cuda_status(cudaGetLastError());
 }
 
