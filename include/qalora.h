@@ -88,7 +88,9 @@ int qalora_packed_bytes(const qalora_desc* desc, size_t* code_bytes, size_t* qpa
 /* Bytes of scratch `workspace` that qalora_forward / qalora_backward need for
  * `m` token rows (host pointer out; may be 0).  The workspace holds the pooled
  * input, the rank-r intermediates and split-K partial sums; its content is
- * undefined on entry and on exit. */
+ * undefined on entry.  On exit its first int32 is a device status word: 0, or
+ * 1 when a bounded wait inside a tensor-core kernel expired (the outputs of
+ * that call are then invalid; nothing hangs or traps). */
 int qalora_workspace_bytes(const qalora_desc* desc, int64_t m, int op, size_t* bytes);
 
 /* Group-wise min-max quantization, Eq. 1 per (group, column) (Section 3.3):

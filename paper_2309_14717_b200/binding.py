@@ -127,7 +127,13 @@ def alloc_packed(d: QaloraDesc, device="cuda"):
 
 
 def alloc_workspace(d: QaloraDesc, m: int, op: int, device="cuda") -> torch.Tensor:
-    return torch.empty(max(qalora_workspace_bytes(d, m, op), 16), dtype=torch.uint8, device=device)
+    return torch.zeros(max(qalora_workspace_bytes(d, m, op), 16), dtype=torch.uint8, device=device)
+
+
+def workspace_status(workspace: torch.Tensor) -> int:
+    """Device status word at the head of a workspace (synchronizes): 0 = ok,
+    1 = a bounded wait inside a tensor-core kernel expired (results invalid)."""
+    return int(workspace[:4].view(torch.int32).item())
 
 
 def qalora_quantize(d: QaloraDesc, W, codes, qparams, dev_status=None, stream=None):

@@ -42,6 +42,7 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   auto take = [&](size_t bytes) { size_t at = off; off += round_up(bytes, 256); return at; };
   const size_t M = (size_t)(m > 0 ? m : 0);
   const bool bwd = op == QALORA_OP_BACKWARD;
+  w.status = take(256);
   w.xp = take(bwd ? M * sh.G * sizeof(float) : 0);
   w.T = take(M * sh.r * sizeof(float));
   w.dT = take(bwd ? M * sh.r * sizeof(float) : 0);
@@ -61,6 +62,9 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
 }  // namespace qalora
 
 using namespace qalora;
+
+// Token counts up to this take the bandwidth-bound small-M path.
+static constexpr int64_t kSmallM = 16;
 
 extern "C" {
 
@@ -159,6 +163,13 @@ int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void
                        nullptr, T, Tb, stream);
     if (st != QALORA_OK) return st;
   }
+  if (m > kSmallM && tc_forward_supported(sh, m)) {
+    int* status = reinterpret_cast<int*>(wsp + ws.status);
+    if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
+    return launch_tc_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
+                             reinterpret_cast<const float2*>(qparams), Tb, static_cast<const __nv_bfloat16*>(B),
+                             static_cast<__nv_bfloat16*>(y), status, stream);
+  }
   return launch_simt_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
                              reinterpret_cast<const float2*>(qparams), T, static_cast<const __nv_bfloat16*>(B),
                              static_cast<__nv_bfloat16*>(y), stream);
@@ -202,7 +213,13 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
   if (dA != nullptr || dB != nullptr) {
     if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
   }
-  if (dx != nullptr) {
+  if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
+    int* status = reinterpret_cast<int*>(wsp + ws.status);
+    if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
+    st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
+                      dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);
+    if (st != QALORA_OK) return st;
+  } else if (dx != nullptr) {
     st = launch_simt_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
                         dT, Ab, static_cast<__nv_bfloat16*>(dx), stream);
     if (st != QALORA_OK) return st;

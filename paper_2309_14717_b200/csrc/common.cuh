@@ -25,6 +25,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Scratch layout shared by forward and backward (offsets in bytes, 256-aligned).
 struct Workspace {
+  size_t status;    // int32  device status word of the tensor-core kernels (first bytes of the workspace)
   size_t xp;        // float  [M][G]   pooled input                      (backward)
   size_t T;         // float  [M][r]   s * pool(x) * A                   (both)
   size_t dT;        // float  [M][r]   s * dy * B^T                      (backward)
@@ -94,6 +95,16 @@ int launch_atb_bf16(int64_t M, int P, int Q, const float* X, const __nv_bfloat16
                     float* partial, size_t partial_bytes, cudaStream_t st);
 int launch_atb_f32(int64_t M, int P, int Q, const float* X, const float* Y, float* out,
                    float* partial, size_t partial_bytes, cudaStream_t st);
+
+// Tensor-core paths (gemm_tc.cu).  Tb / dTb are the bf16 rank-r intermediates.
+bool tc_forward_supported(const Shape& sh, int64_t M);
+bool tc_dx_supported(const Shape& sh, int64_t M);
+int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
+                      const float2* qparams, const __nv_bfloat16* Tb, const __nv_bfloat16* B,
+                      __nv_bfloat16* y, int* status, cudaStream_t st);
+int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint32_t* codes,
+                 const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
+                 __nv_bfloat16* dx, int* status, cudaStream_t st);
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? QALORA_OK : QALORA_ERR_CUDA; }
 

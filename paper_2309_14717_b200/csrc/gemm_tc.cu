@@ -1,0 +1,475 @@
+// Tensor-core kernels of the QA-LoRA layer for sm_100a: the forward product
+// y = x * W~ (+ adapter) and the input gradient dx = dy * W~^T (+ adapter), with
+// the b-bit weights dequantized on the fly.
+//
+// Both are computed transposed, out^T[c][m] = sum_j Wop[c][j] * act[m][j], so that
+// the dequantized weights are the 128-row "A" operand of tcgen05.mma and 256
+// tokens are the "N" extent: every dequantized element is reused 256 times.
+//   forward : c = output channel n, j = input channel k.  A pack unit (32 input
+//             channels of one column) is exactly 32 K-contiguous elements of row
+//             c, so the dequantizing thread writes it straight into TENSOR
+//             MEMORY (tcgen05.st) and the MMA takes A from TMEM.
+//   dx      : c = input channel k, j = output channel n.  A unit is now 32
+//             consecutive ROWS of one j, i.e. 64 contiguous bytes of an
+//             MN-major operand: it goes to shared memory in the 128-byte
+//             swizzled MN-major layout and the MMA takes A from smem.
+// The same packed bytes serve both products.  The adapter is folded in as extra
+// reduction steps of width r: forward appends T = s*pool(x)*A against B, dx
+// appends dT = s*dy*B^T against the group-expanded A.
+//
+// Warp roles (512 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
+// owner, warps 4-11 = dequantizers, warps 12-15 = epilogue.  Stages are handed
+// over with mbarriers; every wait is bounded and a timeout raises a status word
+// instead of hanging.
+#include <mutex>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace qalora {
+
+namespace {
+
+constexpr int TILE_C = 128;      // out channels per tile   (MMA M)
+constexpr int TILE_T = 256;      // tokens per tile         (MMA N)
+constexpr int TILE_J = 64;       // reduction step per stage
+constexpr int THREADS = 512;
+constexpr int TMEM_COLS = 512;
+constexpr int ACC_COL = 0;       // accumulator: columns [0, 256)
+constexpr int A_COL = 256;       // forward A ring: 32 columns per stage
+constexpr uint32_t ACT_BYTES = TILE_T * TILE_J * 2;      // 32 KiB activation tile
+constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx)
+
+enum Mode { FWD = 0, DX = 1 };
+
+struct TcParams {
+  const uint32_t* codes;
+  const float2* qparams;
+  const __nv_bfloat16* lora;   // FWD: B [r][N];  DX: A [G][r]
+  __nv_bfloat16* out;          // FWD: y [M][N];  DX: dx [M][K]
+  long long M;
+  int K, N, g, r;
+  int ld_out;                  // N (FWD) or K (DX)
+  int c_tiles, m_tiles;        // tiles along out channels / tokens
+  int red_iters, lora_iters;   // main / adapter reduction steps per tile
+  int* status;                 // device word: set to 1 when a wait timed out
+};
+
+template <int BITS, int MODE, int STAGES>
+struct Smem {
+  static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
+  static constexpr uint32_t UNITS = MODE == FWD ? 2 * TILE_C : 4 * TILE_J;     // 256 units per stage
+  static constexpr uint32_t CODE_BYTES = UNITS * WORDS * 4;
+  static constexpr uint32_t QP_BYTES = UNITS * 8;
+  static constexpr uint32_t A_BYTES = MODE == DX ? ATILE_BYTES : 0;
+  static constexpr uint32_t STAGE_BYTES = ACT_BYTES + A_BYTES + ((CODE_BYTES + QP_BYTES + 1023) / 1024) * 1024;
+  static constexpr uint32_t OFF_ACT = 0;
+  static constexpr uint32_t OFF_A = ACT_BYTES;
+  static constexpr uint32_t OFF_CODES = ACT_BYTES + A_BYTES;
+  static constexpr uint32_t OFF_QP = OFF_CODES + CODE_BYTES;
+  static constexpr uint32_t BAR_BYTES = 256;
+  static constexpr uint32_t TOTAL = STAGES * STAGE_BYTES + BAR_BYTES + 1024;   // + alignment slack
+};
+
+// ---- dequantization of one pack unit to 16 bf16x2 registers ------------------
+// Position pairs (2p, 2p+1) sit in the low/high half-words of a word, so one
+// shift and one mask give a bf16x2 holding (128 + c_even, 128 + c_odd): the
+// codes are OR-ed into the mantissa of bf16 128.0.  Subtracting 128 is exact;
+// one packed FMA then applies alpha and beta (rounded to bf16).
+__device__ __forceinline__ uint32_t dq_pair(uint32_t v, __nv_bfloat162 a2, __nv_bfloat162 b2) {
+  const __nv_bfloat162 k128 = __floats2bfloat162_rn(128.0f, 128.0f);
+  __nv_bfloat162 c = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&v), k128);
+  c = __hfma2(c, a2, b2);
+  return *reinterpret_cast<uint32_t*>(&c);
+}
+
+template <int WORDS>
+__device__ __forceinline__ void load_unit(const uint32_t* cw, uint32_t* w) {
+  if constexpr (WORDS == 4) {
+    const uint4 t = *reinterpret_cast<const uint4*>(cw);
+    w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+  } else if constexpr (WORDS == 2) {
+    const uint2 t = *reinterpret_cast<const uint2*>(cw);
+    w[0] = t.x; w[1] = t.y;
+  } else {
+#pragma unroll
+    for (int q = 0; q < WORDS; ++q) w[q] = cw[q];
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, uint32_t* out) {
+  const __nv_bfloat162 a2 = __floats2bfloat162_rn(ab.x, ab.x);
+  const __nv_bfloat162 b2 = __floats2bfloat162_rn(ab.y, ab.y);
+  if (BITS == 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+        out[i * 4 + p] = dq_pair(((w[i] >> (4 * p)) & 0x000f000fu) | 0x43004300u, a2, b2);
+  } else if (BITS == 2) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int p = 0; p < 8; ++p)
+        out[i * 8 + p] = dq_pair(((w[i] >> (2 * p)) & 0x00030003u) | 0x43004300u, a2, b2);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        const uint32_t lo = (w[i] >> (2 * p)) & 0x00030003u;
+        const uint32_t hi = ((w[2] >> (8 * i + p)) & 0x00010001u) << 2;
+        out[i * 8 + p] = dq_pair(lo | hi | 0x43004300u, a2, b2);
+      }
+  }
+}
+
+template <int BITS, int MODE, int STAGES>
+__global__ void __launch_bounds__(THREADS, 1)
+qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_constant__ CUtensorMap lora_map,
+                 const TcParams p) {
+  using S = Smem<BITS, MODE, STAGES>;
+  constexpr int WORDS = S::WORDS;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = ptx::smem_u32(smem);
+  uint8_t* bar_area = smem + STAGES * S::STAGE_BYTES;
+  const uint32_t bar_base = smem_base + STAGES * S::STAGE_BYTES;
+  // barrier layout (8 bytes each): full[S], aready[S], empty[S], acc_full, acc_empty
+  auto bar_full = [&](int s) { return bar_base + 8u * s; };
+  auto bar_aready = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto bar_empty = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
+  const uint32_t bar_acc_full = bar_base + 8u * (3 * STAGES);
+  const uint32_t bar_acc_empty = bar_base + 8u * (3 * STAGES + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_area + 8 * (3 * STAGES + 2));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_area + 8 * (3 * STAGES + 2) + 8);
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(bar_full(s), 1);
+      ptx::mbar_init(bar_aready(s), 8);
+      ptx::mbar_init(bar_empty(s), 1);
+    }
+    ptx::mbar_init(bar_acc_full, 1);
+    ptx::mbar_init(bar_acc_empty, 4);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&act_map);
+    if (p.lora_iters > 0) ptx::prefetch_tensormap(&lora_map);
+  }
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int total_tiles = p.c_tiles * p.m_tiles;
+  const int iters = p.red_iters + p.lora_iters;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer ----
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
+        const int c0 = ct * TILE_C, m0 = mt * TILE_T;
+        for (int i = 0; i < iters; ++i, ++it) {
+          const int s = it % STAGES;
+          if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / STAGES) & 1) ^ 1, abort_flag))) break;
+          const uint32_t stage = smem_base + s * S::STAGE_BYTES;
+          if (i < p.red_iters) {
+            ptx::mbar_arrive_expect_tx(bar_full(s), ACT_BYTES + S::CODE_BYTES + S::QP_BYTES);
+            ptx::tma_load_2d(stage + S::OFF_ACT, &act_map, i * TILE_J, m0, bar_full(s));
+            if (MODE == FWD) {
+#pragma unroll
+              for (int b = 0; b < 2; ++b) {
+                const int kb = i * 2 + b;
+                ptx::bulk_load(stage + S::OFF_CODES + b * (TILE_C * WORDS * 4),
+                               p.codes + ((size_t)kb * p.N + c0) * WORDS, TILE_C * WORDS * 4, bar_full(s));
+                ptx::bulk_load(stage + S::OFF_QP + b * (TILE_C * 8),
+                               p.qparams + (size_t)(kb * 32 / p.g) * p.N + c0, TILE_C * 8, bar_full(s));
+              }
+            } else {
+#pragma unroll
+              for (int b = 0; b < 4; ++b) {
+                const int kb = c0 / 32 + b, n0 = i * TILE_J;
+                ptx::bulk_load(stage + S::OFF_CODES + b * (TILE_J * WORDS * 4),
+                               p.codes + ((size_t)kb * p.N + n0) * WORDS, TILE_J * WORDS * 4, bar_full(s));
+                ptx::bulk_load(stage + S::OFF_QP + b * (TILE_J * 8),
+                               p.qparams + (size_t)(kb * 32 / p.g) * p.N + n0, TILE_J * 8, bar_full(s));
+              }
+            }
+          } else {
+            ptx::mbar_arrive_expect_tx(bar_full(s), ACT_BYTES);
+            ptx::tma_load_2d(stage + S::OFF_ACT, &lora_map, (i - p.red_iters) * TILE_J, m0, bar_full(s));
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------- MMA issuer ----
+    if (lane == 0) {
+      constexpr uint32_t IDESC_MAIN = ptx::idesc_bf16(TILE_C, TILE_T, MODE == DX, false);
+      constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(TILE_C, TILE_T, false, false);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
+        ptx::tc_fence_after();
+        for (int i = 0; i < iters; ++i, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!(ok = ptx::mbar_wait(bar_full(s), ph, abort_flag))) break;
+          if (!(ok = ptx::mbar_wait(bar_aready(s), ph, abort_flag))) break;
+          ptx::tc_fence_after();
+          const uint32_t stage = smem_base + s * S::STAGE_BYTES;
+#pragma unroll
+          for (int j = 0; j < TILE_J / 16; ++j) {
+            const uint64_t bdesc = ptx::smem_desc(stage + S::OFF_ACT + j * 32, 16, 1024);
+            const uint32_t acc = (i > 0 || j > 0) ? 1u : 0u;
+            if (MODE == FWD) {
+              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + s * 32 + j * 8, bdesc, IDESC_MAIN, acc);
+            } else if (i < p.red_iters) {
+              // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO)
+              const uint64_t adesc = ptx::smem_desc(stage + S::OFF_A + j * 2048, 8192, 1024);
+              ptx::mma_ss(tmem_base + ACC_COL, adesc, bdesc, IDESC_MAIN, acc);
+            } else {
+              const uint64_t adesc = ptx::smem_desc(stage + S::OFF_A + j * 32, 16, 1024);
+              ptx::mma_ss(tmem_base + ACC_COL, adesc, bdesc, IDESC_LORA, acc);
+            }
+          }
+          ptx::mma_commit(bar_empty(s));
+        }
+        if (ok) ptx::mma_commit(bar_acc_full);
+      }
+    }
+  } else if (warp >= 4 && warp < 12) {
+    // -------------------------------------------------------- dequantizers ----
+    const int dq = threadIdx.x - 128;            // 0..255
+    const int quarter = warp % 4;                // TMEM lane quarter of this warp
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int ct = tile % p.c_tiles;
+      const int c0 = ct * TILE_C;
+      for (int i = 0; i < iters; ++i, ++it) {
+        const int s = it % STAGES;
+        if (!(ok = ptx::mbar_wait(bar_full(s), (it / STAGES) & 1, abort_flag))) break;
+        uint8_t* stage = smem + s * S::STAGE_BYTES;
+        uint32_t v[16];
+        if (MODE == FWD) {
+          const int half = (warp - 4) / 4;       // which 32-channel block of the stage
+          const int row = quarter * 32 + lane;   // out channel within the tile = TMEM lane
+          if (i < p.red_iters) {
+            const uint32_t* cw = reinterpret_cast<const uint32_t*>(stage + S::OFF_CODES) + (half * TILE_C + row) * WORDS;
+            uint32_t w[WORDS];
+            load_unit<WORDS>(cw, w);
+            const float2 ab = reinterpret_cast<const float2*>(stage + S::OFF_QP)[half * TILE_C + row];
+            dequant_unit<BITS>(w, ab, v);
+          } else {
+            // adapter step: row c of the operand is B[r0 + 0..63][c]; this thread packs 32 of them
+            const int r0 = (i - p.red_iters) * TILE_J + half * 32;
+            const __nv_bfloat16* bp = p.lora + (size_t)r0 * p.N + c0 + row;
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+              const int ra = r0 + 2 * q;
+              const uint32_t lo = ra < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q) * p.N) : 0u;
+              const uint32_t hi = ra + 1 < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q + 1) * p.N) : 0u;
+              v[q] = lo | (hi << 16);
+            }
+          }
+          ptx::tmem_st16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL + s * 32 + half * 16, v);
+          ptx::tmem_wait_st();
+          ptx::tc_fence_before();
+        } else {
+          uint8_t* atile = stage + S::OFF_A;
+          if (i < p.red_iters) {
+            const int kbl = dq / TILE_J, nl = dq % TILE_J;       // 32-channel block, column
+            const uint32_t* cw = reinterpret_cast<const uint32_t*>(stage + S::OFF_CODES) + (kbl * TILE_J + nl) * WORDS;
+            uint32_t w[WORDS];
+            load_unit<WORDS>(cw, w);
+            const float2 ab = reinterpret_cast<const float2*>(stage + S::OFF_QP)[kbl * TILE_J + nl];
+            dequant_unit<BITS>(w, ab, v);
+            // MN-major, 128-byte swizzle: row = column nl (128 bytes = 64 channels),
+            // this unit fills chunks (kbl%2)*4 .. +3 of block kbl/2
+            uint8_t* rowp = atile + (kbl / 2) * 8192 + (nl / 8) * 1024 + (nl % 8) * 128;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const int chunk = ((kbl % 2) * 4 + q) ^ (nl % 8);
+              *reinterpret_cast<uint4*>(rowp + chunk * 16) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            }
+          } else {
+            // adapter step, K-major rows: row c holds A[(c0 + c) / g][r0 .. r0 + 63]
+            const int row = dq / 2, halfrow = dq % 2;
+            const int r0 = (i - p.red_iters) * TILE_J + halfrow * 32;
+            const __nv_bfloat16* ap = p.lora + (size_t)((c0 + row) / p.g) * p.r + r0;
+            uint8_t* rowp = atile + (row / 8) * 1024 + (row % 8) * 128;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              uint4 t = make_uint4(0u, 0u, 0u, 0u);
+              if (r0 + q * 8 < p.r) t = *reinterpret_cast<const uint4*>(ap + q * 8);   // r is a multiple of 8
+              const int chunk = (halfrow * 4 + q) ^ (row % 8);
+              *reinterpret_cast<uint4*>(rowp + chunk * 16) = t;
+            }
+          }
+          ptx::fence_proxy_async();              // make the generic-proxy writes visible to the MMA
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_aready(s));
+      }
+    }
+  } else if (warp >= 12) {
+    // ------------------------------------------------------------ epilogue ----
+    const int quarter = warp % 4;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
+      const int c = ct * TILE_C + quarter * 32 + lane;
+      const long long m0 = (long long)mt * TILE_T;
+      if (!(ok = ptx::mbar_wait(bar_acc_full, tcount & 1, abort_flag))) break;
+      ptx::tc_fence_after();
+#pragma unroll 1
+      for (int col = 0; col < TILE_T; col += 32) {
+        uint32_t v[32];
+        ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ACC_COL + col, v);
+        ptx::tmem_wait_ld();
+        __nv_bfloat16* op = p.out + (size_t)(m0 + col) * p.ld_out + c;
+#pragma unroll
+        for (int t = 0; t < 32; ++t)
+          if (m0 + col + t < p.M) op[(size_t)t * p.ld_out] = __float2bfloat16_rn(__uint_as_float(v[t]));
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_acc_empty);
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown ----
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag != 0) atomicExch(p.status, 1);
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------ host side --
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+// bf16 matrix [rows][cols] row-major, box = 64 columns x 256 rows, 128-byte swizzle;
+// out-of-range rows and columns read as zero.
+bool make_act_map(CUtensorMap* map, const void* base, long long rows, int cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {TILE_J, TILE_T};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+template <int BITS, int MODE>
+int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
+  constexpr int STAGES = MODE == FWD ? 5 : 4;
+  using S = Smem<BITS, MODE, STAGES>;
+  static_assert(S::TOTAL <= 232448, "shared memory budget");
+  auto kern = qalora_tc_kernel<BITS, MODE, STAGES>;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
+  if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
+  const int tiles = p.c_tiles * p.m_tiles;
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  {
+    MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
+    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, p);
+  }
+  count_launch();
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+bool tc_forward_supported(const Shape& sh, int64_t M) {
+  return sh.N % TILE_C == 0 && sh.K % TILE_J == 0 && M >= 1 && M <= 0x7fffffffLL / 2 && encode_fn() != nullptr;
+}
+bool tc_dx_supported(const Shape& sh, int64_t M) {
+  return sh.K % TILE_C == 0 && sh.N % TILE_J == 0 && M >= 1 && M <= 0x7fffffffLL / 2 && encode_fn() != nullptr;
+}
+
+// y = x * W~ + Tb * B with Tb = bf16(s * pool(x) * A) precomputed ([M][r]).
+int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
+                      const float2* qparams, const __nv_bfloat16* Tb, const __nv_bfloat16* B,
+                      __nv_bfloat16* y, int* status, cudaStream_t st) {
+  CUtensorMap act, lora;
+  if (!make_act_map(&act, x, M, sh.K)) return QALORA_ERR_CUDA;
+  lora = act;
+  if (sh.r > 0 && !make_act_map(&lora, Tb, M, sh.r)) return QALORA_ERR_CUDA;
+  TcParams p{};
+  p.codes = codes; p.qparams = qparams; p.lora = B; p.out = y;
+  p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.N;
+  p.c_tiles = sh.N / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
+  p.red_iters = sh.K / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
+  p.status = status;
+  if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, p, st);
+  if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, p, st);
+  return launch_tc<2, FWD>(act, lora, p, st);
+}
+
+// dx = dy * W~^T + dTb * expand(A)^T with dTb = bf16(s * dy * B^T) precomputed ([M][r]).
+int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint32_t* codes,
+                 const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
+                 __nv_bfloat16* dx, int* status, cudaStream_t st) {
+  CUtensorMap act, lora;
+  if (!make_act_map(&act, dy, M, sh.N)) return QALORA_ERR_CUDA;
+  lora = act;
+  if (sh.r > 0 && !make_act_map(&lora, dTb, M, sh.r)) return QALORA_ERR_CUDA;
+  TcParams p{};
+  p.codes = codes; p.qparams = qparams; p.lora = A; p.out = dx;
+  p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.K;
+  p.c_tiles = sh.K / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
+  p.red_iters = sh.N / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
+  p.status = status;
+  if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
+  if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);
+  return launch_tc<2, DX>(act, lora, p, st);
+}
+
+}  // namespace qalora

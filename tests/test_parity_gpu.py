@@ -47,6 +47,7 @@ class GpuLayer:
         Q.qalora_forward(d, m, x, self.codes, self.qparams if qparams is None else qparams,
                          self.dev.get("A") if d.rank else None, self.dev.get("B") if d.rank else None, y, ws)
         torch.cuda.synchronize()
+        assert Q.workspace_status(ws) == 0
         return y
 
     def backward(self):
@@ -59,6 +60,7 @@ class GpuLayer:
         Q.qalora_backward(self.d, m, self.dev["x"], self.dev["dy"], self.codes, self.qparams, self.dev["A"],
                           self.dev["B"], dx, dA, dB, ws)
         torch.cuda.synchronize()
+        assert Q.workspace_status(ws) == 0
         return dx, dA, dB
 
     def oracle_quant(self):
@@ -86,6 +88,11 @@ SMALL = [
     ("ragged2", 256, 72, 128, 2, 8, 2.0, 33),
     ("g64_4", 512, 384, 64, 4, 64, 1.0, 200),
     ("colwise", 128, 64, 128, 4, 8, 1.0, 16),
+    # shapes the tensor-core kernels tile (N % 128 == 0, K % 128 == 0), ragged in M
+    ("tc4", 256, 256, 32, 4, 16, 1.0, 300),
+    ("tc3", 384, 256, 64, 3, 24, 0.75, 270),
+    ("tc2", 256, 128, 128, 2, 8, 2.0, 515),
+    ("tc4_r0pad", 1024, 640, 32, 4, 72, 1.0, 1000),
 ]
 
 
