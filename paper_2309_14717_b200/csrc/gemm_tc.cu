@@ -72,15 +72,28 @@ struct Smem {
 };
 
 // ---- dequantization of one pack unit to 16 bf16x2 registers ------------------
-// Position pairs (2p, 2p+1) sit in the low/high half-words of a word, so one
-// shift and one mask give a bf16x2 holding (128 + c_even, 128 + c_odd): the
-// codes are OR-ed into the mantissa of bf16 128.0.  Subtracting 128 is exact;
-// one packed FMA then applies alpha and beta (rounded to bf16).
-__device__ __forceinline__ uint32_t dq_pair(uint32_t v, __nv_bfloat162 a2, __nv_bfloat162 b2) {
-  const __nv_bfloat162 k128 = __floats2bfloat162_rn(128.0f, 128.0f);
-  __nv_bfloat162 c = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&v), k128);
-  c = __hfma2(c, a2, b2);
-  return *reinterpret_cast<uint32_t*>(&c);
+// A b-bit code c is moved to the top of an fp32 mantissa, giving v = 1 + c / 2^b
+// without any int-to-float conversion; then W~ = alpha*c + beta =
+// (2^b alpha) * v + (beta - 2^b alpha) is ONE fp32 FMA per element, and a pair of
+// results is rounded once to bf16x2.  alpha and beta stay in fp32, so the only
+// rounding is that of the final weight (rounding alpha or beta themselves would
+// put a common error on all channels of a group, which the pooled input
+// amplifies).
+template <int SHIFT>   // positive: shift left
+__device__ __forceinline__ uint32_t shift_to(uint32_t w) {
+  if constexpr (SHIFT >= 0) return w << SHIFT; else return w >> (-SHIFT);
+}
+// position e of a word whose codes are BITS wide at bit 16*(e&1) + BITS*(e>>1)
+template <int BITS, int E>
+__device__ __forceinline__ float code_as_1p(uint32_t w) {
+  constexpr int POS = 16 * (E & 1) + BITS * (E >> 1);
+  constexpr int TOP = 23 - BITS;
+  constexpr uint32_t MASK = ((1u << BITS) - 1u) << TOP;
+  return __uint_as_float((shift_to<TOP - POS>(w) & MASK) | 0x3f800000u);
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&t);
 }
 
 template <int WORDS>
@@ -97,32 +110,36 @@ __device__ __forceinline__ void load_unit(const uint32_t* cw, uint32_t* w) {
   }
 }
 
+template <int BITS, int I, int P>
+__device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, float a, float b) {
+  float v0, v1;
+  if constexpr (BITS == 3) {
+    // low two bits from plane word I, the third bit from word 2 (bit 16*(j&1) + (j>>1), j = 16 I + 2 P + h)
+    constexpr int PL = 2 * P, PH = 8 * I + P;
+    v0 = __uint_as_float((shift_to<20 - PL>(w[I]) & 0x00300000u) | (shift_to<22 - PH>(w[2]) & 0x00400000u) | 0x3f800000u);
+    v1 = __uint_as_float((shift_to<20 - (16 + PL)>(w[I]) & 0x00300000u) | (shift_to<22 - (16 + PH)>(w[2]) & 0x00400000u) | 0x3f800000u);
+  } else {
+    v0 = code_as_1p<BITS, 2 * P>(w[I]);
+    v1 = code_as_1p<BITS, 2 * P + 1>(w[I]);
+  }
+  return pack_bf16x2(fmaf(a, v0, b), fmaf(a, v1, b));
+}
+
+template <int BITS, int I, int P>
+__device__ __forceinline__ void dq_all(const uint32_t* w, float a, float b, uint32_t* out) {
+  constexpr int PAIRS = BITS == 4 ? 4 : 8;          // pairs per word
+  constexpr int NWORDS = BITS == 4 ? 4 : 2;         // words that carry the (low) code bits
+  out[I * PAIRS + P] = dq_pair<BITS, I, P>(w, a, b);
+  if constexpr (P + 1 < PAIRS) dq_all<BITS, I, P + 1>(w, a, b, out);
+  else if constexpr (I + 1 < NWORDS) dq_all<BITS, I + 1, 0>(w, a, b, out);
+}
+
+// out[q] = bf16x2 of positions (2q, 2q+1) of the unit, q = 0..15
 template <int BITS>
 __device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, uint32_t* out) {
-  const __nv_bfloat162 a2 = __floats2bfloat162_rn(ab.x, ab.x);
-  const __nv_bfloat162 b2 = __floats2bfloat162_rn(ab.y, ab.y);
-  if (BITS == 4) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int p = 0; p < 4; ++p)
-        out[i * 4 + p] = dq_pair(((w[i] >> (4 * p)) & 0x000f000fu) | 0x43004300u, a2, b2);
-  } else if (BITS == 2) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int p = 0; p < 8; ++p)
-        out[i * 8 + p] = dq_pair(((w[i] >> (2 * p)) & 0x00030003u) | 0x43004300u, a2, b2);
-  } else {
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int p = 0; p < 8; ++p) {
-        const uint32_t lo = (w[i] >> (2 * p)) & 0x00030003u;
-        const uint32_t hi = ((w[2] >> (8 * i + p)) & 0x00010001u) << 2;
-        out[i * 8 + p] = dq_pair(lo | hi | 0x43004300u, a2, b2);
-      }
-  }
+  const float a = ab.x * float(1 << BITS);          // exact
+  const float b = ab.y - a;
+  dq_all<BITS, 0, 0>(w, a, b, out);
 }
 
 template <int BITS, int MODE, int STAGES>
