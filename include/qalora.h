@@ -57,7 +57,9 @@ typedef enum qalora_status {
   QALORA_ERR_UNSUPPORTED_SHAPE = -3,/* see qalora_desc                          */
   QALORA_ERR_MISALIGNED = -4,       /* a pointer is not 16-byte aligned         */
   QALORA_ERR_WORKSPACE_TOO_SMALL = -5,
-  QALORA_ERR_CUDA = -6              /* a CUDA call or launch failed             */
+  QALORA_ERR_CUDA = -6,             /* a CUDA call or launch failed             */
+  QALORA_ERR_STATIC_SCRATCH_EXCEEDED = -7 /* qalora_forward_static: the call needs more
+                                       than QALORA_STATIC_SCRATCH_BYTES of scratch */
 } qalora_status;
 
 /* Shape and hyper-parameters of one layer.  Supported: d_in a multiple of
@@ -137,6 +139,34 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
  * z = -beta/alpha.  qparams_out may alias qparams_in. */
 int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A, const void* B,
                  float* qparams_out, void* cuda_stream);
+
+/* Forward pass for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a convenience of the library).  Some hosts of this code
+ * may not call cudaMalloc at all: a plugin running inside an engine that owns
+ * the whole device heap, code on a real-time or already-capturing path where an
+ * allocation would stall or is forbidden, or a process started with its memory
+ * budget fully handed out.  qalora_forward asks such a caller for a workspace it
+ * has no way to provide.  This variant computes exactly what qalora_forward
+ * computes (same arguments, same kernels, same results) but takes its scratch
+ * from a fixed array of QALORA_STATIC_SCRATCH_BYTES that is part of the
+ * library's device image.  It calls no cudaMalloc/cudaFree and no allocating
+ * routine.
+ *   - Limit: qalora_workspace_bytes(desc, m, QALORA_OP_FORWARD) must not exceed
+ *     QALORA_STATIC_SCRATCH_BYTES (about m * rank * 6 bytes + 1 KiB; e.g. 2048
+ *     tokens at rank 64).  Larger requests return
+ *     QALORA_ERR_STATIC_SCRATCH_EXCEEDED and launch nothing.
+ *   - Cost: every GPU on which the library's device code is loaded holds the
+ *     array until the process exits, whether or not this function is used.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous
+ *     call's contents; the function clears the part that must start at zero.
+ *     Two calls whose GPU work overlaps (different streams, or different
+ *     threads without ordering) race on it: serialize them. */
+#define QALORA_STATIC_SCRATCH_BYTES (1 << 20)
+int qalora_forward_static(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
+                          const float* qparams, const void* A, const void* B, void* y,
+                          void* cuda_stream);
 
 /* ---- Instrumentation (no counterpart in the paper) ------------------------ */
 

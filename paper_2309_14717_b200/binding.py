@@ -20,7 +20,10 @@ EXPORTS = (
     "qalora_version", "qalora_status_string", "qalora_packed_bytes", "qalora_workspace_bytes",
     "qalora_quantize", "qalora_forward", "qalora_backward", "qalora_merge",
     "qalora_kernel_launches", "qalora_profile_next_main_kernel", "qalora_main_kernel_name",
+    "qalora_forward_static",
 )
+
+STATIC_SCRATCH_BYTES = 1 << 20
 
 
 class QaloraDesc(Structure):
@@ -63,6 +66,8 @@ def load() -> ctypes.CDLL:
     lib.qalora_backward.argtypes = [D, c_int64] + [c_void_p] * 9 + [c_void_p, c_size_t, c_void_p]
     lib.qalora_merge.restype = c_int
     lib.qalora_merge.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.qalora_forward_static.restype = c_int
+    lib.qalora_forward_static.argtypes = [D, c_int64] + [c_void_p] * 6 + [c_void_p]
     lib.qalora_kernel_launches.restype = ctypes.c_uint64
     lib.qalora_kernel_launches.argtypes = []
     lib.qalora_profile_next_main_kernel.restype = c_int
@@ -146,6 +151,15 @@ def qalora_forward(d: QaloraDesc, m: int, x, codes, qparams, A, B, y, workspace,
                                                    _ptr(B), _ptr(y), _ptr(workspace),
                                                    workspace.numel() if workspace is not None else 0,
                                                    _stream(stream)))
+
+
+def qalora_forward_static(d: QaloraDesc, m: int, x, codes, qparams, A, B, y, stream=None):
+    """qalora_forward without a workspace argument: the scratch is a fixed array
+    inside the library (STATIC_SCRATCH_BYTES), for callers that cannot allocate
+    device memory.  Raises QaloraError(-7) when m * rank needs more than that.
+    Calls that overlap on the GPU share the array and must be serialized."""
+    _check("qalora_forward_static", load().qalora_forward_static(byref(d), m, _ptr(x), _ptr(codes), _ptr(qparams),
+                                                                 _ptr(A), _ptr(B), _ptr(y), _stream(stream)))
 
 
 def qalora_backward(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, dB, workspace, stream=None):

@@ -89,6 +89,7 @@ const char* qalora_status_string(int status) {
     case QALORA_ERR_MISALIGNED: return "pointer not 16-byte aligned";
     case QALORA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case QALORA_ERR_CUDA: return "CUDA error";
+    case QALORA_ERR_STATIC_SCRATCH_EXCEEDED: return "request exceeds the built-in scratch of qalora_forward_static";
     default: return "unknown status";
   }
 }
