@@ -52,6 +52,10 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   if (bwd) {
     const size_t a = atb_partial_bytes(m, sh.G, sh.r), b = atb_partial_bytes(m, sh.r, sh.N);
     pb = a > b ? a : b;
+    if (sh.r >= 8 && sh.r <= 128) {
+      const size_t c = tc_dB_partial_bytes(sh, m);
+      pb = pb > c ? pb : c;
+    }
   }
   w.partial_bytes = pb;
   w.partial = take(pb);
@@ -210,13 +214,16 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
     if (dB != nullptr && (st = cuda_status(cudaMemsetAsync(dB, 0, (size_t)sh.r * sh.N * sizeof(float), stream)))) return st;
     return QALORA_OK;
   }
-  if ((st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream)) != QALORA_OK) return st;
+  int* status = reinterpret_cast<int*>(wsp + ws.status);
+  if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
+  const bool aux_tc = m > kSmallM && tc_aux_supported(sh, m);
+  if (aux_tc) st = launch_tc_dT(sh, m, dyb, Bb, dT, dTb, status, stream);
+  else st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream);
+  if (st != QALORA_OK) return st;
   if (dA != nullptr || dB != nullptr) {
     if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
   }
   if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
-    int* status = reinterpret_cast<int*>(wsp + ws.status);
-    if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
     st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
                       dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);
     if (st != QALORA_OK) return st;
@@ -230,7 +237,13 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
     if (st != QALORA_OK) return st;
   }
   if (dB != nullptr) {
-    st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial, ws.partial_bytes, stream);
+    if (aux_tc) {
+      int splits = 0;
+      st = launch_tc_dB_partials(sh, m, Tb, dyb, partial, &splits, status, stream);
+      if (st == QALORA_OK) st = launch_sum_partials(partial, dB, (size_t)sh.r * sh.N, splits, stream);
+    } else {
+      st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial, ws.partial_bytes, stream);
+    }
     if (st != QALORA_OK) return st;
   }
   return QALORA_OK;

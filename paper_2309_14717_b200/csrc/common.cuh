@@ -106,6 +106,17 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
                  __nv_bfloat16* dx, int* status, cudaStream_t st);
 
+// out[i] = sum over splits of partial[z][i], added in a fixed order.
+int launch_sum_partials(const float* partial, float* out, size_t count, int splits, cudaStream_t st);
+
+// Tensor-core rank-r side products of the backward pass (aux_tc.cu).
+bool tc_aux_supported(const Shape& sh, int64_t M);
+int launch_tc_dT(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const __nv_bfloat16* B,
+                 float* dT, __nv_bfloat16* dTb, int* status, cudaStream_t st);
+size_t tc_dB_partial_bytes(const Shape& sh, int64_t M);
+int launch_tc_dB_partials(const Shape& sh, int64_t M, const __nv_bfloat16* Tb, const __nv_bfloat16* dy,
+                          float* partial, int* splits_out, int* status, cudaStream_t st);
+
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? QALORA_OK : QALORA_ERR_CUDA; }
 
 // Instrumentation: launch counter and the one-shot event probe around a main kernel.

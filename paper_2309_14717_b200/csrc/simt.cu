@@ -392,6 +392,13 @@ static int launch_atb(int64_t M, int P, int Q, const float* X, const TY* Y, floa
   return cuda_status(cudaGetLastError());
 }
 
+int launch_sum_partials(const float* partial, float* out, size_t count, int splits, cudaStream_t st) {
+  if (count == 0) return QALORA_OK;
+  sum_partials_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(partial, out, count, splits);
+  count_launch();
+  return cuda_status(cudaGetLastError());
+}
+
 int launch_atb_bf16(int64_t M, int P, int Q, const float* X, const __nv_bfloat16* Y, float* out,
                     float* partial, size_t partial_bytes, cudaStream_t st) {
   return launch_atb<__nv_bfloat16>(M, P, Q, X, Y, out, partial, partial_bytes, st);
