@@ -168,6 +168,12 @@ int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void
                        nullptr, T, Tb, stream);
     if (st != QALORA_OK) return st;
   }
+  if (m <= kSmallM && gemv_supported(sh, m)) {
+    return launch_gemv(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
+                       reinterpret_cast<const float2*>(qparams), sh.r > 0 ? T : nullptr,
+                       static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(y),
+                       reinterpret_cast<int*>(wsp + ws.status), stream);
+  }
   if (m > kSmallM && tc_forward_supported(sh, m)) {
     int* status = reinterpret_cast<int*>(wsp + ws.status);
     if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;

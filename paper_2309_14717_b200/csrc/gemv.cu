@@ -1,0 +1,327 @@
+// Few-token forward (M <= 16): y = x * W~ (+ T * B), bound by streaming the packed
+// codes and the (alpha, beta) pairs from HBM exactly once.
+//
+// Design
+//  * One block owns 128 output columns and a slice of the input channels; the
+//    slices of one column tile form a thread-block CLUSTER, and the partial sums
+//    are added through distributed shared memory in a fixed order (no atomics,
+//    no second kernel, no scratch).
+//  * A single thread streams codes, qparams and the x slice into a shared-memory
+//    ring with bulk TMA copies (one per contiguous row of pack units), so that
+//    many tens of KiB per SM are in flight without using registers.
+//  * The products run on mma.sync.m16n8k16 (bf16 in, fp32 accumulate) with the
+//    tokens as the 16 rows: a lane's 32-bit word of packed codes IS its B
+//    fragment after one shift and one mask per pair (the code is OR-ed into the
+//    mantissa of bf16 128.0, no conversion).  The products x * (128 + c) are exact
+//    in fp32; once per quantization group the accumulator is folded as
+//        acc += alpha * D + (beta - 128 alpha) * xp,
+//    where xp (the group sum of x, which the paper's pooling also needs) comes
+//    from one more MMA against a fragment of ones.  alpha and beta stay fp32.
+//  * The same reduction step adds the adapter term T * B (T = s * pool(x) * A is
+//    computed by the pooling kernel) and rounds to bf16.
+#include <cooperative_groups.h>
+
+#include <mutex>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace qalora {
+
+namespace {
+
+constexpr int GV_COLS = 128;        // columns per block
+constexpr int GV_WARPS = 4;         // consumer warps, 32 columns each
+constexpr int GV_THREADS = (GV_WARPS + 1) * 32;   // + 1 producer warp
+constexpr int GV_KBS = 4;           // 32-channel blocks per stage (128 channels)
+constexpr int GV_STAGES = 6;
+constexpr int GV_ROWS = 16;         // token rows of the MMA tile
+
+template <int BITS>
+struct GvSmem {
+  static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
+  static constexpr uint32_t CODE_ROW = GV_COLS * WORDS * 4;             // one k-block row of units
+  static constexpr uint32_t QP_ROW = GV_COLS * 8;
+  static constexpr uint32_t X_BYTES = GV_ROWS * GV_KBS * 32 * 2;        // 16 rows x 128 channels bf16
+  static constexpr uint32_t OFF_CODES = 0;
+  static constexpr uint32_t OFF_QP = GV_KBS * CODE_ROW;
+  static constexpr uint32_t OFF_X = OFF_QP + GV_KBS * QP_ROW;
+  static constexpr uint32_t STAGE_BYTES = ((OFF_X + X_BYTES + 127) / 128) * 128;
+  static constexpr uint32_t OFF_PARTIAL = GV_STAGES * STAGE_BYTES;      // fp32 [16][128]
+  static constexpr uint32_t OFF_BARS = OFF_PARTIAL + GV_ROWS * GV_COLS * 4;
+  static constexpr uint32_t TOTAL = OFF_BARS + 128 + 128;               // + alignment slack
+};
+
+struct GvParams {
+  const uint32_t* codes;
+  const float2* qparams;
+  const float* T;               // fp32 [M][r] (s folded in) or null
+  const __nv_bfloat16* B;       // [r][N]
+  __nv_bfloat16* y;             // [M][N]
+  int M, K, N, g, r;
+  int total_stages;             // K / 128
+  int* status;
+};
+
+__device__ __forceinline__ void mma16816(float* d, const uint32_t* a, uint32_t b0, uint32_t b1, const float* c) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
+}
+
+// The four bf16x2 fragments (128 + c) of the 8 positions 8t .. 8t+7 of a unit, t = lane % 4.
+template <int BITS>
+__device__ __forceinline__ void code_fragments(const uint32_t* unit, int t, uint32_t* f) {
+  constexpr uint32_t MAGIC = 0x43004300u;
+  if (BITS == 4) {
+    const uint32_t w = unit[t];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) f[i] = ((w >> (4 * i)) & 0x000f000fu) | MAGIC;
+  } else if (BITS == 2) {
+    const uint32_t w = unit[t >> 1] >> (8 * (t & 1));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) f[i] = ((w >> (2 * i)) & 0x00030003u) | MAGIC;
+  } else {
+    const uint32_t w = unit[t >> 1] >> (8 * (t & 1));
+    const uint32_t h = unit[2] >> (4 * t);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) f[i] = ((w >> (2 * i)) & 0x00030003u) | (((h >> i) & 0x00010001u) << 2) | MAGIC;
+  }
+}
+
+template <int BITS, bool UPPER>   // UPPER: token rows 8..15 are in use (M > 8)
+__global__ void __launch_bounds__(GV_THREADS, 2)
+qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const GvParams p) {
+  using S = GvSmem<BITS>;
+  constexpr int WORDS = S::WORDS;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+  const uint32_t smem_base = ptx::smem_u32(smem);
+  auto bar_full = [&](int s) { return smem_base + S::OFF_BARS + 8u * s; };
+  auto bar_empty = [&](int s) { return smem_base + S::OFF_BARS + 8u * (GV_STAGES + s); };
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_BARS + 8 * (2 * GV_STAGES));
+  float* partial = reinterpret_cast<float*>(smem + S::OFF_PARTIAL);
+
+  cg::cluster_group cluster = cg::this_cluster();
+  const int splits = (int)cluster.num_blocks();
+  const int rank = (int)cluster.block_rank();
+  const int n0 = (blockIdx.x / splits) * GV_COLS;
+  const int st_beg = (int)((long long)p.total_stages * rank / splits);
+  const int st_end = (int)((long long)p.total_stages * (rank + 1) / splits);
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < GV_STAGES; ++s) {
+      ptx::mbar_init(bar_full(s), 1);
+      ptx::mbar_init(bar_empty(s), GV_WARPS);
+    }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&x_map);
+    if (blockIdx.x == 0) *p.status = 0;     // every block is resident from the start; a timeout is seconds away
+  }
+  __syncthreads();
+
+  if (warp == GV_WARPS) {
+    // ------------------------------------------------------------ producer ----
+    if (lane == 0) {
+      bool ok = true;
+      for (int st = st_beg, it = 0; st < st_end && ok; ++st, ++it) {
+        const int s = it % GV_STAGES;
+        if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / GV_STAGES) & 1) ^ 1, abort_flag))) break;
+        const uint32_t stage = smem_base + s * S::STAGE_BYTES;
+        ptx::mbar_arrive_expect_tx(bar_full(s), GV_KBS * (S::CODE_ROW + S::QP_ROW) + S::X_BYTES);
+#pragma unroll
+        for (int b = 0; b < GV_KBS; ++b) {
+          const int kb = st * GV_KBS + b;
+          ptx::bulk_load(stage + S::OFF_CODES + b * S::CODE_ROW, p.codes + ((size_t)kb * p.N + n0) * WORDS,
+                         S::CODE_ROW, bar_full(s));
+          ptx::bulk_load(stage + S::OFF_QP + b * S::QP_ROW, p.qparams + (size_t)(kb * 32 / p.g) * p.N + n0,
+                         S::QP_ROW, bar_full(s));
+        }
+        ptx::tma_load_2d(stage + S::OFF_X, &x_map, st * GV_KBS * 32, 0, bar_full(s));
+      }
+    }
+  } else {
+    // ----------------------------------------------------------- consumers ----
+    const int gq = lane / 4, t = lane % 4;        // fragment row / column group, quad lane
+    const int kb_per_group = p.g / 32;
+    float acc[4][4], D[4][4], Dx[4];
+    const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { acc[c][i] = 0.f; D[c][i] = 0.f; }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) Dx[i] = 0.f;
+    constexpr uint32_t ONES = 0x3f803f80u;        // bf16x2 (1, 1)
+    bool ok = true;
+    for (int st = st_beg, it = 0; st < st_end && ok; ++st, ++it) {
+      const int s = it % GV_STAGES;
+      if (!(ok = ptx::mbar_wait(bar_full(s), (it / GV_STAGES) & 1, abort_flag))) break;
+      const uint8_t* stage = smem + s * S::STAGE_BYTES;
+#pragma unroll
+      for (int b = 0; b < GV_KBS; ++b) {
+        const int kb = st * GV_KBS + b;
+        // A fragments: x[row][32 b + 8 t .. + 7] for rows gq and gq + 8
+        const uint4 xl = *reinterpret_cast<const uint4*>(stage + S::OFF_X + gq * (GV_KBS * 64) + b * 64 + t * 16);
+        uint4 xh = make_uint4(0u, 0u, 0u, 0u);
+        if (UPPER) xh = *reinterpret_cast<const uint4*>(stage + S::OFF_X + (gq + 8) * (GV_KBS * 64) + b * 64 + t * 16);
+        const uint32_t a0[4] = {xl.x, xh.x, xl.y, xh.y};     // slots (2t,2t+1) | (2t+8,2t+9) of MMA 0
+        const uint32_t a1[4] = {xl.z, xh.z, xl.w, xh.w};     // the same slots of MMA 1
+        const bool first = (kb % kb_per_group) == 0, last = (kb % kb_per_group) == kb_per_group - 1;
+        mma16816(Dx, a0, ONES, ONES, first ? zero4 : Dx);
+        mma16816(Dx, a1, ONES, ONES, Dx);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int col = warp * 32 + c * 8;
+          const uint32_t* unit = reinterpret_cast<const uint32_t*>(stage + S::OFF_CODES + b * S::CODE_ROW) + (col + gq) * WORDS;
+          uint32_t f[4];
+          code_fragments<BITS>(unit, t, f);
+          mma16816(D[c], a0, f[0], f[1], first ? zero4 : D[c]);
+          mma16816(D[c], a1, f[2], f[3], D[c]);
+          if (last) {
+            // accumulator columns of this lane are col + 2t and col + 2t + 1
+            const float4 q = *reinterpret_cast<const float4*>(stage + S::OFF_QP + b * S::QP_ROW + (col + 2 * t) * 8);
+            const float bias0 = fmaf(-128.f, q.x, q.y), bias1 = fmaf(-128.f, q.z, q.w);
+            acc[c][0] = fmaf(q.x, D[c][0], fmaf(bias0, Dx[0], acc[c][0]));
+            acc[c][1] = fmaf(q.z, D[c][1], fmaf(bias1, Dx[1], acc[c][1]));
+            if (UPPER) {
+              acc[c][2] = fmaf(q.x, D[c][2], fmaf(bias0, Dx[2], acc[c][2]));
+              acc[c][3] = fmaf(q.z, D[c][3], fmaf(bias1, Dx[3], acc[c][3]));
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_empty(s));
+    }
+    // partial sums of this block: [16 rows][128 columns]
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int col = warp * 32 + c * 8 + 2 * t;
+      *reinterpret_cast<float2*>(partial + gq * GV_COLS + col) = make_float2(acc[c][0], acc[c][1]);
+      *reinterpret_cast<float2*>(partial + (gq + 8) * GV_COLS + col) = make_float2(acc[c][2], acc[c][3]);
+    }
+  }
+
+  // ---- add the slices in rank order through distributed shared memory ---------
+  cluster.sync();
+  {
+    const int cols_per = GV_COLS / splits;                 // splits is 1, 2, 4 or 8
+    const int outs = p.M * cols_per;
+    for (int o = threadIdx.x; o < outs; o += GV_THREADS) {
+      const int row = o / cols_per, col = rank * cols_per + o % cols_per;
+      float v = 0.f;
+      for (int rk = 0; rk < splits; ++rk) v += cluster.map_shared_rank(partial, rk)[row * GV_COLS + col];
+      if (p.r > 0) {
+        const float* Tr = p.T + (size_t)row * p.r;
+        const __nv_bfloat16* Bc = p.B + n0 + col;
+        float a = 0.f;
+        for (int i = 0; i < p.r; ++i) a = fmaf(Tr[i], __bfloat162float(Bc[(size_t)i * p.N]), a);
+        v += a;
+      }
+      p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v);
+    }
+  }
+  cluster.sync();
+  if (threadIdx.x == 0 && *abort_flag != 0) atomicExch(p.status, 1);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn gv_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+int gv_sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+template <int BITS, bool UPPER>
+int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
+  using S = GvSmem<BITS>;
+  auto kern = qalora_gemv_kernel<BITS, UPPER>;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
+  if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((p.N / GV_COLS) * splits));
+  cfg.blockDim = dim3(GV_THREADS);
+  cfg.dynamicSmemBytes = S::TOTAL;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)splits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e;
+  {
+    MainKernelProbe probe("qalora_gemv_kernel", st);
+    e = cudaLaunchKernelEx(&cfg, kern, xm, p);
+  }
+  count_launch();
+  return cuda_status(e);
+}
+
+}  // namespace
+
+bool gemv_supported(const Shape& sh, int64_t M) {
+  return M >= 1 && M <= GV_ROWS && sh.N % GV_COLS == 0 && sh.K % (GV_KBS * 32) == 0 && (GV_KBS * 32) % sh.g == 0 &&
+         gv_encode_fn() != nullptr;
+}
+
+// y = x * W~ + T * B for M <= 16 rows; T is fp32 [M][r] with s folded in (null when r == 0).
+int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
+                const float* T, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, cudaStream_t st) {
+  EncodeTiledFn fn = gv_encode_fn();
+  CUtensorMap xm;
+  cuuint64_t dims[2] = {(cuuint64_t)sh.K, (cuuint64_t)M};
+  cuuint64_t strides[1] = {(cuuint64_t)sh.K * 2};
+  cuuint32_t box[2] = {GV_KBS * 32, GV_ROWS};
+  cuuint32_t estr[2] = {1, 1};
+  if (fn(&xm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(x), dims, strides, box, estr,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return QALORA_ERR_CUDA;
+  GvParams p{};
+  p.codes = codes; p.qparams = qparams; p.T = T; p.B = B; p.y = y;
+  p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
+  p.total_stages = sh.K / (GV_KBS * 32);
+  p.status = status;
+  // slices per column tile: enough blocks for two per SM, at most 8 (portable cluster size)
+  const int tiles = sh.N / GV_COLS;
+  int splits = 1;
+  while (splits < 8 && tiles * splits < 2 * gv_sm_count() && splits * 2 <= p.total_stages) splits *= 2;
+  const bool upper = M > 8;
+#define QALORA_GV(BITS) (upper ? launch_gemv_t<BITS, true>(xm, p, splits, st) : launch_gemv_t<BITS, false>(xm, p, splits, st))
+  if (sh.bits == 4) return QALORA_GV(4);
+  if (sh.bits == 3) return QALORA_GV(3);
+  return QALORA_GV(2);
+#undef QALORA_GV
+}
+
+}  // namespace qalora

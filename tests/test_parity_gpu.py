@@ -155,6 +155,25 @@ def test_config2_small_m_forward_and_merge(M):
     assert rel_err(layer.forward(qparams=q2, rank=0).float().cpu().numpy(), y_ref) <= TOL
 
 
+@pytest.mark.parametrize("bits,g,M,r", [(4, 32, 1, 16), (4, 128, 8, 0), (3, 32, 16, 24), (3, 64, 3, 8),
+                                       (2, 32, 9, 64), (2, 128, 1, 0), (4, 64, 16, 128)])
+def test_few_token_forward_all_widths(bits, g, M, r):
+    """The bandwidth-bound few-token kernel (N % 128 == 0, K % 128 == 0): every bit
+    width, group sizes 32/64/128, with and without the adapter, M below and above 8."""
+    cfg = LayerConfig("gemv", 1280, 384, g, bits, max(r, 8), 1.25, M, outlier_frac=0.01, seed=bits * 100 + g + M)
+    layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
+    codes, alpha, beta = check_quantize(layer)
+    x, A, B = (to_f64(layer.cpu[k]) for k in ("x", "A", "B"))
+    if r == 0:
+        y_ref = O.forward(x, codes, alpha, beta, g)
+        got = layer.forward(rank=0)
+    else:
+        y_ref = O.forward(x, codes, alpha, beta, g, A, B, cfg.scale)
+        got = layer.forward()
+    assert Q.qalora_main_kernel_name() == "qalora_gemv_kernel"
+    assert rel_err(got.float().cpu().numpy(), y_ref) <= TOL
+
+
 def test_edge_cases():
     cfg = LayerConfig("edge", 64, 64, 32, 4, 8, 1.0, 3, seed=9)
     layer = GpuLayer(cfg)
