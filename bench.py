@@ -383,14 +383,60 @@ def small_m_bandwidth(Q, torch, pk, shape=SMALL_M, ms=(1, 4, 16)):
     return out
 
 
+def run_only(args):
+    """Profiling helper: a few launches of one operation on one shape with a
+    reduced token count (inputs still exceed L2), e.g. for an ncu capture:
+        python bench.py --only fwd --shape cfg3_7b_up --tokens 4096"""
+    import torch
+
+    from paper_2309_14717_b200 import binding as Q
+    from paper_2309_14717_b200 import build as _build
+    from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
+
+    _build.build()
+    cfg = CONFIGS[args.shape].with_(tokens=args.tokens)
+    t = {k: v.cuda() for k, v in make_inputs(cfg).items()}
+    M, K, N, G, r = cfg.tokens, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank
+    d = Q.desc(K, N, cfg.group_size, cfg.bits, r, cfg.scale)
+    codes, qparams = Q.alloc_packed(d)
+    Q.qalora_quantize(d, t["W"], codes, qparams)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dA = torch.empty((G, r), dtype=torch.float32, device="cuda")
+    dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
+    wf, wb = Q.alloc_workspace(d, M, Q.OP_FORWARD), Q.alloc_workspace(d, M, Q.OP_BACKWARD)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    for _ in range(args.steps + 2):
+        e0.record()
+        if args.only in ("fwd", "gemv"):
+            Q.qalora_forward(d, M, t["x"], codes, qparams, t["A"], t["B"], y, wf)
+        elif args.only == "bwd":
+            Q.qalora_backward(d, M, t["x"], t["dy"], codes, qparams, t["A"], t["B"], dx, dA, dB, wb)
+        elif args.only == "quantize":
+            Q.qalora_quantize(d, t["W"], codes, qparams)
+        elif args.only == "merge":
+            Q.qalora_merge(d, qparams, t["A"], t["B"], qparams)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    print(json.dumps({"only": args.only, "shape": args.shape, "tokens": M, "ms": times[2:],
+                      "status": Q.workspace_status(wb if args.only == "bwd" else wf)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--only", default=None, choices=("fwd", "bwd", "gemv", "quantize", "merge"))
+    ap.add_argument("--shape", default="cfg3_7b_up")
+    ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.only is not None:
+        run_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
