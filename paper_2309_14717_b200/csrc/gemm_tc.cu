@@ -17,8 +17,9 @@
 // reduction steps of width r: forward appends T = s*pool(x)*A against B, dx
 // appends dT = s*dy*B^T against the group-expanded A.
 //
-// Warp roles (512 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
-// owner, warps 4-11 = dequantizers, warps 12-15 = epilogue.  Stages are handed
+// Warp roles (768 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
+// owner, warps 4-19 = four dequantizing warpgroups (each owns every fourth
+// reduction step), warps 20-23 = epilogue.  Stages are handed
 // over with mbarriers; every wait is bounded and a timeout raises a status word
 // instead of hanging.
 #include <mutex>
@@ -33,10 +34,11 @@ namespace {
 constexpr int TILE_C = 128;      // out channels per tile   (MMA M)
 constexpr int TILE_T = 256;      // tokens per tile         (MMA N)
 constexpr int TILE_J = 64;       // reduction step per stage
-constexpr int THREADS = 512;
+constexpr int DQ_GROUPS = 4;     // dequantizing warpgroups
+constexpr int THREADS = 128 + 128 * DQ_GROUPS + 128;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_COL = 0;       // accumulator: columns [0, 256)
-constexpr int A_COL = 256;       // forward A ring: 32 columns per stage
+constexpr int A_COL = 256;       // forward operand ring: 8 slots of 32 columns
 constexpr uint32_t ACT_BYTES = TILE_T * TILE_J * 2;      // 32 KiB activation tile
 constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx)
 
@@ -55,20 +57,29 @@ struct TcParams {
   int* status;                 // device word: set to 1 when a wait timed out
 };
 
-template <int BITS, int MODE, int STAGES>
+// Three rings, decoupled so that each covers its own latency:
+//   NX activation tiles (TMA, 32 KiB each)            -> consumed by the MMA
+//   NC code stages (bulk TMA, codes + qparams, ~6 KiB) -> consumed by the dequantizers
+//   NA operand slots (TMEM columns for forward, 16 KiB of smem for dx) written by the
+//      dequantizers, consumed by the MMA.
+// NC and NA are multiples of DQ_GROUPS, so a ring slot always belongs to the same
+// dequantizing warpgroup and its barrier phases are waited on in order.
+template <int BITS, int MODE>
 struct Smem {
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
-  static constexpr uint32_t UNITS = MODE == FWD ? 2 * TILE_C : 4 * TILE_J;     // 256 units per stage
+  static constexpr int NX = 4;
+  static constexpr int NC = MODE == FWD ? 8 : 4;
+  static constexpr int NA = MODE == FWD ? 8 : 4;
+  static constexpr uint32_t UNITS = MODE == FWD ? 2 * TILE_C : 4 * TILE_J;     // 256 units per step
   static constexpr uint32_t CODE_BYTES = UNITS * WORDS * 4;
   static constexpr uint32_t QP_BYTES = UNITS * 8;
-  static constexpr uint32_t A_BYTES = MODE == DX ? ATILE_BYTES : 0;
-  static constexpr uint32_t STAGE_BYTES = ACT_BYTES + A_BYTES + ((CODE_BYTES + QP_BYTES + 1023) / 1024) * 1024;
-  static constexpr uint32_t OFF_ACT = 0;
-  static constexpr uint32_t OFF_A = ACT_BYTES;
-  static constexpr uint32_t OFF_CODES = ACT_BYTES + A_BYTES;
-  static constexpr uint32_t OFF_QP = OFF_CODES + CODE_BYTES;
-  static constexpr uint32_t BAR_BYTES = 256;
-  static constexpr uint32_t TOTAL = STAGES * STAGE_BYTES + BAR_BYTES + 1024;   // + alignment slack
+  static constexpr uint32_t CSTAGE_BYTES = ((CODE_BYTES + QP_BYTES + 127) / 128) * 128;
+  static constexpr uint32_t OFF_X = 0;
+  static constexpr uint32_t OFF_A = NX * ACT_BYTES;                              // dx only
+  static constexpr uint32_t OFF_C = OFF_A + (MODE == DX ? NA * ATILE_BYTES : 0);
+  static constexpr uint32_t OFF_BARS = OFF_C + NC * CSTAGE_BYTES;
+  static constexpr int NBARS = 2 * NX + 2 * NC + 2 * NA + 2;
+  static constexpr uint32_t TOTAL = OFF_BARS + 8 * NBARS + 64 + 1024;            // + alignment slack
 };
 
 // ---- dequantization of one pack unit to 16 bf16x2 registers ------------------
@@ -142,34 +153,34 @@ __device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, uint3
   dq_all<BITS, 0, 0>(w, a, b, out);
 }
 
-template <int BITS, int MODE, int STAGES>
+template <int BITS, int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_constant__ CUtensorMap lora_map,
                  const TcParams p) {
-  using S = Smem<BITS, MODE, STAGES>;
+  using S = Smem<BITS, MODE>;
   constexpr int WORDS = S::WORDS;
+  constexpr int NX = S::NX, NC = S::NC, NA = S::NA;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = ptx::smem_u32(smem);
-  uint8_t* bar_area = smem + STAGES * S::STAGE_BYTES;
-  const uint32_t bar_base = smem_base + STAGES * S::STAGE_BYTES;
-  // barrier layout (8 bytes each): full[S], aready[S], empty[S], acc_full, acc_empty
-  auto bar_full = [&](int s) { return bar_base + 8u * s; };
-  auto bar_aready = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  auto bar_empty = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
-  const uint32_t bar_acc_full = bar_base + 8u * (3 * STAGES);
-  const uint32_t bar_acc_empty = bar_base + 8u * (3 * STAGES + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_area + 8 * (3 * STAGES + 2));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_area + 8 * (3 * STAGES + 2) + 8);
+  const uint32_t bar_base = smem_base + S::OFF_BARS;
+  auto bar_full_x = [&](int s) { return bar_base + 8u * s; };
+  auto bar_empty_x = [&](int s) { return bar_base + 8u * (NX + s); };
+  auto bar_full_c = [&](int s) { return bar_base + 8u * (2 * NX + s); };
+  auto bar_empty_c = [&](int s) { return bar_base + 8u * (2 * NX + NC + s); };
+  auto bar_aready = [&](int s) { return bar_base + 8u * (2 * NX + 2 * NC + s); };
+  auto bar_empty_a = [&](int s) { return bar_base + 8u * (2 * NX + 2 * NC + NA + s); };
+  const uint32_t bar_acc_full = bar_base + 8u * (2 * NX + 2 * NC + 2 * NA);
+  const uint32_t bar_acc_empty = bar_acc_full + 8u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + S::OFF_BARS + 8 * S::NBARS);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_BARS + 8 * S::NBARS + 8);
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(bar_full(s), 1);
-      ptx::mbar_init(bar_aready(s), 8);
-      ptx::mbar_init(bar_empty(s), 1);
-    }
+    for (int s = 0; s < NX; ++s) { ptx::mbar_init(bar_full_x(s), 1); ptx::mbar_init(bar_empty_x(s), 1); }
+    for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4); }
+    for (int s = 0; s < NA; ++s) { ptx::mbar_init(bar_aready(s), 4); ptx::mbar_init(bar_empty_a(s), 1); }
     ptx::mbar_init(bar_acc_full, 1);
     ptx::mbar_init(bar_acc_empty, 4);
     *abort_flag = 0;
@@ -191,42 +202,57 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   const int iters = p.red_iters + p.lora_iters;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ producer ----
+    // ------------------------------------------------- activation producer ----
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
-        const int c0 = ct * TILE_C, m0 = mt * TILE_T;
+        const int m0 = (tile / p.c_tiles) * TILE_T;
         for (int i = 0; i < iters; ++i, ++it) {
-          const int s = it % STAGES;
-          if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / STAGES) & 1) ^ 1, abort_flag))) break;
-          const uint32_t stage = smem_base + s * S::STAGE_BYTES;
-          if (i < p.red_iters) {
-            ptx::mbar_arrive_expect_tx(bar_full(s), ACT_BYTES + S::CODE_BYTES + S::QP_BYTES);
-            ptx::tma_load_2d(stage + S::OFF_ACT, &act_map, i * TILE_J, m0, bar_full(s));
-            if (MODE == FWD) {
+          const int s = it % NX;
+          if (!(ok = ptx::mbar_wait(bar_empty_x(s), ((it / NX) & 1) ^ 1, abort_flag))) break;
+          ptx::mbar_arrive_expect_tx(bar_full_x(s), ACT_BYTES);
+          if (i < p.red_iters)
+            ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &act_map, i * TILE_J, m0, bar_full_x(s));
+          else
+            ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &lora_map, (i - p.red_iters) * TILE_J, m0, bar_full_x(s));
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------- code producer ----
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int c0 = (tile % p.c_tiles) * TILE_C;
+        for (int i = 0; i < iters; ++i, ++it) {
+          const int s = it % NC;
+          if (!(ok = ptx::mbar_wait(bar_empty_c(s), ((it / NC) & 1) ^ 1, abort_flag))) break;
+          const uint32_t stage = smem_base + S::OFF_C + s * S::CSTAGE_BYTES;
+          if (i >= p.red_iters) {                 // adapter step: nothing to stream, just open the phase
+            ptx::mbar_arrive(bar_full_c(s));
+            continue;
+          }
+          ptx::mbar_arrive_expect_tx(bar_full_c(s), S::CODE_BYTES + S::QP_BYTES);
+          if (MODE == FWD) {
 #pragma unroll
-              for (int b = 0; b < 2; ++b) {
-                const int kb = i * 2 + b;
-                ptx::bulk_load(stage + S::OFF_CODES + b * (TILE_C * WORDS * 4),
-                               p.codes + ((size_t)kb * p.N + c0) * WORDS, TILE_C * WORDS * 4, bar_full(s));
-                ptx::bulk_load(stage + S::OFF_QP + b * (TILE_C * 8),
-                               p.qparams + (size_t)(kb * 32 / p.g) * p.N + c0, TILE_C * 8, bar_full(s));
-              }
-            } else {
-#pragma unroll
-              for (int b = 0; b < 4; ++b) {
-                const int kb = c0 / 32 + b, n0 = i * TILE_J;
-                ptx::bulk_load(stage + S::OFF_CODES + b * (TILE_J * WORDS * 4),
-                               p.codes + ((size_t)kb * p.N + n0) * WORDS, TILE_J * WORDS * 4, bar_full(s));
-                ptx::bulk_load(stage + S::OFF_QP + b * (TILE_J * 8),
-                               p.qparams + (size_t)(kb * 32 / p.g) * p.N + n0, TILE_J * 8, bar_full(s));
-              }
+            for (int b = 0; b < 2; ++b) {
+              const int kb = i * 2 + b;
+              ptx::bulk_load(stage + b * (TILE_C * WORDS * 4), p.codes + ((size_t)kb * p.N + c0) * WORDS,
+                             TILE_C * WORDS * 4, bar_full_c(s));
+              ptx::bulk_load(stage + S::CODE_BYTES + b * (TILE_C * 8), p.qparams + (size_t)(kb * 32 / p.g) * p.N + c0,
+                             TILE_C * 8, bar_full_c(s));
             }
           } else {
-            ptx::mbar_arrive_expect_tx(bar_full(s), ACT_BYTES);
-            ptx::tma_load_2d(stage + S::OFF_ACT, &lora_map, (i - p.red_iters) * TILE_J, m0, bar_full(s));
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+              const int kb = c0 / 32 + b, n0 = i * TILE_J;
+              ptx::bulk_load(stage + b * (TILE_J * WORDS * 4), p.codes + ((size_t)kb * p.N + n0) * WORDS,
+                             TILE_J * WORDS * 4, bar_full_c(s));
+              ptx::bulk_load(stage + S::CODE_BYTES + b * (TILE_J * 8), p.qparams + (size_t)(kb * 32 / p.g) * p.N + n0,
+                             TILE_J * 8, bar_full_c(s));
+            }
           }
         }
       }
@@ -242,108 +268,123 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int i = 0; i < iters; ++i, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
-          if (!(ok = ptx::mbar_wait(bar_full(s), ph, abort_flag))) break;
-          if (!(ok = ptx::mbar_wait(bar_aready(s), ph, abort_flag))) break;
+          const int sx = it % NX, sa = it % NA;
+          if (!(ok = ptx::mbar_wait(bar_aready(sa), (it / NA) & 1, abort_flag))) break;
+          if (!(ok = ptx::mbar_wait(bar_full_x(sx), (it / NX) & 1, abort_flag))) break;
           ptx::tc_fence_after();
-          const uint32_t stage = smem_base + s * S::STAGE_BYTES;
+          const uint32_t xs = smem_base + S::OFF_X + sx * ACT_BYTES;
+          const uint32_t as = smem_base + S::OFF_A + sa * ATILE_BYTES;
 #pragma unroll
           for (int j = 0; j < TILE_J / 16; ++j) {
-            const uint64_t bdesc = ptx::smem_desc(stage + S::OFF_ACT + j * 32, 16, 1024);
+            const uint64_t bdesc = ptx::smem_desc(xs + j * 32, 16, 1024);
             const uint32_t acc = (i > 0 || j > 0) ? 1u : 0u;
             if (MODE == FWD) {
-              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + s * 32 + j * 8, bdesc, IDESC_MAIN, acc);
+              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + sa * 32 + j * 8, bdesc, IDESC_MAIN, acc);
             } else if (i < p.red_iters) {
               // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO)
-              const uint64_t adesc = ptx::smem_desc(stage + S::OFF_A + j * 2048, 8192, 1024);
-              ptx::mma_ss(tmem_base + ACC_COL, adesc, bdesc, IDESC_MAIN, acc);
+              ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 2048, 8192, 1024), bdesc, IDESC_MAIN, acc);
             } else {
-              const uint64_t adesc = ptx::smem_desc(stage + S::OFF_A + j * 32, 16, 1024);
-              ptx::mma_ss(tmem_base + ACC_COL, adesc, bdesc, IDESC_LORA, acc);
+              ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 32, 16, 1024), bdesc, IDESC_LORA, acc);
             }
           }
-          ptx::mma_commit(bar_empty(s));
+          ptx::mma_commit(bar_empty_x(sx));
+          ptx::mma_commit(bar_empty_a(sa));
         }
         if (ok) ptx::mma_commit(bar_acc_full);
       }
     }
-  } else if (warp >= 4 && warp < 12) {
+  } else if (warp >= 4 && warp < 4 + 4 * DQ_GROUPS) {
     // -------------------------------------------------------- dequantizers ----
-    const int dq = threadIdx.x - 128;            // 0..255
+    // Warpgroup w owns the reduction steps with it % DQ_GROUPS == w and dequantizes
+    // the whole step (two pack units per thread); the groups work on different
+    // steps at once and hide each other's latencies.
+    const int wg = (warp - 4) / 4;
+    const int tw = threadIdx.x - 128 - wg * 128;  // 0..127 inside the warpgroup
     const int quarter = warp % 4;                // TMEM lane quarter of this warp
     uint32_t it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int ct = tile % p.c_tiles;
-      const int c0 = ct * TILE_C;
+      const int c0 = (tile % p.c_tiles) * TILE_C;
       for (int i = 0; i < iters; ++i, ++it) {
-        const int s = it % STAGES;
-        if (!(ok = ptx::mbar_wait(bar_full(s), (it / STAGES) & 1, abort_flag))) break;
-        uint8_t* stage = smem + s * S::STAGE_BYTES;
-        uint32_t v[16];
+        if ((int)(it % DQ_GROUPS) != wg) continue;
+        const int sc = it % NC, sa = it % NA;
+        if (!(ok = ptx::mbar_wait(bar_full_c(sc), (it / NC) & 1, abort_flag))) break;
+        if (!(ok = ptx::mbar_wait(bar_empty_a(sa), ((it / NA) & 1) ^ 1, abort_flag))) break;
+        const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         if (MODE == FWD) {
-          const int half = (warp - 4) / 4;       // which 32-channel block of the stage
+          ptx::tc_fence_after();
           const int row = quarter * 32 + lane;   // out channel within the tile = TMEM lane
-          if (i < p.red_iters) {
-            const uint32_t* cw = reinterpret_cast<const uint32_t*>(stage + S::OFF_CODES) + (half * TILE_C + row) * WORDS;
-            uint32_t w[WORDS];
-            load_unit<WORDS>(cw, w);
-            const float2 ab = reinterpret_cast<const float2*>(stage + S::OFF_QP)[half * TILE_C + row];
-            dequant_unit<BITS>(w, ab, v);
-          } else {
-            // adapter step: row c of the operand is B[r0 + 0..63][c]; this thread packs 32 of them
-            const int r0 = (i - p.red_iters) * TILE_J + half * 32;
-            const __nv_bfloat16* bp = p.lora + (size_t)r0 * p.N + c0 + row;
 #pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              const int ra = r0 + 2 * q;
-              const uint32_t lo = ra < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q) * p.N) : 0u;
-              const uint32_t hi = ra + 1 < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q + 1) * p.N) : 0u;
-              v[q] = lo | (hi << 16);
+          for (int half = 0; half < 2; ++half) { // the two 32-channel blocks of the step
+            uint32_t v[16];
+            if (i < p.red_iters) {
+              const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (half * TILE_C + row) * WORDS;
+              uint32_t w[WORDS];
+              load_unit<WORDS>(cw, w);
+              const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[half * TILE_C + row];
+              dequant_unit<BITS>(w, ab, v);
+            } else {
+              // adapter step: row c of the operand is B[r0 + 0..63][c]; this thread packs 32 of them
+              const int r0 = (i - p.red_iters) * TILE_J + half * 32;
+              const __nv_bfloat16* bp = p.lora + (size_t)r0 * p.N + c0 + row;
+#pragma unroll
+              for (int q = 0; q < 16; ++q) {
+                const int ra = r0 + 2 * q;
+                const uint32_t lo = ra < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q) * p.N) : 0u;
+                const uint32_t hi = ra + 1 < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q + 1) * p.N) : 0u;
+                v[q] = lo | (hi << 16);
+              }
             }
+            ptx::tmem_st16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL + sa * 32 + half * 16, v);
           }
-          ptx::tmem_st16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL + s * 32 + half * 16, v);
           ptx::tmem_wait_st();
           ptx::tc_fence_before();
         } else {
-          uint8_t* atile = stage + S::OFF_A;
-          if (i < p.red_iters) {
-            const int kbl = dq / TILE_J, nl = dq % TILE_J;       // 32-channel block, column
-            const uint32_t* cw = reinterpret_cast<const uint32_t*>(stage + S::OFF_CODES) + (kbl * TILE_J + nl) * WORDS;
-            uint32_t w[WORDS];
-            load_unit<WORDS>(cw, w);
-            const float2 ab = reinterpret_cast<const float2*>(stage + S::OFF_QP)[kbl * TILE_J + nl];
-            dequant_unit<BITS>(w, ab, v);
-            // MN-major, 128-byte swizzle: row = column nl (128 bytes = 64 channels),
-            // this unit fills chunks (kbl%2)*4 .. +3 of block kbl/2
-            uint8_t* rowp = atile + (kbl / 2) * 8192 + (nl / 8) * 1024 + (nl % 8) * 128;
+          uint8_t* atile = smem + S::OFF_A + sa * ATILE_BYTES;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int chunk = ((kbl % 2) * 4 + q) ^ (nl % 8);
-              *reinterpret_cast<uint4*>(rowp + chunk * 16) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-            }
-          } else {
-            // adapter step, K-major rows: row c holds A[(c0 + c) / g][r0 .. r0 + 63]
-            const int row = dq / 2, halfrow = dq % 2;
-            const int r0 = (i - p.red_iters) * TILE_J + halfrow * 32;
-            const __nv_bfloat16* ap = p.lora + (size_t)((c0 + row) / p.g) * p.r + r0;
-            uint8_t* rowp = atile + (row / 8) * 1024 + (row % 8) * 128;
+          for (int h = 0; h < 2; ++h) {
+            const int dq = tw + 128 * h;         // 0..255: unit (main steps) / half-row (adapter steps)
+            if (i < p.red_iters) {
+              uint32_t v[16];
+              const int kbl = dq / TILE_J, nl = dq % TILE_J;       // 32-channel block, column
+              const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (kbl * TILE_J + nl) * WORDS;
+              uint32_t w[WORDS];
+              load_unit<WORDS>(cw, w);
+              const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[kbl * TILE_J + nl];
+              dequant_unit<BITS>(w, ab, v);
+              // MN-major, 128-byte swizzle: row = column nl (128 bytes = 64 channels),
+              // this unit fills chunks (kbl%2)*4 .. +3 of block kbl/2
+              uint8_t* rowp = atile + (kbl / 2) * 8192 + (nl / 8) * 1024 + (nl % 8) * 128;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint4 t = make_uint4(0u, 0u, 0u, 0u);
-              if (r0 + q * 8 < p.r) t = *reinterpret_cast<const uint4*>(ap + q * 8);   // r is a multiple of 8
-              const int chunk = (halfrow * 4 + q) ^ (row % 8);
-              *reinterpret_cast<uint4*>(rowp + chunk * 16) = t;
+              for (int q = 0; q < 4; ++q) {
+                const int chunk = ((kbl % 2) * 4 + q) ^ (nl % 8);
+                *reinterpret_cast<uint4*>(rowp + chunk * 16) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+              }
+            } else {
+              // adapter step, K-major rows: row c holds A[(c0 + c) / g][r0 .. r0 + 63]
+              const int row = dq / 2, halfrow = dq % 2;
+              const int r0 = (i - p.red_iters) * TILE_J + halfrow * 32;
+              const __nv_bfloat16* ap = p.lora + (size_t)((c0 + row) / p.g) * p.r + r0;
+              uint8_t* rowp = atile + (row / 8) * 1024 + (row % 8) * 128;
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                uint4 t = make_uint4(0u, 0u, 0u, 0u);
+                if (r0 + q * 8 < p.r) t = *reinterpret_cast<const uint4*>(ap + q * 8);   // r is a multiple of 8
+                const int chunk = (halfrow * 4 + q) ^ (row % 8);
+                *reinterpret_cast<uint4*>(rowp + chunk * 16) = t;
+              }
             }
           }
           ptx::fence_proxy_async();              // make the generic-proxy writes visible to the MMA
         }
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar_aready(s));
+        if (lane == 0) {
+          ptx::mbar_arrive(bar_aready(sa));
+          ptx::mbar_arrive(bar_empty_c(sc));
+        }
       }
     }
-  } else if (warp >= 12) {
+  } else if (warp >= 4 + 4 * DQ_GROUPS) {
     // ------------------------------------------------------------ epilogue ----
     const int quarter = warp % 4;
     uint32_t tcount = 0;
@@ -424,10 +465,9 @@ int sm_count() {
 
 template <int BITS, int MODE>
 int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
-  constexpr int STAGES = MODE == FWD ? 5 : 4;
-  using S = Smem<BITS, MODE, STAGES>;
+  using S = Smem<BITS, MODE>;
   static_assert(S::TOTAL <= 232448, "shared memory budget");
-  auto kern = qalora_tc_kernel<BITS, MODE, STAGES>;
+  auto kern = qalora_tc_kernel<BITS, MODE>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
