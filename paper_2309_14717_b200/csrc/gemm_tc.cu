@@ -38,7 +38,7 @@ constexpr int DQ_GROUPS = 4;     // dequantizing warpgroups
 constexpr int THREADS = 128 + 128 * DQ_GROUPS + 128;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_COL = 0;       // accumulator: columns [0, 256)
-constexpr int A_COL = 256;       // forward operand ring: 8 slots of 32 columns
+constexpr int A_COL = 256;       // forward operand ring: 4 slots of 32 columns
 constexpr uint32_t ACT_BYTES = TILE_T * TILE_J * 2;      // 32 KiB activation tile
 constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx)
 
@@ -57,28 +57,30 @@ struct TcParams {
   int* status;                 // device word: set to 1 when a wait timed out
 };
 
-// Three rings, decoupled so that each covers its own latency:
-//   NX activation tiles (TMA, 32 KiB each)            -> consumed by the MMA
-//   NC code stages (bulk TMA, codes + qparams, ~6 KiB) -> consumed by the dequantizers
-//   NA operand slots (TMEM columns for forward, 16 KiB of smem for dx) written by the
-//      dequantizers, consumed by the MMA.
-// NC and NA are multiples of DQ_GROUPS, so a ring slot always belongs to the same
+// Rings, decoupled so that each covers its own latency:
+//   NX activation tiles (TMA, 32 KiB each) and, in lock step with them, NX operand
+//      slots (TMEM columns for forward, 16 KiB of smem for dx) written by the
+//      dequantizers; one tcgen05.commit per reduction step frees both;
+//   NC code stages (bulk TMA, codes + qparams, ~6 KiB) that run further ahead.
+// NX and NC are multiples of DQ_GROUPS, so a ring slot always belongs to the same
 // dequantizing warpgroup and its barrier phases are waited on in order.
 template <int BITS, int MODE>
 struct Smem {
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   static constexpr int NX = 4;
   static constexpr int NC = MODE == FWD ? 8 : 4;
-  static constexpr int NA = MODE == FWD ? 8 : 4;
+  static constexpr int NOUT = MODE == FWD ? 2 : 1;                               // epilogue staging buffers
   static constexpr uint32_t UNITS = MODE == FWD ? 2 * TILE_C : 4 * TILE_J;     // 256 units per step
   static constexpr uint32_t CODE_BYTES = UNITS * WORDS * 4;
   static constexpr uint32_t QP_BYTES = UNITS * 8;
   static constexpr uint32_t CSTAGE_BYTES = ((CODE_BYTES + QP_BYTES + 127) / 128) * 128;
+  static constexpr uint32_t OUT_BYTES = 32 * TILE_C * 2;                         // 32 tokens x 128 channels bf16
   static constexpr uint32_t OFF_X = 0;
   static constexpr uint32_t OFF_A = NX * ACT_BYTES;                              // dx only
-  static constexpr uint32_t OFF_C = OFF_A + (MODE == DX ? NA * ATILE_BYTES : 0);
-  static constexpr uint32_t OFF_BARS = OFF_C + NC * CSTAGE_BYTES;
-  static constexpr int NBARS = 2 * NX + 2 * NC + 2 * NA + 2;
+  static constexpr uint32_t OFF_C = OFF_A + (MODE == DX ? NX * ATILE_BYTES : 0);
+  static constexpr uint32_t OFF_OUT = OFF_C + NC * CSTAGE_BYTES;
+  static constexpr uint32_t OFF_BARS = OFF_OUT + NOUT * OUT_BYTES;
+  static constexpr int NBARS = 2 * NX + 2 * NC + NX + 2;
   static constexpr uint32_t TOTAL = OFF_BARS + 8 * NBARS + 64 + 1024;            // + alignment slack
 };
 
@@ -156,10 +158,10 @@ __device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, uint3
 template <int BITS, int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_constant__ CUtensorMap lora_map,
-                 const TcParams p) {
+                 const __grid_constant__ CUtensorMap out_map, const TcParams p) {
   using S = Smem<BITS, MODE>;
   constexpr int WORDS = S::WORDS;
-  constexpr int NX = S::NX, NC = S::NC, NA = S::NA;
+  constexpr int NX = S::NX, NC = S::NC;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = ptx::smem_u32(smem);
@@ -169,8 +171,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   auto bar_full_c = [&](int s) { return bar_base + 8u * (2 * NX + s); };
   auto bar_empty_c = [&](int s) { return bar_base + 8u * (2 * NX + NC + s); };
   auto bar_aready = [&](int s) { return bar_base + 8u * (2 * NX + 2 * NC + s); };
-  auto bar_empty_a = [&](int s) { return bar_base + 8u * (2 * NX + 2 * NC + NA + s); };
-  const uint32_t bar_acc_full = bar_base + 8u * (2 * NX + 2 * NC + 2 * NA);
+  const uint32_t bar_acc_full = bar_base + 8u * (2 * NX + 2 * NC + NX);
   const uint32_t bar_acc_empty = bar_acc_full + 8u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + S::OFF_BARS + 8 * S::NBARS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_BARS + 8 * S::NBARS + 8);
@@ -180,13 +181,14 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   if (threadIdx.x == 0) {
     for (int s = 0; s < NX; ++s) { ptx::mbar_init(bar_full_x(s), 1); ptx::mbar_init(bar_empty_x(s), 1); }
     for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4); }
-    for (int s = 0; s < NA; ++s) { ptx::mbar_init(bar_aready(s), 4); ptx::mbar_init(bar_empty_a(s), 1); }
+    for (int s = 0; s < NX; ++s) ptx::mbar_init(bar_aready(s), 4);
     ptx::mbar_init(bar_acc_full, 1);
     ptx::mbar_init(bar_acc_empty, 4);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&act_map);
     if (p.lora_iters > 0) ptx::prefetch_tensormap(&lora_map);
+    ptx::prefetch_tensormap(&out_map);
   }
   if (warp == 1) {
     __syncwarp();
@@ -264,22 +266,31 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(TILE_C, TILE_T, false, false);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
+      // the barriers of the coming step are probed while the MMAs of the current one are being issued
+      bool rdy_a = false, rdy_x = false;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
         if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int i = 0; i < iters; ++i, ++it) {
-          const int sx = it % NX, sa = it % NA;
-          if (!(ok = ptx::mbar_wait(bar_aready(sa), (it / NA) & 1, abort_flag))) break;
-          if (!(ok = ptx::mbar_wait(bar_full_x(sx), (it / NX) & 1, abort_flag))) break;
+          const int sx = it % NX;
+          const uint32_t ph = (it / NX) & 1;
+          if (!rdy_a && !(ok = ptx::mbar_wait(bar_aready(sx), ph, abort_flag))) break;
+          if (!rdy_x && !(ok = ptx::mbar_wait(bar_full_x(sx), ph, abort_flag))) break;
           ptx::tc_fence_after();
+          {
+            const int sn = (it + 1) % NX;
+            const uint32_t pn = ((it + 1) / NX) & 1;
+            rdy_a = ptx::mbar_test_wait(bar_aready(sn), pn);
+            rdy_x = ptx::mbar_test_wait(bar_full_x(sn), pn);
+          }
           const uint32_t xs = smem_base + S::OFF_X + sx * ACT_BYTES;
-          const uint32_t as = smem_base + S::OFF_A + sa * ATILE_BYTES;
+          const uint32_t as = smem_base + S::OFF_A + sx * ATILE_BYTES;
 #pragma unroll
           for (int j = 0; j < TILE_J / 16; ++j) {
             const uint64_t bdesc = ptx::smem_desc(xs + j * 32, 16, 1024);
             const uint32_t acc = (i > 0 || j > 0) ? 1u : 0u;
             if (MODE == FWD) {
-              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + sa * 32 + j * 8, bdesc, IDESC_MAIN, acc);
+              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + sx * 32 + j * 8, bdesc, IDESC_MAIN, acc);
             } else if (i < p.red_iters) {
               // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO)
               ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 2048, 8192, 1024), bdesc, IDESC_MAIN, acc);
@@ -287,8 +298,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 32, 16, 1024), bdesc, IDESC_LORA, acc);
             }
           }
-          ptx::mma_commit(bar_empty_x(sx));
-          ptx::mma_commit(bar_empty_a(sa));
+          ptx::mma_commit(bar_empty_x(sx));        // frees the activation tile AND the operand slot
         }
         if (ok) ptx::mma_commit(bar_acc_full);
       }
@@ -307,9 +317,9 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       const int c0 = (tile % p.c_tiles) * TILE_C;
       for (int i = 0; i < iters; ++i, ++it) {
         if ((int)(it % DQ_GROUPS) != wg) continue;
-        const int sc = it % NC, sa = it % NA;
+        const int sc = it % NC, sa = it % NX;
         if (!(ok = ptx::mbar_wait(bar_full_c(sc), (it / NC) & 1, abort_flag))) break;
-        if (!(ok = ptx::mbar_wait(bar_empty_a(sa), ((it / NA) & 1) ^ 1, abort_flag))) break;
+        if (!(ok = ptx::mbar_wait(bar_empty_x(sa), ((it / NX) & 1) ^ 1, abort_flag))) break;
         const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         if (MODE == FWD) {
           ptx::tc_fence_after();
@@ -386,29 +396,45 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     }
   } else if (warp >= 4 + 4 * DQ_GROUPS) {
     // ------------------------------------------------------------ epilogue ----
+    // Each thread owns one out channel (its TMEM lane) and reads 32 tokens at a
+    // time; the bf16 values are transposed through a [32 tokens][128 channels]
+    // staging tile and leave with one TMA store per chunk (rows beyond M are
+    // clipped by the tensor map).  The accumulator is released as soon as its
+    // last column has been read.
     const int quarter = warp % 4;
-    uint32_t tcount = 0;
+    const int et = threadIdx.x - (128 + 128 * DQ_GROUPS);    // 0..127
+    const int ch = quarter * 32 + lane;
+    uint32_t tcount = 0, chunk = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
       const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
-      const int c = ct * TILE_C + quarter * 32 + lane;
-      const long long m0 = (long long)mt * TILE_T;
       if (!(ok = ptx::mbar_wait(bar_acc_full, tcount & 1, abort_flag))) break;
       ptx::tc_fence_after();
 #pragma unroll 1
-      for (int col = 0; col < TILE_T; col += 32) {
+      for (int col = 0; col < TILE_T; col += 32, ++chunk) {
         uint32_t v[32];
         ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ACC_COL + col, v);
         ptx::tmem_wait_ld();
-        __nv_bfloat16* op = p.out + (size_t)(m0 + col) * p.ld_out + c;
+        if (col == TILE_T - 32) {                 // all columns read: hand the accumulator back
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(bar_acc_empty);
+        }
+        uint8_t* stg = smem + S::OFF_OUT + (chunk % S::NOUT) * S::OUT_BYTES;
+        ptx::named_barrier(1, 128);               // the staging tile's previous store has been read out
 #pragma unroll
         for (int t = 0; t < 32; ++t)
-          if (m0 + col + t < p.M) op[(size_t)t * p.ld_out] = __float2bfloat16_rn(__uint_as_float(v[t]));
+          reinterpret_cast<__nv_bfloat16*>(stg)[t * TILE_C + ch] = __float2bfloat16_rn(__uint_as_float(v[t]));
+        ptx::fence_proxy_async();
+        ptx::named_barrier(2, 128);
+        if (et == 0 && (long long)mt * TILE_T + col < p.M) {
+          ptx::tma_store_2d(&out_map, ct * TILE_C, mt * TILE_T + col, ptx::smem_u32(stg));
+          ptx::bulk_commit_group();
+          ptx::bulk_wait_group_read<S::NOUT - 1>();
+        }
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(bar_acc_empty);
     }
+    if (et == 0) ptx::bulk_wait_group<0>();
   }
 
   // ---------------------------------------------------------------- teardown ----
@@ -463,8 +489,22 @@ int sm_count() {
   return n;
 }
 
+// bf16 output [rows][cols] row-major, box = 128 columns x 32 rows, no swizzle (store side)
+bool make_out_map(CUtensorMap* map, void* base, long long rows, int cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {TILE_C, 32};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BITS, int MODE>
 int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
+  CUtensorMap out;
+  if (!make_out_map(&out, p.out, p.M, p.ld_out)) return QALORA_ERR_CUDA;
   using S = Smem<BITS, MODE>;
   static_assert(S::TOTAL <= 232448, "shared memory budget");
   auto kern = qalora_tc_kernel<BITS, MODE>;
@@ -476,7 +516,7 @@ int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p
   const int grid = tiles < sm_count() ? tiles : sm_count();
   {
     MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
-    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, p);
+    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, out, p);
   }
   count_launch();
   return cuda_status(cudaGetLastError());
