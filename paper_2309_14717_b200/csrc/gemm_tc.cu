@@ -54,6 +54,7 @@ struct TcParams {
   int ld_out;                  // N (FWD) or K (DX)
   int c_tiles, m_tiles;        // tiles along out channels / tokens
   int red_iters, lora_iters;   // main / adapter reduction steps per tile
+  int qp_rows;                 // rows of (alpha, beta) per code stage: 128 / g
   int* status;                 // device word: set to 1 when a wait timed out
 };
 
@@ -61,18 +62,23 @@ struct TcParams {
 //   NX activation tiles (TMA, 32 KiB each) and, in lock step with them, NX operand
 //      slots (TMEM columns for forward, 16 KiB of smem for dx) written by the
 //      dequantizers; one tcgen05.commit per reduction step frees both;
-//   NC code stages (bulk TMA, codes + qparams, ~6 KiB) that run further ahead.
+//   NC code stages (two tiled TMA copies each: 4 k-block rows of pack units and the
+//      rows of (alpha, beta) they need; a forward stage feeds two reduction steps)
+//      that run further ahead.
 // NX and NC are multiples of DQ_GROUPS, so a ring slot always belongs to the same
 // dequantizing warpgroup and its barrier phases are waited on in order.
 template <int BITS, int MODE>
 struct Smem {
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   static constexpr int NX = 4;
-  static constexpr int NC = MODE == FWD ? 8 : 4;
+  static constexpr int NC = 4;
+  static constexpr int IPS = MODE == FWD ? 2 : 1;                                // reduction steps per code stage
+  static constexpr int TILE_NC = MODE == FWD ? TILE_C : TILE_J;                  // columns of a code stage
   static constexpr int NOUT = MODE == FWD ? 2 : 1;                               // epilogue staging buffers
-  static constexpr uint32_t UNITS = MODE == FWD ? 2 * TILE_C : 4 * TILE_J;     // 256 units per step
-  static constexpr uint32_t CODE_BYTES = UNITS * WORDS * 4;
-  static constexpr uint32_t QP_BYTES = UNITS * 8;
+  // a code stage = 4 k-block rows x TILE_NC columns of pack units + up to 4 rows of (alpha, beta)
+  static constexpr uint32_t CODE_BYTES = 4 * TILE_NC * WORDS * 4;
+  static constexpr uint32_t QP_ROW_BYTES = TILE_NC * 8;
+  static constexpr uint32_t QP_BYTES = 4 * QP_ROW_BYTES;
   static constexpr uint32_t CSTAGE_BYTES = ((CODE_BYTES + QP_BYTES + 127) / 128) * 128;
   static constexpr uint32_t OUT_BYTES = 32 * TILE_C * 2;                         // 32 tokens x 128 channels bf16
   static constexpr uint32_t OFF_X = 0;
@@ -158,7 +164,8 @@ __device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, uint3
 template <int BITS, int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_constant__ CUtensorMap lora_map,
-                 const __grid_constant__ CUtensorMap out_map, const TcParams p) {
+                 const __grid_constant__ CUtensorMap out_map, const __grid_constant__ CUtensorMap codes_map,
+                 const __grid_constant__ CUtensorMap qp_map, const TcParams p) {
   using S = Smem<BITS, MODE>;
   constexpr int WORDS = S::WORDS;
   constexpr int NX = S::NX, NC = S::NC;
@@ -180,7 +187,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NX; ++s) { ptx::mbar_init(bar_full_x(s), 1); ptx::mbar_init(bar_empty_x(s), 1); }
-    for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4); }
+    for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4 * S::IPS); }
     for (int s = 0; s < NX; ++s) ptx::mbar_init(bar_aready(s), 4);
     ptx::mbar_init(bar_acc_full, 1);
     ptx::mbar_init(bar_acc_empty, 4);
@@ -189,6 +196,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     ptx::prefetch_tensormap(&act_map);
     if (p.lora_iters > 0) ptx::prefetch_tensormap(&lora_map);
     ptx::prefetch_tensormap(&out_map);
+    ptx::prefetch_tensormap(&codes_map);
+    ptx::prefetch_tensormap(&qp_map);
   }
   if (warp == 1) {
     __syncwarp();
@@ -224,38 +233,22 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   } else if (warp == 2) {
     // ------------------------------------------------------- code producer ----
     if (lane == 0) {
-      uint32_t it = 0;
+      constexpr int UPACK = BITS == 4 ? 1 : (BITS == 2 ? 2 : 4);   // units per 16-byte-aligned map element row
+      uint32_t cit = 0;                              // code stages issued so far
       bool ok = true;
+      const int stages_per_tile = p.red_iters / S::IPS;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int c0 = (tile % p.c_tiles) * TILE_C;
-        for (int i = 0; i < iters; ++i, ++it) {
-          const int s = it % NC;
-          if (!(ok = ptx::mbar_wait(bar_empty_c(s), ((it / NC) & 1) ^ 1, abort_flag))) break;
+        for (int cs = 0; cs < stages_per_tile; ++cs, ++cit) {
+          const int s = cit % NC;
+          if (!(ok = ptx::mbar_wait(bar_empty_c(s), ((cit / NC) & 1) ^ 1, abort_flag))) break;
           const uint32_t stage = smem_base + S::OFF_C + s * S::CSTAGE_BYTES;
-          if (i >= p.red_iters) {                 // adapter step: nothing to stream, just open the phase
-            ptx::mbar_arrive(bar_full_c(s));
-            continue;
-          }
-          ptx::mbar_arrive_expect_tx(bar_full_c(s), S::CODE_BYTES + S::QP_BYTES);
-          if (MODE == FWD) {
-#pragma unroll
-            for (int b = 0; b < 2; ++b) {
-              const int kb = i * 2 + b;
-              ptx::bulk_load(stage + b * (TILE_C * WORDS * 4), p.codes + ((size_t)kb * p.N + c0) * WORDS,
-                             TILE_C * WORDS * 4, bar_full_c(s));
-              ptx::bulk_load(stage + S::CODE_BYTES + b * (TILE_C * 8), p.qparams + (size_t)(kb * 32 / p.g) * p.N + c0,
-                             TILE_C * 8, bar_full_c(s));
-            }
-          } else {
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-              const int kb = c0 / 32 + b, n0 = i * TILE_J;
-              ptx::bulk_load(stage + b * (TILE_J * WORDS * 4), p.codes + ((size_t)kb * p.N + n0) * WORDS,
-                             TILE_J * WORDS * 4, bar_full_c(s));
-              ptx::bulk_load(stage + S::CODE_BYTES + b * (TILE_J * 8), p.qparams + (size_t)(kb * 32 / p.g) * p.N + n0,
-                             TILE_J * 8, bar_full_c(s));
-            }
-          }
+          // forward: k-blocks 4 cs .. 4 cs + 3 of columns c0 ..; dx: the tile's 4 k-blocks, columns 64 cs ..
+          const int kb0 = MODE == FWD ? cs * 4 : c0 / 32;
+          const int col0 = MODE == FWD ? c0 : cs * TILE_J;
+          ptx::mbar_arrive_expect_tx(bar_full_c(s), S::CODE_BYTES + p.qp_rows * S::QP_ROW_BYTES);
+          ptx::tma_load_3d(stage, &codes_map, 0, col0 / UPACK, kb0, bar_full_c(s));
+          ptx::tma_load_2d(stage + S::CODE_BYTES, &qp_map, 2 * col0, kb0 * 32 / p.g, bar_full_c(s));
         }
       }
     }
@@ -311,15 +304,21 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     const int wg = (warp - 4) / 4;
     const int tw = threadIdx.x - 128 - wg * 128;  // 0..127 inside the warpgroup
     const int quarter = warp % 4;                // TMEM lane quarter of this warp
-    uint32_t it = 0;
+    uint32_t it = 0, mit0 = 0;                    // reduction steps / main steps before this tile
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+    const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block -> (alpha, beta) row of the stage
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, mit0 += p.red_iters) {
       const int c0 = (tile % p.c_tiles) * TILE_C;
       for (int i = 0; i < iters; ++i, ++it) {
         if ((int)(it % DQ_GROUPS) != wg) continue;
-        const int sc = it % NC, sa = it % NX;
-        if (!(ok = ptx::mbar_wait(bar_full_c(sc), (it / NC) & 1, abort_flag))) break;
+        const int sa = it % NX;
+        // operand slot first: once it is free every earlier step has been multiplied, so
+        // the code ring's previous phase has certainly completed
         if (!(ok = ptx::mbar_wait(bar_empty_x(sa), ((it / NX) & 1) ^ 1, abort_flag))) break;
+        const uint32_t cst = (mit0 + i) / S::IPS;  // code stage counter (main steps only)
+        const int sc = cst % NC;
+        const int kb_base = MODE == FWD ? ((mit0 + i) % S::IPS) * 2 : 0;   // first k-block row of this step
+        if (i < p.red_iters && !(ok = ptx::mbar_wait(bar_full_c(sc), (cst / NC) & 1, abort_flag))) break;
         const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         if (MODE == FWD) {
           ptx::tc_fence_after();
@@ -328,10 +327,11 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           for (int half = 0; half < 2; ++half) { // the two 32-channel blocks of the step
             uint32_t v[16];
             if (i < p.red_iters) {
-              const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (half * TILE_C + row) * WORDS;
+              const int kbl = kb_base + half;
+              const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (kbl * TILE_C + row) * WORDS;
               uint32_t w[WORDS];
               load_unit<WORDS>(cw, w);
-              const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[half * TILE_C + row];
+              const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[(kbl >> qsh) * TILE_C + row];
               dequant_unit<BITS>(w, ab, v);
             } else {
               // adapter step: row c of the operand is B[r0 + 0..63][c]; this thread packs 32 of them
@@ -360,7 +360,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (kbl * TILE_J + nl) * WORDS;
               uint32_t w[WORDS];
               load_unit<WORDS>(cw, w);
-              const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[kbl * TILE_J + nl];
+              const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[(kbl >> qsh) * TILE_J + nl];
               dequant_unit<BITS>(w, ab, v);
               // MN-major, 128-byte swizzle: row = column nl (128 bytes = 64 channels),
               // this unit fills chunks (kbl%2)*4 .. +3 of block kbl/2
@@ -390,7 +390,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         __syncwarp();
         if (lane == 0) {
           ptx::mbar_arrive(bar_aready(sa));
-          ptx::mbar_arrive(bar_empty_c(sc));
+          if (i < p.red_iters) ptx::mbar_arrive(bar_empty_c(sc));
         }
       }
     }
@@ -501,11 +501,40 @@ bool make_out_map(CUtensorMap* map, void* base, long long rows, int cols) {
             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// packed codes uint32 [K/32][N][words] seen as [K/32][N/U][U*words] so that the innermost
+// extent is a multiple of 16 bytes; box = 4 k-block rows x tile_cols columns
+bool make_codes_map(CUtensorMap* map, const uint32_t* codes, int K, int N, int bits, int tile_cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const int words = words_per_unit(bits), upack = bits == 4 ? 1 : (bits == 2 ? 2 : 4);
+  cuuint64_t dims[3] = {(cuuint64_t)(upack * words), (cuuint64_t)(N / upack), (cuuint64_t)(K / 32)};
+  cuuint64_t strides[2] = {(cuuint64_t)upack * words * 4, (cuuint64_t)N * words * 4};
+  cuuint32_t box[3] = {(cuuint32_t)(upack * words), (cuuint32_t)(tile_cols / upack), 4};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint32_t*>(codes), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// (alpha, beta) float32 [G][2N]; box = 2 * tile_cols floats x rows
+bool make_qp_map(CUtensorMap* map, const float2* qp, int G, int N, int tile_cols, int rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)N * 2, (cuuint64_t)G};
+  cuuint64_t strides[1] = {(cuuint64_t)N * 8};
+  cuuint32_t box[2] = {(cuuint32_t)(2 * tile_cols), (cuuint32_t)rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float2*>(qp), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BITS, int MODE>
 int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
-  CUtensorMap out;
-  if (!make_out_map(&out, p.out, p.M, p.ld_out)) return QALORA_ERR_CUDA;
   using S = Smem<BITS, MODE>;
+  CUtensorMap out, cmap, qmap;
+  if (!make_out_map(&out, p.out, p.M, p.ld_out)) return QALORA_ERR_CUDA;
+  if (!make_codes_map(&cmap, p.codes, p.K, p.N, BITS, S::TILE_NC)) return QALORA_ERR_CUDA;
+  if (!make_qp_map(&qmap, p.qparams, p.K / p.g, p.N, S::TILE_NC, p.qp_rows)) return QALORA_ERR_CUDA;
   static_assert(S::TOTAL <= 232448, "shared memory budget");
   auto kern = qalora_tc_kernel<BITS, MODE>;
   static std::once_flag once;
@@ -516,7 +545,7 @@ int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p
   const int grid = tiles < sm_count() ? tiles : sm_count();
   {
     MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
-    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, out, p);
+    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, out, cmap, qmap, p);
   }
   count_launch();
   return cuda_status(cudaGetLastError());
@@ -524,11 +553,13 @@ int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p
 
 }  // namespace
 
+static bool tc_group_ok(int g) { return g == 32 || g == 64 || g == 128; }
+
 bool tc_forward_supported(const Shape& sh, int64_t M) {
-  return sh.N % TILE_C == 0 && sh.K % TILE_J == 0 && M >= 1 && M <= 0x7fffffffLL / 2 && encode_fn() != nullptr;
+  return tc_group_ok(sh.g) && sh.N % TILE_C == 0 && sh.K % (2 * TILE_J) == 0 && M >= 1 && M <= 0x7fffffffLL / 2 && encode_fn() != nullptr;
 }
 bool tc_dx_supported(const Shape& sh, int64_t M) {
-  return sh.K % TILE_C == 0 && sh.N % TILE_J == 0 && M >= 1 && M <= 0x7fffffffLL / 2 && encode_fn() != nullptr;
+  return tc_group_ok(sh.g) && sh.K % TILE_C == 0 && sh.N % TILE_J == 0 && M >= 1 && M <= 0x7fffffffLL / 2 && encode_fn() != nullptr;
 }
 
 // y = x * W~ + Tb * B with Tb = bf16(s * pool(x) * A) precomputed ([M][r]).
@@ -544,7 +575,7 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
   p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.N;
   p.c_tiles = sh.N / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
   p.red_iters = sh.K / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
-  p.status = status;
+  p.status = status; p.qp_rows = 128 / sh.g;
   if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, p, st);
   return launch_tc<2, FWD>(act, lora, p, st);
@@ -563,7 +594,7 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
   p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.K;
   p.c_tiles = sh.K / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
   p.red_iters = sh.N / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
-  p.status = status;
+  p.status = status; p.qp_rows = 128 / sh.g;
   if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);
   return launch_tc<2, DX>(act, lora, p, st);
