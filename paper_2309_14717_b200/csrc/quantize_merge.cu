@@ -97,6 +97,7 @@ merge_kernel(const float2* __restrict__ qin, const __nv_bfloat16* __restrict__ A
   __syncthreads();
   if (n >= N) return;
   float acc = 0.0f;
+#pragma unroll 16                                   // keep 16 loads of B in flight
   for (int i = 0; i < r; ++i) acc = fmaf(a_row[i], bf16_to_float(B[(size_t)i * N + n]), acc);
   float2 p = qin[(size_t)q * N + n];
   p.y = fmaf(s, acc, p.y);

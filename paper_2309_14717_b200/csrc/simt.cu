@@ -50,11 +50,95 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
   }
 }
 
+// Streaming version for many rows and a group size of 32, 64 or 128: eight rows
+// per block, one warp per row.  A lane reads 16 bytes (8 channels) per step, so
+// g / 8 neighbouring lanes hold one group and a few shuffles finish its sum.
+// Then every thread accumulates four rows of T against one column of A, reading
+// each element of A once per block.
+constexpr int POOL8_ROWS = 8;
+
+template <int LANES_PER_GROUP>   // g / 8: 4, 8 or 16
+__global__ void __launch_bounds__(POOL8_ROWS * 32)
+pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
+                   float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
+                   long long M, int K, int G, int r, float s) {
+  extern __shared__ float xps[];                        // [8][G]
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const long long m = (long long)blockIdx.x * POOL8_ROWS + warp;
+  if (m < M) {
+    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)m * K);
+    const int chunks = K / 8;                             // K is a multiple of 32
+    constexpr int BATCH = 8;                              // loads in flight per lane
+    for (int c0 = 0; c0 < chunks; c0 += 32 * BATCH) {     // chunks is a multiple of 32 (K % 256 == 0)
+      uint4 v[BATCH];
+#pragma unroll
+      for (int b = 0; b < BATCH; ++b) {
+        const int c = c0 + b * 32 + lane;
+        v[b] = c < chunks ? xr[c] : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int b = 0; b < BATCH; ++b) {
+        const int c = c0 + b * 32 + lane;
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v[b]);
+        float acc = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __bfloat1622float2(h[i]);
+          acc += f.x + f.y;
+        }
+#pragma unroll
+        for (int o = 1; o < LANES_PER_GROUP; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (c < chunks && (lane % LANES_PER_GROUP) == 0) {
+          const int q = c / LANES_PER_GROUP;
+          xps[warp * G + q] = acc;
+          if (xp_out != nullptr) xp_out[(size_t)m * G + q] = acc;
+        }
+      }
+    }
+  } else {
+    for (int q = lane; q < G; q += 32) xps[warp * G + q] = 0.0f;
+  }
+  __syncthreads();
+  // T: thread -> column i, four rows
+  for (int o = threadIdx.x; o < 2 * r; o += POOL8_ROWS * 32) {
+    const int i = o % r, rg = o / r;                      // rows 4 rg .. 4 rg + 3
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    const float* xr = xps + rg * 4 * G;
+#pragma unroll 8
+    for (int q = 0; q < G; ++q) {
+      const float av = bf16_to_float(A[(size_t)q * r + i]);
+      a0 = fmaf(xr[q], av, a0);
+      a1 = fmaf(xr[G + q], av, a1);
+      a2 = fmaf(xr[2 * G + q], av, a2);
+      a3 = fmaf(xr[3 * G + q], av, a3);
+    }
+    const float acc[4] = {a0 * s, a1 * s, a2 * s, a3 * s};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const long long mm = (long long)blockIdx.x * POOL8_ROWS + rg * 4 + j;
+      if (mm < M) {
+        T[(size_t)mm * r + i] = acc[j];
+        if (Tb != nullptr) Tb[(size_t)mm * r + i] = __float2bfloat16_rn(acc[j]);
+      }
+    }
+  }
+}
+
 int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv_bfloat16* A,
                   float* xp, float* T, __nv_bfloat16* Tb, cudaStream_t st) {
   if (M == 0) return QALORA_OK;
-  pool_T_kernel<<<(unsigned)M, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G,
-                                                                        sh.r, sh.s);
+  const bool rows_path = M >= 64 && (sh.g == 32 || sh.g == 64 || sh.g == 128) && sh.K % 256 == 0 &&
+                         (size_t)POOL8_ROWS * sh.G * sizeof(float) <= 48 * 1024;
+  if (rows_path) {
+    const unsigned grid = (unsigned)((M + POOL8_ROWS - 1) / POOL8_ROWS);
+    const size_t smem = (size_t)POOL8_ROWS * sh.G * sizeof(float);
+    if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
+    else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
+    else pool_T_rows_kernel<16><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
+  } else {
+    pool_T_kernel<<<(unsigned)M, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G,
+                                                                          sh.r, sh.s);
+  }
   count_launch();
   return cuda_status(cudaGetLastError());
 }
