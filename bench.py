@@ -72,7 +72,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -217,8 +217,10 @@ def run_gpu(args):
     shapes = [ShapeState(n, rank, Q, torch) for n in SHAPES]
     stream = torch.cuda.current_stream()
 
-    def device_step(s):
+    def device_step(s, probe=None):
         Q.qalora_quantize(s.d, s.W, s.codes, s.qparams)
+        if probe is not None:                      # events around the forward contraction kernel of this call
+            Q.qalora_profile_next_main_kernel(*probe)
         Q.qalora_forward(s.d, s.cfg.tokens, s.x, s.codes, s.qparams, s.A, s.B, s.y, s.ws_f)
         Q.qalora_backward(s.d, s.cfg.tokens, s.x, s.dy, s.codes, s.qparams, s.A, s.B, s.dx, s.dA, s.dB, s.ws_b)
         if world > 1:
@@ -227,9 +229,11 @@ def run_gpu(args):
         Q.qalora_merge(s.d, s.qparams, s.A, s.B, s.qmerged)
         Q.qalora_forward(s.d0, 1, s.x1, s.codes, s.qmerged, None, None, s.y1, s.ws1)
 
+    probes = []                                     # one event pair per timed step (first shape's forward kernel)
+
     def step():
-        for s in shapes:
-            device_step(s)
+        for j, s in enumerate(shapes):
+            device_step(s, probes.pop() if (j == 0 and probes) else None)
 
     def e2e_step():
         for s in shapes:
@@ -269,30 +273,34 @@ def run_gpu(args):
 
     uuid = str(torch.cuda.get_device_properties(local).uuid)
     uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    probe_pairs = []
+    for _ in range(args.steps):
+        ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ka.record(stream); kb.record(stream)        # creates the underlying CUDA events
+        probe_pairs.append((ka, kb))
+    probes.extend(probe_pairs)
+    torch.cuda.synchronize()
     launches0 = Q.qalora_kernel_launches()
     ms_total, clocks = timed(step, args.steps, ClockSampler(uuid))
+    s0_ = shapes[0]
+    Q.qalora_forward(s0_.d, s0_.cfg.tokens, s0_.x, s0_.codes, s0_.qparams, s0_.A, s0_.B, s0_.y, s0_.ws_f)
+    kernel_name = Q.qalora_main_kernel_name()       # which kernel the library picks for this shape
+    torch.cuda.synchronize()
     launches = (Q.qalora_kernel_launches() - launches0) // max(1, args.steps)
     ms_step = ms_total / args.steps
     flops_step = sum(s.flops for s in shapes) * world
     value = flops_step / (ms_step / 1e3) / 1e12
 
-    # dominant kernel (the forward contraction of the first shape), timed live with
-    # events recorded by the library around that one launch, on the launching stream
+    # dominant kernel: the forward contraction of the first shape, timed live inside the
+    # timed region with events the library records around that one launch on the launch stream
     s0 = shapes[0]
-    ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ka.record(stream); kb.record(stream)            # creates the underlying CUDA events
-    kernel_ms = []
-    for _ in range(max(3, min(args.steps, 10))):
-        Q.qalora_profile_next_main_kernel(ka, kb)
-        Q.qalora_forward(s0.d, s0.cfg.tokens, s0.x, s0.codes, s0.qparams, s0.A, s0.B, s0.y, s0.ws_f)
-        torch.cuda.synchronize()
-        kernel_ms.append(ka.elapsed_time(kb))
-    kms = sum(kernel_ms) / len(kernel_ms)
+    kms = sum(a.elapsed_time(b) for a, b in probe_pairs) / len(probe_pairs)
     pk = peaks()
     achieved = s0.main_flops / (kms / 1e3) / 1e12
-    roofline = {"bound": "tensor", "kernel": Q.qalora_main_kernel_name(), "achieved": achieved, "peak": pk["tensor"],
+    roofline = {"bound": "tensor", "kernel": kernel_name, "achieved": achieved, "peak": pk["tensor"],
                 "unit": "TFLOP/s", "frac": achieved / pk["tensor"], "peak_source": pk["source"] + " (sustained bf16)",
-                "kernel_ms": kms, "traffic": None}
+                "kernel_ms": kms, "launches_timed": len(probe_pairs), "traffic": None,
+                "flops_per_launch": s0.main_flops}
 
     # single-token forward of the merged layer: HBM-bound leg of the metric
     small = small_m_bandwidth(Q, torch, pk)
@@ -430,8 +438,8 @@ def main():
     ap.add_argument("--shape", default="cfg3_7b_up")
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     args = ap.parse_args()
     if args.only is not None:

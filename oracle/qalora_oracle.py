@@ -38,7 +38,7 @@ import numpy as np
 
 __all__ = [
     "levels", "quantize", "quantize_fp64_shadow", "dequantize", "pool",
-    "forward", "backward", "merge", "merge_zero_point", "words_per_unit",
+    "forward", "backward", "backward_adapter", "merge", "merge_zero_point", "words_per_unit",
     "pack", "unpack", "adapter_param_count",
 ]
 
@@ -136,6 +136,22 @@ def forward(x, codes, alpha, beta, g, A=None, B=None, s=0.0) -> np.ndarray:
     return y
 
 
+def backward_adapter(x, dy, g, A, B, s):
+    """The adapter gradients alone (they do not involve W):
+        dT = s * dy @ B^T;  dA = pool(x)^T @ dT;  dB = s * (pool(x) @ A)^T @ dy.
+    Both are sums over token rows, so row blocks can be processed separately and added."""
+    x = np.asarray(x, dtype=np.float64)
+    dy = np.asarray(dy, dtype=np.float64)
+    A = np.asarray(A, dtype=np.float64)
+    B = np.asarray(B, dtype=np.float64)
+    s = float(s)
+    xp = pool(x, g)
+    dT = s * (dy @ B.T)
+    dA = xp.T @ dT
+    dB = s * ((xp @ A).T @ dy)
+    return dA, dB
+
+
 def backward(x, dy, codes, alpha, beta, g, A, B, s):
     """Gradients of l = sum(dy * y) with the base weights frozen (Section 3.1).
 
@@ -151,12 +167,10 @@ def backward(x, dy, codes, alpha, beta, g, A, B, s):
     A = np.asarray(A, dtype=np.float64)
     B = np.asarray(B, dtype=np.float64)
     s = float(s)
-    xp = pool(x, g)
     dT = s * (dy @ B.T)
     dXp = dT @ A.T                                        # [M, G]
     dX = dy @ dequantize(codes, alpha, beta, g).T + np.repeat(dXp, g, axis=1)
-    dA = xp.T @ dT
-    dB = s * ((xp @ A).T @ dy)
+    dA, dB = backward_adapter(x, dy, g, A, B, s)
     return dX, dA, dB
 
 
