@@ -199,6 +199,7 @@ def run_gpu(args):
 
     from paper_2309_14717_b200 import binding as Q
     from paper_2309_14717_b200 import build as _build
+    from paper_2309_14717_b200 import dp
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -224,8 +225,7 @@ def run_gpu(args):
         Q.qalora_forward(s.d, s.cfg.tokens, s.x, s.codes, s.qparams, s.A, s.B, s.y, s.ws_f)
         Q.qalora_backward(s.d, s.cfg.tokens, s.x, s.dy, s.codes, s.qparams, s.A, s.B, s.dx, s.dA, s.dB, s.ws_b)
         if world > 1:
-            dist.all_reduce(s.dA)
-            dist.all_reduce(s.dB)
+            dp.allreduce_adapter_grads(s.dA, s.dB)
         Q.qalora_merge(s.d, s.qparams, s.A, s.B, s.qmerged)
         Q.qalora_forward(s.d0, 1, s.x1, s.codes, s.qmerged, None, None, s.y1, s.ws1)
 

@@ -31,7 +31,8 @@ CASES = [
     ("cfg4_13b_down", {"bits": 2}),
     ("cfg4_13b_attn", {"bits": 2}),
     ("cfg5_65b_attn", {"group_size": 64}),
-    ("cfg5_65b_down", {"group_size": 128, "tokens": 2048}),
+    ("cfg5_65b_down", {"group_size": 128}),
+    ("cfg5_65b_up", {}),
 ]
 
 
