@@ -189,6 +189,7 @@ class ShapeState:
                          "dx": torch.empty((M, K), dtype=torch.bfloat16).pin_memory(),
                          "dA": torch.empty((G, r), dtype=torch.float32).pin_memory(),
                          "dB": torch.empty((r, N), dtype=torch.float32).pin_memory()}
+        self.staging = torch.zeros(Q.qalora_step_host_bytes(self.d, M), dtype=torch.uint8, device="cuda")
         self.flops = fwd_flops(M, K, N, G, r) + bwd_flops(M, K, N, G, r)
         self.main_flops = 2 * M * K * N
 
@@ -236,14 +237,15 @@ def run_gpu(args):
             device_step(s, probes.pop() if (j == 0 and probes) else None)
 
     def e2e_step():
+        # the same step through the C ABI with HOST buffers: x, dy go up and y, dx, dA, dB
+        # come back inside qalora_step_host; quantize, merge and the merged one-token
+        # forward work on resident weights as in the device-resident step
         for s in shapes:
-            s.x.copy_(s.host["x"], non_blocking=True)
-            s.dy.copy_(s.host["dy"], non_blocking=True)
-            device_step(s)
-            s.host_out["y"].copy_(s.y, non_blocking=True)
-            s.host_out["dx"].copy_(s.dx, non_blocking=True)
-            s.host_out["dA"].copy_(s.dA, non_blocking=True)
-            s.host_out["dB"].copy_(s.dB, non_blocking=True)
+            Q.qalora_quantize(s.d, s.W, s.codes, s.qparams)
+            Q.qalora_step_host(s.d, s.cfg.tokens, s.host["x"], s.host["dy"], s.codes, s.qparams, s.A, s.B,
+                               s.host_out["y"], s.host_out["dx"], s.host_out["dA"], s.host_out["dB"], s.staging)
+            Q.qalora_merge(s.d, s.qparams, s.A, s.B, s.qmerged)
+            Q.qalora_forward(s.d0, 1, s.x1, s.codes, s.qmerged, None, None, s.y1, s.ws1)
 
     def timed(fn, steps, sampler=None):
         if world > 1:

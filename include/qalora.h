@@ -140,6 +140,24 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
 int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A, const void* B,
                  float* qparams_out, void* cuda_stream);
 
+/* One fine-tuning step of the layer driven from HOST buffers: copies x and dy to
+ * the device, runs qalora_forward and qalora_backward (Algorithm 1 and its
+ * gradients, as above), and copies y, dx, dA and dB back, all enqueued on
+ * `cuda_stream` (the call returns without synchronizing; the host outputs are
+ * valid once the stream has been synchronized).
+ *   x_host, dy_host   in : HOST memory (pinned for asynchronous copies), bf16 [m][K], [m][N]
+ *   codes, qparams, A, B : DEVICE memory, as for qalora_forward
+ *   y_host, dx_host   out: HOST bf16 [m][N], [m][K];  dA_host, dB_host out: HOST float32
+ *   staging              : DEVICE scratch of qalora_step_host_bytes() bytes (device copies
+ *                          of the inputs and outputs plus the workspaces); its first
+ *                          int32 is the status word described at qalora_workspace_bytes
+ * rank must be > 0. */
+int qalora_step_host_bytes(const qalora_desc* desc, int64_t m, size_t* bytes);
+int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, const void* dy_host,
+                     const void* codes, const float* qparams, const void* A, const void* B,
+                     void* y_host, void* dx_host, float* dA_host, float* dB_host,
+                     void* staging, size_t staging_bytes, void* cuda_stream);
+
 /* Forward pass for callers that cannot allocate device memory (the paper has no
  * counterpart; this is a convenience of the library).  Some hosts of this code
  * may not call cudaMalloc at all: a plugin running inside an engine that owns

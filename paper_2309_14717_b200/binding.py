@@ -20,7 +20,7 @@ EXPORTS = (
     "qalora_version", "qalora_status_string", "qalora_packed_bytes", "qalora_workspace_bytes",
     "qalora_quantize", "qalora_forward", "qalora_backward", "qalora_merge",
     "qalora_kernel_launches", "qalora_profile_next_main_kernel", "qalora_main_kernel_name",
-    "qalora_forward_static",
+    "qalora_forward_static", "qalora_step_host_bytes", "qalora_step_host",
 )
 
 STATIC_SCRATCH_BYTES = 1 << 20
@@ -68,6 +68,10 @@ def load() -> ctypes.CDLL:
     lib.qalora_merge.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.qalora_forward_static.restype = c_int
     lib.qalora_forward_static.argtypes = [D, c_int64] + [c_void_p] * 6 + [c_void_p]
+    lib.qalora_step_host_bytes.restype = c_int
+    lib.qalora_step_host_bytes.argtypes = [D, c_int64, POINTER(c_size_t)]
+    lib.qalora_step_host.restype = c_int
+    lib.qalora_step_host.argtypes = [D, c_int64] + [c_void_p] * 10 + [c_void_p, c_size_t, c_void_p]
     lib.qalora_kernel_launches.restype = ctypes.c_uint64
     lib.qalora_kernel_launches.argtypes = []
     lib.qalora_profile_next_main_kernel.restype = c_int
@@ -160,6 +164,28 @@ def qalora_forward_static(d: QaloraDesc, m: int, x, codes, qparams, A, B, y, str
     Calls that overlap on the GPU share the array and must be serialized."""
     _check("qalora_forward_static", load().qalora_forward_static(byref(d), m, _ptr(x), _ptr(codes), _ptr(qparams),
                                                                  _ptr(A), _ptr(B), _ptr(y), _stream(stream)))
+
+
+def qalora_step_host_bytes(d: QaloraDesc, m: int) -> int:
+    b = c_size_t()
+    _check("qalora_step_host_bytes", load().qalora_step_host_bytes(byref(d), m, byref(b)))
+    return b.value
+
+
+def _hptr(t):
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError("host tensors must be contiguous CPU tensors")
+    return c_void_p(t.data_ptr())
+
+
+def qalora_step_host(d: QaloraDesc, m: int, x_host, dy_host, codes, qparams, A, B, y_host, dx_host, dA_host, dB_host,
+                     staging, stream=None):
+    """Forward + backward from (pinned) host tensors; outputs land in host tensors
+    once the stream is synchronized."""
+    _check("qalora_step_host", load().qalora_step_host(byref(d), m, _hptr(x_host), _hptr(dy_host), _ptr(codes),
+                                                       _ptr(qparams), _ptr(A), _ptr(B), _hptr(y_host), _hptr(dx_host),
+                                                       _hptr(dA_host), _hptr(dB_host), _ptr(staging), staging.numel(),
+                                                       _stream(stream)))
 
 
 def qalora_backward(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, dB, workspace, stream=None):

@@ -255,4 +255,64 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
   return QALORA_OK;
 }
 
+
+namespace {
+struct StepLayout { size_t ws, x, dy, y, dx, dA, dB, total, ws_bytes; };
+StepLayout step_layout(const Shape& sh, int64_t m) {
+  StepLayout L{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t at = off; off += round_up(bytes, 256); return at; };
+  const size_t M = (size_t)m;
+  const size_t wf = workspace_layout(sh, m, QALORA_OP_FORWARD).total, wb = workspace_layout(sh, m, QALORA_OP_BACKWARD).total;
+  L.ws_bytes = wf > wb ? wf : wb;
+  L.ws = take(L.ws_bytes);                         // first: the status word sits at the head of the staging area
+  L.x = take(M * sh.K * 2); L.dy = take(M * sh.N * 2); L.y = take(M * sh.N * 2); L.dx = take(M * sh.K * 2);
+  L.dA = take((size_t)sh.G * sh.r * 4); L.dB = take((size_t)sh.r * sh.N * 4);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+int qalora_step_host_bytes(const qalora_desc* desc, int64_t m, size_t* bytes) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (bytes == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (m < 0) return QALORA_ERR_INVALID_ARG;
+  *bytes = step_layout(sh, m).total;
+  return QALORA_OK;
+}
+
+int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, const void* dy_host,
+                     const void* codes, const float* qparams, const void* A, const void* B,
+                     void* y_host, void* dx_host, float* dA_host, float* dB_host,
+                     void* staging, size_t staging_bytes, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (m < 0 || sh.r == 0) return QALORA_ERR_INVALID_ARG;
+  if (x_host == nullptr || dy_host == nullptr || y_host == nullptr || dx_host == nullptr || dA_host == nullptr ||
+      dB_host == nullptr || staging == nullptr)
+    return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(staging)) return QALORA_ERR_MISALIGNED;
+  const StepLayout L = step_layout(sh, m);
+  if (staging_bytes < L.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* base = static_cast<char*>(staging);
+  const size_t M = (size_t)m;
+  if (cudaMemcpyAsync(base + L.x, x_host, M * sh.K * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess) return QALORA_ERR_CUDA;
+  if (cudaMemcpyAsync(base + L.dy, dy_host, M * sh.N * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess) return QALORA_ERR_CUDA;
+  st = qalora_forward(desc, m, base + L.x, codes, qparams, A, B, base + L.y, base + L.ws, L.ws_bytes, cuda_stream);
+  if (st != QALORA_OK) return st;
+  st = qalora_backward(desc, m, base + L.x, base + L.dy, codes, qparams, A, B, base + L.dx,
+                       reinterpret_cast<float*>(base + L.dA), reinterpret_cast<float*>(base + L.dB), base + L.ws,
+                       L.ws_bytes, cuda_stream);
+  if (st != QALORA_OK) return st;
+  if (cudaMemcpyAsync(y_host, base + L.y, M * sh.N * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
+  if (cudaMemcpyAsync(dx_host, base + L.dx, M * sh.K * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
+  if (cudaMemcpyAsync(dA_host, base + L.dA, (size_t)sh.G * sh.r * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
+  if (cudaMemcpyAsync(dB_host, base + L.dB, (size_t)sh.r * sh.N * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
+  return QALORA_OK;
+}
+
 }  // extern "C"

@@ -206,3 +206,21 @@ def test_results_do_not_depend_on_scheduling():
     assert torch.equal(y1, y2)
     for a, b in zip(b1, b2):
         assert torch.equal(a, b)
+
+
+def test_step_from_host_buffers_matches_device_calls():
+    cfg = LayerConfig("hoststep", 512, 384, 64, 4, 64, 1.0, 300, seed=21)
+    layer = GpuLayer(cfg)
+    y = layer.forward()
+    dx, dA, dB = layer.backward()
+    pin = lambda t: t.pin_memory()
+    hx, hdy = pin(layer.cpu["x"]), pin(layer.cpu["dy"])
+    hy, hdx = pin(torch.empty_like(y, device="cpu")), pin(torch.empty_like(dx, device="cpu"))
+    hdA, hdB = pin(torch.empty_like(dA, device="cpu")), pin(torch.empty_like(dB, device="cpu"))
+    staging = torch.zeros(Q.qalora_step_host_bytes(layer.d, cfg.tokens), dtype=torch.uint8, device="cuda")
+    Q.qalora_step_host(layer.d, cfg.tokens, hx, hdy, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"],
+                       hy, hdx, hdA, hdB, staging)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(staging) == 0
+    assert torch.equal(hy, y.cpu()) and torch.equal(hdx, dx.cpu())
+    assert torch.equal(hdA, dA.cpu()) and torch.equal(hdB, dB.cpu())
