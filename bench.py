@@ -416,8 +416,12 @@ def run_only(args):
     dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
     wf, wb = Q.alloc_workspace(d, M, Q.OP_FORWARD), Q.alloc_workspace(d, M, Q.OP_BACKWARD)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    times = []
+    times, ktimes = [], []
+    ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ka.record(); kb.record()
     for _ in range(args.steps + 2):
+        if args.only in ("fwd", "gemv", "bwd"):
+            Q.qalora_profile_next_main_kernel(ka, kb)
         e0.record()
         if args.only in ("fwd", "gemv"):
             Q.qalora_forward(d, M, t["x"], codes, qparams, t["A"], t["B"], y, wf)
@@ -430,7 +434,10 @@ def run_only(args):
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
+        if args.only in ("fwd", "gemv", "bwd"):
+            ktimes.append(ka.elapsed_time(kb))
     print(json.dumps({"only": args.only, "shape": args.shape, "tokens": M, "ms": times[2:],
+                      "main_kernel": Q.qalora_main_kernel_name(), "main_kernel_ms": ktimes[2:],
                       "status": Q.workspace_status(wb if args.only == "bwd" else wf)}))
 
 

@@ -2,13 +2,14 @@
 // codes and the (alpha, beta) pairs from HBM exactly once.
 //
 // Design
-//  * One block owns 128 output columns and a slice of the input channels; the
+//  * One block (eight consumer warps in two sets that take alternate k-blocks, plus
+//    one producer warp) owns 128 output columns and a slice of the input channels; the
 //    slices of one column tile form a thread-block CLUSTER, and the partial sums
 //    are added through distributed shared memory in a fixed order (no atomics,
 //    no second kernel, no scratch).
 //  * A single thread streams codes, qparams and the x slice into a shared-memory
-//    ring with bulk TMA copies (one per contiguous row of pack units), so that
-//    many tens of KiB per SM are in flight without using registers.
+//    ring with three tiled TMA copies per 128-channel stage, so that many tens of
+//    KiB per SM are in flight without using registers.
 //  * The products run on mma.sync.m16n8k16 (bf16 in, fp32 accumulate) with the
 //    tokens as the 16 rows: a lane's 32-bit word of packed codes IS its B
 //    fragment after one shift and one mask per pair (the code is OR-ed into the
@@ -33,7 +34,8 @@ namespace qalora {
 namespace {
 
 constexpr int GV_COLS = 128;        // columns per block
-constexpr int GV_WARPS = 4;         // consumer warps, 32 columns each
+constexpr int GV_SETS = 2;          // consumer warp sets; set s takes the k-blocks b with b % 2 == s
+constexpr int GV_WARPS = 4 * GV_SETS;   // consumer warps: 4 per set, 32 columns each
 constexpr int GV_THREADS = (GV_WARPS + 1) * 32;   // + 1 producer warp
 constexpr int GV_KBS = 4;           // 32-channel blocks per stage (128 channels)
 constexpr int GV_STAGES = 6;
@@ -49,8 +51,8 @@ struct GvSmem {
   static constexpr uint32_t OFF_QP = GV_KBS * CODE_ROW;
   static constexpr uint32_t OFF_X = OFF_QP + GV_KBS * QP_ROW;
   static constexpr uint32_t STAGE_BYTES = ((OFF_X + X_BYTES + 127) / 128) * 128;
-  static constexpr uint32_t OFF_PARTIAL = GV_STAGES * STAGE_BYTES;      // fp32 [16][128]
-  static constexpr uint32_t OFF_BARS = OFF_PARTIAL + GV_ROWS * GV_COLS * 4;
+  static constexpr uint32_t OFF_PARTIAL = GV_STAGES * STAGE_BYTES;      // fp32 [sets][16][128]
+  static constexpr uint32_t OFF_BARS = OFF_PARTIAL + GV_SETS * GV_ROWS * GV_COLS * 4;
   static constexpr uint32_t TOTAL = OFF_BARS + 128 + 128;               // + alignment slack
 };
 
@@ -94,7 +96,8 @@ __device__ __forceinline__ void code_fragments(const uint32_t* unit, int t, uint
 
 template <int BITS, bool UPPER>   // UPPER: token rows 8..15 are in use (M > 8)
 __global__ void __launch_bounds__(GV_THREADS, 2)
-qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const GvParams p) {
+qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
+                   const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
   using S = GvSmem<BITS>;
   constexpr int WORDS = S::WORDS;
   extern __shared__ uint8_t smem_raw[];
@@ -121,6 +124,8 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const GvParams p) 
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&x_map);
+    ptx::prefetch_tensormap(&codes_map);
+    ptx::prefetch_tensormap(&qp_map);
     if (blockIdx.x == 0) *p.status = 0;     // every block is resident from the start; a timeout is seconds away
   }
   __syncthreads();
@@ -133,30 +138,31 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const GvParams p) 
         const int s = it % GV_STAGES;
         if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / GV_STAGES) & 1) ^ 1, abort_flag))) break;
         const uint32_t stage = smem_base + s * S::STAGE_BYTES;
-        ptx::mbar_arrive_expect_tx(bar_full(s), GV_KBS * (S::CODE_ROW + S::QP_ROW) + S::X_BYTES);
-#pragma unroll
-        for (int b = 0; b < GV_KBS; ++b) {
-          const int kb = st * GV_KBS + b;
-          ptx::bulk_load(stage + S::OFF_CODES + b * S::CODE_ROW, p.codes + ((size_t)kb * p.N + n0) * WORDS,
-                         S::CODE_ROW, bar_full(s));
-          ptx::bulk_load(stage + S::OFF_QP + b * S::QP_ROW, p.qparams + (size_t)(kb * 32 / p.g) * p.N + n0,
-                         S::QP_ROW, bar_full(s));
-        }
+        // three tiled copies per stage: 4 k-block rows of pack units, the rows of
+        // (alpha, beta) they need (128 / g of them) and the x slice
+        constexpr int UPACK = BITS == 4 ? 1 : (BITS == 2 ? 2 : 4);
+        const int qrows = (GV_KBS * 32) / p.g;
+        ptx::mbar_arrive_expect_tx(bar_full(s), GV_KBS * S::CODE_ROW + qrows * S::QP_ROW + S::X_BYTES);
+        ptx::tma_load_3d(stage + S::OFF_CODES, &codes_map, 0, n0 / UPACK, st * GV_KBS, bar_full(s));
+        ptx::tma_load_2d(stage + S::OFF_QP, &qp_map, 2 * n0, st * GV_KBS * 32 / p.g, bar_full(s));
         ptx::tma_load_2d(stage + S::OFF_X, &x_map, st * GV_KBS * 32, 0, bar_full(s));
       }
     }
   } else {
     // ----------------------------------------------------------- consumers ----
+    // Warp w of set s owns columns 32 (w % 4) .. + 31 and the k-blocks b of each stage
+    // with b % GV_SETS == s.  Every k-block is folded on its own (the fold is linear, so
+    // the k-blocks of one quantization group may be folded separately with the same
+    // alpha and beta): acc += alpha * D + (beta - 128 alpha) * xp.
+    const int set = warp / 4, wcol = (warp % 4) * 32;
+    const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block of the stage -> its (alpha, beta) row
     const int gq = lane / 4, t = lane % 4;        // fragment row / column group, quad lane
-    const int kb_per_group = p.g / 32;
-    float acc[4][4], D[4][4], Dx[4];
+    float acc[4][4];
     const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c = 0; c < 4; ++c)
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { acc[c][i] = 0.f; D[c][i] = 0.f; }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) Dx[i] = 0.f;
+      for (int i = 0; i < 4; ++i) acc[c][i] = 0.f;
     constexpr uint32_t ONES = 0x3f803f80u;        // bf16x2 (1, 1)
     bool ok = true;
     for (int st = st_beg, it = 0; st < st_end && ok; ++st, ++it) {
@@ -164,63 +170,70 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const GvParams p) 
       if (!(ok = ptx::mbar_wait(bar_full(s), (it / GV_STAGES) & 1, abort_flag))) break;
       const uint8_t* stage = smem + s * S::STAGE_BYTES;
 #pragma unroll
-      for (int b = 0; b < GV_KBS; ++b) {
-        const int kb = st * GV_KBS + b;
+      for (int bb = 0; bb < GV_KBS / GV_SETS; ++bb) {
+        const int b = bb * GV_SETS + set;
         // A fragments: x[row][32 b + 8 t .. + 7] for rows gq and gq + 8
         const uint4 xl = *reinterpret_cast<const uint4*>(stage + S::OFF_X + gq * (GV_KBS * 64) + b * 64 + t * 16);
         uint4 xh = make_uint4(0u, 0u, 0u, 0u);
         if (UPPER) xh = *reinterpret_cast<const uint4*>(stage + S::OFF_X + (gq + 8) * (GV_KBS * 64) + b * 64 + t * 16);
         const uint32_t a0[4] = {xl.x, xh.x, xl.y, xh.y};     // slots (2t,2t+1) | (2t+8,2t+9) of MMA 0
         const uint32_t a1[4] = {xl.z, xh.z, xl.w, xh.w};     // the same slots of MMA 1
-        const bool first = (kb % kb_per_group) == 0, last = (kb % kb_per_group) == kb_per_group - 1;
-        mma16816(Dx, a0, ONES, ONES, first ? zero4 : Dx);
+        float Dx[4];
+        mma16816(Dx, a0, ONES, ONES, zero4);
         mma16816(Dx, a1, ONES, ONES, Dx);
+        const uint8_t* crow = stage + S::OFF_CODES + b * S::CODE_ROW;
+        const uint8_t* qrow = stage + S::OFF_QP + (b >> qsh) * S::QP_ROW;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const int col = warp * 32 + c * 8;
-          const uint32_t* unit = reinterpret_cast<const uint32_t*>(stage + S::OFF_CODES + b * S::CODE_ROW) + (col + gq) * WORDS;
+          const int col = wcol + c * 8;
           uint32_t f[4];
-          code_fragments<BITS>(unit, t, f);
-          mma16816(D[c], a0, f[0], f[1], first ? zero4 : D[c]);
-          mma16816(D[c], a1, f[2], f[3], D[c]);
-          if (last) {
-            // accumulator columns of this lane are col + 2t and col + 2t + 1
-            const float4 q = *reinterpret_cast<const float4*>(stage + S::OFF_QP + b * S::QP_ROW + (col + 2 * t) * 8);
-            const float bias0 = fmaf(-128.f, q.x, q.y), bias1 = fmaf(-128.f, q.z, q.w);
-            acc[c][0] = fmaf(q.x, D[c][0], fmaf(bias0, Dx[0], acc[c][0]));
-            acc[c][1] = fmaf(q.z, D[c][1], fmaf(bias1, Dx[1], acc[c][1]));
-            if (UPPER) {
-              acc[c][2] = fmaf(q.x, D[c][2], fmaf(bias0, Dx[2], acc[c][2]));
-              acc[c][3] = fmaf(q.z, D[c][3], fmaf(bias1, Dx[3], acc[c][3]));
-            }
+          code_fragments<BITS>(reinterpret_cast<const uint32_t*>(crow) + (col + gq) * WORDS, t, f);
+          float D[4];
+          mma16816(D, a0, f[0], f[1], zero4);
+          mma16816(D, a1, f[2], f[3], D);
+          // accumulator columns of this lane are col + 2t and col + 2t + 1
+          const float4 q = *reinterpret_cast<const float4*>(qrow + (col + 2 * t) * 8);
+          const float bias0 = fmaf(-128.f, q.x, q.y), bias1 = fmaf(-128.f, q.z, q.w);
+          acc[c][0] = fmaf(q.x, D[0], fmaf(bias0, Dx[0], acc[c][0]));
+          acc[c][1] = fmaf(q.z, D[1], fmaf(bias1, Dx[1], acc[c][1]));
+          if (UPPER) {
+            acc[c][2] = fmaf(q.x, D[2], fmaf(bias0, Dx[2], acc[c][2]));
+            acc[c][3] = fmaf(q.z, D[3], fmaf(bias1, Dx[3], acc[c][3]));
           }
         }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar_empty(s));
     }
-    // partial sums of this block: [16 rows][128 columns]
+    // partial sums of this warp set: [16 rows][128 columns]
+    float* mine = partial + set * (GV_ROWS * GV_COLS);
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-      const int col = warp * 32 + c * 8 + 2 * t;
-      *reinterpret_cast<float2*>(partial + gq * GV_COLS + col) = make_float2(acc[c][0], acc[c][1]);
-      *reinterpret_cast<float2*>(partial + (gq + 8) * GV_COLS + col) = make_float2(acc[c][2], acc[c][3]);
+      const int col = wcol + c * 8 + 2 * t;
+      *reinterpret_cast<float2*>(mine + gq * GV_COLS + col) = make_float2(acc[c][0], acc[c][1]);
+      *reinterpret_cast<float2*>(mine + (gq + 8) * GV_COLS + col) = make_float2(acc[c][2], acc[c][3]);
     }
   }
 
   // ---- add the slices in rank order through distributed shared memory ---------
   cluster.sync();
   {
-    const int cols_per = GV_COLS / splits;                 // splits is 1, 2, 4 or 8
+    const int col_beg = GV_COLS * rank / splits, col_end = GV_COLS * (rank + 1) / splits;
+    const int cols_per = col_end - col_beg;
     const int outs = p.M * cols_per;
     for (int o = threadIdx.x; o < outs; o += GV_THREADS) {
-      const int row = o / cols_per, col = rank * cols_per + o % cols_per;
+      const int row = o / cols_per, col = col_beg + o % cols_per;
       float v = 0.f;
-      for (int rk = 0; rk < splits; ++rk) v += cluster.map_shared_rank(partial, rk)[row * GV_COLS + col];
+      for (int rk = 0; rk < splits; ++rk) {
+        const float* remote = cluster.map_shared_rank(partial, rk);
+#pragma unroll
+        for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (GV_ROWS * GV_COLS) + row * GV_COLS + col];
+      }
       if (p.r > 0) {
         const float* Tr = p.T + (size_t)row * p.r;
         const __nv_bfloat16* Bc = p.B + n0 + col;
         float a = 0.f;
+#pragma unroll 8
         for (int i = 0; i < p.r; ++i) a = fmaf(Tr[i], __bfloat162float(Bc[(size_t)i * p.N]), a);
         v += a;
       }
@@ -260,6 +273,30 @@ int gv_sm_count() {
 
 template <int BITS, bool UPPER>
 int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
+  EncodeTiledFn fn = gv_encode_fn();
+  CUtensorMap cm, qm;
+  {
+    // packed codes uint32 [K/32][N][words] seen as [K/32][N/U][U*words] (innermost extent a
+    // multiple of 16 bytes); box = 4 k-block rows x 128 columns
+    constexpr int W = GvSmem<BITS>::WORDS, U = BITS == 4 ? 1 : (BITS == 2 ? 2 : 4);
+    cuuint64_t dims[3] = {(cuuint64_t)(U * W), (cuuint64_t)(p.N / U), (cuuint64_t)(p.K / 32)};
+    cuuint64_t strides[2] = {(cuuint64_t)U * W * 4, (cuuint64_t)p.N * W * 4};
+    cuuint32_t box[3] = {(cuuint32_t)(U * W), (cuuint32_t)(GV_COLS / U), GV_KBS};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (fn(&cm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint32_t*>(p.codes), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return QALORA_ERR_CUDA;
+    // (alpha, beta) float32 [G][2N]; box = 256 floats x (128 / g) rows
+    cuuint64_t qdims[2] = {(cuuint64_t)p.N * 2, (cuuint64_t)(p.K / p.g)};
+    cuuint64_t qstrides[1] = {(cuuint64_t)p.N * 8};
+    cuuint32_t qbox[2] = {2 * GV_COLS, (cuuint32_t)((GV_KBS * 32) / p.g)};
+    cuuint32_t qestr[2] = {1, 1};
+    if (fn(&qm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float2*>(p.qparams), qdims, qstrides, qbox, qestr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return QALORA_ERR_CUDA;
+  }
   using S = GvSmem<BITS>;
   auto kern = qalora_gemv_kernel<BITS, UPPER>;
   static std::once_flag once;
@@ -281,7 +318,7 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   cudaError_t e;
   {
     MainKernelProbe probe("qalora_gemv_kernel", st);
-    e = cudaLaunchKernelEx(&cfg, kern, xm, p);
+    e = cudaLaunchKernelEx(&cfg, kern, xm, cm, qm, p);
   }
   count_launch();
   return cuda_status(e);
@@ -290,7 +327,8 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
 }  // namespace
 
 bool gemv_supported(const Shape& sh, int64_t M) {
-  return M >= 1 && M <= GV_ROWS && sh.N % GV_COLS == 0 && sh.K % (GV_KBS * 32) == 0 && (GV_KBS * 32) % sh.g == 0 &&
+  return M >= 1 && M <= GV_ROWS && sh.N % GV_COLS == 0 && sh.K % (GV_KBS * 32) == 0 &&
+         (sh.g == 32 || sh.g == 64 || sh.g == 128) &&
          gv_encode_fn() != nullptr;
 }
 
@@ -312,10 +350,16 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;
-  // slices per column tile: enough blocks for two per SM, at most 8 (portable cluster size)
-  const int tiles = sh.N / GV_COLS;
+  // slices per column tile (= cluster size, at most 8): the count whose blocks fill whole
+  // waves of two resident blocks per SM best; ties go to fewer slices
+  const int tiles = sh.N / GV_COLS, capacity = 2 * gv_sm_count();
   int splits = 1;
-  while (splits < 8 && tiles * splits < 2 * gv_sm_count() && splits * 2 <= p.total_stages) splits *= 2;
+  double best = 0.0;
+  for (int sp = 1; sp <= 8 && sp <= p.total_stages; ++sp) {
+    const int blocks = tiles * sp, waves = (blocks + capacity - 1) / capacity;
+    const double eff = (double)blocks / ((double)waves * capacity);
+    if (eff > best + 0.02) { best = eff; splits = sp; }
+  }
   const bool upper = M > 8;
 #define QALORA_GV(BITS) (upper ? launch_gemv_t<BITS, true>(xm, p, splits, st) : launch_gemv_t<BITS, false>(xm, p, splits, st))
   if (sh.bits == 4) return QALORA_GV(4);
