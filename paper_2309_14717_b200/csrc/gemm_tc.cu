@@ -233,7 +233,6 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   } else if (warp == 2) {
     // ------------------------------------------------------- code producer ----
     if (lane == 0) {
-      constexpr int UPACK = BITS == 4 ? 1 : (BITS == 2 ? 2 : 4);   // units per 16-byte-aligned map element row
       uint32_t cit = 0;                              // code stages issued so far
       bool ok = true;
       const int stages_per_tile = p.red_iters / S::IPS;
@@ -247,7 +246,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           const int kb0 = MODE == FWD ? cs * 4 : c0 / 32;
           const int col0 = MODE == FWD ? c0 : cs * TILE_J;
           ptx::mbar_arrive_expect_tx(bar_full_c(s), S::CODE_BYTES + p.qp_rows * S::QP_ROW_BYTES);
-          ptx::tma_load_3d(stage, &codes_map, 0, col0 / UPACK, kb0, bar_full_c(s));
+          ptx::tma_load_2d(stage, &codes_map, col0 * WORDS / 2, kb0, bar_full_c(s));
           ptx::tma_load_2d(stage + S::CODE_BYTES, &qp_map, 2 * col0, kb0 * 32 / p.g, bar_full_c(s));
         }
       }
@@ -501,17 +500,17 @@ bool make_out_map(CUtensorMap* map, void* base, long long rows, int cols) {
             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// packed codes uint32 [K/32][N][words] seen as [K/32][N/U][U*words] so that the innermost
-// extent is a multiple of 16 bytes; box = 4 k-block rows x tile_cols columns
+// packed codes [K/32][N][words] uint32 seen as a 2-D matrix of 8-byte elements, so that one
+// box row is the whole contiguous run of tile_cols pack units; box = 4 k-block rows
 bool make_codes_map(CUtensorMap* map, const uint32_t* codes, int K, int N, int bits, int tile_cols) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
-  const int words = words_per_unit(bits), upack = bits == 4 ? 1 : (bits == 2 ? 2 : 4);
-  cuuint64_t dims[3] = {(cuuint64_t)(upack * words), (cuuint64_t)(N / upack), (cuuint64_t)(K / 32)};
-  cuuint64_t strides[2] = {(cuuint64_t)upack * words * 4, (cuuint64_t)N * words * 4};
-  cuuint32_t box[3] = {(cuuint32_t)(upack * words), (cuuint32_t)(tile_cols / upack), 4};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint32_t*>(codes), dims, strides, box, estr,
+  const int words = words_per_unit(bits);
+  cuuint64_t dims[2] = {(cuuint64_t)N * words / 2, (cuuint64_t)(K / 32)};
+  cuuint64_t strides[1] = {(cuuint64_t)N * words * 4};
+  cuuint32_t box[2] = {(cuuint32_t)(tile_cols * words / 2), 4};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<uint32_t*>(codes), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -75,22 +75,21 @@ __device__ __forceinline__ void mma16816(float* d, const uint32_t* a, uint32_t b
 }
 
 // The four bf16x2 fragments (128 + c) of the 8 positions 8t .. 8t+7 of a unit, t = lane % 4.
+// `lo` is the word that holds the (low) code bits of those positions, already shifted so
+// that they start at bit 0 of each half-word; `hi` (3-bit codes only) the third-bit word
+// shifted likewise.
 template <int BITS>
-__device__ __forceinline__ void code_fragments(const uint32_t* unit, int t, uint32_t* f) {
+__device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, uint32_t* f) {
   constexpr uint32_t MAGIC = 0x43004300u;
   if (BITS == 4) {
-    const uint32_t w = unit[t];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) f[i] = ((w >> (4 * i)) & 0x000f000fu) | MAGIC;
+    for (int i = 0; i < 4; ++i) f[i] = ((lo >> (4 * i)) & 0x000f000fu) | MAGIC;
   } else if (BITS == 2) {
-    const uint32_t w = unit[t >> 1] >> (8 * (t & 1));
 #pragma unroll
-    for (int i = 0; i < 4; ++i) f[i] = ((w >> (2 * i)) & 0x00030003u) | MAGIC;
+    for (int i = 0; i < 4; ++i) f[i] = ((lo >> (2 * i)) & 0x00030003u) | MAGIC;
   } else {
-    const uint32_t w = unit[t >> 1] >> (8 * (t & 1));
-    const uint32_t h = unit[2] >> (4 * t);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) f[i] = ((w >> (2 * i)) & 0x00030003u) | (((h >> i) & 0x00010001u) << 2) | MAGIC;
+    for (int i = 0; i < 4; ++i) f[i] = ((lo >> (2 * i)) & 0x00030003u) | (((hi >> i) & 0x00010001u) << 2) | MAGIC;
   }
 }
 
@@ -140,10 +139,9 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         const uint32_t stage = smem_base + s * S::STAGE_BYTES;
         // three tiled copies per stage: 4 k-block rows of pack units, the rows of
         // (alpha, beta) they need (128 / g of them) and the x slice
-        constexpr int UPACK = BITS == 4 ? 1 : (BITS == 2 ? 2 : 4);
         const int qrows = (GV_KBS * 32) / p.g;
         ptx::mbar_arrive_expect_tx(bar_full(s), GV_KBS * S::CODE_ROW + qrows * S::QP_ROW + S::X_BYTES);
-        ptx::tma_load_3d(stage + S::OFF_CODES, &codes_map, 0, n0 / UPACK, st * GV_KBS, bar_full(s));
+        ptx::tma_load_2d(stage + S::OFF_CODES, &codes_map, n0 * WORDS / 2, st * GV_KBS, bar_full(s));
         ptx::tma_load_2d(stage + S::OFF_QP, &qp_map, 2 * n0, st * GV_KBS * 32 / p.g, bar_full(s));
         ptx::tma_load_2d(stage + S::OFF_X, &x_map, st * GV_KBS * 32, 0, bar_full(s));
       }
@@ -157,6 +155,13 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int set = warp / 4, wcol = (warp % 4) * 32;
     const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block of the stage -> its (alpha, beta) row
     const int gq = lane / 4, t = lane % 4;        // fragment row / column group, quad lane
+    // per-thread byte offsets inside a stage; everything else is a compile-time constant
+    const uint32_t x_off = S::OFF_X + gq * (GV_KBS * 64) + t * 16 + set * 64;
+    const uint32_t lo_word = BITS == 4 ? t : (t >> 1);
+    const uint32_t lo_shift = BITS == 4 ? 0 : 8 * (t & 1);
+    const uint32_t c_off = S::OFF_CODES + set * S::CODE_ROW + ((wcol + gq) * WORDS + lo_word) * 4;
+    const uint32_t h_off = S::OFF_CODES + set * S::CODE_ROW + ((wcol + gq) * WORDS + 2) * 4;   // 3-bit codes: third-bit word
+    const uint32_t q_off = S::OFF_QP + (wcol + 2 * t) * 8;
     float acc[4][4];
     const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -171,28 +176,28 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       const uint8_t* stage = smem + s * S::STAGE_BYTES;
 #pragma unroll
       for (int bb = 0; bb < GV_KBS / GV_SETS; ++bb) {
-        const int b = bb * GV_SETS + set;
-        // A fragments: x[row][32 b + 8 t .. + 7] for rows gq and gq + 8
-        const uint4 xl = *reinterpret_cast<const uint4*>(stage + S::OFF_X + gq * (GV_KBS * 64) + b * 64 + t * 16);
+        // this set's k-block b = bb * GV_SETS + set; A fragments: x[row][32 b + 8 t .. + 7], rows gq and gq + 8
+        const uint4 xl = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64);
         uint4 xh = make_uint4(0u, 0u, 0u, 0u);
-        if (UPPER) xh = *reinterpret_cast<const uint4*>(stage + S::OFF_X + (gq + 8) * (GV_KBS * 64) + b * 64 + t * 16);
+        if (UPPER) xh = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64 + 8 * (GV_KBS * 64));
         const uint32_t a0[4] = {xl.x, xh.x, xl.y, xh.y};     // slots (2t,2t+1) | (2t+8,2t+9) of MMA 0
         const uint32_t a1[4] = {xl.z, xh.z, xl.w, xh.w};     // the same slots of MMA 1
         float Dx[4];
         mma16816(Dx, a0, ONES, ONES, zero4);
         mma16816(Dx, a1, ONES, ONES, Dx);
-        const uint8_t* crow = stage + S::OFF_CODES + b * S::CODE_ROW;
-        const uint8_t* qrow = stage + S::OFF_QP + (b >> qsh) * S::QP_ROW;
+        const uint8_t* qrow = stage + q_off + (((bb * GV_SETS + set) >> qsh) * S::QP_ROW);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const int col = wcol + c * 8;
+          const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> lo_shift;
+          uint32_t hi = 0;
+          if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> (4 * t);
           uint32_t f[4];
-          code_fragments<BITS>(reinterpret_cast<const uint32_t*>(crow) + (col + gq) * WORDS, t, f);
+          code_fragments<BITS>(lo, hi, f);
           float D[4];
           mma16816(D, a0, f[0], f[1], zero4);
           mma16816(D, a1, f[2], f[3], D);
           // accumulator columns of this lane are col + 2t and col + 2t + 1
-          const float4 q = *reinterpret_cast<const float4*>(qrow + (col + 2 * t) * 8);
+          const float4 q = *reinterpret_cast<const float4*>(qrow + c * 64);
           const float bias0 = fmaf(-128.f, q.x, q.y), bias1 = fmaf(-128.f, q.z, q.w);
           acc[c][0] = fmaf(q.x, D[0], fmaf(bias0, Dx[0], acc[c][0]));
           acc[c][1] = fmaf(q.z, D[1], fmaf(bias1, Dx[1], acc[c][1]));
@@ -276,14 +281,14 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   EncodeTiledFn fn = gv_encode_fn();
   CUtensorMap cm, qm;
   {
-    // packed codes uint32 [K/32][N][words] seen as [K/32][N/U][U*words] (innermost extent a
-    // multiple of 16 bytes); box = 4 k-block rows x 128 columns
-    constexpr int W = GvSmem<BITS>::WORDS, U = BITS == 4 ? 1 : (BITS == 2 ? 2 : 4);
-    cuuint64_t dims[3] = {(cuuint64_t)(U * W), (cuuint64_t)(p.N / U), (cuuint64_t)(p.K / 32)};
-    cuuint64_t strides[2] = {(cuuint64_t)U * W * 4, (cuuint64_t)p.N * W * 4};
-    cuuint32_t box[3] = {(cuuint32_t)(U * W), (cuuint32_t)(GV_COLS / U), GV_KBS};
-    cuuint32_t estr[3] = {1, 1, 1};
-    if (fn(&cm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint32_t*>(p.codes), dims, strides, box, estr,
+    // packed codes [K/32][N][words] uint32 seen as a 2-D matrix of 8-byte elements, so that
+    // one box row is the whole contiguous run of 128 pack units (2 KiB at 4 bits)
+    constexpr int W = GvSmem<BITS>::WORDS;
+    cuuint64_t dims[2] = {(cuuint64_t)p.N * W / 2, (cuuint64_t)(p.K / 32)};
+    cuuint64_t strides[1] = {(cuuint64_t)p.N * W * 4};
+    cuuint32_t box[2] = {(cuuint32_t)(GV_COLS * W / 2), GV_KBS};
+    cuuint32_t estr[2] = {1, 1};
+    if (fn(&cm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<uint32_t*>(p.codes), dims, strides, box, estr,
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return QALORA_ERR_CUDA;
