@@ -58,7 +58,8 @@ aux_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__
   using C = AuxCfg<MODE>;
   constexpr int STAGES = C::STAGES;
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // aligned by pointer arithmetic on the __shared__ array, so that the accesses stay shared-space loads/stores
+  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t smem_base = ptx::smem_u32(smem);
   uint8_t* bar_area = smem + STAGES * C::STAGE_BYTES;
   const uint32_t bar_base = smem_base + STAGES * C::STAGE_BYTES;

@@ -170,7 +170,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   constexpr int WORDS = S::WORDS;
   constexpr int NX = S::NX, NC = S::NC;
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // aligned by pointer arithmetic on the __shared__ array, so that the accesses stay shared-space loads/stores
+  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = smem_base + S::OFF_BARS;
   auto bar_full_x = [&](int s) { return bar_base + 8u * s; };

@@ -67,8 +67,9 @@ struct GvParams {
   int* status;
 };
 
+// (not volatile: a pure function of its operands, so that independent MMAs can be interleaved)
 __device__ __forceinline__ void mma16816(float* d, const uint32_t* a, uint32_t b0, uint32_t b1, const float* c) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
       : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
@@ -100,7 +101,8 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
   using S = GvSmem<BITS>;
   constexpr int WORDS = S::WORDS;
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+  // aligned by pointer arithmetic on the __shared__ array, so that the accesses stay shared-space loads/stores
+  uint8_t* smem = smem_raw + ((128u - (ptx::smem_u32(smem_raw) & 127u)) & 127u);
   const uint32_t smem_base = ptx::smem_u32(smem);
   auto bar_full = [&](int s) { return smem_base + S::OFF_BARS + 8u * s; };
   auto bar_empty = [&](int s) { return smem_base + S::OFF_BARS + 8u * (GV_STAGES + s); };
@@ -186,24 +188,31 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         mma16816(Dx, a0, ONES, ONES, zero4);
         mma16816(Dx, a1, ONES, ONES, Dx);
         const uint8_t* qrow = stage + q_off + (((bb * GV_SETS + set) >> qsh) * S::QP_ROW);
+        // the four column groups are independent: issue their loads, then their first
+        // MMAs, then their second MMAs, so that the tensor-pipe latencies overlap
+        uint32_t f[4][4];
+        float4 q[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> lo_shift;
           uint32_t hi = 0;
           if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> (4 * t);
-          uint32_t f[4];
-          code_fragments<BITS>(lo, hi, f);
-          float D[4];
-          mma16816(D, a0, f[0], f[1], zero4);
-          mma16816(D, a1, f[2], f[3], D);
-          // accumulator columns of this lane are col + 2t and col + 2t + 1
-          const float4 q = *reinterpret_cast<const float4*>(qrow + c * 64);
-          const float bias0 = fmaf(-128.f, q.x, q.y), bias1 = fmaf(-128.f, q.z, q.w);
-          acc[c][0] = fmaf(q.x, D[0], fmaf(bias0, Dx[0], acc[c][0]));
-          acc[c][1] = fmaf(q.z, D[1], fmaf(bias1, Dx[1], acc[c][1]));
+          code_fragments<BITS>(lo, hi, f[c]);
+          q[c] = *reinterpret_cast<const float4*>(qrow + c * 64);   // accumulator columns col + 2t, col + 2t + 1
+        }
+        float D[4][4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) mma16816(D[c], a0, f[c][0], f[c][1], zero4);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) mma16816(D[c], a1, f[c][2], f[c][3], D[c]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const float bias0 = fmaf(-128.f, q[c].x, q[c].y), bias1 = fmaf(-128.f, q[c].z, q[c].w);
+          acc[c][0] = fmaf(q[c].x, D[c][0], fmaf(bias0, Dx[0], acc[c][0]));
+          acc[c][1] = fmaf(q[c].z, D[c][1], fmaf(bias1, Dx[1], acc[c][1]));
           if (UPPER) {
-            acc[c][2] = fmaf(q.x, D[2], fmaf(bias0, Dx[2], acc[c][2]));
-            acc[c][3] = fmaf(q.z, D[3], fmaf(bias1, Dx[3], acc[c][3]));
+            acc[c][2] = fmaf(q[c].x, D[c][2], fmaf(bias0, Dx[2], acc[c][2]));
+            acc[c][3] = fmaf(q[c].z, D[c][3], fmaf(bias1, Dx[3], acc[c][3]));
           }
         }
       }
@@ -355,16 +364,14 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;
-  // slices per column tile (= cluster size, at most 8): the count whose blocks fill whole
-  // waves of two resident blocks per SM best; ties go to fewer slices
+  // slices per column tile (= cluster size, at most 8): as many as still fit in ONE wave of
+  // two resident blocks per SM.  A block pays several microseconds of fixed cost (launch,
+  // barrier set-up, first-byte latency, two cluster barriers), so blocks must live long.
   const int tiles = sh.N / GV_COLS, capacity = 2 * gv_sm_count();
-  int splits = 1;
-  double best = 0.0;
-  for (int sp = 1; sp <= 8 && sp <= p.total_stages; ++sp) {
-    const int blocks = tiles * sp, waves = (blocks + capacity - 1) / capacity;
-    const double eff = (double)blocks / ((double)waves * capacity);
-    if (eff > best + 0.02) { best = eff; splits = sp; }
-  }
+  int splits = capacity / tiles;
+  if (splits > 8) splits = 8;
+  if (splits > p.total_stages) splits = p.total_stages;
+  if (splits < 1) splits = 1;
   const bool upper = M > 8;
 #define QALORA_GV(BITS) (upper ? launch_gemv_t<BITS, true>(xm, p, splits, st) : launch_gemv_t<BITS, false>(xm, p, splits, st))
   if (sh.bits == 4) return QALORA_GV(4);
