@@ -38,7 +38,7 @@ constexpr int GV_SETS = 2;          // consumer warp sets; set s takes the k-blo
 constexpr int GV_WARPS = 4 * GV_SETS;   // consumer warps: 4 per set, 32 columns each
 constexpr int GV_THREADS = (GV_WARPS + 1) * 32;   // + 1 producer warp
 constexpr int GV_KBS = 4;           // 32-channel blocks per stage (128 channels)
-constexpr int GV_STAGES = 6;
+constexpr int GV_STAGES = 3;
 constexpr int GV_ROWS = 16;         // token rows of the MMA tile
 
 template <int BITS>
@@ -95,7 +95,7 @@ __device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, uint32_
 }
 
 template <int BITS, bool UPPER>   // UPPER: token rows 8..15 are in use (M > 8)
-__global__ void __launch_bounds__(GV_THREADS, 2)
+__global__ void __launch_bounds__(GV_THREADS, 3)
 qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
                    const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
   using S = GvSmem<BITS>;
@@ -188,31 +188,36 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         mma16816(Dx, a0, ONES, ONES, zero4);
         mma16816(Dx, a1, ONES, ONES, Dx);
         const uint8_t* qrow = stage + q_off + (((bb * GV_SETS + set) >> qsh) * S::QP_ROW);
-        // the four column groups are independent: issue their loads, then their first
-        // MMAs, then their second MMAs, so that the tensor-pipe latencies overlap
-        uint32_t f[4][4];
-        float4 q[4];
+        // column groups are independent: two at a time, loads first, then their first MMAs,
+        // then their second MMAs, so that the tensor-pipe latencies overlap
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> lo_shift;
-          uint32_t hi = 0;
-          if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> (4 * t);
-          code_fragments<BITS>(lo, hi, f[c]);
-          q[c] = *reinterpret_cast<const float4*>(qrow + c * 64);   // accumulator columns col + 2t, col + 2t + 1
-        }
-        float D[4][4];
+        for (int ch = 0; ch < 4; ch += 2) {
+          uint32_t f[2][4];
+          float4 q[2];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) mma16816(D[c], a0, f[c][0], f[c][1], zero4);
+          for (int j = 0; j < 2; ++j) {
+            const int c = ch + j;
+            const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> lo_shift;
+            uint32_t hi = 0;
+            if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> (4 * t);
+            code_fragments<BITS>(lo, hi, f[j]);
+            q[j] = *reinterpret_cast<const float4*>(qrow + c * 64);   // accumulator columns col + 2t, col + 2t + 1
+          }
+          float D[2][4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) mma16816(D[c], a1, f[c][2], f[c][3], D[c]);
+          for (int j = 0; j < 2; ++j) mma16816(D[j], a0, f[j][0], f[j][1], zero4);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const float bias0 = fmaf(-128.f, q[c].x, q[c].y), bias1 = fmaf(-128.f, q[c].z, q[c].w);
-          acc[c][0] = fmaf(q[c].x, D[c][0], fmaf(bias0, Dx[0], acc[c][0]));
-          acc[c][1] = fmaf(q[c].z, D[c][1], fmaf(bias1, Dx[1], acc[c][1]));
-          if (UPPER) {
-            acc[c][2] = fmaf(q[c].x, D[c][2], fmaf(bias0, Dx[2], acc[c][2]));
-            acc[c][3] = fmaf(q[c].z, D[c][3], fmaf(bias1, Dx[3], acc[c][3]));
+          for (int j = 0; j < 2; ++j) mma16816(D[j], a1, f[j][2], f[j][3], D[j]);
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const int c = ch + j;
+            const float bias0 = fmaf(-128.f, q[j].x, q[j].y), bias1 = fmaf(-128.f, q[j].z, q[j].w);
+            acc[c][0] = fmaf(q[j].x, D[j][0], fmaf(bias0, Dx[0], acc[c][0]));
+            acc[c][1] = fmaf(q[j].z, D[j][1], fmaf(bias1, Dx[1], acc[c][1]));
+            if (UPPER) {
+              acc[c][2] = fmaf(q[j].x, D[j][2], fmaf(bias0, Dx[2], acc[c][2]));
+              acc[c][3] = fmaf(q[j].z, D[j][3], fmaf(bias1, Dx[3], acc[c][3]));
+            }
           }
         }
       }
@@ -364,14 +369,17 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;
-  // slices per column tile (= cluster size, at most 8): as many as still fit in ONE wave of
-  // two resident blocks per SM.  A block pays several microseconds of fixed cost (launch,
-  // barrier set-up, first-byte latency, two cluster barriers), so blocks must live long.
-  const int tiles = sh.N / GV_COLS, capacity = 2 * gv_sm_count();
-  int splits = capacity / tiles;
-  if (splits > 8) splits = 8;
-  if (splits > p.total_stages) splits = p.total_stages;
-  if (splits < 1) splits = 1;
+  // slices per column tile (= cluster size): the count among {1,2,3,4,6,8} that brings the
+  // grid closest to two blocks per SM.  Three blocks fit on an SM, so the grid stays one
+  // wave with room for imbalance, while a block still streams enough bytes to amortize its
+  // fixed cost (launch, barrier set-up, first-byte latency, two cluster barriers).
+  const int tiles = sh.N / GV_COLS, target = 2 * gv_sm_count();
+  int splits = 1, best = 1 << 30;
+  for (int sp : {1, 2, 3, 4, 6, 8}) {
+    if (sp > p.total_stages) break;
+    const int miss = tiles * sp > target ? tiles * sp - target : target - tiles * sp;
+    if (miss < best) { best = miss; splits = sp; }
+  }
   const bool upper = M > 8;
 #define QALORA_GV(BITS) (upper ? launch_gemv_t<BITS, true>(xm, p, splits, st) : launch_gemv_t<BITS, false>(xm, p, splits, st))
   if (sh.bits == 4) return QALORA_GV(4);
