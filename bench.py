@@ -306,6 +306,7 @@ def run_gpu(args):
 
     # single-token forward of the merged layer: HBM-bound leg of the metric
     small = small_m_bandwidth(Q, torch, pk)
+    small_65b = small_m_bandwidth(Q, torch, pk, shape="cfg5_65b_up", ms=(1,)) if rank == 0 else None
 
     e2e_ms, _ = timed(e2e_step, args.steps)
     e2e_ms /= args.steps
@@ -326,7 +327,7 @@ def run_gpu(args):
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": flops_step / (e2e_ms / 1e3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "roofline": roofline, "small_m": small,
+            "roofline": roofline, "small_m": small, "small_m_65b": small_65b,
             "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc,
                              "seconds": dt},
         }

@@ -6,8 +6,9 @@
 namespace qalora {
 
 // ------------------------------------------------------------ pool and T -----
-// One block per token row: xp[q] = sum of the g channels of group q
-// (Appendix B Eq. 3), then T[i] = s * sum_q xp[q] * A[q][i].
+// One token row per blockIdx.x: xp[q] = sum of the g channels of group q
+// (Appendix B Eq. 3), then T[i] = s * sum_q xp[q] * A[q][i] for the 32 adapter
+// columns of blockIdx.y (every block pools the row again: it is a few KiB).
 constexpr int POOL_THREADS = 256;
 
 __global__ void __launch_bounds__(POOL_THREADS)
@@ -37,16 +38,29 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
     acc += __shfl_xor_sync(0xffffffffu, acc, 2);
     if (lane4 == 0 && q < G) {
       xp[q] = acc;
-      if (xp_out != nullptr) xp_out[m * (size_t)G + q] = acc;
+      if (xp_out != nullptr && blockIdx.y == 0) xp_out[m * (size_t)G + q] = acc;
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < r; i += POOL_THREADS) {
-    float acc = 0.0f;
-    for (int q = 0; q < G; ++q) acc = fmaf(xp[q], bf16_to_float(A[(size_t)q * r + i]), acc);
-    acc *= s;
-    T[m * (size_t)r + i] = acc;
-    if (Tb != nullptr) Tb[m * (size_t)r + i] = __float2bfloat16_rn(acc);
+  // this block's 32 adapter columns (blockIdx.y); 8 threads share a column, each taking
+  // every eighth group, so that the loads of A of one column are spread over 8 lanes
+  __shared__ float part[8][33];
+  const int il = threadIdx.x % 32, pr = threadIdx.x / 32;
+  const int i = blockIdx.y * 32 + il;
+  float acc = 0.0f;
+  if (i < r) {
+#pragma unroll 4
+    for (int q = pr; q < G; q += 8) acc = fmaf(xp[q], bf16_to_float(A[(size_t)q * r + i]), acc);
+  }
+  part[pr][il] = acc;
+  __syncthreads();
+  if (pr == 0 && i < r) {
+    float t = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) t += part[k][il];
+    t *= s;
+    T[m * (size_t)r + i] = t;
+    if (Tb != nullptr) Tb[m * (size_t)r + i] = __float2bfloat16_rn(t);
   }
 }
 
@@ -136,8 +150,8 @@ int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv
     else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
     else pool_T_rows_kernel<16><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
   } else {
-    pool_T_kernel<<<(unsigned)M, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G,
-                                                                          sh.r, sh.s);
+    dim3 grid((unsigned)M, (unsigned)((sh.r + 31) / 32 > 0 ? (sh.r + 31) / 32 : 1));
+    pool_T_kernel<<<grid, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G, sh.r, sh.s);
   }
   count_launch();
   return cuda_status(cudaGetLastError());
