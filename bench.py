@@ -109,12 +109,8 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------- CPU reference --
-def oracle_sample(rows=32):
-    """Times the CPU oracle (as it stands) on `rows` token rows of the first
-    shape: forward + backward.  Returns (TFLOP/s, seconds, description)."""
-    import numpy as np
-    import torch
-
+def oracle_setup(rows):
+    """Inputs of the CPU-oracle sample: `rows` token rows of the first shape, quantized once."""
     from oracle import qalora_oracle as O
     from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs, to_f64
 
@@ -122,32 +118,44 @@ def oracle_sample(rows=32):
     t = make_inputs(cfg)
     codes, alpha, beta = O.quantize(t["W"].numpy(), cfg.group_size, cfg.bits)
     x, A, B, dy = (to_f64(t[k]) for k in ("x", "A", "B", "dy"))
+    fl = fwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank) + bwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank)
+    desc = (f"fp64 numpy oracle, forward+backward on {rows} of 8192 token rows of {SHAPES[0]} "
+            f"(each call dequantizes the full {cfg.d_in}x{cfg.d_out} weight); quantize excluded")
+    return (O, cfg, codes, alpha, beta, x, A, B, dy), fl, desc
+
+
+def oracle_run(state):
+    O, cfg, codes, alpha, beta, x, A, B, dy = state
     t0 = time.perf_counter()
     O.forward(x, codes, alpha, beta, cfg.group_size, A, B, cfg.scale)
     O.backward(x, dy, codes, alpha, beta, cfg.group_size, A, B, cfg.scale)
-    dt = time.perf_counter() - t0
-    fl = fwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank) + bwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank)
-    cores = torch.get_num_threads()
-    desc = (f"fp64 numpy oracle, forward+backward on {rows} of 8192 token rows of {SHAPES[0]} "
-            f"(each call dequantizes the full {cfg.d_in}x{cfg.d_out} weight); quantize excluded")
-    return fl / dt / 1e12, dt, desc, cores
+    return time.perf_counter() - t0
+
+
+def oracle_sample(rows=32):
+    """Times the CPU oracle (as it stands) on `rows` token rows of the first
+    shape: forward + backward.  Returns (TFLOP/s, seconds, description, threads)."""
+    import torch
+    state, fl, desc = oracle_setup(rows)
+    dt = oracle_run(state)
+    return fl / dt / 1e12, dt, desc, torch.get_num_threads()
 
 
 def run_reference(args):
+    """The reference arm: the CPU oracle, one bounded sample of the workload per step."""
+    import torch
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    times, val, desc, cores = [], 0.0, "", 0
+    state, fl, desc = oracle_setup(16)
+    times = []
     for i in range(args.warmup + args.steps):
-        v, dt, desc, cores = oracle_sample(rows=16)
+        dt = oracle_run(state)
         if i >= args.warmup:
             times.append(dt)
     ms = 1e3 * sum(times) / max(1, len(times))
-    cfg_rows = 16
-    from paper_2309_14717_b200.synthetic import CONFIGS
-    c = CONFIGS[SHAPES[0]]
-    fl = fwd_flops(cfg_rows, c.d_in, c.d_out, c.groups, c.rank) + bwd_flops(cfg_rows, c.d_in, c.d_out, c.groups, c.rank)
     value = fl / (ms / 1e3) / 1e12
+    cores = torch.get_num_threads()
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
