@@ -67,8 +67,7 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
 // Streaming version for many rows and a group size of 32, 64 or 128: eight rows
 // per block, one warp per row.  A lane reads 16 bytes (8 channels) per step, so
 // g / 8 neighbouring lanes hold one group and a few shuffles finish its sum.
-// Then every thread accumulates four rows of T against one column of A, reading
-// each element of A once per block.
+// Then every thread accumulates two rows of T against one column of A.
 constexpr int POOL8_ROWS = 8;
 
 template <int LANES_PER_GROUP>   // g / 8: 4, 8 or 16
@@ -113,23 +112,21 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
     for (int q = lane; q < G; q += 32) xps[warp * G + q] = 0.0f;
   }
   __syncthreads();
-  // T: thread -> column i, four rows
-  for (int o = threadIdx.x; o < 2 * r; o += POOL8_ROWS * 32) {
-    const int i = o % r, rg = o / r;                      // rows 4 rg .. 4 rg + 3
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    const float* xr = xps + rg * 4 * G;
-#pragma unroll 8
+  // T: thread -> column i, two rows; each element of A is read once per two rows
+  for (int o = threadIdx.x; o < 4 * r; o += POOL8_ROWS * 32) {
+    const int i = o % r, rg = o / r;                      // rows 2 rg, 2 rg + 1
+    float a0 = 0.f, a1 = 0.f;
+    const float* xr = xps + rg * 2 * G;
+#pragma unroll 16
     for (int q = 0; q < G; ++q) {
       const float av = bf16_to_float(A[(size_t)q * r + i]);
       a0 = fmaf(xr[q], av, a0);
       a1 = fmaf(xr[G + q], av, a1);
-      a2 = fmaf(xr[2 * G + q], av, a2);
-      a3 = fmaf(xr[3 * G + q], av, a3);
     }
-    const float acc[4] = {a0 * s, a1 * s, a2 * s, a3 * s};
+    const float acc[2] = {a0 * s, a1 * s};
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const long long mm = (long long)blockIdx.x * POOL8_ROWS + rg * 4 + j;
+    for (int j = 0; j < 2; ++j) {
+      const long long mm = (long long)blockIdx.x * POOL8_ROWS + rg * 2 + j;
       if (mm < M) {
         T[(size_t)mm * r + i] = acc[j];
         if (Tb != nullptr) Tb[(size_t)mm * r + i] = __float2bfloat16_rn(acc[j]);
