@@ -10,14 +10,16 @@
 //  * A single thread streams codes, qparams and the x slice into a shared-memory
 //    ring with three tiled TMA copies per 128-channel stage, so that many tens of
 //    KiB per SM are in flight without using registers.
-//  * The products run on mma.sync.m16n8k16 (bf16 in, fp32 accumulate) with the
-//    tokens as the 16 rows: a lane's 32-bit word of packed codes IS its B
-//    fragment after one shift and one mask per pair (the code is OR-ed into the
-//    mantissa of bf16 128.0, no conversion).  The products x * (128 + c) are exact
-//    in fp32; once per quantization group the accumulator is folded as
-//        acc += alpha * D + (beta - 128 alpha) * xp,
+//  * The products run on mma.sync.m16n8k16 (bf16 in, fp32 accumulate) with 16
+//    columns of W as the rows and 8 tokens as the columns: a lane's 32-bit words
+//    of packed codes ARE its A fragments after one shift and one mask per pair
+//    (the code is OR-ed into the mantissa of bf16 128.0, no conversion), and its
+//    16-byte load of x is its B fragments.  The products x * (128 + c) are exact
+//    in fp32; the MMAs of a 32-channel block start from C = -128 xp, so that
+//    D = sum c x, and the block is folded as
+//        acc += alpha * D + beta * xp,
 //    where xp (the group sum of x, which the paper's pooling also needs) comes
-//    from one more MMA against a fragment of ones.  alpha and beta stay fp32.
+//    from one more MMA with ones as the A operand.  alpha and beta stay fp32.
 //  * The same reduction step adds the adapter term T * B (T = s * pool(x) * A is
 //    computed by the pooling kernel) and rounds to bf16.
 #include <cooperative_groups.h>
@@ -151,26 +153,34 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
   } else {
     // ----------------------------------------------------------- consumers ----
     // Warp w of set s owns columns 32 (w % 4) .. + 31 and the k-blocks b of each stage
-    // with b % GV_SETS == s.  Every k-block is folded on its own (the fold is linear, so
-    // the k-blocks of one quantization group may be folded separately with the same
-    // alpha and beta): acc += alpha * D + (beta - 128 alpha) * xp.
+    // with b % GV_SETS == s.  The weights are the A operand (16 columns x 16 channels per
+    // MMA) and the tokens the B operand (8 token columns), so that a lane's fragments of x
+    // are the register pairs its 16-byte load delivered and the code fragments are built
+    // in place.  Every k-block is folded on its own (the fold is linear, so the k-blocks
+    // of one quantization group may be folded separately with the same alpha and beta).
+    // The MMAs of a k-block start from C = -128 xp, which takes the offset of the raw
+    // codes out again: D = sum c x, and acc += alpha * D + beta * xp.
     const int set = warp / 4, wcol = (warp % 4) * 32;
     const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block of the stage -> its (alpha, beta) row
-    const int gq = lane / 4, t = lane % 4;        // fragment row / column group, quad lane
+    const int gq = lane / 4, t = lane % 4;        // fragment row (column of W, token), quad lane
+    constexpr int NTS = UPPER ? 2 : 1;            // sets of 8 tokens
     // per-thread byte offsets inside a stage; everything else is a compile-time constant
     const uint32_t x_off = S::OFF_X + gq * (GV_KBS * 64) + t * 16 + set * 64;
     const uint32_t lo_word = BITS == 4 ? t : (t >> 1);
     const uint32_t lo_shift = BITS == 4 ? 0 : 8 * (t & 1);
     const uint32_t c_off = S::OFF_CODES + set * S::CODE_ROW + ((wcol + gq) * WORDS + lo_word) * 4;
     const uint32_t h_off = S::OFF_CODES + set * S::CODE_ROW + ((wcol + gq) * WORDS + 2) * 4;   // 3-bit codes: third-bit word
-    const uint32_t q_off = S::OFF_QP + (wcol + 2 * t) * 8;
-    float acc[4][4];
+    const uint32_t q_off = S::OFF_QP + (wcol + gq) * 8;
+    float acc[2][NTS][4];                         // [16-column group][token set][(col gq | gq + 8) x (token 2t | 2t + 1)]
     const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
+    for (int c = 0; c < 2; ++c)
 #pragma unroll
-      for (int i = 0; i < 4; ++i) acc[c][i] = 0.f;
+      for (int ts = 0; ts < NTS; ++ts)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[c][ts][i] = 0.f;
     constexpr uint32_t ONES = 0x3f803f80u;        // bf16x2 (1, 1)
+    const uint32_t ones4[4] = {ONES, ONES, ONES, ONES};
     bool ok = true;
     for (int st = st_beg, it = 0; st < st_end && ok; ++st, ++it) {
       const int s = it % GV_STAGES;
@@ -178,60 +188,66 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       const uint8_t* stage = smem + s * S::STAGE_BYTES;
 #pragma unroll
       for (int bb = 0; bb < GV_KBS / GV_SETS; ++bb) {
-        // this set's k-block b = bb * GV_SETS + set; A fragments: x[row][32 b + 8 t .. + 7], rows gq and gq + 8
-        const uint4 xl = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64);
-        uint4 xh = make_uint4(0u, 0u, 0u, 0u);
-        if (UPPER) xh = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64 + 8 * (GV_KBS * 64));
-        const uint32_t a0[4] = {xl.x, xh.x, xl.y, xh.y};     // slots (2t,2t+1) | (2t+8,2t+9) of MMA 0
-        const uint32_t a1[4] = {xl.z, xh.z, xl.w, xh.w};     // the same slots of MMA 1
-        float Dx[4];
-        mma16816(Dx, a0, ONES, ONES, zero4);
-        mma16816(Dx, a1, ONES, ONES, Dx);
+        // this set's k-block b = bb * GV_SETS + set; B fragments: x[token gq (+ 8)][32 b + 8 t .. + 7]:
+        // the lane's k slots (2t, 2t+1 | 2t+8, 2t+9) of MMA 0 are channels 8t .. 8t+3, those of MMA 1 8t+4 .. 8t+7
+        uint4 xs[NTS];
+        xs[0] = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64);
+        if (UPPER) xs[NTS - 1] = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64 + 8 * (GV_KBS * 64));
+        // xp of the tokens (ones as the A operand: every row of the product holds the sums), then C = -128 xp
+        float cinit[NTS][4], xp[NTS][2];
+#pragma unroll
+        for (int ts = 0; ts < NTS; ++ts) {
+          mma16816(cinit[ts], ones4, xs[ts].x, xs[ts].y, zero4);
+          mma16816(cinit[ts], ones4, xs[ts].z, xs[ts].w, cinit[ts]);
+          xp[ts][0] = cinit[ts][0];
+          xp[ts][1] = cinit[ts][1];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) cinit[ts][i] *= -128.f;
+        }
         const uint8_t* qrow = stage + q_off + (((bb * GV_SETS + set) >> qsh) * S::QP_ROW);
-        // column groups are independent: two at a time, loads first, then their first MMAs,
-        // then their second MMAs, so that the tensor-pipe latencies overlap
 #pragma unroll
-        for (int ch = 0; ch < 4; ch += 2) {
+        for (int cg = 0; cg < 2; ++cg) {
+          // columns wcol + 16 cg + gq (fragment rows 0..7) and + 8 (rows 8..15)
           uint32_t f[2][4];
-          float4 q[2];
+          float2 q[2];
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
-            const int c = ch + j;
-            const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> lo_shift;
+            const uint32_t coff = bb * GV_SETS * S::CODE_ROW + (cg * 16 + j * 8) * WORDS * 4;
+            const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + coff) >> lo_shift;
             uint32_t hi = 0;
-            if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + bb * GV_SETS * S::CODE_ROW + c * 8 * WORDS * 4) >> (4 * t);
+            if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t);
             code_fragments<BITS>(lo, hi, f[j]);
-            q[j] = *reinterpret_cast<const float4*>(qrow + c * 64);   // accumulator columns col + 2t, col + 2t + 1
+            q[j] = *reinterpret_cast<const float2*>(qrow + (cg * 16 + j * 8) * 8);
           }
-          float D[2][4];
+          const uint32_t a0[4] = {f[0][0], f[1][0], f[0][1], f[1][1]};
+          const uint32_t a1[4] = {f[0][2], f[1][2], f[0][3], f[1][3]};
 #pragma unroll
-          for (int j = 0; j < 2; ++j) mma16816(D[j], a0, f[j][0], f[j][1], zero4);
-#pragma unroll
-          for (int j = 0; j < 2; ++j) mma16816(D[j], a1, f[j][2], f[j][3], D[j]);
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const int c = ch + j;
-            const float bias0 = fmaf(-128.f, q[j].x, q[j].y), bias1 = fmaf(-128.f, q[j].z, q[j].w);
-            acc[c][0] = fmaf(q[j].x, D[j][0], fmaf(bias0, Dx[0], acc[c][0]));
-            acc[c][1] = fmaf(q[j].z, D[j][1], fmaf(bias1, Dx[1], acc[c][1]));
-            if (UPPER) {
-              acc[c][2] = fmaf(q[j].x, D[j][2], fmaf(bias0, Dx[2], acc[c][2]));
-              acc[c][3] = fmaf(q[j].z, D[j][3], fmaf(bias1, Dx[3], acc[c][3]));
-            }
+          for (int ts = 0; ts < NTS; ++ts) {
+            float D[4];
+            mma16816(D, a0, xs[ts].x, xs[ts].y, cinit[ts]);
+            mma16816(D, a1, xs[ts].z, xs[ts].w, D);
+            acc[cg][ts][0] = fmaf(q[0].x, D[0], fmaf(q[0].y, xp[ts][0], acc[cg][ts][0]));
+            acc[cg][ts][1] = fmaf(q[0].x, D[1], fmaf(q[0].y, xp[ts][1], acc[cg][ts][1]));
+            acc[cg][ts][2] = fmaf(q[1].x, D[2], fmaf(q[1].y, xp[ts][0], acc[cg][ts][2]));
+            acc[cg][ts][3] = fmaf(q[1].x, D[3], fmaf(q[1].y, xp[ts][1], acc[cg][ts][3]));
           }
         }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar_empty(s));
     }
-    // partial sums of this warp set: [16 rows][128 columns]
+    // partial sums of this warp set: [16 token rows][128 columns]
     float* mine = partial + set * (GV_ROWS * GV_COLS);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const int col = wcol + c * 8 + 2 * t;
-      *reinterpret_cast<float2*>(mine + gq * GV_COLS + col) = make_float2(acc[c][0], acc[c][1]);
-      *reinterpret_cast<float2*>(mine + (gq + 8) * GV_COLS + col) = make_float2(acc[c][2], acc[c][3]);
-    }
+    for (int cg = 0; cg < 2; ++cg)
+#pragma unroll
+      for (int ts = 0; ts < NTS; ++ts) {
+        const int col = wcol + cg * 16 + gq, row = ts * 8 + 2 * t;
+        mine[row * GV_COLS + col] = acc[cg][ts][0];
+        mine[(row + 1) * GV_COLS + col] = acc[cg][ts][1];
+        mine[row * GV_COLS + col + 8] = acc[cg][ts][2];
+        mine[(row + 1) * GV_COLS + col + 8] = acc[cg][ts][3];
+      }
   }
 
   // ---- add the slices in rank order through distributed shared memory ---------
