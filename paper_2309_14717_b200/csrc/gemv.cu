@@ -40,21 +40,22 @@ constexpr int GV_SETS = 2;          // consumer warp sets; set s takes the k-blo
 constexpr int GV_WARPS = 4 * GV_SETS;   // consumer warps: 4 per set, 32 columns each
 constexpr int GV_THREADS = (GV_WARPS + 1) * 32;   // + 1 producer warp
 constexpr int GV_KBS = 4;           // 32-channel blocks per stage (128 channels)
-constexpr int GV_STAGES = 3;
-constexpr int GV_ROWS = 16;         // token rows of the MMA tile
+constexpr int GV_ROWS = 16;         // most token rows
 
-template <int BITS>
+template <int BITS, bool UPPER>   // UPPER: more than 8 token rows
 struct GvSmem {
+  static constexpr int ROWS = UPPER ? 16 : 8;                           // token rows held in shared memory
+  static constexpr int STAGES = UPPER ? 3 : 4;                          // three blocks per SM either way
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   static constexpr uint32_t CODE_ROW = GV_COLS * WORDS * 4;             // one k-block row of units
   static constexpr uint32_t QP_ROW = GV_COLS * 8;
-  static constexpr uint32_t X_BYTES = GV_ROWS * GV_KBS * 32 * 2;        // 16 rows x 128 channels bf16
+  static constexpr uint32_t X_BYTES = ROWS * GV_KBS * 32 * 2;           // rows x 128 channels bf16
   static constexpr uint32_t OFF_CODES = 0;
   static constexpr uint32_t OFF_QP = GV_KBS * CODE_ROW;
   static constexpr uint32_t OFF_X = OFF_QP + GV_KBS * QP_ROW;
   static constexpr uint32_t STAGE_BYTES = ((OFF_X + X_BYTES + 127) / 128) * 128;
-  static constexpr uint32_t OFF_PARTIAL = GV_STAGES * STAGE_BYTES;      // fp32 [sets][16][128]
-  static constexpr uint32_t OFF_BARS = OFF_PARTIAL + GV_SETS * GV_ROWS * GV_COLS * 4;
+  static constexpr uint32_t OFF_PARTIAL = STAGES * STAGE_BYTES;         // fp32 [sets][rows][128]
+  static constexpr uint32_t OFF_BARS = OFF_PARTIAL + GV_SETS * ROWS * GV_COLS * 4;
   static constexpr uint32_t TOTAL = OFF_BARS + 128 + 128;               // + alignment slack
 };
 
@@ -100,8 +101,9 @@ template <int BITS, bool UPPER>   // UPPER: token rows 8..15 are in use (M > 8)
 __global__ void __launch_bounds__(GV_THREADS, 3)
 qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
                    const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
-  using S = GvSmem<BITS>;
+  using S = GvSmem<BITS, UPPER>;
   constexpr int WORDS = S::WORDS;
+  constexpr int GV_STAGES = S::STAGES;
   extern __shared__ uint8_t smem_raw[];
   // aligned by pointer arithmetic on the __shared__ array, so that the accesses stay shared-space loads/stores
   uint8_t* smem = smem_raw + ((128u - (ptx::smem_u32(smem_raw) & 127u)) & 127u);
@@ -237,7 +239,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       if (lane == 0) ptx::mbar_arrive(bar_empty(s));
     }
     // partial sums of this warp set: [16 token rows][128 columns]
-    float* mine = partial + set * (GV_ROWS * GV_COLS);
+    float* mine = partial + set * (S::ROWS * GV_COLS);
 #pragma unroll
     for (int cg = 0; cg < 2; ++cg)
 #pragma unroll
@@ -262,7 +264,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       for (int rk = 0; rk < splits; ++rk) {
         const float* remote = cluster.map_shared_rank(partial, rk);
 #pragma unroll
-        for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (GV_ROWS * GV_COLS) + row * GV_COLS + col];
+        for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
       }
       if (p.r > 0) {
         const float* Tr = p.T + (size_t)row * p.r;
@@ -313,7 +315,7 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   {
     // packed codes [K/32][N][words] uint32 seen as a 2-D matrix of 8-byte elements, so that
     // one box row is the whole contiguous run of 128 pack units (2 KiB at 4 bits)
-    constexpr int W = GvSmem<BITS>::WORDS;
+    constexpr int W = GvSmem<BITS, UPPER>::WORDS;
     cuuint64_t dims[2] = {(cuuint64_t)p.N * W / 2, (cuuint64_t)(p.K / 32)};
     cuuint64_t strides[1] = {(cuuint64_t)p.N * W * 4};
     cuuint32_t box[2] = {(cuuint32_t)(GV_COLS * W / 2), GV_KBS};
@@ -332,7 +334,7 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return QALORA_ERR_CUDA;
   }
-  using S = GvSmem<BITS>;
+  using S = GvSmem<BITS, UPPER>;
   auto kern = qalora_gemv_kernel<BITS, UPPER>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -374,7 +376,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   CUtensorMap xm;
   cuuint64_t dims[2] = {(cuuint64_t)sh.K, (cuuint64_t)M};
   cuuint64_t strides[1] = {(cuuint64_t)sh.K * 2};
-  cuuint32_t box[2] = {GV_KBS * 32, GV_ROWS};
+  cuuint32_t box[2] = {GV_KBS * 32, (cuuint32_t)(M > 8 ? 16 : 8)};   // the token rows the kernel keeps
   cuuint32_t estr[2] = {1, 1};
   if (fn(&xm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(x), dims, strides, box, estr,
          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
