@@ -82,18 +82,35 @@ __device__ __forceinline__ void mma16816(float* d, const uint32_t* a, uint32_t b
 // `lo` is the word that holds the (low) code bits of those positions, already shifted so
 // that they start at bit 0 of each half-word; `hi` (3-bit codes only) the third-bit word
 // shifted likewise.
+//
+// The logic/shift pipe is what this kernel runs out of first, so the extraction is spelled
+// out: the constants live in registers (FragConsts; a LOP3 takes one immediate at most, and
+// with two it becomes two instructions) and "(a & mask) | magic" is one LOP3.  (Shifting by
+// mul.hi on the multiplier pipe instead was measured slower.)
+struct FragConsts {
+  uint32_t mask, magic;
+};
 template <int BITS>
-__device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, uint32_t* f) {
-  constexpr uint32_t MAGIC = 0x43004300u;
-  if (BITS == 4) {
+__device__ __forceinline__ FragConsts frag_consts() {
+  FragConsts c;
+  // asm volatile: the values stay opaque, so that they are not turned back into immediates
+  asm volatile("mov.b32 %0, %1;" : "=r"(c.mask) : "n"(BITS == 4 ? 0x000f000f : 0x00030003));
+  asm volatile("mov.b32 %0, 0x43004300;" : "=r"(c.magic));
+  return c;
+}
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {   // (a & b) | c
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+template <int BITS>
+__device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, const FragConsts& k, uint32_t* f) {
+  constexpr int W = BITS == 4 ? 4 : 2;          // field width of the (low) code bits
 #pragma unroll
-    for (int i = 0; i < 4; ++i) f[i] = ((lo >> (4 * i)) & 0x000f000fu) | MAGIC;
-  } else if (BITS == 2) {
+  for (int i = 0; i < 4; ++i) f[i] = and_or(lo >> (W * i), k.mask, k.magic);
+  if (BITS == 3) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) f[i] = ((lo >> (2 * i)) & 0x00030003u) | MAGIC;
-  } else {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) f[i] = ((lo >> (2 * i)) & 0x00030003u) | (((hi >> i) & 0x00010001u) << 2) | MAGIC;
+    for (int i = 0; i < 4; ++i) f[i] |= ((hi >> i) & 0x00010001u) << 2;
   }
 }
 
@@ -181,6 +198,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       for (int ts = 0; ts < NTS; ++ts)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[c][ts][i] = 0.f;
+    const FragConsts fk = frag_consts<BITS>();
     constexpr uint32_t ONES = 0x3f803f80u;        // bf16x2 (1, 1)
     const uint32_t ones4[4] = {ONES, ONES, ONES, ONES};
     bool ok = true;
@@ -218,7 +236,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
             const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + coff) >> lo_shift;
             uint32_t hi = 0;
             if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t);
-            code_fragments<BITS>(lo, hi, f[j]);
+            code_fragments<BITS>(lo, hi, fk, f[j]);
             q[j] = *reinterpret_cast<const float2*>(qrow + (cg * 16 + j * 8) * 8);
           }
           const uint32_t a0[4] = {f[0][0], f[1][0], f[0][1], f[1][1]};
