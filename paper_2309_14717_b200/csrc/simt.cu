@@ -64,20 +64,49 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
   }
 }
 
-// Streaming version for many rows and a group size of 32, 64 or 128: eight rows
+// Streaming version for many rows and a group size of 32, 64 or 128: sixteen rows
 // per block, one warp per row.  A lane reads 16 bytes (8 channels) per step, so
 // g / 8 neighbouring lanes hold one group and a few shuffles finish its sum.
-// Then every thread accumulates two rows of T against one column of A.
-constexpr int POOL8_ROWS = 8;
+// T = xp * A then runs on mma.sync.m16n8k16 with the block's 16 rows as the MMA rows
+// and the groups as the reduction dimension; xp enters as a bf16 pair hi + lo
+// (hi = xp rounded, lo = the remainder rounded: 16 significant bits together), so that
+// T keeps fp32-like accuracy although the operands are bf16.
+constexpr int POOL16_ROWS = 16;
+
+__device__ __forceinline__ void mma_bf16_16816(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Row stride (in 32-bit words) of the bf16 [16][Gp] arrays in shared memory: at least
+// Gp / 2 and = 4 mod 32, so that the eight rows x four words of a fragment load fall into
+// 32 different banks.
+__host__ __device__ inline int pool16_stride_words(int G) {
+  const int gp = (G + 15) / 16 * 16;
+  int w = gp / 2;
+  w += (4 - (w % 32) + 32) % 32;
+  return w;
+}
 
 template <int LANES_PER_GROUP>   // g / 8: 4, 8 or 16
-__global__ void __launch_bounds__(POOL8_ROWS * 32)
+__global__ void __launch_bounds__(POOL16_ROWS * 32)
 pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
                    float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
                    long long M, int K, int G, int r, float s) {
-  extern __shared__ float xps[];                        // [8][G]
+  extern __shared__ __align__(16) uint32_t pool_smem[];
+  const int SW = pool16_stride_words(G);                 // row stride of the two bf16 arrays, in words
+  __nv_bfloat16* xhi = reinterpret_cast<__nv_bfloat16*>(pool_smem);                 // [16][2 SW]
+  __nv_bfloat16* xlo = reinterpret_cast<__nv_bfloat16*>(pool_smem + POOL16_ROWS * SW);
+  float* part = reinterpret_cast<float*>(pool_smem + 2 * POOL16_ROWS * SW);        // [ksplit][16][r]
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const long long m = (long long)blockIdx.x * POOL8_ROWS + warp;
+  const long long m = (long long)blockIdx.x * POOL16_ROWS + warp;
+  const int Gp = (G + 15) / 16 * 16;
+  // the padding groups G .. Gp - 1 and the rows beyond M count as zero
+  for (int q = (m < M ? G : 0) + lane; q < Gp; q += 32) {
+    xhi[warp * 2 * SW + q] = __float2bfloat16_rn(0.f);
+    xlo[warp * 2 * SW + q] = __float2bfloat16_rn(0.f);
+  }
   if (m < M) {
     const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)m * K);
     const int chunks = K / 8;                             // K is a multiple of 32
@@ -103,49 +132,90 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
         for (int o = 1; o < LANES_PER_GROUP; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (c < chunks && (lane % LANES_PER_GROUP) == 0) {
           const int q = c / LANES_PER_GROUP;
-          xps[warp * G + q] = acc;
+          const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
+          xhi[warp * 2 * SW + q] = hi;
+          xlo[warp * 2 * SW + q] = __float2bfloat16_rn(acc - __bfloat162float(hi));
           if (xp_out != nullptr) xp_out[(size_t)m * G + q] = acc;
         }
       }
     }
-  } else {
-    for (int q = lane; q < G; q += 32) xps[warp * G + q] = 0.0f;
   }
   __syncthreads();
-  // T: thread -> column i, two rows; each element of A is read once per two rows
-  for (int o = threadIdx.x; o < 4 * r; o += POOL8_ROWS * 32) {
-    const int i = o % r, rg = o / r;                      // rows 2 rg, 2 rg + 1
-    float a0 = 0.f, a1 = 0.f;
-    const float* xr = xps + rg * 2 * G;
-#pragma unroll 16
-    for (int q = 0; q < G; ++q) {
-      const float av = bf16_to_float(A[(size_t)q * r + i]);
-      a0 = fmaf(xr[q], av, a0);
-      a1 = fmaf(xr[G + q], av, a1);
-    }
-    const float acc[2] = {a0 * s, a1 * s};
+  // T tile of 16 rows x 8 adapter columns per job; with few column tiles the groups are split
+  // over several warps (ksplit parts), whose sums meet in shared memory
+  const int ntiles = r / 8;                               // r is a multiple of 8
+  int ksplit = 1;
+  while (ksplit * 2 * ntiles <= POOL16_ROWS) ksplit *= 2;
+  const int gq = lane / 4, t = lane % 4;
+  const uint32_t* hi32 = pool_smem;
+  const uint32_t* lo32 = pool_smem + POOL16_ROWS * SW;
+  const uint16_t* A16 = reinterpret_cast<const uint16_t*>(A);
+  for (int job = warp; job < ntiles * ksplit; job += POOL16_ROWS) {
+    const int nt = job % ntiles, part_i = job / ntiles;
+    const int n = nt * 8 + gq;                            // this lane's column of A
+    float d[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int ks = part_i; ks < Gp / 16; ks += ksplit) {
+      const int k0 = ks * 16 + 2 * t;                     // groups k0, k0 + 1 | k0 + 8, k0 + 9
+      uint32_t bw[4];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const long long mm = (long long)blockIdx.x * POOL8_ROWS + rg * 2 + j;
-      if (mm < M) {
-        T[(size_t)mm * r + i] = acc[j];
-        if (Tb != nullptr) Tb[(size_t)mm * r + i] = __float2bfloat16_rn(acc[j]);
+      for (int e = 0; e < 4; ++e) {
+        const int q = k0 + (e & 1) + 8 * (e >> 1);
+        bw[e] = q < G ? A16[(size_t)q * r + n] : 0u;
       }
+      const uint32_t b0 = bw[0] | (bw[1] << 16), b1 = bw[2] | (bw[3] << 16);
+      const int w0 = ks * 8 + t;                          // word of (k0, k0 + 1) in a row
+      const uint32_t ah[4] = {hi32[gq * SW + w0], hi32[(gq + 8) * SW + w0], hi32[gq * SW + w0 + 4], hi32[(gq + 8) * SW + w0 + 4]};
+      const uint32_t al[4] = {lo32[gq * SW + w0], lo32[(gq + 8) * SW + w0], lo32[gq * SW + w0 + 4], lo32[(gq + 8) * SW + w0 + 4]};
+      mma_bf16_16816(d, ah, b0, b1);
+      mma_bf16_16816(d, al, b0, b1);
+    }
+    float* pp = part + (size_t)part_i * POOL16_ROWS * r;
+    const int col = nt * 8 + 2 * t;
+    pp[gq * r + col] = d[0];
+    pp[gq * r + col + 1] = d[1];
+    pp[(gq + 8) * r + col] = d[2];
+    pp[(gq + 8) * r + col + 1] = d[3];
+  }
+  __syncthreads();
+  for (int o = threadIdx.x; o < POOL16_ROWS * r; o += POOL16_ROWS * 32) {
+    const long long mm = (long long)blockIdx.x * POOL16_ROWS + o / r;
+    float v = 0.f;
+    for (int pi = 0; pi < ksplit; ++pi) v += part[(size_t)pi * POOL16_ROWS * r + o];
+    v *= s;
+    if (mm < M) {
+      T[(size_t)mm * r + o % r] = v;
+      if (Tb != nullptr) Tb[(size_t)mm * r + o % r] = __float2bfloat16_rn(v);
     }
   }
+}
+
+// shared memory of pool_T_rows_kernel (up to kPool16MaxSmem)
+constexpr size_t kPool16MaxSmem = 96 * 1024;
+static size_t pool16_smem_bytes(int G, int r) {
+  const int ntiles = r / 8;
+  int ksplit = 1;
+  while (ksplit * 2 * ntiles <= POOL16_ROWS) ksplit *= 2;
+  return (size_t)2 * POOL16_ROWS * pool16_stride_words(G) * 4 + (size_t)ksplit * POOL16_ROWS * r * 4;
 }
 
 int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv_bfloat16* A,
                   float* xp, float* T, __nv_bfloat16* Tb, cudaStream_t st) {
   if (M == 0) return QALORA_OK;
+  const size_t smem = sh.r >= 8 ? pool16_smem_bytes(sh.G, sh.r) : 0;
   const bool rows_path = M >= 64 && (sh.g == 32 || sh.g == 64 || sh.g == 128) && sh.K % 256 == 0 &&
-                         (size_t)POOL8_ROWS * sh.G * sizeof(float) <= 48 * 1024;
+                         sh.r >= 8 && smem <= kPool16MaxSmem;
   if (rows_path) {
-    const unsigned grid = (unsigned)((M + POOL8_ROWS - 1) / POOL8_ROWS);
-    const size_t smem = (size_t)POOL8_ROWS * sh.G * sizeof(float);
-    if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
-    else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
-    else pool_T_rows_kernel<16><<<grid, POOL8_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
+    static const cudaError_t attr_err = [] {             // once: allow more than the default 48 KiB
+      cudaError_t e = cudaFuncSetAttribute(pool_T_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPool16MaxSmem);
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(pool_T_rows_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPool16MaxSmem);
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(pool_T_rows_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPool16MaxSmem);
+      return e;
+    }();
+    if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
+    const unsigned grid = (unsigned)((M + POOL16_ROWS - 1) / POOL16_ROWS);
+    if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
+    else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
+    else pool_T_rows_kernel<16><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
   } else {
     dim3 grid((unsigned)M, (unsigned)((sh.r + 31) / 32 > 0 ? (sh.r + 31) / 32 : 1));
     pool_T_kernel<<<grid, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G, sh.r, sh.s);
