@@ -12,8 +12,12 @@ constexpr int QCOLS = 128;   // columns (threads) per block
 
 // Each thread: two passes over its g weights.  Pass 1 finds min/max, pass 2
 // re-reads (L1/L2 hits), rounds and packs one 32-channel unit at a time.  Every
-// floating-point step is a single IEEE fp32 operation (no FMA contraction, no
-// reciprocal), so the integer decision is reproducible bit for bit on a CPU.
+// floating-point step is a single IEEE fp32 operation (no FMA contraction), so
+// the integer decision is reproducible bit for bit on a CPU.  The division
+// t = (w - beta) / alpha is the expensive one; the code only needs rint(t), so the
+// kernel first takes t' = (w - beta) * (1 / alpha), which is within 2e-6 of t for
+// t in [0, 15], and falls back to the IEEE division only where t' lies within 1e-4
+// of a rounding boundary (a half-integer): everywhere else rint(t') = rint(t).
 template <int BITS>
 __global__ void __launch_bounds__(QCOLS)
 quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
@@ -43,6 +47,7 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
   qparams[(size_t)q * N + n] = make_float2(alpha, beta);
   if (bad && dev_status != nullptr) atomicOr(dev_status, 1);
 
+  const float inv_alpha = __frcp_rn(alpha);
   const int kb0 = q * (g / 32);
   for (int k0 = 0; k0 < g; k0 += 32) {
     float v[32];
@@ -53,7 +58,9 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
     for (int i = 0; i < WORDS; ++i) u[i] = 0u;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-      const float t = __fdiv_rn(__fsub_rn(v[j], beta), alpha);
+      const float d = __fsub_rn(v[j], beta);
+      float t = __fmul_rn(d, inv_alpha);
+      if (fabsf(fabsf(t - rintf(t)) - 0.5f) < 1e-4f) t = __fdiv_rn(d, alpha);   // near a boundary (or a tie): exact
       float c = rintf(t);                              // round half to even
       c = fminf(fmaxf(c, 0.0f), QMAX);
       unit_insert<BITS>(u, j, (uint32_t)(int)c);
