@@ -59,9 +59,9 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
       const float d = __fsub_rn(v[j], beta);
-      float t = __fmul_rn(d, inv_alpha);
-      if (fabsf(fabsf(t - rintf(t)) - 0.5f) < 1e-4f) t = __fdiv_rn(d, alpha);   // near a boundary (or a tie): exact
+      const float t = __fmul_rn(d, inv_alpha);
       float c = rintf(t);                              // round half to even
+      if (fabsf(t - c) > 0.4999f) c = rintf(__fdiv_rn(d, alpha));   // near a boundary (or a tie): exact
       c = fminf(fmaxf(c, 0.0f), QMAX);
       unit_insert<BITS>(u, j, (uint32_t)(int)c);
     }
