@@ -178,7 +178,6 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   auto bar_empty_x = [&](int s) { return bar_base + 8u * (NX + s); };
   auto bar_full_c = [&](int s) { return bar_base + 8u * (2 * NX + s); };
   auto bar_empty_c = [&](int s) { return bar_base + 8u * (2 * NX + NC + s); };
-  auto bar_aready = [&](int s) { return bar_base + 8u * (2 * NX + 2 * NC + s); };
   const uint32_t bar_acc_full = bar_base + 8u * (2 * NX + 2 * NC + NX);
   const uint32_t bar_acc_empty = bar_acc_full + 8u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + S::OFF_BARS + 8 * S::NBARS);
@@ -187,9 +186,10 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NX; ++s) { ptx::mbar_init(bar_full_x(s), 1); ptx::mbar_init(bar_empty_x(s), 1); }
+    // full_x: the activation tile has landed (producer's arrive + its bytes) AND the four
+    // dequantizer warps have written the operand slot: one wait per step for the MMA issuer
+    for (int s = 0; s < NX; ++s) { ptx::mbar_init(bar_full_x(s), 1 + 4); ptx::mbar_init(bar_empty_x(s), 1); }
     for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4 * S::IPS); }
-    for (int s = 0; s < NX; ++s) ptx::mbar_init(bar_aready(s), 4);
     ptx::mbar_init(bar_acc_full, 1);
     ptx::mbar_init(bar_acc_empty, 4);
     *abort_flag = 0;
@@ -259,23 +259,17 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(TILE_C, TILE_T, false, false);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      // the barriers of the coming step are probed while the MMAs of the current one are being issued
-      bool rdy_a = false, rdy_x = false;
+      // Issuing one tcgen05.mma costs this thread about 110 cycles and the four MMAs of a step
+      // keep the tensor pipe busy for 512, so everything else in this loop has to stay short:
+      // one barrier wait, one fence, one commit per step.
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
         if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int i = 0; i < iters; ++i, ++it) {
           const int sx = it % NX;
           const uint32_t ph = (it / NX) & 1;
-          if (!rdy_a && !(ok = ptx::mbar_wait(bar_aready(sx), ph, abort_flag))) break;
-          if (!rdy_x && !(ok = ptx::mbar_wait(bar_full_x(sx), ph, abort_flag))) break;
+          if (!(ok = ptx::mbar_wait(bar_full_x(sx), ph, abort_flag))) break;
           ptx::tc_fence_after();
-          {
-            const int sn = (it + 1) % NX;
-            const uint32_t pn = ((it + 1) / NX) & 1;
-            rdy_a = ptx::mbar_test_wait(bar_aready(sn), pn);
-            rdy_x = ptx::mbar_test_wait(bar_full_x(sn), pn);
-          }
           const uint32_t xs = smem_base + S::OFF_X + sx * ACT_BYTES;
           const uint32_t as = smem_base + S::OFF_A + sx * ATILE_BYTES;
 #pragma unroll
@@ -389,7 +383,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         }
         __syncwarp();
         if (lane == 0) {
-          ptx::mbar_arrive(bar_aready(sa));
+          ptx::mbar_arrive(bar_full_x(sa));
           if (i < p.red_iters) ptx::mbar_arrive(bar_empty_c(sc));
         }
       }
