@@ -38,7 +38,7 @@ constexpr int DQ_GROUPS = 4;     // dequantizing warpgroups
 constexpr int THREADS = 128 + 128 * DQ_GROUPS + 128;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_COL = 0;       // accumulator: columns [0, 256)
-constexpr int A_COL = 256;       // forward operand ring: 4 slots of 32 columns
+constexpr int A_COL = 256;       // forward operand ring: 8 slots of 32 columns
 constexpr uint32_t ACT_BYTES = TILE_T * TILE_J * 2;      // 32 KiB activation tile
 constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx)
 
@@ -59,18 +59,22 @@ struct TcParams {
 };
 
 // Rings, decoupled so that each covers its own latency:
-//   NX activation tiles (TMA, 32 KiB each) and, in lock step with them, NX operand
-//      slots (TMEM columns for forward, 16 KiB of smem for dx) written by the
-//      dequantizers; one tcgen05.commit per reduction step frees both;
+//   NX activation tiles (TMA, 32 KiB each);
+//   NB operand slots written by the dequantizers (TMEM columns for forward: eight, so that
+//      a warpgroup can fill its next slot while its last one is still being multiplied;
+//      16 KiB of smem each for dx: four), each with a "ready" and a "free" barrier that
+//      step it uses at index it % NB; the step's activation tile completes the same "ready"
+//      barrier, and one tcgen05.commit per step frees the slot AND the tile;
 //   NC code stages (two tiled TMA copies each: 4 k-block rows of pack units and the
 //      rows of (alpha, beta) they need; a forward stage feeds two reduction steps)
 //      that run further ahead.
-// NX and NC are multiples of DQ_GROUPS, so a ring slot always belongs to the same
+// NB and NC are multiples of DQ_GROUPS, so a ring slot always belongs to the same
 // dequantizing warpgroup and its barrier phases are waited on in order.
 template <int BITS, int MODE>
 struct Smem {
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   static constexpr int NX = 4;
+  static constexpr int NB = MODE == FWD ? 8 : 4;
   static constexpr int NC = 4;
   static constexpr int IPS = MODE == FWD ? 2 : 1;                                // reduction steps per code stage
   static constexpr int TILE_NC = MODE == FWD ? TILE_C : TILE_J;                  // columns of a code stage
@@ -86,7 +90,7 @@ struct Smem {
   static constexpr uint32_t OFF_C = OFF_A + (MODE == DX ? NX * ATILE_BYTES : 0);
   static constexpr uint32_t OFF_OUT = OFF_C + NC * CSTAGE_BYTES;
   static constexpr uint32_t OFF_BARS = OFF_OUT + NOUT * OUT_BYTES;
-  static constexpr int NBARS = 2 * NX + 2 * NC + NX + 2;
+  static constexpr int NBARS = 2 * NB + 2 * NC + 2;
   static constexpr uint32_t TOTAL = OFF_BARS + 8 * NBARS + 64 + 1024;            // + alignment slack
 };
 
@@ -168,17 +172,17 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
                  const __grid_constant__ CUtensorMap qp_map, const TcParams p) {
   using S = Smem<BITS, MODE>;
   constexpr int WORDS = S::WORDS;
-  constexpr int NX = S::NX, NC = S::NC;
+  constexpr int NX = S::NX, NB = S::NB, NC = S::NC;
   extern __shared__ uint8_t smem_raw[];
   // aligned by pointer arithmetic on the __shared__ array, so that the accesses stay shared-space loads/stores
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = smem_base + S::OFF_BARS;
   auto bar_full_x = [&](int s) { return bar_base + 8u * s; };
-  auto bar_empty_x = [&](int s) { return bar_base + 8u * (NX + s); };
-  auto bar_full_c = [&](int s) { return bar_base + 8u * (2 * NX + s); };
-  auto bar_empty_c = [&](int s) { return bar_base + 8u * (2 * NX + NC + s); };
-  const uint32_t bar_acc_full = bar_base + 8u * (2 * NX + 2 * NC + NX);
+  auto bar_empty_x = [&](int s) { return bar_base + 8u * (NB + s); };
+  auto bar_full_c = [&](int s) { return bar_base + 8u * (2 * NB + s); };
+  auto bar_empty_c = [&](int s) { return bar_base + 8u * (2 * NB + NC + s); };
+  const uint32_t bar_acc_full = bar_base + 8u * (2 * NB + 2 * NC);
   const uint32_t bar_acc_empty = bar_acc_full + 8u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + S::OFF_BARS + 8 * S::NBARS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_BARS + 8 * S::NBARS + 8);
@@ -188,7 +192,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   if (threadIdx.x == 0) {
     // full_x: the activation tile has landed (producer's arrive + its bytes) AND the four
     // dequantizer warps have written the operand slot: one wait per step for the MMA issuer
-    for (int s = 0; s < NX; ++s) { ptx::mbar_init(bar_full_x(s), 1 + 4); ptx::mbar_init(bar_empty_x(s), 1); }
+    for (int s = 0; s < NB; ++s) { ptx::mbar_init(bar_full_x(s), 1 + 4); ptx::mbar_init(bar_empty_x(s), 1); }
     for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4 * S::IPS); }
     ptx::mbar_init(bar_acc_full, 1);
     ptx::mbar_init(bar_acc_empty, 4);
@@ -221,13 +225,14 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile / p.c_tiles) * TILE_T;
         for (int i = 0; i < iters; ++i, ++it) {
-          const int s = it % NX;
-          if (!(ok = ptx::mbar_wait(bar_empty_x(s), ((it / NX) & 1) ^ 1, abort_flag))) break;
-          ptx::mbar_arrive_expect_tx(bar_full_x(s), ACT_BYTES);
+          const int s = it % NX, sb = it % NB;
+          // the tile slot was last used by step it - NX: wait until that step has been multiplied
+          if (it >= (uint32_t)NX && !(ok = ptx::mbar_wait(bar_empty_x((it - NX) % NB), ((it - NX) / NB) & 1, abort_flag))) break;
+          ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES);
           if (i < p.red_iters)
-            ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &act_map, i * TILE_J, m0, bar_full_x(s));
+            ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &act_map, i * TILE_J, m0, bar_full_x(sb));
           else
-            ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &lora_map, (i - p.red_iters) * TILE_J, m0, bar_full_x(s));
+            ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &lora_map, (i - p.red_iters) * TILE_J, m0, bar_full_x(sb));
         }
       }
     }
@@ -266,18 +271,18 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int i = 0; i < iters; ++i, ++it) {
-          const int sx = it % NX;
-          const uint32_t ph = (it / NX) & 1;
-          if (!(ok = ptx::mbar_wait(bar_full_x(sx), ph, abort_flag))) break;
+          const int sx = it % NX, sb = it % NB;
+          const uint32_t ph = (it / NB) & 1;
+          if (!(ok = ptx::mbar_wait(bar_full_x(sb), ph, abort_flag))) break;
           ptx::tc_fence_after();
           const uint32_t xs = smem_base + S::OFF_X + sx * ACT_BYTES;
-          const uint32_t as = smem_base + S::OFF_A + sx * ATILE_BYTES;
+          const uint32_t as = smem_base + S::OFF_A + sb * ATILE_BYTES;     // dx: NB == NX
 #pragma unroll
           for (int j = 0; j < TILE_J / 16; ++j) {
             const uint64_t bdesc = ptx::smem_desc(xs + j * 32, 16, 1024);
             const uint32_t acc = (i > 0 || j > 0) ? 1u : 0u;
             if (MODE == FWD) {
-              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + sx * 32 + j * 8, bdesc, IDESC_MAIN, acc);
+              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + sb * 32 + j * 8, bdesc, IDESC_MAIN, acc);
             } else if (i < p.red_iters) {
               // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO)
               ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 2048, 8192, 1024), bdesc, IDESC_MAIN, acc);
@@ -285,7 +290,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 32, 16, 1024), bdesc, IDESC_LORA, acc);
             }
           }
-          ptx::mma_commit(bar_empty_x(sx));        // frees the activation tile AND the operand slot
+          ptx::mma_commit(bar_empty_x(sb));        // frees the activation tile AND the operand slot
         }
         if (ok) ptx::mma_commit(bar_acc_full);
       }
@@ -305,10 +310,10 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       const int c0 = (tile % p.c_tiles) * TILE_C;
       for (int i = 0; i < iters; ++i, ++it) {
         if ((int)(it % DQ_GROUPS) != wg) continue;
-        const int sa = it % NX;
+        const int sa = it % NB;
         // operand slot first: once it is free every earlier step has been multiplied, so
         // the code ring's previous phase has certainly completed
-        if (!(ok = ptx::mbar_wait(bar_empty_x(sa), ((it / NX) & 1) ^ 1, abort_flag))) break;
+        if (!(ok = ptx::mbar_wait(bar_empty_x(sa), ((it / NB) & 1) ^ 1, abort_flag))) break;
         const uint32_t cst = (mit0 + i) / S::IPS;  // code stage counter (main steps only)
         const int sc = cst % NC;
         const int kb_base = MODE == FWD ? ((mit0 + i) % S::IPS) * 2 : 0;   // first k-block row of this step
