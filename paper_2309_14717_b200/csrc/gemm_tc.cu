@@ -95,24 +95,42 @@ struct Smem {
 };
 
 // ---- dequantization of one pack unit to 16 bf16x2 registers ------------------
-// A b-bit code c is moved to the top of an fp32 mantissa, giving v = 1 + c / 2^b
-// without any int-to-float conversion; then W~ = alpha*c + beta =
-// (2^b alpha) * v + (beta - 2^b alpha) is ONE fp32 FMA per element, and a pair of
-// results is rounded once to bf16x2.  alpha and beta stay in fp32, so the only
-// rounding is that of the final weight (rounding alpha or beta themselves would
-// put a common error on all channels of a group, which the pooled input
+// The two codes of a pair sit at the same bit offset of the two half-words, so one shift
+// and one LOP3 turn them into the bf16 pair (128 + c0, 128 + c1): the code is OR-ed into
+// the mantissa of bf16 128.0, no int-to-float conversion.  Widening each half to fp32 is
+// one more logic op, then W~ = alpha * (128 + c) + (beta - 128 alpha) is ONE fp32 FMA per
+// element, and the pair is rounded once to bf16x2.  alpha and beta stay in fp32, so the
+// only rounding that matters is that of the final weight (rounding alpha or beta
+// themselves would put a common error on all channels of a group, which the pooled input
 // amplifies).
+// The logic/shift pipe is the busiest one in these kernels.  A LOP3 takes at most one
+// immediate, so the masks live in registers (DqConsts, made opaque to the compiler):
+// "(a & mask) | magic" then is one instruction instead of two.
+struct DqConsts {
+  uint32_t mask, magic, himask, third;
+};
+template <int BITS>
+__device__ __forceinline__ DqConsts dq_consts() {
+  DqConsts c;
+  asm volatile("mov.b32 %0, %1;" : "=r"(c.mask) : "n"(BITS == 4 ? 0x000f000f : 0x00030003));
+  asm volatile("mov.b32 %0, 0x43004300;" : "=r"(c.magic));
+  asm volatile("mov.b32 %0, 0xffff0000;" : "=r"(c.himask));
+  asm volatile("mov.b32 %0, 0x00040004;" : "=r"(c.third));
+  return c;
+}
+__device__ __forceinline__ uint32_t lop_and_or(uint32_t a, uint32_t b, uint32_t c) {   // (a & b) | c
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t lop_and(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("and.b32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
 template <int SHIFT>   // positive: shift left
 __device__ __forceinline__ uint32_t shift_to(uint32_t w) {
   if constexpr (SHIFT >= 0) return w << SHIFT; else return w >> (-SHIFT);
-}
-// position e of a word whose codes are BITS wide at bit 16*(e&1) + BITS*(e>>1)
-template <int BITS, int E>
-__device__ __forceinline__ float code_as_1p(uint32_t w) {
-  constexpr int POS = 16 * (E & 1) + BITS * (E >> 1);
-  constexpr int TOP = 23 - BITS;
-  constexpr uint32_t MASK = ((1u << BITS) - 1u) << TOP;
-  return __uint_as_float((shift_to<TOP - POS>(w) & MASK) | 0x3f800000u);
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
@@ -133,36 +151,34 @@ __device__ __forceinline__ void load_unit(const uint32_t* cw, uint32_t* w) {
   }
 }
 
+// pair P of word I: positions (2P, 2P+1) of that word's codes
 template <int BITS, int I, int P>
-__device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, float a, float b) {
-  float v0, v1;
+__device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, float a, float b, const DqConsts& k) {
+  constexpr int W = BITS == 4 ? 4 : 2;             // width of the (low) code bits
+  uint32_t pr = lop_and_or(w[I] >> (W * P), k.mask, k.magic);
   if constexpr (BITS == 3) {
-    // low two bits from plane word I, the third bit from word 2 (bit 16*(j&1) + (j>>1), j = 16 I + 2 P + h)
-    constexpr int PL = 2 * P, PH = 8 * I + P;
-    v0 = __uint_as_float((shift_to<20 - PL>(w[I]) & 0x00300000u) | (shift_to<22 - PH>(w[2]) & 0x00400000u) | 0x3f800000u);
-    v1 = __uint_as_float((shift_to<20 - (16 + PL)>(w[I]) & 0x00300000u) | (shift_to<22 - (16 + PH)>(w[2]) & 0x00400000u) | 0x3f800000u);
-  } else {
-    v0 = code_as_1p<BITS, 2 * P>(w[I]);
-    v1 = code_as_1p<BITS, 2 * P + 1>(w[I]);
+    // third bits of the pair: bits PH and 16 + PH of word 2, PH = 8 I + P; they go to bit 2 of each half
+    constexpr int PH = 8 * I + P;
+    pr = lop_and_or(shift_to<2 - PH>(w[2]), k.third, pr);
   }
+  const float v0 = __uint_as_float(pr << 16), v1 = __uint_as_float(lop_and(pr, k.himask));   // 128 + c, exactly
   return pack_bf16x2(fmaf(a, v0, b), fmaf(a, v1, b));
 }
 
 template <int BITS, int I, int P>
-__device__ __forceinline__ void dq_all(const uint32_t* w, float a, float b, uint32_t* out) {
+__device__ __forceinline__ void dq_all(const uint32_t* w, float a, float b, const DqConsts& k, uint32_t* out) {
   constexpr int PAIRS = BITS == 4 ? 4 : 8;          // pairs per word
   constexpr int NWORDS = BITS == 4 ? 4 : 2;         // words that carry the (low) code bits
-  out[I * PAIRS + P] = dq_pair<BITS, I, P>(w, a, b);
-  if constexpr (P + 1 < PAIRS) dq_all<BITS, I, P + 1>(w, a, b, out);
-  else if constexpr (I + 1 < NWORDS) dq_all<BITS, I + 1, 0>(w, a, b, out);
+  out[I * PAIRS + P] = dq_pair<BITS, I, P>(w, a, b, k);
+  if constexpr (P + 1 < PAIRS) dq_all<BITS, I, P + 1>(w, a, b, k, out);
+  else if constexpr (I + 1 < NWORDS) dq_all<BITS, I + 1, 0>(w, a, b, k, out);
 }
 
 // out[q] = bf16x2 of positions (2q, 2q+1) of the unit, q = 0..15
 template <int BITS>
-__device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, uint32_t* out) {
-  const float a = ab.x * float(1 << BITS);          // exact
-  const float b = ab.y - a;
-  dq_all<BITS, 0, 0>(w, a, b, out);
+__device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, const DqConsts& k, uint32_t* out) {
+  const float b = fmaf(-128.f, ab.x, ab.y);
+  dq_all<BITS, 0, 0>(w, ab.x, b, k, out);
 }
 
 template <int BITS, int MODE>
@@ -303,6 +319,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     const int wg = (warp - 4) / 4;
     const int tw = threadIdx.x - 128 - wg * 128;  // 0..127 inside the warpgroup
     const int quarter = warp % 4;                // TMEM lane quarter of this warp
+    const DqConsts dk = dq_consts<BITS>();
     uint32_t it = 0, mit0 = 0;                    // reduction steps / main steps before this tile
     bool ok = true;
     const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block -> (alpha, beta) row of the stage
@@ -331,7 +348,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               uint32_t w[WORDS];
               load_unit<WORDS>(cw, w);
               const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[(kbl >> qsh) * TILE_C + row];
-              dequant_unit<BITS>(w, ab, v);
+              dequant_unit<BITS>(w, ab, dk, v);
             } else {
               // adapter step: row c of the operand is B[r0 + 0..63][c]; this thread packs 32 of them
               const int r0 = (i - p.red_iters) * TILE_J + half * 32;
@@ -360,7 +377,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               uint32_t w[WORDS];
               load_unit<WORDS>(cw, w);
               const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[(kbl >> qsh) * TILE_J + nl];
-              dequant_unit<BITS>(w, ab, v);
+              dequant_unit<BITS>(w, ab, dk, v);
               // MN-major, 128-byte swizzle: row = column nl (128 bytes = 64 channels),
               // this unit fills chunks (kbl%2)*4 .. +3 of block kbl/2
               uint8_t* rowp = atile + (kbl / 2) * 8192 + (nl / 8) * 1024 + (nl % 8) * 128;
