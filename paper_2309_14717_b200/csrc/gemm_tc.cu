@@ -282,31 +282,36 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       bool ok = true;
       // Issuing one tcgen05.mma costs this thread about 110 cycles and the four MMAs of a step
       // keep the tensor pipe busy for 512, so everything else in this loop has to stay short:
-      // one barrier wait, one fence, one commit per step.
+      // per step one fence and one block of instructions that probes the NEXT step's barrier,
+      // issues the four MMAs and the commit and then reads the probe (whose latency thus hides
+      // behind the issue); the blocking wait runs only when the probe said "not yet".
+      static_assert(TILE_J == 64, "the step helpers issue four K = 16 MMAs");
+      bool ready = false;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
         if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int i = 0; i < iters; ++i, ++it) {
           const int sx = it % NX, sb = it % NB;
           const uint32_t ph = (it / NB) & 1;
-          if (!(ok = ptx::mbar_wait(bar_full_x(sb), ph, abort_flag))) break;
+          if (!ready && !(ok = ptx::mbar_wait(bar_full_x(sb), ph, abort_flag))) break;
           ptx::tc_fence_after();
           const uint32_t xs = smem_base + S::OFF_X + sx * ACT_BYTES;
           const uint32_t as = smem_base + S::OFF_A + sb * ATILE_BYTES;     // dx: NB == NX
-#pragma unroll
-          for (int j = 0; j < TILE_J / 16; ++j) {
-            const uint64_t bdesc = ptx::smem_desc(xs + j * 32, 16, 1024);
-            const uint32_t acc = (i > 0 || j > 0) ? 1u : 0u;
-            if (MODE == FWD) {
-              ptx::mma_ts(tmem_base + ACC_COL, tmem_base + A_COL + sb * 32 + j * 8, bdesc, IDESC_MAIN, acc);
-            } else if (i < p.red_iters) {
-              // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO)
-              ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 2048, 8192, 1024), bdesc, IDESC_MAIN, acc);
-            } else {
-              ptx::mma_ss(tmem_base + ACC_COL, ptx::smem_desc(as + j * 32, 16, 1024), bdesc, IDESC_LORA, acc);
-            }
+          const uint64_t bdesc = ptx::smem_desc(xs, 16, 1024);             // + 32 bytes per K = 16 step
+          const uint32_t next_bar = bar_full_x((it + 1) % NB), next_par = ((it + 1) / NB) & 1;
+          const uint32_t acc = i > 0 ? 1u : 0u;
+          // the commit frees the activation tile AND the operand slot
+          if (MODE == FWD) {
+            ready = ptx::mma4_ts_commit_probe<2>(tmem_base + ACC_COL, tmem_base + A_COL + sb * 32, bdesc, IDESC_MAIN, acc,
+                                                 bar_empty_x(sb), next_bar, next_par) != 0;
+          } else if (i < p.red_iters) {
+            // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO); 2 KiB per step
+            ready = ptx::mma4_ss_commit_probe<128, 2>(tmem_base + ACC_COL, ptx::smem_desc(as, 8192, 1024), bdesc, IDESC_MAIN,
+                                                      acc, bar_empty_x(sb), next_bar, next_par) != 0;
+          } else {
+            ready = ptx::mma4_ss_commit_probe<2, 2>(tmem_base + ACC_COL, ptx::smem_desc(as, 16, 1024), bdesc, IDESC_LORA, acc,
+                                                    bar_empty_x(sb), next_bar, next_par) != 0;
           }
-          ptx::mma_commit(bar_empty_x(sb));        // frees the activation tile AND the operand slot
         }
         if (ok) ptx::mma_commit(bar_acc_full);
       }

@@ -188,6 +188,61 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// One reduction step in one instruction block: probe `next_bar` (the barrier the NEXT step
+// will need), issue four MMAs whose operands advance by fixed steps, commit to `commit_bar`,
+// and only then read the probe's answer.  A barrier probe takes a few hundred cycles to come
+// back; issued first and consumed last, its latency hides behind the MMA issue.
+// Returns non-zero if the phase `next_parity` of `next_bar` was already complete.
+// TS: A from TMEM (address step 8 columns per MMA), B descriptor step `B_STEP` (16-byte units).
+template <int B_STEP>
+__device__ __forceinline__ uint32_t mma4_ts_commit_probe(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                         uint32_t accumulate_first, uint32_t commit_bar,
+                                                         uint32_t next_bar, uint32_t next_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred p, q, t;\n\t.reg .b32 a1, a2, a3;\n\t.reg .b64 b1, b2, b3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 q, [%7], %8;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "setp.eq.b32 t, 0, 0;\n\t"
+      "add.u32 a1, %2, 8;\n\tadd.u32 a2, %2, 16;\n\tadd.u32 a3, %2, 24;\n\t"
+      "add.u64 b1, %3, %9;\n\tadd.u64 b2, b1, %9;\n\tadd.u64 b3, b2, %9;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], [%2], %3, %4, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], [a1], b1, %4, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], [a2], b2, %4, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], [a3], b3, %4, t;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];\n\t"
+      "selp.b32 %0, 1, 0, q;\n\t}"
+      : "=r"(ready)
+      : "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate_first), "r"(commit_bar), "r"(next_bar),
+        "r"(next_parity), "n"(B_STEP)
+      : "memory");
+  return ready;
+}
+// SS: A and B descriptors advance by `A_STEP` / `B_STEP` (16-byte units) per MMA.
+template <int A_STEP, int B_STEP>
+__device__ __forceinline__ uint32_t mma4_ss_commit_probe(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                         uint32_t accumulate_first, uint32_t commit_bar,
+                                                         uint32_t next_bar, uint32_t next_parity) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred p, q, t;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 q, [%7], %8;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "setp.eq.b32 t, 0, 0;\n\t"
+      "add.u64 a1, %2, %9;\n\tadd.u64 a2, a1, %9;\n\tadd.u64 a3, a2, %9;\n\t"
+      "add.u64 b1, %3, %10;\n\tadd.u64 b2, b1, %10;\n\tadd.u64 b3, b2, %10;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], a1, b1, %4, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], a2, b2, %4, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], a3, b3, %4, t;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];\n\t"
+      "selp.b32 %0, 1, 0, q;\n\t}"
+      : "=r"(ready)
+      : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate_first), "r"(commit_bar), "r"(next_bar),
+        "r"(next_parity), "n"(A_STEP), "n"(B_STEP)
+      : "memory");
+  return ready;
+}
 // Arrives on `bar` once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
