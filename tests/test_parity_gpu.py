@@ -93,6 +93,10 @@ SMALL = [
     ("tc3", 384, 256, 64, 3, 24, 0.75, 270),
     ("tc2", 256, 128, 128, 2, 8, 2.0, 515),
     ("tc4_r0pad", 1024, 640, 32, 4, 72, 1.0, 1000),
+    # many-row pooling kernel (M >= 64, K % 256 == 0) with few, many and more-than-a-block's adapter columns
+    ("pool_r8", 512, 256, 32, 4, 8, 1.0, 100),
+    ("pool_r128", 768, 256, 64, 4, 128, 0.5, 70),
+    ("pool_r256", 1024, 128, 128, 2, 256, 1.0, 65),
 ]
 
 
