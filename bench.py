@@ -347,14 +347,14 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-def small_m_bandwidth(Q, torch, pk, shape=SMALL_M, ms=(1, 4, 16)):
+def small_m_bandwidth(Q, torch, pk, shape=SMALL_M, ms=(1, 4, 16), cfg=None):
     """Few-token forward of one layer shape, rotating over enough weight copies
     (> 4 x L2) that the codes stream from HBM.  The rotation is captured once in
     a CUDA graph and replayed, so that the GPU and not the host's launch rate is
     timed.  Reported for the adapted layer (pool/adapter pre-kernel + main
     kernel per call) and for the merged, deployed layer (one kernel per call)."""
     from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
-    cfg = CONFIGS[shape]
+    cfg = CONFIGS[shape] if cfg is None else cfg
     t = make_inputs(cfg.with_(tokens=max(ms)), need=("W", "x", "A", "B"))
     d = Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, cfg.rank, cfg.scale)
     d0 = Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, 0, cfg.scale)
@@ -453,8 +453,77 @@ def run_only(args):
                       "status": Q.workspace_status(wb if args.only == "bwd" else wf)}))
 
 
+def run_table(args):
+    """Every benchmark configuration in turn (one layer at a time): forward and backward
+    at the configuration's token count, and the merged one-token forward of the 65B shapes
+    per group size.  Prints a markdown table; times are medians of CUDA-event timed calls."""
+    import statistics
+
+    import torch
+
+    from paper_2309_14717_b200 import binding as Q
+    from paper_2309_14717_b200 import build as _build
+    from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
+
+    _build.build()
+    pk = peaks()
+    cases = [(CONFIGS[n], 8192) for n in ("cfg3_7b_up", "cfg3_7b_down")]
+    for bits in (3, 2):
+        cases += [(CONFIGS[n].with_(bits=bits), 4096) for n in ("cfg4_13b_up", "cfg4_13b_down", "cfg4_13b_attn")]
+    for g in (32, 64, 128):
+        cases += [(CONFIGS[n].with_(group_size=g), 8192) for n in ("cfg5_65b_up", "cfg5_65b_down", "cfg5_65b_attn")]
+    print("| layer | bits | g | M | forward ms | TFLOP/s | of sustained bf16 peak | backward ms | TFLOP/s | of peak | fwd+bwd TFLOP/s | of peak |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for cfg0, M in cases:
+        cfg = cfg0.with_(tokens=M)
+        t = {k: v.cuda() for k, v in make_inputs(cfg).items()}
+        K, N, G, r = cfg.d_in, cfg.d_out, cfg.groups, cfg.rank
+        d = Q.desc(K, N, cfg.group_size, cfg.bits, r, cfg.scale)
+        codes, qparams = Q.alloc_packed(d)
+        Q.qalora_quantize(d, t["W"], codes, qparams)
+        del t["W"]
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dA = torch.empty((G, r), dtype=torch.float32, device="cuda")
+        dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
+        wf, wb = Q.alloc_workspace(d, M, Q.OP_FORWARD), Q.alloc_workspace(d, M, Q.OP_BACKWARD)
+        res = {}
+        for op in ("fwd", "bwd"):
+            ts = []
+            for _ in range(3 + 7):
+                e0.record()
+                if op == "fwd":
+                    Q.qalora_forward(d, M, t["x"], codes, qparams, t["A"], t["B"], y, wf)
+                else:
+                    Q.qalora_backward(d, M, t["x"], t["dy"], codes, qparams, t["A"], t["B"], dx, dA, dB, wb)
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            res[op] = statistics.median(ts[3:])
+        assert Q.workspace_status(wf) == 0 and Q.workspace_status(wb) == 0
+        ff, fb = fwd_flops(M, K, N, G, r), bwd_flops(M, K, N, G, r)
+        tf, tb = ff / res["fwd"] / 1e9, fb / res["bwd"] / 1e9
+        tt = (ff + fb) / (res["fwd"] + res["bwd"]) / 1e9
+        print(f"| {cfg.name} | {cfg.bits} | {cfg.group_size} | {M} | {res['fwd']:.3f} | {tf:.0f} | {tf / pk['tensor']:.2f} | "
+              f"{res['bwd']:.3f} | {tb:.0f} | {tb / pk['tensor']:.2f} | {tt:.0f} | {tt / pk['tensor']:.2f} |", flush=True)
+        del t, codes, qparams, y, dx, wf, wb
+        torch.cuda.empty_cache()
+    print()
+    print("| layer | g | merged M = 1 forward us | GB/s | of measured copy bandwidth |")
+    print("|---|---|---|---|---|")
+    for g in (32, 64, 128):
+        for n in ("cfg5_65b_up", "cfg5_65b_down", "cfg5_65b_attn"):
+            rr = small_m_bandwidth(Q, torch, pk, ms=(1,), cfg=CONFIGS[n].with_(group_size=g))["M1_merged"]
+            print(f"| {n} | {g} | {rr['us_per_call']:.1f} | {rr['GB/s']:.0f} | {rr['frac_of_hbm']:.2f} |", flush=True)
+            torch.cuda.empty_cache()
+    print()
+    print(f"peaks: bf16 {pk['tensor']:.0f} TFLOP/s, HBM {pk['hbm']:.0f} GB/s ({pk['source']})")
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--table", action="store_true", help="per-configuration throughput table (markdown)")
     ap.add_argument("--only", default=None, choices=("fwd", "bwd", "gemv", "quantize", "merge"))
     ap.add_argument("--shape", default="cfg3_7b_up")
     ap.add_argument("--tokens", type=int, default=4096)
@@ -463,7 +532,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     args = ap.parse_args()
-    if args.only is not None:
+    if args.table:
+        run_table(args)
+    elif args.only is not None:
         run_only(args)
     elif args.impl == "reference":
         run_reference(args)
