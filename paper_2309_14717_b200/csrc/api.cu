@@ -36,6 +36,9 @@ int check_desc(const qalora_desc* d, Shape* sh) {
   return QALORA_OK;
 }
 
+// Token counts up to this take the bandwidth-bound small-M path.
+static constexpr int64_t kSmallM = 16;
+
 Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   Workspace w{};
   size_t off = 0;
@@ -59,6 +62,7 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   }
   w.partial_bytes = pb;
   w.partial = take(pb);
+  w.fwd_parts = take(!bwd && m > kSmallM && tc_forward_supported(sh, m) ? tc_forward_partial_bytes(sh, m) : 0);
   w.total = off;
   return w;
 }
@@ -67,8 +71,6 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
 
 using namespace qalora;
 
-// Token counts up to this take the bandwidth-bound small-M path.
-static constexpr int64_t kSmallM = 16;
 
 extern "C" {
 
@@ -179,7 +181,7 @@ int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void
     if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
     return launch_tc_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
                              reinterpret_cast<const float2*>(qparams), Tb, static_cast<const __nv_bfloat16*>(B),
-                             static_cast<__nv_bfloat16*>(y), status, stream);
+                             static_cast<__nv_bfloat16*>(y), reinterpret_cast<float*>(wsp + ws.fwd_parts), status, stream);
   }
   return launch_simt_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
                              reinterpret_cast<const float2*>(qparams), T, static_cast<const __nv_bfloat16*>(B),

@@ -33,6 +33,7 @@ struct Workspace {
   size_t dTb;       // bf16   [M][r]   dT rounded
   size_t partial;   // float  split-K / split-M partial sums
   size_t partial_bytes;
+  size_t fwd_parts; // float  [parts][M][N] partial results of a forward reduction cut into parts (forward)
   size_t total;
 };
 Workspace workspace_layout(const Shape& sh, int64_t m, int op);
@@ -99,9 +100,10 @@ int launch_atb_f32(int64_t M, int P, int Q, const float* X, const float* Y, floa
 // Tensor-core paths (gemm_tc.cu).  Tb / dTb are the bf16 rank-r intermediates.
 bool tc_forward_supported(const Shape& sh, int64_t M);
 bool tc_dx_supported(const Shape& sh, int64_t M);
+size_t tc_forward_partial_bytes(const Shape& sh, int64_t M);   // scratch for a reduction cut into parts (few tokens)
 int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
                       const float2* qparams, const __nv_bfloat16* Tb, const __nv_bfloat16* B,
-                      __nv_bfloat16* y, int* status, cudaStream_t st);
+                      __nv_bfloat16* y, float* partial, int* status, cudaStream_t st);
 int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint32_t* codes,
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
                  __nv_bfloat16* dx, int* status, cudaStream_t st);

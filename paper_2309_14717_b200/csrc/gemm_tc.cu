@@ -33,13 +33,13 @@ namespace {
 
 constexpr int TILE_C = 128;      // out channels per tile   (MMA M)
 constexpr int TILE_T = 256;      // tokens per tile         (MMA N)
+constexpr int TILE_T_FEW = 64;   // tokens per tile of the forward variant for at most 64 tokens
 constexpr int TILE_J = 64;       // reduction step per stage
 constexpr int DQ_GROUPS = 4;     // dequantizing warpgroups
 constexpr int THREADS = 128 + 128 * DQ_GROUPS + 128;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_COL = 0;       // accumulator: columns [0, 256)
 constexpr int A_COL = 256;       // forward operand ring: 8 slots of 32 columns
-constexpr uint32_t ACT_BYTES = TILE_T * TILE_J * 2;      // 32 KiB activation tile
 constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx)
 
 enum Mode { FWD = 0, DX = 1 };
@@ -55,8 +55,41 @@ struct TcParams {
   int c_tiles, m_tiles;        // tiles along out channels / tokens
   int red_iters, lora_iters;   // main / adapter reduction steps per tile
   int qp_rows;                 // rows of (alpha, beta) per code stage: 128 / g
+  int ksplit;                  // parts the reduction of a tile is cut into (1: none)
+  int tile_t;                  // tokens per tile: TILE_T, or TILE_T_FEW (forward, M <= 64; always with parts)
+  float* partial;              // ksplit > 1: fp32 [ksplit][M][ld_out] partial results
   int* status;                 // device word: set to 1 when a wait timed out
 };
+
+// Work item of a block: part `sp` of tile `tile`, i.e. the main steps mb .. mb + n_main - 1
+// and, for the last part, the adapter steps; n_steps in all.  Parts begin on even steps (a
+// forward code stage feeds two).
+struct TcSegment {
+  int tile, sp, mb, n_main, n_steps;
+};
+template <bool PARTS>
+__device__ __forceinline__ TcSegment tc_segment(const TcParams& p, int vt) {
+  TcSegment g;
+  g.tile = PARTS ? vt / p.ksplit : vt;
+  g.sp = PARTS ? vt % p.ksplit : 0;
+  if (!PARTS) {
+    g.mb = 0;
+    g.n_main = p.red_iters;
+    g.n_steps = p.red_iters + p.lora_iters;
+  } else {
+    const long long pairs = p.red_iters / 2;
+    g.mb = 2 * (int)(pairs * g.sp / p.ksplit);
+    g.n_main = 2 * (int)(pairs * (g.sp + 1) / p.ksplit) - g.mb;
+    g.n_steps = g.n_main + (g.sp == p.ksplit - 1 ? p.lora_iters : 0);
+  }
+  return g;
+}
+// j-th step of a segment -> step index of the tile (main steps 0 .. red_iters - 1, then the adapter steps)
+template <bool PARTS>
+__device__ __forceinline__ int tc_step(const TcParams& p, const TcSegment& g, int j) {
+  if (!PARTS) return j;
+  return j < g.n_main ? g.mb + j : p.red_iters + (j - g.n_main);
+}
 
 // Rings, decoupled so that each covers its own latency:
 //   NX activation tiles (TMA, 32 KiB each);
@@ -70,12 +103,13 @@ struct TcParams {
 //      that run further ahead.
 // NB and NC are multiples of DQ_GROUPS, so a ring slot always belongs to the same
 // dequantizing warpgroup and its barrier phases are waited on in order.
-template <int BITS, int MODE>
+template <int BITS, int MODE, int TT = TILE_T>   // TT: tokens per tile (MMA N): 256, or 64 for the few-token variant
 struct Smem {
+  static constexpr uint32_t ACT_BYTES = TT * TILE_J * 2;                         // activation tile: 32 KiB (8 KiB)
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   static constexpr int NX = 4;
   static constexpr int NB = MODE == FWD ? 8 : 4;
-  static constexpr int NC = 4;
+  static constexpr int NC = TT == TILE_T ? 4 : 12;                               // small activation tiles leave room for a deep code ring
   static constexpr int IPS = MODE == FWD ? 2 : 1;                                // reduction steps per code stage
   static constexpr int TILE_NC = MODE == FWD ? TILE_C : TILE_J;                  // columns of a code stage
   static constexpr int NOUT = MODE == FWD ? 2 : 1;                               // epilogue staging buffers
@@ -181,14 +215,16 @@ __device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, const
   dq_all<BITS, 0, 0>(w, ab.x, b, k, out);
 }
 
-template <int BITS, int MODE>
+// PARTS: every tile's reduction is cut into p.ksplit parts.  TT: tokens per tile.
+template <int BITS, int MODE, bool PARTS, int TT>
 __global__ void __launch_bounds__(THREADS, 1)
 qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_constant__ CUtensorMap lora_map,
                  const __grid_constant__ CUtensorMap out_map, const __grid_constant__ CUtensorMap codes_map,
                  const __grid_constant__ CUtensorMap qp_map, const TcParams p) {
-  using S = Smem<BITS, MODE>;
+  using S = Smem<BITS, MODE, TT>;
   constexpr int WORDS = S::WORDS;
   constexpr int NX = S::NX, NB = S::NB, NC = S::NC;
+  constexpr uint32_t ACT_BYTES = S::ACT_BYTES;
   extern __shared__ uint8_t smem_raw[];
   // aligned by pointer arithmetic on the __shared__ array, so that the accesses stay shared-space loads/stores
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -230,17 +266,18 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int total_tiles = p.c_tiles * p.m_tiles;
-  const int iters = p.red_iters + p.lora_iters;
+  const int total_tiles = p.c_tiles * p.m_tiles * (PARTS ? p.ksplit : 1);      // work items: (tile, part)
 
   if (warp == 0) {
     // ------------------------------------------------- activation producer ----
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile / p.c_tiles) * TILE_T;
-        for (int i = 0; i < iters; ++i, ++it) {
+      for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x) {
+        const TcSegment sg = tc_segment<PARTS>(p, vt);
+        const int m0 = (sg.tile / p.c_tiles) * TT;
+        for (int j = 0; j < sg.n_steps; ++j, ++it) {
+          const int i = tc_step<PARTS>(p, sg, j);
           const int s = it % NX, sb = it % NB;
           // the tile slot was last used by step it - NX: wait until that step has been multiplied
           if (it >= (uint32_t)NX && !(ok = ptx::mbar_wait(bar_empty_x((it - NX) % NB), ((it - NX) / NB) & 1, abort_flag))) break;
@@ -257,10 +294,11 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     if (lane == 0) {
       uint32_t cit = 0;                              // code stages issued so far
       bool ok = true;
-      const int stages_per_tile = p.red_iters / S::IPS;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int c0 = (tile % p.c_tiles) * TILE_C;
-        for (int cs = 0; cs < stages_per_tile; ++cs, ++cit) {
+      for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x) {
+        const TcSegment sg = tc_segment<PARTS>(p, vt);
+        const int c0 = (sg.tile % p.c_tiles) * TILE_C;
+        const int cs_end = (sg.mb + sg.n_main) / S::IPS;
+        for (int cs = sg.mb / S::IPS; cs < cs_end; ++cs, ++cit) {
           const int s = cit % NC;
           if (!(ok = ptx::mbar_wait(bar_empty_c(s), ((cit / NC) & 1) ^ 1, abort_flag))) break;
           const uint32_t stage = smem_base + S::OFF_C + s * S::CSTAGE_BYTES;
@@ -276,8 +314,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer ----
     if (lane == 0) {
-      constexpr uint32_t IDESC_MAIN = ptx::idesc_bf16(TILE_C, TILE_T, MODE == DX, false);
-      constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(TILE_C, TILE_T, false, false);
+      constexpr uint32_t IDESC_MAIN = ptx::idesc_bf16(TILE_C, TT, MODE == DX, false);
+      constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(TILE_C, TT, false, false);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       // Issuing one tcgen05.mma costs this thread about 110 cycles and the four MMAs of a step
@@ -287,10 +325,11 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       // behind the issue); the blocking wait runs only when the probe said "not yet".
       static_assert(TILE_J == 64, "the step helpers issue four K = 16 MMAs");
       bool ready = false;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x, ++tcount) {
+        const TcSegment sg = tc_segment<PARTS>(p, vt);
         if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
-        for (int i = 0; i < iters; ++i, ++it) {
+        for (int j = 0; j < sg.n_steps; ++j, ++it) {
           const int sx = it % NX, sb = it % NB;
           const uint32_t ph = (it / NB) & 1;
           if (!ready && !(ok = ptx::mbar_wait(bar_full_x(sb), ph, abort_flag))) break;
@@ -299,12 +338,12 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           const uint32_t as = smem_base + S::OFF_A + sb * ATILE_BYTES;     // dx: NB == NX
           const uint64_t bdesc = ptx::smem_desc(xs, 16, 1024);             // + 32 bytes per K = 16 step
           const uint32_t next_bar = bar_full_x((it + 1) % NB), next_par = ((it + 1) / NB) & 1;
-          const uint32_t acc = i > 0 ? 1u : 0u;
+          const uint32_t acc = j > 0 ? 1u : 0u;
           // the commit frees the activation tile AND the operand slot
           if (MODE == FWD) {
             ready = ptx::mma4_ts_commit_probe<2>(tmem_base + ACC_COL, tmem_base + A_COL + sb * 32, bdesc, IDESC_MAIN, acc,
                                                  bar_empty_x(sb), next_bar, next_par) != 0;
-          } else if (i < p.red_iters) {
+          } else if (j < sg.n_main) {
             // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO); 2 KiB per step
             ready = ptx::mma4_ss_commit_probe<128, 2>(tmem_base + ACC_COL, ptx::smem_desc(as, 8192, 1024), bdesc, IDESC_MAIN,
                                                       acc, bar_empty_x(sb), next_bar, next_par) != 0;
@@ -328,17 +367,19 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     uint32_t it = 0, mit0 = 0;                    // reduction steps / main steps before this tile
     bool ok = true;
     const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block -> (alpha, beta) row of the stage
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, mit0 += p.red_iters) {
-      const int c0 = (tile % p.c_tiles) * TILE_C;
-      for (int i = 0; i < iters; ++i, ++it) {
+    for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x) {
+      const TcSegment sg = tc_segment<PARTS>(p, vt);
+      const int c0 = (sg.tile % p.c_tiles) * TILE_C;
+      for (int j = 0; j < sg.n_steps; ++j, ++it) {
         if ((int)(it % DQ_GROUPS) != wg) continue;
+        const int i = tc_step<PARTS>(p, sg, j);
         const int sa = it % NB;
         // operand slot first: once it is free every earlier step has been multiplied, so
         // the code ring's previous phase has certainly completed
         if (!(ok = ptx::mbar_wait(bar_empty_x(sa), ((it / NB) & 1) ^ 1, abort_flag))) break;
-        const uint32_t cst = (mit0 + i) / S::IPS;  // code stage counter (main steps only)
+        const uint32_t cst = (mit0 + j) / S::IPS;  // code stage counter (main steps only; mit0 stays even)
         const int sc = cst % NC;
-        const int kb_base = MODE == FWD ? ((mit0 + i) % S::IPS) * 2 : 0;   // first k-block row of this step
+        const int kb_base = MODE == FWD ? ((mit0 + j) % S::IPS) * 2 : 0;   // first k-block row of this step
         if (i < p.red_iters && !(ok = ptx::mbar_wait(bar_full_c(sc), (cst / NC) & 1, abort_flag))) break;
         const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         if (MODE == FWD) {
@@ -414,6 +455,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           if (i < p.red_iters) ptx::mbar_arrive(bar_empty_c(sc));
         }
       }
+      mit0 += sg.n_main;
     }
   } else if (warp >= 4 + 4 * DQ_GROUPS) {
     // ------------------------------------------------------------ epilogue ----
@@ -427,19 +469,29 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     const int ch = quarter * 32 + lane;
     uint32_t tcount = 0, chunk = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+    for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x, ++tcount) {
+      const int tile = PARTS ? vt / p.ksplit : vt, sp = PARTS ? vt % p.ksplit : 0;
       const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
       if (!(ok = ptx::mbar_wait(bar_acc_full, tcount & 1, abort_flag))) break;
       ptx::tc_fence_after();
 #pragma unroll 1
-      for (int col = 0; col < TILE_T; col += 32, ++chunk) {
+      for (int col = 0; col < TT; col += 32, ++chunk) {
         uint32_t v[32];
         ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ACC_COL + col, v);
         ptx::tmem_wait_ld();
-        if (col == TILE_T - 32) {                 // all columns read: hand the accumulator back
+        if (col == TT - 32) {                     // all columns read: hand the accumulator back
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(bar_acc_empty);
+        }
+        if constexpr (PARTS) {
+          // a part of the reduction: fp32 partial results [part][token][channel], added up by
+          // sum_parts_kernel; a warp writes 32 neighbouring channels of one token per store
+          float* dst = p.partial + ((size_t)sp * p.M + (size_t)mt * TT + col) * p.ld_out + ct * TILE_C + ch;
+#pragma unroll
+          for (int t = 0; t < 32; ++t)
+            if ((long long)mt * TT + col + t < p.M) dst[(size_t)t * p.ld_out] = __uint_as_float(v[t]);
+          continue;
         }
         uint8_t* stg = smem + S::OFF_OUT + (chunk % S::NOUT) * S::OUT_BYTES;
         ptx::named_barrier(1, 128);               // the staging tile's previous store has been read out
@@ -448,8 +500,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           reinterpret_cast<__nv_bfloat16*>(stg)[t * TILE_C + ch] = __float2bfloat16_rn(__uint_as_float(v[t]));
         ptx::fence_proxy_async();
         ptx::named_barrier(2, 128);
-        if (et == 0 && (long long)mt * TILE_T + col < p.M) {
-          ptx::tma_store_2d(&out_map, ct * TILE_C, mt * TILE_T + col, ptx::smem_u32(stg));
+        if (et == 0 && (long long)mt * TT + col < p.M) {
+          ptx::tma_store_2d(&out_map, ct * TILE_C, mt * TT + col, ptx::smem_u32(stg));
           ptx::bulk_commit_group();
           ptx::bulk_wait_group_read<S::NOUT - 1>();
         }
@@ -486,14 +538,14 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 matrix [rows][cols] row-major, box = 64 columns x 256 rows, 128-byte swizzle;
+// bf16 matrix [rows][cols] row-major, box = 64 columns x `box_rows` rows, 128-byte swizzle;
 // out-of-range rows and columns read as zero.
-bool make_act_map(CUtensorMap* map, const void* base, long long rows, int cols) {
+bool make_act_map(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows = TILE_T) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {TILE_J, TILE_T};
+  cuuint32_t box[2] = {TILE_J, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -549,27 +601,58 @@ bool make_qp_map(CUtensorMap* map, const float2* qp, int G, int N, int tile_cols
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BITS, int MODE>
-int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
-  using S = Smem<BITS, MODE>;
+// out[i] = bf16(sum over parts of partial[part][i]), added in part order; 8 elements per thread
+__global__ void __launch_bounds__(256)
+sum_parts_kernel(const float* __restrict__ partial, __nv_bfloat16* __restrict__ out, size_t count, int parts) {
+  const size_t i0 = ((size_t)blockIdx.x * 256 + threadIdx.x) * 8;
+  if (i0 >= count) return;                                   // count is a multiple of 8
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int s = 0; s < parts; ++s) {
+    const float4 a = *reinterpret_cast<const float4*>(partial + (size_t)s * count + i0);
+    const float4 b = *reinterpret_cast<const float4*>(partial + (size_t)s * count + i0 + 4);
+    acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+    acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+  }
+  uint4 o;
+  o.x = pack_bf16x2(acc[0], acc[1]); o.y = pack_bf16x2(acc[2], acc[3]);
+  o.z = pack_bf16x2(acc[4], acc[5]); o.w = pack_bf16x2(acc[6], acc[7]);
+  *reinterpret_cast<uint4*>(out + i0) = o;
+}
+
+template <int BITS, int MODE, bool PARTS, int TT>
+int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
+  using S = Smem<BITS, MODE, TT>;
   CUtensorMap out, cmap, qmap;
   if (!make_out_map(&out, p.out, p.M, p.ld_out)) return QALORA_ERR_CUDA;
   if (!make_codes_map(&cmap, p.codes, p.K, p.N, BITS, S::TILE_NC)) return QALORA_ERR_CUDA;
   if (!make_qp_map(&qmap, p.qparams, p.K / p.g, p.N, S::TILE_NC, p.qp_rows)) return QALORA_ERR_CUDA;
   static_assert(S::TOTAL <= 232448, "shared memory budget");
-  auto kern = qalora_tc_kernel<BITS, MODE>;
+  auto kern = qalora_tc_kernel<BITS, MODE, PARTS, TT>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
   if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
-  const int tiles = p.c_tiles * p.m_tiles;
+  const int tiles = p.c_tiles * p.m_tiles * p.ksplit;
   const int grid = tiles < sm_count() ? tiles : sm_count();
   {
     MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
     kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, out, cmap, qmap, p);
   }
   count_launch();
+  if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
+  if (PARTS) {
+    const size_t count = (size_t)p.M * p.ld_out;
+    sum_parts_kernel<<<(unsigned)((count / 8 + 255) / 256), 256, 0, st>>>(p.partial, p.out, count, p.ksplit);
+    count_launch();
+  }
   return cuda_status(cudaGetLastError());
+}
+
+template <int BITS, int MODE>
+int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
+  if (MODE == FWD && p.tile_t == TILE_T_FEW) return launch_tc_t<BITS, FWD, true, TILE_T_FEW>(act, lora, p, st);
+  if (MODE == FWD && p.ksplit > 1) return launch_tc_t<BITS, FWD, true, TILE_T>(act, lora, p, st);
+  return launch_tc_t<BITS, MODE, false, TILE_T>(act, lora, p, st);
 }
 
 }  // namespace
@@ -583,20 +666,61 @@ bool tc_dx_supported(const Shape& sh, int64_t M) {
   return tc_group_ok(sh.g) && sh.K % TILE_C == 0 && sh.N % TILE_J == 0 && M >= 1 && M <= 0x7fffffffLL / 2 && encode_fn() != nullptr;
 }
 
+// Parts the forward reduction is cut into.  With few tokens a layer has fewer (or not many
+// more) 128 x 256 tiles than the GPU has SMs; cutting every tile's reduction into parts fills
+// the SMs and evens out the last wave.  The parts meet as fp32 partial results in scratch.
+int tc_forward_parts(const Shape& sh, int64_t M) {
+  if (M > 512) return 1;
+  if (M <= TILE_T_FEW && sh.K / TILE_J >= 8) {
+    // the 64-token variant always writes partial results; as many parts as fill the SMs evenly
+    const long long tiles = sh.N / TILE_C;
+    const int steps = sh.K / TILE_J, sms = sm_count();
+    int best = 1;
+    double best_cost = 1e30;
+    for (int ks = 1; ks <= 8; ++ks) {
+      if (ks > 1 && steps / ks < 8) break;
+      const double cost = (double)((tiles * ks + sms - 1) / sms) / ks + 0.02 * ks;
+      if (cost < best_cost - 1e-9) { best_cost = cost; best = ks; }
+    }
+    return -best;                                              // negative: the 64-token variant
+  }
+  const long long tiles = (long long)(sh.N / TILE_C) * ((M + TILE_T - 1) / TILE_T);
+  const int steps = sh.K / TILE_J, sms = sm_count();
+  if (tiles * 4 > sms) return 1;          // enough tiles: the parts' extra epilogues and scratch traffic cost more than they save
+  int best = 1;
+  double best_cost = (double)((tiles + sms - 1) / sms);          // waves x (share of a tile per wave)
+  for (int ks = 2; ks <= 6; ++ks) {
+    if (steps / ks < 8) break;
+    if ((size_t)ks * M * sh.N * sizeof(float) > ((size_t)256 << 20)) break;
+    const double cost = (double)((tiles * ks + sms - 1) / sms) / ks + 0.02 * ks;   // + per-part start-up
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = ks; }
+  }
+  return best;
+}
+size_t tc_forward_partial_bytes(const Shape& sh, int64_t M) {
+  const int ks = tc_forward_parts(sh, M);
+  if (ks < 0) return (size_t)(-ks) * M * sh.N * sizeof(float);
+  return ks > 1 ? (size_t)ks * M * sh.N * sizeof(float) : 0;
+}
+
 // y = x * W~ + Tb * B with Tb = bf16(s * pool(x) * A) precomputed ([M][r]).
+// `partial`: tc_forward_partial_bytes() of scratch.
 int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
                       const float2* qparams, const __nv_bfloat16* Tb, const __nv_bfloat16* B,
-                      __nv_bfloat16* y, int* status, cudaStream_t st) {
+                      __nv_bfloat16* y, float* partial, int* status, cudaStream_t st) {
+  const int parts = tc_forward_parts(sh, M);
+  const int tile_t = parts < 0 ? TILE_T_FEW : TILE_T;
   CUtensorMap act, lora;
-  if (!make_act_map(&act, x, M, sh.K)) return QALORA_ERR_CUDA;
+  if (!make_act_map(&act, x, M, sh.K, tile_t)) return QALORA_ERR_CUDA;
   lora = act;
-  if (sh.r > 0 && !make_act_map(&lora, Tb, M, sh.r)) return QALORA_ERR_CUDA;
+  if (sh.r > 0 && !make_act_map(&lora, Tb, M, sh.r, tile_t)) return QALORA_ERR_CUDA;
   TcParams p{};
   p.codes = codes; p.qparams = qparams; p.lora = B; p.out = y;
   p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.N;
-  p.c_tiles = sh.N / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
+  p.c_tiles = sh.N / TILE_C; p.m_tiles = (int)((M + tile_t - 1) / tile_t);
   p.red_iters = sh.K / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
   p.status = status; p.qp_rows = 128 / sh.g;
+  p.ksplit = parts < 0 ? -parts : parts; p.tile_t = tile_t; p.partial = partial;
   if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, p, st);
   return launch_tc<2, FWD>(act, lora, p, st);
@@ -616,6 +740,7 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
   p.c_tiles = sh.K / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
   p.red_iters = sh.N / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
   p.status = status; p.qp_rows = 128 / sh.g;
+  p.ksplit = 1; p.tile_t = TILE_T; p.partial = nullptr;
   if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);
   return launch_tc<2, DX>(act, lora, p, st);

@@ -97,6 +97,10 @@ SMALL = [
     ("pool_r8", 512, 256, 32, 4, 8, 1.0, 100),
     ("pool_r128", 768, 256, 64, 4, 128, 0.5, 70),
     ("pool_r256", 1024, 128, 128, 2, 256, 1.0, 65),
+    # few tokens and a long reduction: the forward contraction is cut into parts that meet in scratch
+    ("parts4", 2048, 256, 32, 4, 16, 1.0, 40),
+    ("parts3", 1536, 384, 64, 3, 24, 0.75, 300),
+    ("parts2", 4096, 128, 128, 2, 8, 1.5, 17),
 ]
 
 
