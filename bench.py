@@ -36,6 +36,15 @@ SMALL_M = "cfg2_7b_attn"
 
 
 # ----------------------------------------------------------- work accounting --
+# DRAM traffic of ONE launch of the forward contraction kernel at the benchmark size
+# (4096 -> 11008, M = 8192), from a one-pass ncu capture of
+#   python bench.py --only fwd --tokens 8192 --steps 3
+# with --metrics dram__bytes_read.sum,dram__bytes_write.sum (156.8 MB read + 155.6 MB
+# written; algorithmic 282.7 MB).  Counters of the kernel as it stands; set to None when
+# qalora_tc_kernel changes until they have been taken again.
+FWD_KERNEL_DRAM_BYTES = 312.4e6
+
+
 def fwd_flops(M, K, N, G, r):
     return 2 * M * K * N + M * K + 2 * M * G * r + 2 * M * r * N
 
@@ -309,7 +318,8 @@ def run_gpu(args):
     achieved = s0.main_flops / (kms / 1e3) / 1e12
     roofline = {"bound": "tensor", "kernel": kernel_name, "achieved": achieved, "peak": pk["tensor"],
                 "unit": "TFLOP/s", "frac": achieved / pk["tensor"], "peak_source": pk["source"] + " (sustained bf16)",
-                "kernel_ms": kms, "launches_timed": len(probe_pairs), "traffic": None,
+                "kernel_ms": kms, "launches_timed": len(probe_pairs), "traffic": FWD_KERNEL_DRAM_BYTES,
+                "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum)",
                 "flops_per_launch": s0.main_flops}
 
     # single-token forward of the merged layer: HBM-bound leg of the metric
