@@ -101,6 +101,10 @@ SMALL = [
     ("parts4", 2048, 256, 32, 4, 16, 1.0, 40),
     ("parts3", 1536, 384, 64, 3, 24, 0.75, 300),
     ("parts2", 4096, 128, 128, 2, 8, 1.5, 17),
+    # many tokens, several channel tiles, ragged token count
+    ("pair4", 512, 256, 32, 4, 16, 1.0, 700),
+    ("pair3", 384, 512, 64, 3, 24, 0.75, 530),
+    ("pair2", 256, 768, 128, 2, 8, 2.0, 1100),
 ]
 
 
