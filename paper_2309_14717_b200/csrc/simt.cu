@@ -90,7 +90,7 @@ __host__ __device__ inline int pool16_stride_words(int G) {
 }
 
 template <int LANES_PER_GROUP>   // g / 8: 4, 8 or 16
-__global__ void __launch_bounds__(POOL16_ROWS * 32)
+__global__ void __launch_bounds__(POOL16_ROWS * 32, 2)
 pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
                    float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
                    long long M, int K, int G, int r, float s) {
@@ -110,18 +110,22 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
   if (m < M) {
     const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)m * K);
     const int chunks = K / 8;                             // K is a multiple of 32
-    constexpr int BATCH = 8;                              // loads in flight per lane
-    for (int c0 = 0; c0 < chunks; c0 += 32 * BATCH) {     // chunks is a multiple of 32 (K % 256 == 0)
-      uint4 v[BATCH];
+    constexpr int BATCH = 4;                              // 16-byte loads per lane and batch
+    // two batches in flight: the loads of batch k + 1 are issued before batch k is summed, so
+    // that the rows keep streaming while the warp computes (chunks is a multiple of 32: K % 256 == 0)
+    uint4 v[2][BATCH];
+    auto load_batch = [&](int c0, uint4* dst) {
 #pragma unroll
       for (int b = 0; b < BATCH; ++b) {
         const int c = c0 + b * 32 + lane;
-        v[b] = c < chunks ? xr[c] : make_uint4(0u, 0u, 0u, 0u);
+        dst[b] = c < chunks ? xr[c] : make_uint4(0u, 0u, 0u, 0u);
       }
+    };
+    auto sum_batch = [&](int c0, const uint4* src) {
 #pragma unroll
       for (int b = 0; b < BATCH; ++b) {
         const int c = c0 + b * 32 + lane;
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v[b]);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&src[b]);
         float acc = 0.0f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -138,6 +142,13 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
           if (xp_out != nullptr) xp_out[(size_t)m * G + q] = acc;
         }
       }
+    };
+    load_batch(0, v[0]);
+    for (int c0 = 0; c0 < chunks; c0 += 2 * 32 * BATCH) {
+      load_batch(c0 + 32 * BATCH, v[1]);
+      sum_batch(c0, v[0]);
+      load_batch(c0 + 2 * 32 * BATCH, v[0]);
+      sum_batch(c0 + 32 * BATCH, v[1]);
     }
   }
   __syncthreads();
