@@ -91,32 +91,50 @@ int launch_quantize(const Shape& sh, const float* W, uint32_t* codes, float2* qp
 }
 
 // beta'[q][n] = beta[q][n] + s * sum_i A[q][i] * B[i][n]; alpha is copied.
-// One thread per (group, column); the row of A sits in shared memory.  In-place
-// use is safe: a thread reads only the element it then writes.
+// One thread per column and MERGE_GROUPS consecutive groups, whose rows of A sit in shared
+// memory: an element of B is loaded once and used for all of them.  In-place use is safe: a
+// thread reads only the elements it then writes.
+constexpr int MERGE_GROUPS = 8;
+
 __global__ void __launch_bounds__(QCOLS)
 merge_kernel(const float2* __restrict__ qin, const __nv_bfloat16* __restrict__ A,
              const __nv_bfloat16* __restrict__ B, float2* __restrict__ qout,
-             int N, int r, float s, int ntiles) {
-  extern __shared__ float a_row[];
-  const int q = blockIdx.x / ntiles;
+             int G, int N, int r, float s, int ntiles) {
+  extern __shared__ float a_rows[];                 // [MERGE_GROUPS][r]
+  const int q0 = (blockIdx.x / ntiles) * MERGE_GROUPS;
   const int n = (blockIdx.x % ntiles) * QCOLS + threadIdx.x;
-  for (int i = threadIdx.x; i < r; i += QCOLS) a_row[i] = bf16_to_float(A[(size_t)q * r + i]);
+  for (int i = threadIdx.x; i < MERGE_GROUPS * r; i += QCOLS) {
+    const int q = q0 + i / r;
+    a_rows[i] = q < G ? bf16_to_float(A[(size_t)q * r + i % r]) : 0.0f;
+  }
   __syncthreads();
   if (n >= N) return;
-  float acc = 0.0f;
-#pragma unroll 16                                   // keep 16 loads of B in flight
-  for (int i = 0; i < r; ++i) acc = fmaf(a_row[i], bf16_to_float(B[(size_t)i * N + n]), acc);
-  float2 p = qin[(size_t)q * N + n];
-  p.y = fmaf(s, acc, p.y);
-  qout[(size_t)q * N + n] = p;
+  float acc[MERGE_GROUPS];
+#pragma unroll
+  for (int j = 0; j < MERGE_GROUPS; ++j) acc[j] = 0.0f;
+#pragma unroll 8                                    // keep 8 loads of B in flight
+  for (int i = 0; i < r; ++i) {
+    const float b = bf16_to_float(B[(size_t)i * N + n]);
+#pragma unroll
+    for (int j = 0; j < MERGE_GROUPS; ++j) acc[j] = fmaf(a_rows[j * r + i], b, acc[j]);
+  }
+#pragma unroll
+  for (int j = 0; j < MERGE_GROUPS; ++j) {
+    const int q = q0 + j;
+    if (q < G) {
+      float2 p = qin[(size_t)q * N + n];
+      p.y = fmaf(s, acc[j], p.y);
+      qout[(size_t)q * N + n] = p;
+    }
+  }
 }
 
 int launch_merge(const Shape& sh, const float2* qin, const __nv_bfloat16* A, const __nv_bfloat16* B,
                  float2* qout, cudaStream_t st) {
   const int ntiles = (sh.N + QCOLS - 1) / QCOLS;
-  const long long blocks = (long long)sh.G * ntiles;
+  const long long blocks = (long long)((sh.G + MERGE_GROUPS - 1) / MERGE_GROUPS) * ntiles;
   if (blocks > 0x7fffffffLL) return QALORA_ERR_UNSUPPORTED_SHAPE;
-  merge_kernel<<<(unsigned)blocks, QCOLS, sh.r * sizeof(float), st>>>(qin, A, B, qout, sh.N, sh.r, sh.s, ntiles);
+  merge_kernel<<<(unsigned)blocks, QCOLS, MERGE_GROUPS * sh.r * sizeof(float), st>>>(qin, A, B, qout, sh.G, sh.N, sh.r, sh.s, ntiles);
   count_launch();
   return cuda_status(cudaGetLastError());
 }
