@@ -118,17 +118,18 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------- CPU reference --
-def oracle_setup(rows):
-    """Inputs of the CPU-oracle sample: `rows` token rows of the first shape, quantized once."""
+def oracle_setup(rows, shape=None):
+    """Inputs of the CPU-oracle sample: `rows` token rows of one shape (the first by default), quantized once."""
     from oracle import qalora_oracle as O
     from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs, to_f64
 
-    cfg = CONFIGS[SHAPES[0]].with_(tokens=rows)
+    shape = SHAPES[0] if shape is None else shape
+    cfg = CONFIGS[shape].with_(tokens=rows)
     t = make_inputs(cfg)
     codes, alpha, beta = O.quantize(t["W"].numpy(), cfg.group_size, cfg.bits)
     x, A, B, dy = (to_f64(t[k]) for k in ("x", "A", "B", "dy"))
     fl = fwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank) + bwd_flops(rows, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank)
-    desc = (f"fp64 numpy oracle, forward+backward on {rows} of 8192 token rows of {SHAPES[0]} "
+    desc = (f"fp64 numpy oracle, forward+backward on {rows} of 8192 token rows of {shape} "
             f"(each call dequantizes the full {cfg.d_in}x{cfg.d_out} weight); quantize excluded")
     return (O, cfg, codes, alpha, beta, x, A, B, dy), fl, desc
 
@@ -142,12 +143,17 @@ def oracle_run(state):
 
 
 def oracle_sample(rows=32):
-    """Times the CPU oracle (as it stands) on `rows` token rows of the first
-    shape: forward + backward.  Returns (TFLOP/s, seconds, description, threads)."""
+    """Times the CPU oracle (as it stands) on `rows` token rows of every shape of the
+    step: forward + backward.  Returns (TFLOP/s, seconds, description, threads)."""
     import torch
-    state, fl, desc = oracle_setup(rows)
-    dt = oracle_run(state)
-    return fl / dt / 1e12, dt, desc, torch.get_num_threads()
+    fl_sum, dt_sum, descs = 0.0, 0.0, []
+    for shape in SHAPES:
+        state, fl, desc = oracle_setup(rows, shape)
+        dt_sum += oracle_run(state)
+        fl_sum += fl
+        descs.append(desc)
+        del state
+    return fl_sum / dt_sum / 1e12, dt_sum, "; ".join(descs), torch.get_num_threads()
 
 
 def run_reference(args):
