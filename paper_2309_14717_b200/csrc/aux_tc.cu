@@ -144,29 +144,28 @@ aux_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__
     if (lane == 0) {
       constexpr uint32_t IDESC = ptx::idesc_bf16(ROWS_A, C::TILE_N, MODE == AUX_DB, MODE == AUX_DB);
       uint32_t it = 0, tcount = 0;
-      bool ok = true;
+      bool ok = true, ready = false;
       for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++tcount) {
         const int iters = item_iters(item);
         if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int i = 0; i < iters; ++i, ++it) {
           const int s = it % STAGES;
-          if (!(ok = ptx::mbar_wait(bar_full(s), (it / STAGES) & 1, abort_flag))) break;
+          // the next stage's barrier is probed inside the block that issues this stage's MMAs
+          if (!ready && !(ok = ptx::mbar_wait(bar_full(s), (it / STAGES) & 1, abort_flag))) break;
           ptx::tc_fence_after();
           const uint32_t stage = smem_base + s * C::STAGE_BYTES;
-#pragma unroll
-          for (int j = 0; j < STEP / 16; ++j) {
-            uint64_t adesc, bdesc;
-            if (MODE == AUX_DT) {
-              adesc = ptx::smem_desc(stage + j * 32, 16, 1024);
-              bdesc = ptx::smem_desc(stage + C::A_BYTES + j * 32, 16, 1024);
-            } else {   // MN-major: 64-wide blocks 8 KiB apart, 8-row groups 1 KiB apart
-              adesc = ptx::smem_desc(stage + j * 2048, 8192, 1024);
-              bdesc = ptx::smem_desc(stage + C::A_BYTES + j * 2048, 8192, 1024);
-            }
-            ptx::mma_ss(tmem_base, adesc, bdesc, IDESC, (i > 0 || j > 0) ? 1u : 0u);
+          const uint32_t next_bar = bar_full((it + 1) % STAGES), next_par = ((it + 1) / STAGES) & 1;
+          static_assert(STEP == 64, "the step helper issues four K = 16 MMAs");
+          if (MODE == AUX_DT) {
+            ready = ptx::mma4_ss_commit_probe<2, 2>(tmem_base, ptx::smem_desc(stage, 16, 1024),
+                                                    ptx::smem_desc(stage + C::A_BYTES, 16, 1024), IDESC, i > 0 ? 1u : 0u,
+                                                    bar_empty(s), next_bar, next_par) != 0;
+          } else {   // MN-major: 64-wide blocks 8 KiB apart, 8-row groups 1 KiB apart; 2 KiB per K = 16 step
+            ready = ptx::mma4_ss_commit_probe<128, 128>(tmem_base, ptx::smem_desc(stage, 8192, 1024),
+                                                        ptx::smem_desc(stage + C::A_BYTES, 8192, 1024), IDESC,
+                                                        i > 0 ? 1u : 0u, bar_empty(s), next_bar, next_par) != 0;
           }
-          ptx::mma_commit(bar_empty(s));
         }
         if (ok) ptx::mma_commit(bar_acc_full);
       }
