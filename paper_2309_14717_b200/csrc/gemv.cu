@@ -2,7 +2,7 @@
 // codes and the (alpha, beta) pairs from HBM exactly once.
 //
 // Design
-//  * One block (eight consumer warps in two sets that take alternate k-blocks, plus
+//  * One block (eight consumer warps in two sets that take two k-blocks of a stage each, plus
 //    one producer warp) owns 128 output columns and a slice of the input channels; the
 //    slices of one column tile form a thread-block CLUSTER, and the partial sums
 //    are added through distributed shared memory in a fixed order (no atomics,
@@ -20,6 +20,8 @@
 //        acc += alpha * D + beta * xp,
 //    where xp (the group sum of x, which the paper's pooling also needs) comes
 //    from one more MMA with ones as the A operand.  alpha and beta stay fp32.
+//    With group sizes 64 and 128 a set's two k-blocks share (alpha, beta): they go into
+//    one accumulator chain and are folded once.
 //  * The same reduction step adds the adapter term T * B (T = s * pool(x) * A is
 //    computed by the pooling kernel) and rounds to bf16.
 #include <cooperative_groups.h>
@@ -114,7 +116,9 @@ __device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, const F
   }
 }
 
-template <int BITS, bool UPPER>   // UPPER: token rows 8..15 are in use (M > 8)
+// UPPER: token rows 8..15 are in use (M > 8).  CHAIN: the group size is 64 or 128, so the two
+// k-blocks a warp set takes from a stage share (alpha, beta) and are folded together.
+template <int BITS, bool UPPER, bool CHAIN>
 __global__ void __launch_bounds__(GV_THREADS, 3)
 qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
                    const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
@@ -184,11 +188,11 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int gq = lane / 4, t = lane % 4;        // fragment row (column of W, token), quad lane
     constexpr int NTS = UPPER ? 2 : 1;            // sets of 8 tokens
     // per-thread byte offsets inside a stage; everything else is a compile-time constant
-    const uint32_t x_off = S::OFF_X + gq * (GV_KBS * 64) + t * 16 + set * 64;
+    const uint32_t x_off = S::OFF_X + gq * (GV_KBS * 64) + t * 16 + set * (GV_KBS / GV_SETS) * 64;
     const uint32_t lo_word = BITS == 4 ? t : (t >> 1);
     const uint32_t lo_shift = BITS == 4 ? 0 : 8 * (t & 1);
-    const uint32_t c_off = S::OFF_CODES + set * S::CODE_ROW + ((wcol + gq) * WORDS + lo_word) * 4;
-    const uint32_t h_off = S::OFF_CODES + set * S::CODE_ROW + ((wcol + gq) * WORDS + 2) * 4;   // 3-bit codes: third-bit word
+    const uint32_t c_off = S::OFF_CODES + set * (GV_KBS / GV_SETS) * S::CODE_ROW + ((wcol + gq) * WORDS + lo_word) * 4;
+    const uint32_t h_off = S::OFF_CODES + set * (GV_KBS / GV_SETS) * S::CODE_ROW + ((wcol + gq) * WORDS + 2) * 4;   // 3-bit codes: third-bit word
     const uint32_t q_off = S::OFF_QP + (wcol + gq) * 8;
     float acc[2][NTS][4];                         // [16-column group][token set][(col gq | gq + 8) x (token 2t | 2t + 1)]
     const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -206,13 +210,68 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       const int s = it % GV_STAGES;
       if (!(ok = ptx::mbar_wait(bar_full(s), (it / GV_STAGES) & 1, abort_flag))) break;
       const uint8_t* stage = smem + s * S::STAGE_BYTES;
+      if constexpr (CHAIN) {
+        // the set's two k-blocks lie in one quantization group: one accumulator chain over
+        // both (four MMAs per 16 columns), one fold, one (alpha, beta) load
+        uint4 xs[2][NTS];
+#pragma unroll
+        for (int bb = 0; bb < 2; ++bb) {
+          xs[bb][0] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64);
+          if (UPPER) xs[bb][NTS - 1] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + 8 * (GV_KBS * 64));
+        }
+        float cinit[NTS][4], xp[NTS][2];
+#pragma unroll
+        for (int ts = 0; ts < NTS; ++ts) {
+          mma16816(cinit[ts], ones4, xs[0][ts].x, xs[0][ts].y, zero4);
+          mma16816(cinit[ts], ones4, xs[0][ts].z, xs[0][ts].w, cinit[ts]);
+          mma16816(cinit[ts], ones4, xs[1][ts].x, xs[1][ts].y, cinit[ts]);
+          mma16816(cinit[ts], ones4, xs[1][ts].z, xs[1][ts].w, cinit[ts]);
+          xp[ts][0] = cinit[ts][0];
+          xp[ts][1] = cinit[ts][1];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) cinit[ts][i] *= -128.f;
+        }
+        const uint8_t* qrow = stage + q_off + (((set * (GV_KBS / GV_SETS)) >> qsh) * S::QP_ROW);
+#pragma unroll
+        for (int cg = 0; cg < 2; ++cg) {
+          float D[NTS][4];
+#pragma unroll
+          for (int bb = 0; bb < 2; ++bb) {
+            uint32_t f[2][4];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              const uint32_t coff = bb * S::CODE_ROW + (cg * 16 + j * 8) * WORDS * 4;
+              const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + coff) >> lo_shift;
+              uint32_t hi = 0;
+              if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t);
+              code_fragments<BITS>(lo, hi, fk, f[j]);
+            }
+            const uint32_t a0[4] = {f[0][0], f[1][0], f[0][1], f[1][1]};
+            const uint32_t a1[4] = {f[0][2], f[1][2], f[0][3], f[1][3]};
+#pragma unroll
+            for (int ts = 0; ts < NTS; ++ts) {
+              mma16816(D[ts], a0, xs[bb][ts].x, xs[bb][ts].y, bb == 0 ? cinit[ts] : D[ts]);
+              mma16816(D[ts], a1, xs[bb][ts].z, xs[bb][ts].w, D[ts]);
+            }
+          }
+          const float2 q0 = *reinterpret_cast<const float2*>(qrow + (cg * 16) * 8);
+          const float2 q1 = *reinterpret_cast<const float2*>(qrow + (cg * 16 + 8) * 8);
+#pragma unroll
+          for (int ts = 0; ts < NTS; ++ts) {
+            acc[cg][ts][0] = fmaf(q0.x, D[ts][0], fmaf(q0.y, xp[ts][0], acc[cg][ts][0]));
+            acc[cg][ts][1] = fmaf(q0.x, D[ts][1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
+            acc[cg][ts][2] = fmaf(q1.x, D[ts][2], fmaf(q1.y, xp[ts][0], acc[cg][ts][2]));
+            acc[cg][ts][3] = fmaf(q1.x, D[ts][3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
+          }
+        }
+      } else {
 #pragma unroll
       for (int bb = 0; bb < GV_KBS / GV_SETS; ++bb) {
-        // this set's k-block b = bb * GV_SETS + set; B fragments: x[token gq (+ 8)][32 b + 8 t .. + 7]:
+        // this set's k-block b = 2 set + bb; B fragments: x[token gq (+ 8)][32 b + 8 t .. + 7]:
         // the lane's k slots (2t, 2t+1 | 2t+8, 2t+9) of MMA 0 are channels 8t .. 8t+3, those of MMA 1 8t+4 .. 8t+7
         uint4 xs[NTS];
-        xs[0] = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64);
-        if (UPPER) xs[NTS - 1] = *reinterpret_cast<const uint4*>(stage + x_off + bb * GV_SETS * 64 + 8 * (GV_KBS * 64));
+        xs[0] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64);
+        if (UPPER) xs[NTS - 1] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + 8 * (GV_KBS * 64));
         // xp of the tokens (ones as the A operand: every row of the product holds the sums), then C = -128 xp
         float cinit[NTS][4], xp[NTS][2];
 #pragma unroll
@@ -224,7 +283,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
 #pragma unroll
           for (int i = 0; i < 4; ++i) cinit[ts][i] *= -128.f;
         }
-        const uint8_t* qrow = stage + q_off + (((bb * GV_SETS + set) >> qsh) * S::QP_ROW);
+        const uint8_t* qrow = stage + q_off + (((set * (GV_KBS / GV_SETS) + bb) >> qsh) * S::QP_ROW);
 #pragma unroll
         for (int cg = 0; cg < 2; ++cg) {
           // columns wcol + 16 cg + gq (fragment rows 0..7) and + 8 (rows 8..15)
@@ -232,7 +291,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
           float2 q[2];
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
-            const uint32_t coff = bb * GV_SETS * S::CODE_ROW + (cg * 16 + j * 8) * WORDS * 4;
+            const uint32_t coff = bb * S::CODE_ROW + (cg * 16 + j * 8) * WORDS * 4;
             const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + coff) >> lo_shift;
             uint32_t hi = 0;
             if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t);
@@ -252,6 +311,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
             acc[cg][ts][3] = fmaf(q[1].x, D[3], fmaf(q[1].y, xp[ts][1], acc[cg][ts][3]));
           }
         }
+      }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar_empty(s));
@@ -326,7 +386,7 @@ int gv_sm_count() {
   return n;
 }
 
-template <int BITS, bool UPPER>
+template <int BITS, bool UPPER, bool CHAIN>
 int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
   EncodeTiledFn fn = gv_encode_fn();
   CUtensorMap cm, qm;
@@ -353,7 +413,7 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
       return QALORA_ERR_CUDA;
   }
   using S = GvSmem<BITS, UPPER>;
-  auto kern = qalora_gemv_kernel<BITS, UPPER>;
+  auto kern = qalora_gemv_kernel<BITS, UPPER, CHAIN>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
@@ -417,7 +477,10 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
     if (miss < best) { best = miss; splits = sp; }
   }
   const bool upper = M > 8;
-#define QALORA_GV(BITS) (upper ? launch_gemv_t<BITS, true>(xm, p, splits, st) : launch_gemv_t<BITS, false>(xm, p, splits, st))
+  const bool chain = sh.g >= 64;
+#define QALORA_GV(BITS)                                                                                              \
+  (upper ? (chain ? launch_gemv_t<BITS, true, true>(xm, p, splits, st) : launch_gemv_t<BITS, true, false>(xm, p, splits, st))   \
+         : (chain ? launch_gemv_t<BITS, false, true>(xm, p, splits, st) : launch_gemv_t<BITS, false, false>(xm, p, splits, st)))
   if (sh.bits == 4) return QALORA_GV(4);
   if (sh.bits == 3) return QALORA_GV(3);
   return QALORA_GV(2);
