@@ -142,9 +142,17 @@ int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A
 
 /* One fine-tuning step of the layer driven from HOST buffers: copies x and dy to
  * the device, runs qalora_forward and qalora_backward (Algorithm 1 and its
- * gradients, as above), and copies y, dx, dA and dB back, all enqueued on
- * `cuda_stream` (the call returns without synchronizing; the host outputs are
- * valid once the stream has been synchronized).
+ * gradients, as above), and copies y, dx, dA and dB back.  The call returns
+ * without synchronizing; everything it enqueues starts after the work already on
+ * `cuda_stream`, and `cuda_stream` ends after the last copy, so the host outputs
+ * are valid once that stream has been synchronized.  Batches of 2048 rows and
+ * more are cut into up to 8 row chunks (multiples of 256 rows, at least 1024):
+ * the copies run on two streams of the library's own (made on first use, one
+ * pair per device), so that a chunk's inputs arrive while the previous chunk
+ * computes and the one before that returns.  y and dx are the same bits as from
+ * one qalora_forward / qalora_backward over all rows; dA and dB are then the sums
+ * of the chunks' results in chunk order (a different, fixed, summation order).
+ * Calls from several host threads are serialized by the library.
  *   x_host, dy_host   in : HOST memory (pinned for asynchronous copies), bf16 [m][K], [m][N]
  *   codes, qparams, A, B : DEVICE memory, as for qalora_forward
  *   y_host, dx_host   out: HOST bf16 [m][N], [m][K];  dA_host, dB_host out: HOST float32

@@ -1,5 +1,6 @@
 // C-ABI entry points: argument checks, scratch layout and kernel dispatch.
 #include <atomic>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -259,19 +260,74 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
 
 
 namespace {
-struct StepLayout { size_t ws, x, dy, y, dx, dA, dB, total, ws_bytes; };
+// qalora_step_host cuts the rows into chunks so that the copy of one chunk to the
+// device, the kernels of another and the copy of a third back to the host run at
+// the same time (the link is full duplex).  A chunk is a multiple of 256 rows and at
+// least kStepChunkMin rows long, so that every chunk takes the same large-M kernels
+// as the whole batch would; batches below two such chunks stay in one piece.
+constexpr int kStepMaxChunks = 8;
+constexpr int64_t kStepChunkMin = 1024;
+int64_t step_chunk_rows(int64_t m) {
+  if (m < 2 * kStepChunkMin) return m > 0 ? m : 1;
+  int64_t rows = round_up((size_t)((m + kStepMaxChunks - 1) / kStepMaxChunks), 256);
+  return rows < kStepChunkMin ? kStepChunkMin : rows;
+}
+
+struct StepLayout { size_t ws, x, dy, y, dx, dA, dB, dA_parts, dB_parts, total, ws_bytes; int chunks; int64_t rows; };
 StepLayout step_layout(const Shape& sh, int64_t m) {
   StepLayout L{};
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t at = off; off += round_up(bytes, 256); return at; };
   const size_t M = (size_t)m;
-  const size_t wf = workspace_layout(sh, m, QALORA_OP_FORWARD).total, wb = workspace_layout(sh, m, QALORA_OP_BACKWARD).total;
+  L.rows = step_chunk_rows(m);
+  L.chunks = m > 0 ? (int)((m + L.rows - 1) / L.rows) : 1;
+  const size_t wf = workspace_layout(sh, L.rows, QALORA_OP_FORWARD).total,
+               wb = workspace_layout(sh, L.rows, QALORA_OP_BACKWARD).total;
   L.ws_bytes = wf > wb ? wf : wb;
   L.ws = take(L.ws_bytes);                         // first: the status word sits at the head of the staging area
   L.x = take(M * sh.K * 2); L.dy = take(M * sh.N * 2); L.y = take(M * sh.N * 2); L.dx = take(M * sh.K * 2);
   L.dA = take((size_t)sh.G * sh.r * 4); L.dB = take((size_t)sh.r * sh.N * 4);
+  L.dA_parts = take(L.chunks > 1 ? (size_t)L.chunks * sh.G * sh.r * 4 : 0);
+  L.dB_parts = take(L.chunks > 1 ? (size_t)L.chunks * sh.r * sh.N * 4 : 0);
   L.total = off;
   return L;
+}
+
+// Copy streams and events of one device, made on first use and kept for the life of
+// the process.  An event may be recorded again while an earlier wait on it is still
+// pending: a wait refers to the record that preceded it.
+struct StepPipes {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, done = nullptr;
+  cudaEvent_t x[kStepMaxChunks], dy[kStepMaxChunks], fwd[kStepMaxChunks], bwd[kStepMaxChunks];
+};
+constexpr int kMaxDevices = 64;
+std::mutex g_step_mutex;
+StepPipes g_step_pipes[kMaxDevices];
+
+StepPipes* step_pipes_locked() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  StepPipes& P = g_step_pipes[dev];
+  if (P.ready) return &P;
+  bool ok = cudaStreamCreateWithFlags(&P.in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&P.out, cudaStreamNonBlocking) == cudaSuccess;
+  auto make = [&](cudaEvent_t* e) { ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+  make(&P.start); make(&P.done);
+  for (int i = 0; i < kStepMaxChunks; ++i) { make(&P.x[i]); make(&P.dy[i]); make(&P.fwd[i]); make(&P.bwd[i]); }
+  if (!ok) return nullptr;
+  P.ready = true;
+  return &P;
+}
+
+// out[i] = sum over chunks of parts[c][i], in chunk order (deterministic).
+__global__ void sum_chunks_kernel(float* __restrict__ out, const float* __restrict__ parts, size_t n, int chunks) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float acc = 0.f;
+  for (int c = 0; c < chunks; ++c) acc += parts[(size_t)c * n + i];
+  out[i] = acc;
 }
 }  // namespace
 
@@ -301,19 +357,54 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
   if (staging_bytes < L.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   char* base = static_cast<char*>(staging);
-  const size_t M = (size_t)m;
-  if (cudaMemcpyAsync(base + L.x, x_host, M * sh.K * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess) return QALORA_ERR_CUDA;
-  if (cudaMemcpyAsync(base + L.dy, dy_host, M * sh.N * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess) return QALORA_ERR_CUDA;
-  st = qalora_forward(desc, m, base + L.x, codes, qparams, A, B, base + L.y, base + L.ws, L.ws_bytes, cuda_stream);
-  if (st != QALORA_OK) return st;
-  st = qalora_backward(desc, m, base + L.x, base + L.dy, codes, qparams, A, B, base + L.dx,
-                       reinterpret_cast<float*>(base + L.dA), reinterpret_cast<float*>(base + L.dB), base + L.ws,
-                       L.ws_bytes, cuda_stream);
-  if (st != QALORA_OK) return st;
-  if (cudaMemcpyAsync(y_host, base + L.y, M * sh.N * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
-  if (cudaMemcpyAsync(dx_host, base + L.dx, M * sh.K * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
-  if (cudaMemcpyAsync(dA_host, base + L.dA, (size_t)sh.G * sh.r * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
-  if (cudaMemcpyAsync(dB_host, base + L.dB, (size_t)sh.r * sh.N * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return QALORA_ERR_CUDA;
+  const size_t nA = (size_t)sh.G * sh.r, nB = (size_t)sh.r * sh.N;
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+
+  std::lock_guard<std::mutex> lock(g_step_mutex);
+  StepPipes* P = step_pipes_locked();
+  if (P == nullptr) return QALORA_ERR_CUDA;
+  // The copy streams start after everything already enqueued on the caller's stream.
+  if (!ok(cudaEventRecord(P->start, stream)) || !ok(cudaStreamWaitEvent(P->in, P->start, 0)) ||
+      !ok(cudaStreamWaitEvent(P->out, P->start, 0)))
+    return QALORA_ERR_CUDA;
+  for (int c = 0; c < L.chunks; ++c) {
+    const size_t r0 = (size_t)c * L.rows;
+    const int64_t rows = (int64_t)((size_t)m - r0 < (size_t)L.rows ? (size_t)m - r0 : (size_t)L.rows);
+    const size_t xo = r0 * sh.K * 2, yo = r0 * sh.N * 2, xb = (size_t)rows * sh.K * 2, yb = (size_t)rows * sh.N * 2;
+    float* dA_c = reinterpret_cast<float*>(base + (L.chunks > 1 ? L.dA_parts + c * nA * 4 : L.dA));
+    float* dB_c = reinterpret_cast<float*>(base + (L.chunks > 1 ? L.dB_parts + c * nB * 4 : L.dB));
+    if (!ok(cudaMemcpyAsync(base + L.x + xo, static_cast<const char*>(x_host) + xo, xb, cudaMemcpyHostToDevice, P->in)) ||
+        !ok(cudaEventRecord(P->x[c], P->in)) ||
+        !ok(cudaMemcpyAsync(base + L.dy + yo, static_cast<const char*>(dy_host) + yo, yb, cudaMemcpyHostToDevice, P->in)) ||
+        !ok(cudaEventRecord(P->dy[c], P->in)) || !ok(cudaStreamWaitEvent(stream, P->x[c], 0)))
+      return QALORA_ERR_CUDA;
+    st = qalora_forward(desc, rows, base + L.x + xo, codes, qparams, A, B, base + L.y + yo, base + L.ws, L.ws_bytes,
+                        cuda_stream);
+    if (st != QALORA_OK) return st;
+    if (!ok(cudaEventRecord(P->fwd[c], stream)) || !ok(cudaStreamWaitEvent(stream, P->dy[c], 0))) return QALORA_ERR_CUDA;
+    st = qalora_backward(desc, rows, base + L.x + xo, base + L.dy + yo, codes, qparams, A, B, base + L.dx + xo, dA_c, dB_c,
+                         base + L.ws, L.ws_bytes, cuda_stream);
+    if (st != QALORA_OK) return st;
+    if (!ok(cudaEventRecord(P->bwd[c], stream)) || !ok(cudaStreamWaitEvent(P->out, P->fwd[c], 0)) ||
+        !ok(cudaMemcpyAsync(static_cast<char*>(y_host) + yo, base + L.y + yo, yb, cudaMemcpyDeviceToHost, P->out)) ||
+        !ok(cudaStreamWaitEvent(P->out, P->bwd[c], 0)) ||
+        !ok(cudaMemcpyAsync(static_cast<char*>(dx_host) + xo, base + L.dx + xo, xb, cudaMemcpyDeviceToHost, P->out)))
+      return QALORA_ERR_CUDA;
+  }
+  if (L.chunks > 1) {
+    const int threads = 256;
+    sum_chunks_kernel<<<(unsigned)((nA + threads - 1) / threads), threads, 0, stream>>>(
+        reinterpret_cast<float*>(base + L.dA), reinterpret_cast<const float*>(base + L.dA_parts), nA, L.chunks);
+    sum_chunks_kernel<<<(unsigned)((nB + threads - 1) / threads), threads, 0, stream>>>(
+        reinterpret_cast<float*>(base + L.dB), reinterpret_cast<const float*>(base + L.dB_parts), nB, L.chunks);
+    count_launch(2);
+    if (!ok(cudaGetLastError())) return QALORA_ERR_CUDA;
+  }
+  if (!ok(cudaMemcpyAsync(dA_host, base + L.dA, nA * 4, cudaMemcpyDeviceToHost, stream)) ||
+      !ok(cudaMemcpyAsync(dB_host, base + L.dB, nB * 4, cudaMemcpyDeviceToHost, stream)))
+    return QALORA_ERR_CUDA;
+  // The caller's stream ends after the last copy back to the host.
+  if (!ok(cudaEventRecord(P->done, P->out)) || !ok(cudaStreamWaitEvent(stream, P->done, 0))) return QALORA_ERR_CUDA;
   return QALORA_OK;
 }
 

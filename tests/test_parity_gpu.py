@@ -236,3 +236,30 @@ def test_step_from_host_buffers_matches_device_calls():
     assert Q.workspace_status(staging) == 0
     assert torch.equal(hy, y.cpu()) and torch.equal(hdx, dx.cpu())
     assert torch.equal(hdA, dA.cpu()) and torch.equal(hdB, dB.cpu())
+
+
+def test_chunked_step_from_host_buffers():
+    # 2348 rows: three pipelined chunks (1024, 1024 and a ragged 300).  Rows are independent in y
+    # and dx, so those match the whole-batch device calls bit for bit; dA and dB are sums over the
+    # chunks and are held to the oracle's tolerance.
+    cfg = LayerConfig("hostchunks", 512, 384, 64, 4, 64, 1.0, 2348, seed=22)
+    layer = GpuLayer(cfg)
+    y = layer.forward()
+    dx, dA, dB = layer.backward()
+    pin = lambda t: t.pin_memory()
+    hx, hdy = pin(layer.cpu["x"]), pin(layer.cpu["dy"])
+    hy, hdx = pin(torch.empty_like(y, device="cpu")), pin(torch.empty_like(dx, device="cpu"))
+    hdA, hdB = pin(torch.empty_like(dA, device="cpu")), pin(torch.empty_like(dB, device="cpu"))
+    staging = torch.zeros(Q.qalora_step_host_bytes(layer.d, cfg.tokens), dtype=torch.uint8, device="cuda")
+    codes, alpha, beta = check_quantize(layer)
+    xf, Af, Bf, dyf = (to_f64(layer.cpu[k]) for k in ("x", "A", "B", "dy"))
+    _, dA_ref, dB_ref = O.backward(xf, dyf, codes, alpha, beta, cfg.group_size, Af, Bf, cfg.scale)
+    for _ in range(2):  # the second call reuses the library's streams and events
+        hy.zero_(); hdx.zero_(); hdA.zero_(); hdB.zero_()
+        Q.qalora_step_host(layer.d, cfg.tokens, hx, hdy, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"],
+                           hy, hdx, hdA, hdB, staging)
+        torch.cuda.synchronize()
+        assert Q.workspace_status(staging) == 0
+        assert torch.equal(hy, y.cpu()) and torch.equal(hdx, dx.cpu())
+        assert rel_err(hdA.numpy(), dA_ref) <= TOL and rel_err(hdB.numpy(), dB_ref) <= TOL
+        assert rel_err(hdA.numpy(), dA.cpu().numpy()) <= 1e-5 and rel_err(hdB.numpy(), dB.cpu().numpy()) <= 1e-5
