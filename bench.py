@@ -332,6 +332,8 @@ def run_gpu(args):
     small = small_m_bandwidth(Q, torch, pk)
     small_65b = small_m_bandwidth(Q, torch, pk, shape="cfg5_65b_up", ms=(1,)) if rank == 0 else None
 
+    adamw = adapter_update_bandwidth(Q, torch, pk) if rank == 0 else None
+
     e2e_ms, _ = timed(e2e_step, args.steps)
     e2e_ms /= args.steps
     h2d = sum(s.host["x"].numel() * 2 + s.host["dy"].numel() * 2 for s in shapes)
@@ -356,11 +358,39 @@ def run_gpu(args):
             "e2e": {"value": flops_step / (e2e_ms / 1e3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "roofline": roofline, "small_m": small, "small_m_65b": small_65b,
-            "cpu_baseline": cpu,
+            "adapter_update": adamw, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def adapter_update_bandwidth(Q, torch, pk, reps=10):
+    """Clipped AdamW (Section 4.1) over all adapter values of a LLaMA-7B sized model
+    (32 blocks x 7 projections, rank 64, group size 32): one flat array of about 80 M values,
+    far larger than L2.  Algorithmic bytes per value: 4 (norm pass) + 16 read + 14 written."""
+    r, g, d, f = 64, 32, 4096, 11008
+    per_block = 4 * (d // g * r + r * d) + 2 * (d // g * r + r * f) + (f // g * r + r * d)
+    n = 32 * per_block
+    grad = torch.randn(n, device="cuda") * 1e-3
+    param = torch.randn(n, device="cuda") * 0.02
+    m, v = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    pb = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(Q.qalora_adamw_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    norm = torch.zeros(2, device="cuda")
+    for t in range(1, 4):
+        Q.qalora_adamw_step(Q.adamw_hyper(t, 2e-5), n, grad, param, m, v, pb, norm, ws)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for t in range(4, 4 + reps):
+        Q.qalora_adamw_step(Q.adamw_hyper(t, 2e-5), n, grad, param, m, v, pb, norm, ws)
+    b.record()
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) * 1e3 / reps
+    gbs = n * 34 / (us * 1e-6) / 1e9
+    return {"values": n, "us_per_step": us, "GB/s": gbs, "frac_of_hbm": gbs / pk["hbm"], "bytes_per_value": 34,
+            "launches": 2}
 
 
 def small_m_bandwidth(Q, torch, pk, shape=SMALL_M, ms=(1, 4, 16), cfg=None):

@@ -166,6 +166,37 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
                      void* y_host, void* dx_host, float* dA_host, float* dB_host,
                      void* staging, size_t staging_bytes, void* cuda_stream);
 
+/* Adapter update of one fine-tuning step (Section 4.1, training details: AdamW with a
+ * maximum gradient norm of 0.3 and a constant learning rate; only A and B are trained,
+ * Section 3.3).  All trained values of the step lie in ONE flat array of n float32
+ * (the caller lays the layers' A and B out in it, e.g. as the all-reduce bucket of a
+ * data-parallel step), so the gradient norm is the joint norm over all of them:
+ *     norm = ||grad||_2,  coef = max_grad_norm > 0 ? min(1, max_grad_norm / (norm + 1e-6)) : 1
+ *     g = coef * grad;  param *= 1 - lr * weight_decay
+ *     m = beta1 * m + (1 - beta1) * g;  v = beta2 * v + (1 - beta2) * g * g
+ *     param -= lr * (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps)
+ *     param_bf16 = bf16(param)           (round to nearest even; what qalora_forward reads)
+ * The paper does not state beta1, beta2, eps or weight_decay; they are the caller's.
+ *   hyper        in : HOST struct; step counts from 1
+ *   grad         in : DEVICE float32 [n]
+ *   param, exp_avg, exp_avg_sq  in/out: DEVICE float32 [n] (master copy and both moments)
+ *   param_bf16   out: DEVICE bf16 [n]
+ *   norm_out     out: DEVICE float32 [2] = {norm, coef}, or NULL
+ *   workspace       : DEVICE scratch of qalora_adamw_workspace_bytes() bytes, caller-owned
+ * All device pointers 16-byte aligned.  Two launches on `cuda_stream`, no synchronization,
+ * no allocation; results are reproducible bit for bit for a given n and device.
+ * Errors: QALORA_ERR_NULL_POINTER, QALORA_ERR_MISALIGNED, QALORA_ERR_INVALID_ARG (n < 0,
+ * step < 1, a beta outside [0, 1), lr, eps or weight_decay negative or not finite),
+ * QALORA_ERR_WORKSPACE_TOO_SMALL, QALORA_ERR_CUDA. */
+typedef struct qalora_adamw_hyper {
+  float lr, beta1, beta2, eps, weight_decay, max_grad_norm;
+  int64_t step;
+} qalora_adamw_hyper;
+int qalora_adamw_workspace_bytes(size_t* bytes);
+int qalora_adamw_step(const qalora_adamw_hyper* hyper, int64_t n, const float* grad, float* param,
+                      float* exp_avg, float* exp_avg_sq, void* param_bf16, float* norm_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Forward pass for callers that cannot allocate device memory (the paper has no
  * counterpart; this is a convenience of the library).  Some hosts of this code
  * may not call cudaMalloc at all: a plugin running inside an engine that owns

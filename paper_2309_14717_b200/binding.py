@@ -21,6 +21,7 @@ EXPORTS = (
     "qalora_quantize", "qalora_forward", "qalora_backward", "qalora_merge",
     "qalora_kernel_launches", "qalora_profile_next_main_kernel", "qalora_main_kernel_name",
     "qalora_forward_static", "qalora_step_host_bytes", "qalora_step_host",
+    "qalora_adamw_workspace_bytes", "qalora_adamw_step",
 )
 
 STATIC_SCRATCH_BYTES = 1 << 20
@@ -29,6 +30,11 @@ STATIC_SCRATCH_BYTES = 1 << 20
 class QaloraDesc(Structure):
     _fields_ = [("d_in", c_int32), ("d_out", c_int32), ("group_size", c_int32), ("bits", c_int32),
                 ("rank", c_int32), ("scale", c_float)]
+
+
+class AdamwHyper(Structure):
+    _fields_ = [("lr", c_float), ("beta1", c_float), ("beta2", c_float), ("eps", c_float),
+                ("weight_decay", c_float), ("max_grad_norm", c_float), ("step", c_int64)]
 
 
 class QaloraError(RuntimeError):
@@ -72,6 +78,10 @@ def load() -> ctypes.CDLL:
     lib.qalora_step_host_bytes.argtypes = [D, c_int64, POINTER(c_size_t)]
     lib.qalora_step_host.restype = c_int
     lib.qalora_step_host.argtypes = [D, c_int64] + [c_void_p] * 10 + [c_void_p, c_size_t, c_void_p]
+    lib.qalora_adamw_workspace_bytes.restype = c_int
+    lib.qalora_adamw_workspace_bytes.argtypes = [POINTER(c_size_t)]
+    lib.qalora_adamw_step.restype = c_int
+    lib.qalora_adamw_step.argtypes = [POINTER(AdamwHyper), c_int64] + [c_void_p] * 6 + [c_void_p, c_size_t, c_void_p]
     lib.qalora_kernel_launches.restype = ctypes.c_uint64
     lib.qalora_kernel_launches.argtypes = []
     lib.qalora_profile_next_main_kernel.restype = c_int
@@ -199,6 +209,27 @@ def qalora_backward(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, 
 def qalora_merge(d: QaloraDesc, qparams_in, A, B, qparams_out, stream=None):
     _check("qalora_merge", load().qalora_merge(byref(d), _ptr(qparams_in), _ptr(A), _ptr(B), _ptr(qparams_out),
                                                _stream(stream)))
+
+
+def qalora_adamw_workspace_bytes() -> int:
+    b = c_size_t()
+    _check("qalora_adamw_workspace_bytes", load().qalora_adamw_workspace_bytes(byref(b)))
+    return b.value
+
+
+def adamw_hyper(step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                weight_decay: float = 0.0, max_grad_norm: float = 0.3) -> AdamwHyper:
+    return AdamwHyper(lr, beta1, beta2, eps, weight_decay, max_grad_norm, step)
+
+
+def qalora_adamw_step(hyper: AdamwHyper, n: int, grad, param, exp_avg, exp_avg_sq, param_bf16, norm_out, workspace,
+                      stream=None):
+    """Clipped AdamW over one flat array of n trained values (all on the device)."""
+    _check("qalora_adamw_step", load().qalora_adamw_step(byref(hyper), n, _ptr(grad), _ptr(param), _ptr(exp_avg),
+                                                         _ptr(exp_avg_sq), _ptr(param_bf16), _ptr(norm_out),
+                                                         _ptr(workspace),
+                                                         workspace.numel() * workspace.element_size()
+                                                         if workspace is not None else 0, _stream(stream)))
 
 
 def qalora_kernel_launches() -> int:

@@ -321,14 +321,6 @@ StepPipes* step_pipes_locked() {
   return &P;
 }
 
-// out[i] = sum over chunks of parts[c][i], in chunk order (deterministic).
-__global__ void sum_chunks_kernel(float* __restrict__ out, const float* __restrict__ parts, size_t n, int chunks) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  float acc = 0.f;
-  for (int c = 0; c < chunks; ++c) acc += parts[(size_t)c * n + i];
-  out[i] = acc;
-}
 }  // namespace
 
 int qalora_step_host_bytes(const qalora_desc* desc, int64_t m, size_t* bytes) {
@@ -391,14 +383,13 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
         !ok(cudaMemcpyAsync(static_cast<char*>(dx_host) + xo, base + L.dx + xo, xb, cudaMemcpyDeviceToHost, P->out)))
       return QALORA_ERR_CUDA;
   }
-  if (L.chunks > 1) {
-    const int threads = 256;
-    sum_chunks_kernel<<<(unsigned)((nA + threads - 1) / threads), threads, 0, stream>>>(
-        reinterpret_cast<float*>(base + L.dA), reinterpret_cast<const float*>(base + L.dA_parts), nA, L.chunks);
-    sum_chunks_kernel<<<(unsigned)((nB + threads - 1) / threads), threads, 0, stream>>>(
-        reinterpret_cast<float*>(base + L.dB), reinterpret_cast<const float*>(base + L.dB_parts), nB, L.chunks);
-    count_launch(2);
-    if (!ok(cudaGetLastError())) return QALORA_ERR_CUDA;
+  if (L.chunks > 1) {   // dA, dB = the chunks' results added in chunk order
+    st = launch_sum_partials(reinterpret_cast<const float*>(base + L.dA_parts), reinterpret_cast<float*>(base + L.dA), nA,
+                             L.chunks, stream);
+    if (st != QALORA_OK) return st;
+    st = launch_sum_partials(reinterpret_cast<const float*>(base + L.dB_parts), reinterpret_cast<float*>(base + L.dB), nB,
+                             L.chunks, stream);
+    if (st != QALORA_OK) return st;
   }
   if (!ok(cudaMemcpyAsync(dA_host, base + L.dA, nA * 4, cudaMemcpyDeviceToHost, stream)) ||
       !ok(cudaMemcpyAsync(dB_host, base + L.dB, nB * 4, cudaMemcpyDeviceToHost, stream)))
@@ -406,6 +397,34 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
   // The caller's stream ends after the last copy back to the host.
   if (!ok(cudaEventRecord(P->done, P->out)) || !ok(cudaStreamWaitEvent(stream, P->done, 0))) return QALORA_ERR_CUDA;
   return QALORA_OK;
+}
+
+int qalora_adamw_workspace_bytes(size_t* bytes) {
+  if (bytes == nullptr) return QALORA_ERR_NULL_POINTER;
+  *bytes = adamw_workspace_bytes();
+  return QALORA_OK;
+}
+
+int qalora_adamw_step(const qalora_adamw_hyper* hyper, int64_t n, const float* grad, float* param,
+                      float* exp_avg, float* exp_avg_sq, void* param_bf16, float* norm_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (hyper == nullptr) return QALORA_ERR_NULL_POINTER;
+  auto finite_nonneg = [](float v) { return v >= 0.f && v <= 3.0e38f; };   // false for NaN
+  if (n < 0 || hyper->step < 1 || !(hyper->beta1 >= 0.f && hyper->beta1 < 1.f) ||
+      !(hyper->beta2 >= 0.f && hyper->beta2 < 1.f) || !finite_nonneg(hyper->lr) || !finite_nonneg(hyper->eps) ||
+      !finite_nonneg(hyper->weight_decay) || !(hyper->max_grad_norm == hyper->max_grad_norm))
+    return QALORA_ERR_INVALID_ARG;
+  if (n == 0) return QALORA_OK;
+  if (grad == nullptr || param == nullptr || exp_avg == nullptr || exp_avg_sq == nullptr || param_bf16 == nullptr ||
+      workspace == nullptr)
+    return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(grad) || !aligned16(param) || !aligned16(exp_avg) || !aligned16(exp_avg_sq) || !aligned16(param_bf16) ||
+      !aligned16(workspace) || (norm_out != nullptr && (reinterpret_cast<uintptr_t>(norm_out) & 3u)))
+    return QALORA_ERR_MISALIGNED;
+  if (workspace_bytes < adamw_workspace_bytes()) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  AdamwArgs a{hyper->lr, hyper->beta1, hyper->beta2, hyper->eps, hyper->weight_decay, hyper->max_grad_norm, hyper->step};
+  return launch_adamw(a, n, grad, param, exp_avg, exp_avg_sq, static_cast<__nv_bfloat16*>(param_bf16),
+                      static_cast<float*>(workspace), norm_out, static_cast<cudaStream_t>(cuda_stream));
 }
 
 }  // extern "C"

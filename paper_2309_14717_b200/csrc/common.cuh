@@ -124,6 +124,12 @@ size_t tc_dB_partial_bytes(const Shape& sh, int64_t M);
 int launch_tc_dB_partials(const Shape& sh, int64_t M, const __nv_bfloat16* Tb, const __nv_bfloat16* dy,
                           float* partial, int* splits_out, int* status, cudaStream_t st);
 
+// Adapter update (optimizer.cu): clipped AdamW over one flat array, two launches.
+struct AdamwArgs { float lr, beta1, beta2, eps, weight_decay, max_grad_norm; int64_t step; };
+size_t adamw_workspace_bytes();
+int launch_adamw(const AdamwArgs& a, int64_t n, const float* grad, float* param, float* exp_avg, float* exp_avg_sq,
+                 __nv_bfloat16* param_bf16, float* parts, float* norm_out, cudaStream_t st);
+
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? QALORA_OK : QALORA_ERR_CUDA; }
 
 // Instrumentation: launch counter and the one-shot event probe around a main kernel.

@@ -92,3 +92,15 @@ def make_inputs(cfg: LayerConfig, need=("W", "x", "A", "B", "dy")) -> dict:
 def to_f64(t: torch.Tensor):
     """Exact widening of a stored tensor to a numpy fp64 array."""
     return t.detach().cpu().to(torch.float64).numpy()
+
+
+def make_optimizer_inputs(n: int, steps: int, seed: int = 0, grad_scales=(1e-4, 1.0)) -> dict:
+    """Seeded inputs for the adapter update: float32 parameters N(0, 0.02^2) and one
+    gradient array per step, N(0, scale^2) with the scales taken in turn (a small one
+    keeps the joint norm below the clipping bound of 0.3 for short arrays, a large one
+    exceeds it), so that both branches of the clipping rule are visited."""
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    param = torch.randn(n, generator=gen, dtype=torch.float32) * 0.02
+    grads = [torch.randn(n, generator=gen, dtype=torch.float32) * grad_scales[t % len(grad_scales)]
+             for t in range(steps)]
+    return {"param": param, "grads": grads}

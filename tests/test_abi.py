@@ -87,3 +87,22 @@ def test_null_and_misaligned_pointers_are_rejected_without_a_launch():
     d0 = Q.desc(512, 512, 32, 4, 0, 1.0)
     assert lib.qalora_backward(r(d0), 8, p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), 1 << 30, None) == -1
     assert lib.qalora_forward(r(d), 0, None, None, None, None, None, None, None, 0, None) == 0
+
+
+def test_adamw_argument_checks_need_no_gpu():
+    lib = Q.load()
+    p = ctypes.c_void_p
+    buf = ctypes.create_string_buffer(64)          # host memory: must never be dereferenced
+    a16 = (ctypes.addressof(buf) + 15) // 16 * 16
+    r = ctypes.byref
+    good = Q.adamw_hyper(1, 2e-5)
+    args = lambda h, n=8, g=a16, ws=1 << 20: (r(h) if h is not None else None, n, p(g), p(a16), p(a16), p(a16), p(a16),
+                                              None, p(a16), ws, None)
+    assert lib.qalora_adamw_step(*args(None)) == -2
+    assert lib.qalora_adamw_step(*args(Q.adamw_hyper(0, 2e-5))) == -1
+    assert lib.qalora_adamw_step(*args(Q.adamw_hyper(1, 2e-5, beta2=1.0))) == -1
+    assert lib.qalora_adamw_step(*args(good, n=-1)) == -1
+    assert lib.qalora_adamw_step(*args(good, g=a16 + 4)) == -4
+    assert lib.qalora_adamw_step(*args(good, ws=8)) == -5
+    assert lib.qalora_adamw_step(*args(good, n=0)) == 0
+    assert Q.qalora_adamw_workspace_bytes() >= 4096

@@ -70,3 +70,65 @@ def test_row_slices_tile_the_batch(m, world):
     assert max(sizes) - min(sizes) <= 1
     with pytest.raises(ValueError):
         dp.shard_rows(m, world, world)
+
+
+LAYERS = [(4, 8, 48), (6, 16, 24), (4, 8, 40)]        # (G, r, N) of three layers
+
+
+def _bucket_worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        b = dp.AdapterBucket(LAYERS)
+        for i in range(len(LAYERS)):
+            dA, dB = b.grads(i)
+            g = torch.Generator().manual_seed(100 * rank + i)
+            dA.copy_(torch.randn(dA.shape, generator=g)); dB.copy_(torch.randn(dB.shape, generator=g))
+        b.reduce()
+        if rank == 0:
+            out.put(b.grad.numpy().copy())
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.timeout(120)
+def test_bucket_views_and_single_allreduce():
+    b = dp.AdapterBucket(LAYERS)
+    assert b.n == sum(G * r + r * N for G, r, N in LAYERS)
+    spans = []
+    for i, (G, r, N) in enumerate(LAYERS):
+        dA, dB = b.grads(i)
+        A, B = b.factors(i)
+        assert dA.shape == (G, r) == A.shape and dB.shape == (r, N) == B.shape
+        assert dA.data_ptr() % 16 == 0 and dB.data_ptr() % 16 == 0 and A.data_ptr() % 16 == 0 and B.data_ptr() % 16 == 0
+        spans += [(dA.data_ptr(), dA.numel() * 4), (dB.data_ptr(), dB.numel() * 4)]
+    spans.sort()
+    assert spans[0][0] == b.grad.data_ptr() and sum(s for _, s in spans) == b.n * 4
+    for (p, s), (q, _) in zip(spans, spans[1:]):
+        assert p + s == q                                # the views tile the bucket without gaps
+    with pytest.raises(ValueError):
+        dp.AdapterBucket([(4, 12, 48)])
+    with pytest.raises(RuntimeError):
+        b.update(2e-5)                                   # no CPU path for the optimizer
+    world = 2
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_bucket_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = out.get(timeout=90)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    want = np.zeros(b.n, dtype=np.float32)
+    for rank in range(world):
+        off = 0
+        for i, (G, r, N) in enumerate(LAYERS):
+            g = torch.Generator().manual_seed(100 * rank + i)
+            for shape in ((G, r), (r, N)):
+                t = torch.randn(shape, generator=g).numpy().ravel()
+                want[off:off + t.size] += t
+                off += t.size
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-6)
