@@ -462,6 +462,9 @@ def run_only(args):
     from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
 
     _build.build()
+    if args.only == "adamw":   # the adapter update on the 7B-sized flat array (--steps timed calls inside)
+        print(json.dumps({"only": "adamw", **adapter_update_bandwidth(Q, torch, peaks(), reps=max(1, args.steps))}))
+        return
     cfg = CONFIGS[args.shape].with_(tokens=args.tokens)
     t = {k: v.cuda() for k, v in make_inputs(cfg).items()}
     M, K, N, G, r = cfg.tokens, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank
@@ -570,7 +573,7 @@ def run_table(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", action="store_true", help="per-configuration throughput table (markdown)")
-    ap.add_argument("--only", default=None, choices=("fwd", "bwd", "gemv", "quantize", "merge"))
+    ap.add_argument("--only", default=None, choices=("fwd", "bwd", "gemv", "quantize", "merge", "adamw"))
     ap.add_argument("--shape", default="cfg3_7b_up")
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gpus", type=int, default=1)
