@@ -38,7 +38,8 @@ import numpy as np
 
 __all__ = [
     "levels", "quantize", "quantize_fp64_shadow", "dequantize", "pool",
-    "forward", "backward", "backward_adapter", "merge", "merge_zero_point", "words_per_unit",
+    "forward", "backward", "backward_adapter", "merge", "merge_zero_point", "zero_point_from_beta",
+    "beta_from_zero_point", "dequantize_zero_point", "words_per_unit",
     "pack", "unpack", "adapter_param_count",
 ]
 
@@ -193,6 +194,32 @@ def merge_zero_point(z, alpha, A, B, s) -> np.ndarray:
     alpha = np.asarray(alpha, dtype=np.float64)
     P = np.asarray(A, dtype=np.float64) @ np.asarray(B, dtype=np.float64)
     return z - float(s) * P / alpha
+
+
+def zero_point_from_beta(alpha, beta) -> np.ndarray:
+    """z = -beta / alpha: the zero POINT of Algorithm 1's form W~ = alpha * (c - z) that
+    describes the same weights as Eq. 1's additive zero beta (W~ = alpha * c + beta)."""
+    alpha = np.asarray(alpha, dtype=np.float64)
+    if np.any(alpha == 0):
+        raise ValueError("alpha must be non-zero")
+    return -np.asarray(beta, dtype=np.float64) / alpha
+
+
+def beta_from_zero_point(alpha, z) -> np.ndarray:
+    """beta = -alpha * z: Eq. 1's additive zero for a layer stored in Algorithm 1's
+    zero-point form (an integer z from an asymmetric integer quantizer, or the real z'
+    left by Algorithm 1's merge)."""
+    return -np.asarray(alpha, dtype=np.float64) * np.asarray(z, dtype=np.float64)
+
+
+def dequantize_zero_point(codes: np.ndarray, alpha: np.ndarray, z: np.ndarray, g: int) -> np.ndarray:
+    """W~[k, n] = alpha[k // g, n] * (c[k, n] - z[k // g, n])  (Algorithm 1, pre_quantization)."""
+    K, N = codes.shape
+    G = _check_group(K, g)
+    a = np.asarray(alpha, dtype=np.float64).reshape(G, 1, N)
+    zz = np.asarray(z, dtype=np.float64).reshape(G, 1, N)
+    c = codes.astype(np.float64).reshape(G, g, N)
+    return (a * (c - zz)).reshape(K, N)
 
 
 # ----------------------------------------------------------------------------

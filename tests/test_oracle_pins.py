@@ -300,3 +300,27 @@ def test_param_counts_reproduce_table_2(row):
     qlora = layers * sum(O.adapter_param_count(K, N, 1, 64) for K, N in linears)
     assert round(qalora / 1e6) == int(qalora_m)
     assert round(qlora / 1e6) == int(qlora_m)
+
+
+def test_zero_point_form_of_algorithm_1():
+    """Algorithm 1 writes the layer as alpha * (c - z); Eq. 1 as alpha * c + beta.  A hand-worked
+    asymmetric INT4 example with an integer zero point, the conversion in both directions, and
+    a sign error that must be caught."""
+    # scale 0.5, integer zero point 6: codes 0, 6, 15 stand for -3, 0 and 4.5
+    codes = np.array([[0], [6], [15], [8]], dtype=np.uint8)
+    alpha, z = np.array([[0.5]]), np.array([[6.0]])
+    np.testing.assert_array_equal(O.dequantize_zero_point(codes, alpha, z, 4).ravel(), [-3.0, 0.0, 4.5, 1.0])
+    beta = O.beta_from_zero_point(alpha, z)
+    assert beta[0, 0] == -3.0                                  # the weight that code 0 stands for
+    np.testing.assert_array_equal(O.dequantize(codes, alpha, beta, 4).ravel(), [-3.0, 0.0, 4.5, 1.0])
+    assert O.zero_point_from_beta(alpha, beta)[0, 0] == 6.0
+    # random layers: both forms give the same weights, and the round trip is the identity
+    rng = np.random.default_rng(77)
+    W, codes, alpha, beta, *_ = _rand_layer(rng, 64, 12, 32, 4, 4, 3)
+    z = O.zero_point_from_beta(alpha, beta)
+    ref = O.dequantize(codes, alpha, beta, 32)
+    assert np.max(np.abs(O.dequantize_zero_point(codes, alpha, z, 32) - ref)) <= 1e-12 * np.max(np.abs(ref))
+    np.testing.assert_allclose(O.beta_from_zero_point(alpha, z), beta, rtol=1e-14)
+    assert np.max(np.abs(O.dequantize_zero_point(codes, alpha, -z, 32) - ref)) > 1e-3      # planted sign error
+    with pytest.raises(ValueError):
+        O.zero_point_from_beta(np.zeros((1, 1)), np.ones((1, 1)))
