@@ -166,6 +166,28 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
                      void* y_host, void* dx_host, float* dA_host, float* dB_host,
                      void* staging, size_t staging_bytes, void* cuda_stream);
 
+/* Dequantizes the whole weight matrix, W~[k][n] = alpha[k/g][n] * c[k][n] + beta[k/g][n]
+ * (Eq. 1), e.g. to export a merged layer or to feed a 16-bit baseline.
+ *   codes, qparams in : DEVICE, as written by qalora_quantize / qalora_merge
+ *   W              out: DEVICE [d_in][d_out] row-major, float32 (out_bf16 == 0) or bf16
+ *                       (out_bf16 != 0; the float32 value rounded to nearest even)
+ * Pointers 16-byte aligned.  One launch on `cuda_stream`, no synchronization. */
+int qalora_dequantize(const qalora_desc* desc, const void* codes, const float* qparams, void* W,
+                      int out_bf16, void* cuda_stream);
+
+/* The zero-point form of Algorithm 1 (pre_quantization / merge_with_quantization):
+ * W~ = alpha * (c - z), against Eq. 1's W~ = alpha * c + beta; the two describe the same
+ * weights when beta = -alpha * z.  qalora_qparams_from_zero_point imports scales and zero
+ * points (integer ones of an asymmetric integer quantizer, stored as float32, or the real
+ * ones Algorithm 1's merge leaves) into the library's qparams; qalora_qparams_to_zero_point
+ * exports them, z = -beta / alpha (alpha is never 0 in qparams written by this library).
+ *   alpha, zero : DEVICE float32 [G][d_out];  qparams : DEVICE float32 [G][d_out][2]
+ * Pointers 16-byte aligned.  One launch each on `cuda_stream`, no synchronization. */
+int qalora_qparams_from_zero_point(const qalora_desc* desc, const float* alpha, const float* zero,
+                                   float* qparams, void* cuda_stream);
+int qalora_qparams_to_zero_point(const qalora_desc* desc, const float* qparams, float* alpha,
+                                 float* zero, void* cuda_stream);
+
 /* Adapter update of one fine-tuning step (Section 4.1, training details: AdamW with a
  * maximum gradient norm of 0.3 and a constant learning rate; only A and B are trained,
  * Section 3.3).  All trained values of the step lie in ONE flat array of n float32

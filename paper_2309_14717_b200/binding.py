@@ -22,6 +22,7 @@ EXPORTS = (
     "qalora_kernel_launches", "qalora_profile_next_main_kernel", "qalora_main_kernel_name",
     "qalora_forward_static", "qalora_step_host_bytes", "qalora_step_host",
     "qalora_adamw_workspace_bytes", "qalora_adamw_step",
+    "qalora_dequantize", "qalora_qparams_from_zero_point", "qalora_qparams_to_zero_point",
 )
 
 STATIC_SCRATCH_BYTES = 1 << 20
@@ -78,6 +79,12 @@ def load() -> ctypes.CDLL:
     lib.qalora_step_host_bytes.argtypes = [D, c_int64, POINTER(c_size_t)]
     lib.qalora_step_host.restype = c_int
     lib.qalora_step_host.argtypes = [D, c_int64] + [c_void_p] * 10 + [c_void_p, c_size_t, c_void_p]
+    lib.qalora_dequantize.restype = c_int
+    lib.qalora_dequantize.argtypes = [D, c_void_p, c_void_p, c_void_p, c_int, c_void_p]
+    lib.qalora_qparams_from_zero_point.restype = c_int
+    lib.qalora_qparams_from_zero_point.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.qalora_qparams_to_zero_point.restype = c_int
+    lib.qalora_qparams_to_zero_point.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.qalora_adamw_workspace_bytes.restype = c_int
     lib.qalora_adamw_workspace_bytes.argtypes = [POINTER(c_size_t)]
     lib.qalora_adamw_step.restype = c_int
@@ -209,6 +216,25 @@ def qalora_backward(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, 
 def qalora_merge(d: QaloraDesc, qparams_in, A, B, qparams_out, stream=None):
     _check("qalora_merge", load().qalora_merge(byref(d), _ptr(qparams_in), _ptr(A), _ptr(B), _ptr(qparams_out),
                                                _stream(stream)))
+
+
+def qalora_dequantize(d: QaloraDesc, codes, qparams, W, stream=None):
+    """W [d_in][d_out] (float32 or bfloat16, by W's dtype) = alpha * codes + beta."""
+    import torch
+    if W.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("W must be float32 or bfloat16")
+    _check("qalora_dequantize", load().qalora_dequantize(byref(d), _ptr(codes), _ptr(qparams), _ptr(W),
+                                                         1 if W.dtype == torch.bfloat16 else 0, _stream(stream)))
+
+
+def qalora_qparams_from_zero_point(d: QaloraDesc, alpha, zero, qparams, stream=None):
+    _check("qalora_qparams_from_zero_point", load().qalora_qparams_from_zero_point(
+        byref(d), _ptr(alpha), _ptr(zero), _ptr(qparams), _stream(stream)))
+
+
+def qalora_qparams_to_zero_point(d: QaloraDesc, qparams, alpha, zero, stream=None):
+    _check("qalora_qparams_to_zero_point", load().qalora_qparams_to_zero_point(
+        byref(d), _ptr(qparams), _ptr(alpha), _ptr(zero), _stream(stream)))
 
 
 def qalora_adamw_workspace_bytes() -> int:

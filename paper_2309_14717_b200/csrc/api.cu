@@ -399,6 +399,37 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
   return QALORA_OK;
 }
 
+int qalora_dequantize(const qalora_desc* desc, const void* codes, const float* qparams, void* W,
+                      int out_bf16, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (codes == nullptr || qparams == nullptr || W == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(codes) || !aligned16(qparams) || !aligned16(W)) return QALORA_ERR_MISALIGNED;
+  return launch_dequantize(sh, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams), W,
+                           out_bf16 != 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int qalora_qparams_from_zero_point(const qalora_desc* desc, const float* alpha, const float* zero,
+                                   float* qparams, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (alpha == nullptr || zero == nullptr || qparams == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(alpha) || !aligned16(zero) || !aligned16(qparams)) return QALORA_ERR_MISALIGNED;
+  return launch_from_zero_point(sh, alpha, zero, reinterpret_cast<float2*>(qparams), static_cast<cudaStream_t>(cuda_stream));
+}
+
+int qalora_qparams_to_zero_point(const qalora_desc* desc, const float* qparams, float* alpha,
+                                 float* zero, void* cuda_stream) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (alpha == nullptr || zero == nullptr || qparams == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(alpha) || !aligned16(zero) || !aligned16(qparams)) return QALORA_ERR_MISALIGNED;
+  return launch_to_zero_point(sh, reinterpret_cast<const float2*>(qparams), alpha, zero, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int qalora_adamw_workspace_bytes(size_t* bytes) {
   if (bytes == nullptr) return QALORA_ERR_NULL_POINTER;
   *bytes = adamw_workspace_bytes();

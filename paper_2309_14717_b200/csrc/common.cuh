@@ -124,6 +124,11 @@ size_t tc_dB_partial_bytes(const Shape& sh, int64_t M);
 int launch_tc_dB_partials(const Shape& sh, int64_t M, const __nv_bfloat16* Tb, const __nv_bfloat16* dy,
                           float* partial, int* splits_out, int* status, cudaStream_t st);
 
+// Format conversions (formats.cu): whole-matrix dequantization and Algorithm 1's zero-point form.
+int launch_dequantize(const Shape& sh, const uint32_t* codes, const float2* qparams, void* W, bool bf16_out, cudaStream_t st);
+int launch_from_zero_point(const Shape& sh, const float* alpha, const float* zero, float2* qparams, cudaStream_t st);
+int launch_to_zero_point(const Shape& sh, const float2* qparams, float* alpha, float* zero, cudaStream_t st);
+
 // Adapter update (optimizer.cu): clipped AdamW over one flat array, two launches.
 struct AdamwArgs { float lr, beta1, beta2, eps, weight_decay, max_grad_norm; int64_t step; };
 size_t adamw_workspace_bytes();
