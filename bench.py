@@ -570,8 +570,117 @@ def run_table(args):
     print(f"peaks: bf16 {pk['tensor']:.0f} TFLOP/s, HBM {pk['hbm']:.0f} GB/s ({pk['source']})")
 
 
+def run_baselines(args):
+    """The paper's Table 2 comparison restated on this GPU, one layer at a time: a 16-bit LoRA
+    layer (library GEMMs on a bf16 weight, adapter on the un-pooled input), a QLoRA-style layer
+    (dequantize the 4-bit weight to bf16, then the same GEMMs) and this library's QA-LoRA layer.
+    The two baselines are written with torch.matmul (cuBLAS): they are context, not product."""
+    import statistics
+
+    import torch
+
+    from paper_2309_14717_b200 import binding as Q
+    from paper_2309_14717_b200 import build as _build
+    from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
+
+    _build.build()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def med(fn, reps=7, warm=3):
+        ts = []
+        for _ in range(warm + reps):
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts[warm:])
+
+    print("| layer | M | 16-bit LoRA fwd+bwd ms | dequantize + 16-bit fwd+bwd ms | QA-LoRA fwd+bwd ms | QA-LoRA / LoRA | QA-LoRA / dequantize-first |")
+    print("|---|---|---|---|---|---|---|")
+    rows1 = []
+    for name in ("cfg3_7b_up", "cfg3_7b_down", "cfg5_65b_up", "cfg5_65b_down", "cfg5_65b_attn"):
+        M = 8192
+        cfg = CONFIGS[name].with_(tokens=M)
+        t = {k: v.cuda() for k, v in make_inputs(cfg).items()}
+        K, N, G, r, s = cfg.d_in, cfg.d_out, cfg.groups, cfg.rank, cfg.scale
+        d = Q.desc(K, N, cfg.group_size, cfg.bits, r, s)
+        codes, qparams = Q.alloc_packed(d)
+        Q.qalora_quantize(d, t["W"], codes, qparams)
+        del t["W"]
+        x, dy, B = t["x"], t["dy"], t["B"]
+        W16 = torch.empty((K, N), dtype=torch.bfloat16, device="cuda")
+        Q.qalora_dequantize(d, codes, qparams, W16)
+        A_full = (torch.randn(K, r, device="cuda") * 0.02).to(torch.bfloat16)      # LoRA's A spans D_in
+
+        def lora_step(W):
+            T = x @ A_full
+            y = torch.addmm(x @ W, T, B, alpha=s)
+            dT = (dy @ B.t()) * s
+            dx = torch.addmm(dy @ W.t(), dT, A_full.t())
+            dA = x.t() @ dT
+            dB = (T.t() @ dy) * s
+            return y, dx, dA, dB
+
+        def qlora_step():
+            Q.qalora_dequantize(d, codes, qparams, W16)      # forward
+            T = x @ A_full
+            y = torch.addmm(x @ W16, T, B, alpha=s)
+            Q.qalora_dequantize(d, codes, qparams, W16)      # backward dequantizes again
+            dT = (dy @ B.t()) * s
+            dx = torch.addmm(dy @ W16.t(), dT, A_full.t())
+            return y, dx, x.t() @ dT, (T.t() @ dy) * s
+
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dA = torch.empty((G, r), dtype=torch.float32, device="cuda")
+        dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
+        wf, wb = Q.alloc_workspace(d, M, Q.OP_FORWARD), Q.alloc_workspace(d, M, Q.OP_BACKWARD)
+
+        def qalora_step():
+            Q.qalora_forward(d, M, x, codes, qparams, t["A"], B, y, wf)
+            Q.qalora_backward(d, M, x, dy, codes, qparams, t["A"], B, dx, dA, dB, wb)
+
+        # one-token serving first (before the long GEMMs heat the part): merged INT4 layer against
+        # a bf16 matrix-vector product
+        time.sleep(1.0)
+        x1 = x[:1].contiguous()
+        y1 = torch.empty((1, N), dtype=torch.bfloat16, device="cuda")
+        d0 = Q.desc(K, N, cfg.group_size, cfg.bits, 0, s)
+        w1 = Q.alloc_workspace(d0, 1, Q.OP_FORWARD)
+        copies = max(8, int(5 * 126e6 // (K * N // 2)) + 1)     # even the 4-bit copies total > 4 x L2
+        W16s = [W16.clone() for _ in range(copies)]
+        Cs = [(codes.clone(), qparams.clone()) for _ in range(copies)]
+
+        def graph_us(fn):
+            g = torch.cuda.CUDAGraph()
+            fn(0)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g):
+                for i in range(copies):
+                    fn(i)
+
+            def five():
+                for _ in range(5):
+                    g.replay()
+            return med(five, reps=3, warm=1) * 1e3 / (5 * copies)
+
+        t16 = graph_us(lambda i: torch.matmul(x1, W16s[i], out=y1))
+        t4 = graph_us(lambda i: Q.qalora_forward(d0, 1, x1, Cs[i][0], Cs[i][1], None, None, y1, w1,
+                                                 torch.cuda.current_stream()))
+        rows1.append(f"| {name} | {t16:.1f} | {t4:.1f} | {t16 / t4:.2f} |")
+        a, b, c = med(lambda: lora_step(W16)), med(qlora_step), med(qalora_step)
+        del W16s, Cs
+        print(f"| {name} | {M} | {a:.3f} | {b:.3f} | {c:.3f} | {c / a:.2f} | {c / b:.2f} |", flush=True)
+        del t, W16, codes, qparams, y, dx, wf, wb, x, dy
+        torch.cuda.empty_cache()
+    print()
+    print("| layer | bf16 weight, M = 1 forward us | merged INT4 QA-LoRA, M = 1 forward us | speed-up |")
+    print("|---|---|---|---|")
+    print("\n".join(rows1))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--baselines", action="store_true", help="16-bit LoRA and dequantize-first layers beside QA-LoRA (markdown)")
     ap.add_argument("--table", action="store_true", help="per-configuration throughput table (markdown)")
     ap.add_argument("--only", default=None, choices=("fwd", "bwd", "gemv", "quantize", "merge", "adamw"))
     ap.add_argument("--shape", default="cfg3_7b_up")
@@ -583,6 +692,8 @@ def main():
     args = ap.parse_args()
     if args.table:
         run_table(args)
+    elif args.baselines:
+        run_baselines(args)
     elif args.only is not None:
         run_only(args)
     elif args.impl == "reference":
