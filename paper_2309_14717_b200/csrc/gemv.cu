@@ -336,23 +336,55 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int col_beg = GV_COLS * rank / splits, col_end = GV_COLS * (rank + 1) / splits;
     const int cols_per = col_end - col_beg;
     const int outs = p.M * cols_per;
-    for (int o = threadIdx.x; o < outs; o += GV_THREADS) {
-      const int row = o / cols_per, col = col_beg + o % cols_per;
-      float v = 0.f;
-      for (int rk = 0; rk < splits; ++rk) {
-        const float* remote = cluster.map_shared_rank(partial, rk);
-#pragma unroll
-        for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
-      }
-      if (p.r > 0) {
-        const float* Tr = p.T + (size_t)row * p.r;
-        const __nv_bfloat16* Bc = p.B + n0 + col;
-        float a = 0.f;
+    if (p.r > 0) {
+      // T is written by the pooling kernel, which this kernel is allowed to overtake (it is
+      // launched with programmatic stream serialization): wait for it only now.  A no-op when
+      // the launch carried no such attribute.
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      // P neighbouring lanes share an output (P = 8, 4, 2 or 1: as many as the eight consumer
+      // warps have to spare, so that one pass covers the block's outputs whenever it can) and
+      // split the adapter rows between them, i = l (mod P), so that their loads of B are in
+      // flight together; shuffles add the lanes' parts in a fixed order and lane 0 of them
+      // adds the slices.
+      constexpr int EPI_THREADS = GV_WARPS * 32;
+      int P = 1;
+      while (P < 8 && outs * (2 * P) <= EPI_THREADS) P *= 2;
+      if (threadIdx.x < EPI_THREADS) {
+        const int lp = threadIdx.x & (P - 1);
+        for (int o0 = 0; o0 < outs; o0 += EPI_THREADS / P) {      // uniform trip count: the shuffles see whole warps
+          const int o = o0 + threadIdx.x / P;
+          const bool live = o < outs;
+          const int row = live ? o / cols_per : 0, col = col_beg + (live ? o % cols_per : 0);
+          const float* Tr = p.T + (size_t)row * p.r;
+          const __nv_bfloat16* Bc = p.B + n0 + col;
+          float a = 0.f;
 #pragma unroll 8
-        for (int i = 0; i < p.r; ++i) a = fmaf(Tr[i], __bfloat162float(Bc[(size_t)i * p.N]), a);
-        v += a;
+          for (int i = lp; i < p.r; i += P) a = fmaf(Tr[i], __bfloat162float(Bc[(size_t)i * p.N]), a);
+          if (P > 1) a += __shfl_xor_sync(0xffffffffu, a, 1);
+          if (P > 2) a += __shfl_xor_sync(0xffffffffu, a, 2);
+          if (P > 4) a += __shfl_xor_sync(0xffffffffu, a, 4);
+          if (live && lp == 0) {
+            float v = 0.f;
+            for (int rk = 0; rk < splits; ++rk) {
+              const float* remote = cluster.map_shared_rank(partial, rk);
+#pragma unroll
+              for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
+            }
+            p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v + a);
+          }
+        }
       }
-      p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v);
+    } else {
+      for (int o = threadIdx.x; o < outs; o += GV_THREADS) {
+        const int row = o / cols_per, col = col_beg + o % cols_per;
+        float v = 0.f;
+        for (int rk = 0; rk < splits; ++rk) {
+          const float* remote = cluster.map_shared_rank(partial, rk);
+#pragma unroll
+          for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
+        }
+        p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v);
+      }
     }
   }
   cluster.sync();
@@ -423,13 +455,18 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   cfg.blockDim = dim3(GV_THREADS);
   cfg.dynamicSmemBytes = S::TOTAL;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // With an adapter the kernel before this one in the stream is the pooling kernel that
+  // writes T, which is read only at the very end: let this kernel start beside it.  (With
+  // more than 8 token rows the pooling kernel is larger and the overlap measured slower.)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (p.T != nullptr && !UPPER) ? 2 : 1;
   cudaError_t e;
   {
     MainKernelProbe probe("qalora_gemv_kernel", st);

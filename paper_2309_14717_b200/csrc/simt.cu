@@ -16,6 +16,9 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
               float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
               int K, int g, int G, int r, float s) {
   extern __shared__ float xp[];                       // [G]
+  // The few-token forward kernel that follows needs T only at its very end: let it start now
+  // (it waits for this grid before it reads T).  Without such a dependent launch this does nothing.
+  asm volatile("griddepcontrol.launch_dependents;");
   const size_t m = blockIdx.x;
   const __nv_bfloat16* xr = x + m * (size_t)K;
   // four lanes per group, 8 channels (16 bytes) per lane and step; g is a multiple of 32
