@@ -228,8 +228,6 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
           mma16816(cinit[ts], ones4, xs[1][ts].z, xs[1][ts].w, cinit[ts]);
           xp[ts][0] = cinit[ts][0];
           xp[ts][1] = cinit[ts][1];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) cinit[ts][i] *= -128.f;
         }
         const uint8_t* qrow = stage + q_off + (((set * (GV_KBS / GV_SETS)) >> qsh) * S::QP_ROW);
 #pragma unroll
@@ -250,12 +248,14 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
             const uint32_t a1[4] = {f[0][2], f[1][2], f[0][3], f[1][3]};
 #pragma unroll
             for (int ts = 0; ts < NTS; ++ts) {
-              mma16816(D[ts], a0, xs[bb][ts].x, xs[bb][ts].y, bb == 0 ? cinit[ts] : D[ts]);
+              mma16816(D[ts], a0, xs[bb][ts].x, xs[bb][ts].y, bb == 0 ? zero4 : D[ts]);
               mma16816(D[ts], a1, xs[bb][ts].z, xs[bb][ts].w, D[ts]);
             }
           }
-          const float2 q0 = *reinterpret_cast<const float2*>(qrow + (cg * 16) * 8);
-          const float2 q1 = *reinterpret_cast<const float2*>(qrow + (cg * 16 + 8) * 8);
+          float2 q0 = *reinterpret_cast<const float2*>(qrow + (cg * 16) * 8);
+          float2 q1 = *reinterpret_cast<const float2*>(qrow + (cg * 16 + 8) * 8);
+          q0.y = fmaf(-128.f, q0.x, q0.y);      // D holds sum (128 + c) x: the offset goes into the xp term
+          q1.y = fmaf(-128.f, q1.x, q1.y);
 #pragma unroll
           for (int ts = 0; ts < NTS; ++ts) {
             acc[cg][ts][0] = fmaf(q0.x, D[ts][0], fmaf(q0.y, xp[ts][0], acc[cg][ts][0]));
@@ -280,8 +280,6 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
           mma16816(cinit[ts], ones4, xs[ts].z, xs[ts].w, cinit[ts]);
           xp[ts][0] = cinit[ts][0];
           xp[ts][1] = cinit[ts][1];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) cinit[ts][i] *= -128.f;
         }
         const uint8_t* qrow = stage + q_off + (((set * (GV_KBS / GV_SETS) + bb) >> qsh) * S::QP_ROW);
 #pragma unroll
@@ -297,13 +295,14 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
             if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t);
             code_fragments<BITS>(lo, hi, fk, f[j]);
             q[j] = *reinterpret_cast<const float2*>(qrow + (cg * 16 + j * 8) * 8);
+            q[j].y = fmaf(-128.f, q[j].x, q[j].y);    // D holds sum (128 + c) x: the offset goes into the xp term
           }
           const uint32_t a0[4] = {f[0][0], f[1][0], f[0][1], f[1][1]};
           const uint32_t a1[4] = {f[0][2], f[1][2], f[0][3], f[1][3]};
 #pragma unroll
           for (int ts = 0; ts < NTS; ++ts) {
             float D[4];
-            mma16816(D, a0, xs[ts].x, xs[ts].y, cinit[ts]);
+            mma16816(D, a0, xs[ts].x, xs[ts].y, zero4);
             mma16816(D, a1, xs[ts].z, xs[ts].w, D);
             acc[cg][ts][0] = fmaf(q[0].x, D[0], fmaf(q[0].y, xp[ts][0], acc[cg][ts][0]));
             acc[cg][ts][1] = fmaf(q[0].x, D[1], fmaf(q[0].y, xp[ts][1], acc[cg][ts][1]));
