@@ -186,6 +186,39 @@ def test_few_token_forward_all_widths(bits, g, M, r):
     assert rel_err(got.float().cpu().numpy(), y_ref) <= TOL
 
 
+@pytest.mark.parametrize("M", [1, 8])
+def test_few_token_forward_back_to_back_calls_share_a_workspace(M):
+    """The few-token kernel starts while the pooling kernel that writes T = s pool(x) A is still
+    running and may read T only once that kernel is complete.  Many calls in a row on one stream,
+    with one workspace and inputs that change from call to call (a large layer, so that the main
+    kernel is still streaming when the next call is queued): every output must be its own
+    input's, never a mix with the neighbouring call's T."""
+    cfg = LayerConfig("gemv_b2b", 4096, 1024, 32, 4, 64, 4.0, M, seed=77)
+    layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
+    codes, alpha, beta = check_quantize(layer)
+    gen = torch.Generator(device="cpu").manual_seed(1234)
+    calls = 6
+    # large adapter weights make the adapter term as large as the base term, so that a stale T shows
+    A = (torch.randn((cfg.groups, cfg.rank), generator=gen) * 0.5).to(torch.bfloat16)
+    B = (torch.randn((cfg.rank, cfg.d_out), generator=gen) * 0.5).to(torch.bfloat16)
+    xs = [(torch.randn((M, cfg.d_in), generator=gen) * (1.0 + i)).to(torch.bfloat16) for i in range(calls)]
+    Ad, Bd = A.cuda(), B.cuda()
+    xd = [x.cuda() for x in xs]
+    ys = [torch.empty((M, cfg.d_out), dtype=torch.bfloat16, device="cuda") for _ in range(calls)]
+    ws = Q.alloc_workspace(layer.d, M, Q.OP_FORWARD)
+    torch.cuda.synchronize()
+    for i in range(calls):
+        Q.qalora_forward(layer.d, M, xd[i], layer.codes, layer.qparams, Ad, Bd, ys[i], ws)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(ws) == 0
+    for i in range(calls):
+        y_ref = O.forward(to_f64(xs[i]), codes, alpha, beta, cfg.group_size, to_f64(A), to_f64(B), cfg.scale)
+        adapter = O.forward(to_f64(xs[i]), codes, alpha, beta, cfg.group_size, to_f64(A), to_f64(B), cfg.scale) - \
+            O.forward(to_f64(xs[i]), codes, alpha, beta, cfg.group_size)
+        assert np.max(np.abs(adapter)) > 0.2 * np.max(np.abs(y_ref))     # the case does exercise T
+        assert rel_err(ys[i].float().cpu().numpy(), y_ref) <= TOL, i
+
+
 def test_edge_cases():
     cfg = LayerConfig("edge", 64, 64, 32, 4, 8, 1.0, 3, seed=9)
     layer = GpuLayer(cfg)
