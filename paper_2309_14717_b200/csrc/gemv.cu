@@ -42,15 +42,12 @@ constexpr int GV_SETS = 2;          // consumer warp sets; set s takes the k-blo
 constexpr int GV_WARPS = 4 * GV_SETS;   // consumer warps: 4 per set, 32 columns each
 constexpr int GV_THREADS = (GV_WARPS + 1) * 32;   // + 1 producer warp
 constexpr int GV_KBS = 4;           // 32-channel blocks per stage (128 channels)
-#ifndef GV_NST
-#define GV_NST 4
-#endif
 constexpr int GV_ROWS = 16;         // most token rows
 
 template <int BITS, bool UPPER>   // UPPER: more than 8 token rows
 struct GvSmem {
   static constexpr int ROWS = UPPER ? 16 : 8;                           // token rows held in shared memory
-  static constexpr int STAGES = UPPER ? 3 : GV_NST;                        // three blocks per SM either way
+  static constexpr int STAGES = UPPER ? 3 : 4;                          // three blocks per SM either way
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   static constexpr uint32_t CODE_ROW = GV_COLS * WORDS * 4;             // one k-block row of units
   static constexpr uint32_t QP_ROW = GV_COLS * 8;
