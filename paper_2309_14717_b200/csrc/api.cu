@@ -39,6 +39,8 @@ int check_desc(const qalora_desc* d, Shape* sh) {
 
 // Token counts up to this take the bandwidth-bound small-M path.
 static constexpr int64_t kSmallM = 16;
+// The forward pass alone keeps the few-token kernel up to this many tokens (where its shapes allow).
+static constexpr int64_t kFewTokenM = 32;
 
 Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   Workspace w{};
@@ -171,13 +173,14 @@ int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void
                        nullptr, T, Tb, stream);
     if (st != QALORA_OK) return st;
   }
-  if (m <= kSmallM && gemv_supported(sh, m)) {
+  const bool few = m <= kFewTokenM && gemv_supported(sh, m);
+  if (few) {
     return launch_gemv(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
                        reinterpret_cast<const float2*>(qparams), sh.r > 0 ? T : nullptr,
                        static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(y),
                        reinterpret_cast<int*>(wsp + ws.status), stream);
   }
-  if (m > kSmallM && tc_forward_supported(sh, m)) {
+  if (!few && m > kSmallM && tc_forward_supported(sh, m)) {
     int* status = reinterpret_cast<int*>(wsp + ws.status);
     if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
     return launch_tc_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),

@@ -42,12 +42,12 @@ constexpr int GV_SETS = 2;          // consumer warp sets; set s takes the k-blo
 constexpr int GV_WARPS = 4 * GV_SETS;   // consumer warps: 4 per set, 32 columns each
 constexpr int GV_THREADS = (GV_WARPS + 1) * 32;   // + 1 producer warp
 constexpr int GV_KBS = 4;           // 32-channel blocks per stage (128 channels)
-constexpr int GV_ROWS = 16;         // most token rows
+constexpr int GV_ROWS = 32;         // most token rows
 
-template <int BITS, bool UPPER>   // UPPER: more than 8 token rows
+template <int BITS, int NTS>      // NTS: sets of 8 token rows (1, 2 or 4)
 struct GvSmem {
-  static constexpr int ROWS = UPPER ? 16 : 8;                           // token rows held in shared memory
-  static constexpr int STAGES = UPPER ? 3 : 4;                          // three blocks per SM either way
+  static constexpr int ROWS = 8 * NTS;                                  // token rows held in shared memory
+  static constexpr int STAGES = NTS == 1 ? 4 : 3;                       // three blocks per SM (two with 32 rows)
   static constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   static constexpr uint32_t CODE_ROW = GV_COLS * WORDS * 4;             // one k-block row of units
   static constexpr uint32_t QP_ROW = GV_COLS * 8;
@@ -116,13 +116,13 @@ __device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, const F
   }
 }
 
-// UPPER: token rows 8..15 are in use (M > 8).  CHAIN: the group size is 64 or 128, so the two
+// NTS: sets of 8 token rows in use (M <= 8 NTS).  CHAIN: the group size is 64 or 128, so the two
 // k-blocks a warp set takes from a stage share (alpha, beta) and are folded together.
-template <int BITS, bool UPPER, bool CHAIN>
-__global__ void __launch_bounds__(GV_THREADS, 3)
+template <int BITS, int NTS, bool CHAIN>
+__global__ void __launch_bounds__(GV_THREADS, NTS == 4 ? 2 : 3)
 qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
                    const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
-  using S = GvSmem<BITS, UPPER>;
+  using S = GvSmem<BITS, NTS>;
   constexpr int WORDS = S::WORDS;
   constexpr int GV_STAGES = S::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -186,7 +186,6 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int set = warp / 4, wcol = (warp % 4) * 32;
     const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block of the stage -> its (alpha, beta) row
     const int gq = lane / 4, t = lane % 4;        // fragment row (column of W, token), quad lane
-    constexpr int NTS = UPPER ? 2 : 1;            // sets of 8 tokens
     // per-thread byte offsets inside a stage; everything else is a compile-time constant
     const uint32_t x_off = S::OFF_X + gq * (GV_KBS * 64) + t * 16 + set * (GV_KBS / GV_SETS) * 64;
     const uint32_t lo_word = BITS == 4 ? t : (t >> 1);
@@ -216,8 +215,9 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         uint4 xs[2][NTS];
 #pragma unroll
         for (int bb = 0; bb < 2; ++bb) {
-          xs[bb][0] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64);
-          if (UPPER) xs[bb][NTS - 1] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + 8 * (GV_KBS * 64));
+#pragma unroll
+          for (int ts = 0; ts < NTS; ++ts)
+            xs[bb][ts] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + ts * 8 * (GV_KBS * 64));
         }
         float cinit[NTS][4], xp[NTS][2];
 #pragma unroll
@@ -270,8 +270,9 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         // this set's k-block b = 2 set + bb; B fragments: x[token gq (+ 8)][32 b + 8 t .. + 7]:
         // the lane's k slots (2t, 2t+1 | 2t+8, 2t+9) of MMA 0 are channels 8t .. 8t+3, those of MMA 1 8t+4 .. 8t+7
         uint4 xs[NTS];
-        xs[0] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64);
-        if (UPPER) xs[NTS - 1] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + 8 * (GV_KBS * 64));
+#pragma unroll
+        for (int ts = 0; ts < NTS; ++ts)
+          xs[ts] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + ts * 8 * (GV_KBS * 64));
         // xp of the tokens (ones as the A operand: every row of the product holds the sums), then C = -128 xp
         float cinit[NTS][4], xp[NTS][2];
 #pragma unroll
@@ -417,14 +418,14 @@ int gv_sm_count() {
   return n;
 }
 
-template <int BITS, bool UPPER, bool CHAIN>
+template <int BITS, int NTS, bool CHAIN>
 int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
   EncodeTiledFn fn = gv_encode_fn();
   CUtensorMap cm, qm;
   {
     // packed codes [K/32][N][words] uint32 seen as a 2-D matrix of 8-byte elements, so that
     // one box row is the whole contiguous run of 128 pack units (2 KiB at 4 bits)
-    constexpr int W = GvSmem<BITS, UPPER>::WORDS;
+    constexpr int W = GvSmem<BITS, NTS>::WORDS;
     cuuint64_t dims[2] = {(cuuint64_t)p.N * W / 2, (cuuint64_t)(p.K / 32)};
     cuuint64_t strides[1] = {(cuuint64_t)p.N * W * 4};
     cuuint32_t box[2] = {(cuuint32_t)(GV_COLS * W / 2), GV_KBS};
@@ -443,8 +444,8 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return QALORA_ERR_CUDA;
   }
-  using S = GvSmem<BITS, UPPER>;
-  auto kern = qalora_gemv_kernel<BITS, UPPER, CHAIN>;
+  using S = GvSmem<BITS, NTS>;
+  auto kern = qalora_gemv_kernel<BITS, NTS, CHAIN>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
@@ -465,7 +466,7 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (p.T != nullptr && !UPPER) ? 2 : 1;
+  cfg.numAttrs = (p.T != nullptr && NTS == 1) ? 2 : 1;
   cudaError_t e;
   {
     MainKernelProbe probe("qalora_gemv_kernel", st);
@@ -477,10 +478,44 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
 
 }  // namespace
 
+// Slices per column tile (= cluster size): the count among {1,2,3,4,6,8} that brings the
+// grid closest to two blocks per SM.  Three blocks fit on an SM, so the grid stays one
+// wave with room for imbalance, while a block still streams enough bytes to amortize its
+// fixed cost (launch, barrier set-up, first-byte latency, two cluster barriers).  With more
+// than 16 token rows only two blocks fit on an SM: there the grid must not exceed two blocks
+// per SM, or a second wave would follow.
+static int gv_slices(const Shape& sh, int64_t M) {
+  const int tiles = sh.N / GV_COLS, total_stages = sh.K / (GV_KBS * 32), target = 2 * gv_sm_count();
+  const bool capped = M > 16;
+  int splits = 1, best = 1 << 30;
+  for (int sp : {1, 2, 3, 4, 6, 8}) {
+    if (sp > total_stages) break;
+    if (capped && sp > 1 && tiles * sp > target) break;
+    const int miss = tiles * sp > target ? tiles * sp - target : target - tiles * sp;
+    if (miss < best) { best = miss; splits = sp; }
+  }
+  return splits;
+}
+
 bool gemv_supported(const Shape& sh, int64_t M) {
-  return M >= 1 && M <= GV_ROWS && sh.N % GV_COLS == 0 && sh.K % (GV_KBS * 32) == 0 &&
-         (sh.g == 32 || sh.g == 64 || sh.g == 128) &&
-         gv_encode_fn() != nullptr;
+  if (!(M >= 1 && M <= GV_ROWS && sh.N % GV_COLS == 0 && sh.K % (GV_KBS * 32) == 0 &&
+        (sh.g == 32 || sh.g == 64 || sh.g == 128) && gv_encode_fn() != nullptr))
+    return false;
+  if (M > 16) {
+    // 17..32 rows: the tensor-pipe work per code grows with the rows and only two blocks fit
+    // on an SM, so this kernel beats the 64-token tensor-core tile only where its grid fills
+    // the SMs evenly (measured, merged layers: 15 against 20 us for a 4096 x 4096 layer whose
+    // 256 blocks fill 86 % of two per SM; 116 against 88 us for 8192 x 22016, whose 172 blocks
+    // fill 58 %), and only for a layer without adapter: the tensor-core kernel folds the
+    // adapter into its MMA steps, while here T * B is summed per output at the end, which
+    // costs more than the streaming saves once there are thousands of outputs per block.
+    if (sh.r > 0) return false;
+    const int sms = gv_sm_count();
+    const long long blocks = (long long)(sh.N / GV_COLS) * gv_slices(sh, M);
+    const long long waves = (blocks + sms - 1) / sms;
+    if (blocks > sms && (waves > 2 || blocks * 4 < waves * sms * 3)) return false;
+  }
+  return true;
 }
 
 // y = x * W~ + T * B for M <= 16 rows; T is fp32 [M][r] with s folded in (null when r == 0).
@@ -490,7 +525,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   CUtensorMap xm;
   cuuint64_t dims[2] = {(cuuint64_t)sh.K, (cuuint64_t)M};
   cuuint64_t strides[1] = {(cuuint64_t)sh.K * 2};
-  cuuint32_t box[2] = {GV_KBS * 32, (cuuint32_t)(M > 8 ? 16 : 8)};   // the token rows the kernel keeps
+  cuuint32_t box[2] = {GV_KBS * 32, (cuuint32_t)(M > 16 ? 32 : (M > 8 ? 16 : 8))};   // the token rows the kernel keeps
   cuuint32_t estr[2] = {1, 1};
   if (fn(&xm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(x), dims, strides, box, estr,
          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -501,26 +536,17 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;
-  // slices per column tile (= cluster size): the count among {1,2,3,4,6,8} that brings the
-  // grid closest to two blocks per SM.  Three blocks fit on an SM, so the grid stays one
-  // wave with room for imbalance, while a block still streams enough bytes to amortize its
-  // fixed cost (launch, barrier set-up, first-byte latency, two cluster barriers).
-  const int tiles = sh.N / GV_COLS, target = 2 * gv_sm_count();
-  int splits = 1, best = 1 << 30;
-  for (int sp : {1, 2, 3, 4, 6, 8}) {
-    if (sp > p.total_stages) break;
-    const int miss = tiles * sp > target ? tiles * sp - target : target - tiles * sp;
-    if (miss < best) { best = miss; splits = sp; }
-  }
-  const bool upper = M > 8;
+  const int splits = gv_slices(sh, M);
+  const int nts = M > 16 ? 4 : (M > 8 ? 2 : 1);
   const bool chain = sh.g >= 64;
-#define QALORA_GV(BITS)                                                                                              \
-  (upper ? (chain ? launch_gemv_t<BITS, true, true>(xm, p, splits, st) : launch_gemv_t<BITS, true, false>(xm, p, splits, st))   \
-         : (chain ? launch_gemv_t<BITS, false, true>(xm, p, splits, st) : launch_gemv_t<BITS, false, false>(xm, p, splits, st)))
+#define QALORA_GV_N(BITS, NTS) (chain ? launch_gemv_t<BITS, NTS, true>(xm, p, splits, st) : launch_gemv_t<BITS, NTS, false>(xm, p, splits, st))
+// (32 rows: the per-k-block fold for every group size; the chained form runs out of registers there)
+#define QALORA_GV(BITS) (nts == 4 ? launch_gemv_t<BITS, 4, false>(xm, p, splits, st) : (nts == 2 ? QALORA_GV_N(BITS, 2) : QALORA_GV_N(BITS, 1)))
   if (sh.bits == 4) return QALORA_GV(4);
   if (sh.bits == 3) return QALORA_GV(3);
   return QALORA_GV(2);
 #undef QALORA_GV
+#undef QALORA_GV_N
 }
 
 }  // namespace qalora

@@ -100,7 +100,7 @@ SMALL = [
     # few tokens and a long reduction: the forward contraction is cut into parts that meet in scratch
     ("parts4", 2048, 256, 32, 4, 16, 1.0, 40),
     ("parts3", 1536, 384, 64, 3, 24, 0.75, 300),
-    ("parts2", 4096, 128, 128, 2, 8, 1.5, 17),
+    ("parts2", 4096, 128, 128, 2, 8, 1.5, 33),
     # many tokens, several channel tiles, ragged token count
     ("pair4", 512, 256, 32, 4, 16, 1.0, 700),
     ("pair3", 384, 512, 64, 3, 24, 0.75, 530),
@@ -168,10 +168,12 @@ def test_config2_small_m_forward_and_merge(M):
 
 
 @pytest.mark.parametrize("bits,g,M,r", [(4, 32, 1, 16), (4, 128, 8, 0), (3, 32, 16, 24), (3, 64, 3, 8),
-                                       (2, 32, 9, 64), (2, 128, 1, 0), (4, 64, 16, 128)])
+                                       (2, 32, 9, 64), (2, 128, 1, 0), (4, 64, 16, 128),
+                                       (4, 32, 17, 0), (4, 128, 32, 0), (3, 64, 25, 0), (2, 32, 32, 0)])
 def test_few_token_forward_all_widths(bits, g, M, r):
     """The bandwidth-bound few-token kernel (N % 128 == 0, K % 128 == 0): every bit
-    width, group sizes 32/64/128, with and without the adapter, M below and above 8."""
+    width, group sizes 32/64/128, with and without the adapter, M in every set of eight rows
+    up to 32 (17..32 rows: layers without adapter only; adapted ones take the tensor-core kernel)."""
     cfg = LayerConfig("gemv", 1280, 384, g, bits, max(r, 8), 1.25, M, outlier_frac=0.01, seed=bits * 100 + g + M)
     layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
     codes, alpha, beta = check_quantize(layer)
