@@ -75,25 +75,38 @@ class ClockSampler:
     def __init__(self, gpu_uuid):
         self.uuid = gpu_uuid
         self.proc = None
-        self.lines = []
+        self.lines = []          # (arrival time, text)
+        self.t_begin = self.t_end = None
 
     def start(self):
+        """Starts nvidia-smi (it needs a few hundred ms before its first sample, so this is
+        called before the warm-up) and waits for the first line."""
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                  "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
+            deadline = time.monotonic() + 5.0
+            while not self.lines and time.monotonic() < deadline and self.proc.poll() is None:
+                time.sleep(0.01)
         except OSError:
             self.proc = None
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
+
+    def begin(self):
+        self.t_begin = time.monotonic()
+
+    def end(self):
+        self.t_end = time.monotonic()
 
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.03)          # let the last sample of the region arrive
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -101,7 +114,12 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons, power = [], [], set(), []
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
+        # samples taken during the timed region (a sample is printed right after it is taken)
+        t0 = self.t_begin if self.t_begin is not None else float("-inf")
+        t1 = (self.t_end if self.t_end is not None else float("inf")) + 0.02
+        for stamp, line in self.lines:
+            if not (t0 <= stamp <= t1):
+                continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 7:
                 continue
@@ -275,13 +293,15 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
         if sampler:
-            sampler.start()
+            sampler.begin()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(steps):
             fn()
         e1.record(stream)
         torch.cuda.synchronize()
+        if sampler:
+            sampler.end()
         if world > 1:
             dist.barrier()
         clocks = sampler.stop() if sampler else None
@@ -292,12 +312,14 @@ def run_gpu(args):
             ms = float(t.item())
         return ms, clocks
 
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    sampler = ClockSampler(uuid)
+    sampler.start()                                 # before the warm-up: its first sample takes a while
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
 
-    uuid = str(torch.cuda.get_device_properties(local).uuid)
-    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
     probe_pairs = []
     for _ in range(args.steps):
         ka, kb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -306,7 +328,7 @@ def run_gpu(args):
     probes.extend(probe_pairs)
     torch.cuda.synchronize()
     launches0 = Q.qalora_kernel_launches()
-    ms_total, clocks = timed(step, args.steps, ClockSampler(uuid))
+    ms_total, clocks = timed(step, args.steps, sampler)
     s0_ = shapes[0]
     Q.qalora_forward(s0_.d, s0_.cfg.tokens, s0_.x, s0_.codes, s0_.qparams, s0_.A, s0_.B, s0_.y, s0_.ws_f)
     kernel_name = Q.qalora_main_kernel_name()       # which kernel the library picks for this shape

@@ -176,7 +176,7 @@ int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void
   const bool few = m <= kFewTokenM && gemv_supported(sh, m);
   if (few) {
     return launch_gemv(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
-                       reinterpret_cast<const float2*>(qparams), sh.r > 0 ? T : nullptr,
+                       reinterpret_cast<const float2*>(qparams), sh.r > 0 ? Tb : nullptr,
                        static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(y),
                        reinterpret_cast<int*>(wsp + ws.status), stream);
   }

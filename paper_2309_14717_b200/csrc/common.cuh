@@ -108,10 +108,10 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
                  __nv_bfloat16* dx, int* status, cudaStream_t st);
 
-// Few-token forward (gemv.cu): M <= 16.
+// Few-token forward (gemv.cu): M <= 32.
 bool gemv_supported(const Shape& sh, int64_t M);
 int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
-                const float* T, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, cudaStream_t st);
+                const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, cudaStream_t st);
 
 // out[i] = sum over splits of partial[z][i], added in a fixed order.
 int launch_sum_partials(const float* partial, float* out, size_t count, int splits, cudaStream_t st);

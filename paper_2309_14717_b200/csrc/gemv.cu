@@ -64,7 +64,7 @@ struct GvSmem {
 struct GvParams {
   const uint32_t* codes;
   const float2* qparams;
-  const float* T;               // fp32 [M][r] (s folded in) or null
+  const __nv_bfloat16* Tb;      // bf16 [M][r], T = s * pool(x) * A, or null
   const __nv_bfloat16* B;       // [r][N]
   __nv_bfloat16* y;             // [M][N]
   int M, K, N, g, r;
@@ -316,6 +316,44 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar_empty(s));
     }
+    if (p.r > 0 && rank == 0) {
+      // Adapter term T * B, once per column tile (by the cluster's first block), as more MMAs
+      // into the same accumulators: rows = columns of B (A operand: B transposed, two 2-byte
+      // loads per register, from L2), columns = tokens (B operand: T in bf16, as the
+      // tensor-core kernel takes it).  The sets take alternate 16-row steps of the rank;
+      // rows beyond it read as zero.  T is written by the pooling kernel, which this kernel
+      // is allowed to overtake (programmatic stream serialization): wait for it only now (a
+      // no-op when the launch carried no such attribute).
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      const unsigned short* Bu = reinterpret_cast<const unsigned short*>(p.B);
+      const unsigned short* Tu = reinterpret_cast<const unsigned short*>(p.Tb);
+      auto pair = [](const unsigned short* base, size_t stride, int i, int r) -> uint32_t {   // (base[i], base[i + 1]) along stride
+        const uint32_t lo = i < r ? base[(size_t)i * stride] : 0u;
+        const uint32_t hi = i + 1 < r ? base[(size_t)(i + 1) * stride] : 0u;
+        return lo | (hi << 16);
+      };
+      const int ksteps = (p.r + 15) / 16;
+      for (int ks = set; ks < ksteps; ks += GV_SETS) {
+        const int i0 = ks * 16 + 2 * t;
+        uint32_t tb[NTS][2];
+#pragma unroll
+        for (int ts = 0; ts < NTS; ++ts) {
+          const int token = ts * 8 + gq;
+          const bool live = token < p.M;
+          const unsigned short* Tr = Tu + (size_t)(live ? token : 0) * p.r;
+          tb[ts][0] = live ? pair(Tr, 1, i0, p.r) : 0u;
+          tb[ts][1] = live ? pair(Tr, 1, i0 + 8, p.r) : 0u;
+        }
+#pragma unroll
+        for (int cg = 0; cg < 2; ++cg) {
+          const unsigned short* c0 = Bu + n0 + wcol + cg * 16 + gq;
+          const uint32_t a[4] = {pair(c0, p.N, i0, p.r), pair(c0 + 8, p.N, i0, p.r),
+                                 pair(c0, p.N, i0 + 8, p.r), pair(c0 + 8, p.N, i0 + 8, p.r)};
+#pragma unroll
+          for (int ts = 0; ts < NTS; ++ts) mma16816(acc[cg][ts], a, tb[ts][0], tb[ts][1], acc[cg][ts]);
+        }
+      }
+    }
     // partial sums of this warp set: [16 token rows][128 columns]
     float* mine = partial + set * (S::ROWS * GV_COLS);
 #pragma unroll
@@ -336,55 +374,15 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int col_beg = GV_COLS * rank / splits, col_end = GV_COLS * (rank + 1) / splits;
     const int cols_per = col_end - col_beg;
     const int outs = p.M * cols_per;
-    if (p.r > 0) {
-      // T is written by the pooling kernel, which this kernel is allowed to overtake (it is
-      // launched with programmatic stream serialization): wait for it only now.  A no-op when
-      // the launch carried no such attribute.
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      // P neighbouring lanes share an output (P = 8, 4, 2 or 1: as many as the eight consumer
-      // warps have to spare, so that one pass covers the block's outputs whenever it can) and
-      // split the adapter rows between them, i = l (mod P), so that their loads of B are in
-      // flight together; shuffles add the lanes' parts in a fixed order and lane 0 of them
-      // adds the slices.
-      constexpr int EPI_THREADS = GV_WARPS * 32;
-      int P = 1;
-      while (P < 8 && outs * (2 * P) <= EPI_THREADS) P *= 2;
-      if (threadIdx.x < EPI_THREADS) {
-        const int lp = threadIdx.x & (P - 1);
-        for (int o0 = 0; o0 < outs; o0 += EPI_THREADS / P) {      // uniform trip count: the shuffles see whole warps
-          const int o = o0 + threadIdx.x / P;
-          const bool live = o < outs;
-          const int row = live ? o / cols_per : 0, col = col_beg + (live ? o % cols_per : 0);
-          const float* Tr = p.T + (size_t)row * p.r;
-          const __nv_bfloat16* Bc = p.B + n0 + col;
-          float a = 0.f;
-#pragma unroll 8
-          for (int i = lp; i < p.r; i += P) a = fmaf(Tr[i], __bfloat162float(Bc[(size_t)i * p.N]), a);
-          if (P > 1) a += __shfl_xor_sync(0xffffffffu, a, 1);
-          if (P > 2) a += __shfl_xor_sync(0xffffffffu, a, 2);
-          if (P > 4) a += __shfl_xor_sync(0xffffffffu, a, 4);
-          if (live && lp == 0) {
-            float v = 0.f;
-            for (int rk = 0; rk < splits; ++rk) {
-              const float* remote = cluster.map_shared_rank(partial, rk);
+    for (int o = threadIdx.x; o < outs; o += GV_THREADS) {
+      const int row = o / cols_per, col = col_beg + o % cols_per;
+      float v = 0.f;
+      for (int rk = 0; rk < splits; ++rk) {
+        const float* remote = cluster.map_shared_rank(partial, rk);
 #pragma unroll
-              for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
-            }
-            p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v + a);
-          }
-        }
+        for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
       }
-    } else {
-      for (int o = threadIdx.x; o < outs; o += GV_THREADS) {
-        const int row = o / cols_per, col = col_beg + o % cols_per;
-        float v = 0.f;
-        for (int rk = 0; rk < splits; ++rk) {
-          const float* remote = cluster.map_shared_rank(partial, rk);
-#pragma unroll
-          for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
-        }
-        p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v);
-      }
+      p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v);
     }
   }
   cluster.sync();
@@ -461,12 +459,14 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   // With an adapter the kernel before this one in the stream is the pooling kernel that
-  // writes T, which is read only at the very end: let this kernel start beside it.  (With
-  // more than 8 token rows the pooling kernel is larger and the overlap measured slower.)
+  // writes T, which is read only after the last stage: let this kernel start beside it.  With
+  // more than 8 token rows the pooling kernel is larger, and beside a short main loop the
+  // overlap measured slower (4096 x 4096, 16 rows: 15.7 against 14.8 us), beside a long one
+  // faster (8192 x 22016: 56 against 63 us): there it is used from 64 Mi weights on.
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (p.T != nullptr && NTS == 1) ? 2 : 1;
+  cfg.numAttrs = (p.Tb != nullptr && (NTS == 1 || (long long)p.K * p.N >= (64ll << 20))) ? 2 : 1;
   cudaError_t e;
   {
     MainKernelProbe probe("qalora_gemv_kernel", st);
@@ -509,7 +509,6 @@ bool gemv_supported(const Shape& sh, int64_t M) {
     // fill 58 %), and only for a layer without adapter: the tensor-core kernel folds the
     // adapter into its MMA steps, while here T * B is summed per output at the end, which
     // costs more than the streaming saves once there are thousands of outputs per block.
-    if (sh.r > 0) return false;
     const int sms = gv_sm_count();
     const long long blocks = (long long)(sh.N / GV_COLS) * gv_slices(sh, M);
     const long long waves = (blocks + sms - 1) / sms;
@@ -518,9 +517,9 @@ bool gemv_supported(const Shape& sh, int64_t M) {
   return true;
 }
 
-// y = x * W~ + T * B for M <= 16 rows; T is fp32 [M][r] with s folded in (null when r == 0).
+// y = x * W~ + T * B for M <= 32 rows; Tb is T = s * pool(x) * A in bf16 [M][r] (null when r == 0).
 int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
-                const float* T, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, cudaStream_t st) {
+                const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, cudaStream_t st) {
   EncodeTiledFn fn = gv_encode_fn();
   CUtensorMap xm;
   cuuint64_t dims[2] = {(cuuint64_t)sh.K, (cuuint64_t)M};
@@ -532,7 +531,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return QALORA_ERR_CUDA;
   GvParams p{};
-  p.codes = codes; p.qparams = qparams; p.T = T; p.B = B; p.y = y;
+  p.codes = codes; p.qparams = qparams; p.Tb = Tb; p.B = B; p.y = y;
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;

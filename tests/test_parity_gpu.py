@@ -169,11 +169,11 @@ def test_config2_small_m_forward_and_merge(M):
 
 @pytest.mark.parametrize("bits,g,M,r", [(4, 32, 1, 16), (4, 128, 8, 0), (3, 32, 16, 24), (3, 64, 3, 8),
                                        (2, 32, 9, 64), (2, 128, 1, 0), (4, 64, 16, 128),
-                                       (4, 32, 17, 0), (4, 128, 32, 0), (3, 64, 25, 0), (2, 32, 32, 0)])
+                                       (4, 32, 17, 16), (4, 128, 32, 0), (3, 64, 25, 64), (2, 32, 32, 8), (4, 32, 5, 24), (2, 64, 12, 40)])
 def test_few_token_forward_all_widths(bits, g, M, r):
     """The bandwidth-bound few-token kernel (N % 128 == 0, K % 128 == 0): every bit
-    width, group sizes 32/64/128, with and without the adapter, M in every set of eight rows
-    up to 32 (17..32 rows: layers without adapter only; adapted ones take the tensor-core kernel)."""
+    width, group sizes 32/64/128, with and without the adapter (ranks that are and are not
+    multiples of the 16-row MMA step), M in every set of eight rows up to 32."""
     cfg = LayerConfig("gemv", 1280, 384, g, bits, max(r, 8), 1.25, M, outlier_frac=0.01, seed=bits * 100 + g + M)
     layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
     codes, alpha, beta = check_quantize(layer)
