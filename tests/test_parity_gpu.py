@@ -221,6 +221,39 @@ def test_few_token_forward_back_to_back_calls_share_a_workspace(M):
         assert rel_err(ys[i].float().cpu().numpy(), y_ref) <= TOL, i
 
 
+def test_few_token_forward_replayed_from_a_cuda_graph():
+    """The adapted few-token forward is two launches, the second one started beside the first
+    (programmatic dependent launch).  Captured once into a CUDA graph and replayed with new
+    input values in the same buffers, it must give each replay's own result."""
+    cfg = LayerConfig("gemv_graph", 2048, 512, 64, 4, 32, 2.0, 4, seed=31)
+    layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
+    codes, alpha, beta = check_quantize(layer)
+    A, B = to_f64(layer.cpu["A"]), to_f64(layer.cpu["B"])
+    M = cfg.tokens
+    x_static = torch.zeros((M, cfg.d_in), dtype=torch.bfloat16, device="cuda")
+    y_static = torch.empty((M, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+    ws = Q.alloc_workspace(layer.d, M, Q.OP_FORWARD)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):                     # first call outside the capture: sets kernel attributes
+        Q.qalora_forward(layer.d, M, x_static, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"], y_static, ws)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for _ in range(3):                            # several calls in one graph, as a decoding loop would hold
+            Q.qalora_forward(layer.d, M, x_static, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"], y_static, ws)
+    gen = torch.Generator(device="cpu").manual_seed(5)
+    for rep in range(3):
+        x = (torch.randn((M, cfg.d_in), generator=gen) * (rep + 1)).to(torch.bfloat16)
+        x_static.copy_(x.cuda())
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert Q.workspace_status(ws) == 0
+        y_ref = O.forward(to_f64(x), codes, alpha, beta, cfg.group_size, A, B, cfg.scale)
+        assert rel_err(y_static.float().cpu().numpy(), y_ref) <= TOL, rep
+
+
 def test_edge_cases():
     cfg = LayerConfig("edge", 64, 64, 32, 4, 8, 1.0, 3, seed=9)
     layer = GpuLayer(cfg)
