@@ -24,6 +24,24 @@ MainKernelProbe::~MainKernelProbe() {
   if (stop != nullptr) cudaEventRecord(stop, st);
 }
 
+int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
+int device_sm_count() {
+  static std::atomic<int> cached[kMaxDevices];       // zero-initialized: 0 = not asked yet
+  const int dev = current_device();
+  if (dev < 0) return 148;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+
 int check_desc(const qalora_desc* d, Shape* sh) {
   if (d == nullptr) return QALORA_ERR_NULL_POINTER;
   if (d->d_in <= 0 || d->d_out <= 0 || d->group_size <= 0 || d->rank < 0) return QALORA_ERR_INVALID_ARG;
@@ -65,9 +83,140 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   }
   w.partial_bytes = pb;
   w.partial = take(pb);
-  w.fwd_parts = take(!bwd && m > kSmallM && tc_forward_supported(sh, m) ? tc_forward_partial_bytes(sh, m) : 0);
+  // partial results of the tensor-core forward whose reduction is cut into parts; none where the
+  // dispatcher takes the few-token kernel (same predicate as in forward_launch)
+  const bool few = m <= kFewTokenM && gemv_supported(sh, m);
+  w.fwd_parts = take(!bwd && !few && m > kSmallM && tc_forward_supported(sh, m) ? tc_forward_partial_bytes(sh, m) : 0);
   w.total = off;
   return w;
+}
+
+
+// Argument checks of the forward pass: everything qalora_forward rejects, nothing launched.
+int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
+                     const void* A, const void* B, const void* y, const void* workspace, size_t workspace_bytes) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (m < 0) return QALORA_ERR_INVALID_ARG;
+  if (m == 0) return QALORA_OK;
+  if (x == nullptr || codes == nullptr || qparams == nullptr || y == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (sh.r > 0 && (A == nullptr || B == nullptr)) return QALORA_ERR_NULL_POINTER;
+  const Workspace ws = workspace_layout(sh, m, QALORA_OP_FORWARD);
+  if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) || !aligned16(B) ||
+      !aligned16(y) || !aligned16(workspace))
+    return QALORA_ERR_MISALIGNED;
+  return QALORA_OK;
+}
+
+// The forward pass proper, on arguments forward_validate has accepted (m > 0).  The status
+// word at the head of the workspace is zeroed before the first kernel that can raise it when
+// `reset_status` is set (a public call); qalora_step_host zeroes it once for all its chunks
+// and passes false, so that a time-out raised by an earlier chunk survives to the end.
+int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
+                   const void* A, const void* B, void* y, void* workspace, void* cuda_stream, bool reset_status) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  const Workspace ws = workspace_layout(sh, m, QALORA_OP_FORWARD);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* wsp = static_cast<char*>(workspace);
+  float* T = reinterpret_cast<float*>(wsp + ws.T);
+  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
+  int* status = reinterpret_cast<int*>(wsp + ws.status);
+  const bool few = m <= kFewTokenM && gemv_supported(sh, m);
+  // The few-token kernel clears the word itself (its first block, long before any wait can
+  // expire): a memset node between the pooling kernel and it would undo their overlap.
+  if (reset_status && !few && (st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
+  if (sh.r > 0) {
+    st = launch_pool_T(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(A),
+                       nullptr, T, Tb, stream);
+    if (st != QALORA_OK) return st;
+  }
+  if (few) {
+    return launch_gemv(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
+                       reinterpret_cast<const float2*>(qparams), sh.r > 0 ? Tb : nullptr,
+                       static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(y), status, reset_status, stream);
+  }
+  if (m > kSmallM && tc_forward_supported(sh, m)) {
+    return launch_tc_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
+                             reinterpret_cast<const float2*>(qparams), Tb, static_cast<const __nv_bfloat16*>(B),
+                             static_cast<__nv_bfloat16*>(y), reinterpret_cast<float*>(wsp + ws.fwd_parts), status, stream);
+  }
+  return launch_simt_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
+                             reinterpret_cast<const float2*>(qparams), T, static_cast<const __nv_bfloat16*>(B),
+                             static_cast<__nv_bfloat16*>(y), stream);
+}
+
+int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
+                  const void* codes, const float* qparams, const void* A, const void* B,
+                  void* dx, float* dA, float* dB,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status) {
+  Shape sh;
+  int st = check_desc(desc, &sh);
+  if (st != QALORA_OK) return st;
+  if (m < 0 || sh.r == 0) return QALORA_ERR_INVALID_ARG;
+  if (x == nullptr || dy == nullptr || codes == nullptr || qparams == nullptr || A == nullptr || B == nullptr)
+    return QALORA_ERR_NULL_POINTER;
+  const Workspace ws = workspace_layout(sh, m, QALORA_OP_BACKWARD);
+  if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(x) || !aligned16(dy) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) ||
+      !aligned16(B) || !aligned16(dx) || !aligned16(dA) || !aligned16(dB) || !aligned16(workspace))
+    return QALORA_ERR_MISALIGNED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* wsp = static_cast<char*>(workspace);
+  float* xp = reinterpret_cast<float*>(wsp + ws.xp);
+  float* T = reinterpret_cast<float*>(wsp + ws.T);
+  float* dT = reinterpret_cast<float*>(wsp + ws.dT);
+  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
+  __nv_bfloat16* dTb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.dTb);
+  float* partial = reinterpret_cast<float*>(wsp + ws.partial);
+  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+  const __nv_bfloat16* dyb = static_cast<const __nv_bfloat16*>(dy);
+  const __nv_bfloat16* Ab = static_cast<const __nv_bfloat16*>(A);
+  const __nv_bfloat16* Bb = static_cast<const __nv_bfloat16*>(B);
+
+  if (m == 0) {
+    if (dA != nullptr && (st = cuda_status(cudaMemsetAsync(dA, 0, (size_t)sh.G * sh.r * sizeof(float), stream)))) return st;
+    if (dB != nullptr && (st = cuda_status(cudaMemsetAsync(dB, 0, (size_t)sh.r * sh.N * sizeof(float), stream)))) return st;
+    return QALORA_OK;
+  }
+  int* status = reinterpret_cast<int*>(wsp + ws.status);
+  if (reset_status && (st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
+  const bool aux_tc = m > kSmallM && tc_aux_supported(sh, m);
+  if (aux_tc) st = launch_tc_dT(sh, m, dyb, Bb, dT, dTb, status, stream);
+  else st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream);
+  if (st != QALORA_OK) return st;
+  if (dA != nullptr || dB != nullptr) {
+    if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
+  }
+  if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
+    st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
+                      dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);
+    if (st != QALORA_OK) return st;
+  } else if (dx != nullptr) {
+    st = launch_simt_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
+                        dT, Ab, static_cast<__nv_bfloat16*>(dx), stream);
+    if (st != QALORA_OK) return st;
+  }
+  if (dA != nullptr) {
+    st = launch_atb_f32(m, sh.G, sh.r, xp, dT, dA, partial, ws.partial_bytes, stream);
+    if (st != QALORA_OK) return st;
+  }
+  if (dB != nullptr) {
+    if (aux_tc) {
+      int splits = 0;
+      st = launch_tc_dB_partials(sh, m, Tb, dyb, partial, &splits, status, stream);
+      if (st == QALORA_OK) st = launch_sum_partials(partial, dB, (size_t)sh.r * sh.N, splits, stream);
+    } else {
+      st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial, ws.partial_bytes, stream);
+    }
+    if (st != QALORA_OK) return st;
+  }
+  return QALORA_OK;
 }
 
 }  // namespace qalora
@@ -88,6 +237,17 @@ int qalora_profile_next_main_kernel(void* start_event, void* stop_event) {
 }
 
 const char* qalora_main_kernel_name(void) { return t_main_kernel; }
+
+// Test hook, deliberately not declared in the public header.  Arms the NEXT few-token
+// forward launch of this process so that each of its producers stops after `stages` stages
+// and its waits give up after `limit_ns` nanoseconds: the consumers' bounded waits then
+// expire, the status word is raised and the kernel leaves in the ordinary way.  Nothing
+// faults, traps or spins without bound.
+int qalora_debug_expire_next_few_token_wait(int stages, uint64_t limit_ns) {
+  if (limit_ns == 0 || limit_ns > 2000000000ull) return QALORA_ERR_INVALID_ARG;
+  arm_few_token_wait_expiry(stages, limit_ns);
+  return QALORA_OK;
+}
 
 const char* qalora_status_string(int status) {
   switch (status) {
@@ -151,114 +311,17 @@ int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A
 int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
                    const float* qparams, const void* A, const void* B, void* y,
                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  Shape sh;
-  int st = check_desc(desc, &sh);
-  if (st != QALORA_OK) return st;
-  if (m < 0) return QALORA_ERR_INVALID_ARG;
-  if (m == 0) return QALORA_OK;
-  if (x == nullptr || codes == nullptr || qparams == nullptr || y == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (sh.r > 0 && (A == nullptr || B == nullptr)) return QALORA_ERR_NULL_POINTER;
-  const Workspace ws = workspace_layout(sh, m, QALORA_OP_FORWARD);
-  if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
-  if (!aligned16(x) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) || !aligned16(B) ||
-      !aligned16(y) || !aligned16(workspace))
-    return QALORA_ERR_MISALIGNED;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  char* wsp = static_cast<char*>(workspace);
-  float* T = reinterpret_cast<float*>(wsp + ws.T);
-  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
-  if (sh.r > 0) {
-    st = launch_pool_T(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(A),
-                       nullptr, T, Tb, stream);
-    if (st != QALORA_OK) return st;
-  }
-  const bool few = m <= kFewTokenM && gemv_supported(sh, m);
-  if (few) {
-    return launch_gemv(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
-                       reinterpret_cast<const float2*>(qparams), sh.r > 0 ? Tb : nullptr,
-                       static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(y),
-                       reinterpret_cast<int*>(wsp + ws.status), stream);
-  }
-  if (!few && m > kSmallM && tc_forward_supported(sh, m)) {
-    int* status = reinterpret_cast<int*>(wsp + ws.status);
-    if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
-    return launch_tc_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
-                             reinterpret_cast<const float2*>(qparams), Tb, static_cast<const __nv_bfloat16*>(B),
-                             static_cast<__nv_bfloat16*>(y), reinterpret_cast<float*>(wsp + ws.fwd_parts), status, stream);
-  }
-  return launch_simt_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
-                             reinterpret_cast<const float2*>(qparams), T, static_cast<const __nv_bfloat16*>(B),
-                             static_cast<__nv_bfloat16*>(y), stream);
+  int st = forward_validate(desc, m, x, codes, qparams, A, B, y, workspace, workspace_bytes);
+  if (st != QALORA_OK || m == 0) return st;
+  return forward_launch(desc, m, x, codes, qparams, A, B, y, workspace, cuda_stream, /*reset_status=*/true);
 }
 
 int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
                     const void* codes, const float* qparams, const void* A, const void* B,
                     void* dx, float* dA, float* dB,
                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  Shape sh;
-  int st = check_desc(desc, &sh);
-  if (st != QALORA_OK) return st;
-  if (m < 0 || sh.r == 0) return QALORA_ERR_INVALID_ARG;
-  if (x == nullptr || dy == nullptr || codes == nullptr || qparams == nullptr || A == nullptr || B == nullptr)
-    return QALORA_ERR_NULL_POINTER;
-  const Workspace ws = workspace_layout(sh, m, QALORA_OP_BACKWARD);
-  if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
-  if (!aligned16(x) || !aligned16(dy) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) ||
-      !aligned16(B) || !aligned16(dx) || !aligned16(dA) || !aligned16(dB) || !aligned16(workspace))
-    return QALORA_ERR_MISALIGNED;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  char* wsp = static_cast<char*>(workspace);
-  float* xp = reinterpret_cast<float*>(wsp + ws.xp);
-  float* T = reinterpret_cast<float*>(wsp + ws.T);
-  float* dT = reinterpret_cast<float*>(wsp + ws.dT);
-  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
-  __nv_bfloat16* dTb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.dTb);
-  float* partial = reinterpret_cast<float*>(wsp + ws.partial);
-  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
-  const __nv_bfloat16* dyb = static_cast<const __nv_bfloat16*>(dy);
-  const __nv_bfloat16* Ab = static_cast<const __nv_bfloat16*>(A);
-  const __nv_bfloat16* Bb = static_cast<const __nv_bfloat16*>(B);
-
-  if (m == 0) {
-    if (dA != nullptr && (st = cuda_status(cudaMemsetAsync(dA, 0, (size_t)sh.G * sh.r * sizeof(float), stream)))) return st;
-    if (dB != nullptr && (st = cuda_status(cudaMemsetAsync(dB, 0, (size_t)sh.r * sh.N * sizeof(float), stream)))) return st;
-    return QALORA_OK;
-  }
-  int* status = reinterpret_cast<int*>(wsp + ws.status);
-  if ((st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
-  const bool aux_tc = m > kSmallM && tc_aux_supported(sh, m);
-  if (aux_tc) st = launch_tc_dT(sh, m, dyb, Bb, dT, dTb, status, stream);
-  else st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream);
-  if (st != QALORA_OK) return st;
-  if (dA != nullptr || dB != nullptr) {
-    if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
-  }
-  if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
-    st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
-                      dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);
-    if (st != QALORA_OK) return st;
-  } else if (dx != nullptr) {
-    st = launch_simt_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
-                        dT, Ab, static_cast<__nv_bfloat16*>(dx), stream);
-    if (st != QALORA_OK) return st;
-  }
-  if (dA != nullptr) {
-    st = launch_atb_f32(m, sh.G, sh.r, xp, dT, dA, partial, ws.partial_bytes, stream);
-    if (st != QALORA_OK) return st;
-  }
-  if (dB != nullptr) {
-    if (aux_tc) {
-      int splits = 0;
-      st = launch_tc_dB_partials(sh, m, Tb, dyb, partial, &splits, status, stream);
-      if (st == QALORA_OK) st = launch_sum_partials(partial, dB, (size_t)sh.r * sh.N, splits, stream);
-    } else {
-      st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial, ws.partial_bytes, stream);
-    }
-    if (st != QALORA_OK) return st;
-  }
-  return QALORA_OK;
+  return backward_impl(desc, m, x, dy, codes, qparams, A, B, dx, dA, dB, workspace, workspace_bytes, cuda_stream,
+                       /*reset_status=*/true);
 }
 
 
@@ -358,6 +421,8 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
   std::lock_guard<std::mutex> lock(g_step_mutex);
   StepPipes* P = step_pipes_locked();
   if (P == nullptr) return QALORA_ERR_CUDA;
+  // one status word for the whole call: cleared here, only ever raised by the chunks' kernels
+  if (!ok(cudaMemsetAsync(base + L.ws, 0, sizeof(int), stream))) return QALORA_ERR_CUDA;
   // The copy streams start after everything already enqueued on the caller's stream.
   if (!ok(cudaEventRecord(P->start, stream)) || !ok(cudaStreamWaitEvent(P->in, P->start, 0)) ||
       !ok(cudaStreamWaitEvent(P->out, P->start, 0)))
@@ -373,12 +438,14 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
         !ok(cudaMemcpyAsync(base + L.dy + yo, static_cast<const char*>(dy_host) + yo, yb, cudaMemcpyHostToDevice, P->in)) ||
         !ok(cudaEventRecord(P->dy[c], P->in)) || !ok(cudaStreamWaitEvent(stream, P->x[c], 0)))
       return QALORA_ERR_CUDA;
-    st = qalora_forward(desc, rows, base + L.x + xo, codes, qparams, A, B, base + L.y + yo, base + L.ws, L.ws_bytes,
-                        cuda_stream);
+    st = forward_validate(desc, rows, base + L.x + xo, codes, qparams, A, B, base + L.y + yo, base + L.ws, L.ws_bytes);
+    if (st == QALORA_OK)
+      st = forward_launch(desc, rows, base + L.x + xo, codes, qparams, A, B, base + L.y + yo, base + L.ws, cuda_stream,
+                          /*reset_status=*/false);
     if (st != QALORA_OK) return st;
     if (!ok(cudaEventRecord(P->fwd[c], stream)) || !ok(cudaStreamWaitEvent(stream, P->dy[c], 0))) return QALORA_ERR_CUDA;
-    st = qalora_backward(desc, rows, base + L.x + xo, base + L.dy + yo, codes, qparams, A, B, base + L.dx + xo, dA_c, dB_c,
-                         base + L.ws, L.ws_bytes, cuda_stream);
+    st = backward_impl(desc, rows, base + L.x + xo, base + L.dy + yo, codes, qparams, A, B, base + L.dx + xo, dA_c, dB_c,
+                       base + L.ws, L.ws_bytes, cuda_stream, /*reset_status=*/false);
     if (st != QALORA_OK) return st;
     if (!ok(cudaEventRecord(P->bwd[c], stream)) || !ok(cudaStreamWaitEvent(P->out, P->fwd[c], 0)) ||
         !ok(cudaMemcpyAsync(static_cast<char*>(y_host) + yo, base + L.y + yo, yb, cudaMemcpyDeviceToHost, P->out)) ||

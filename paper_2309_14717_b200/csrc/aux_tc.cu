@@ -255,26 +255,15 @@ bool make_map(CUtensorMap* map, const void* base, long long rows, int cols, int 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int aux_sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
-
 template <int MODE>
 int launch_aux(const CUtensorMap& a, const CUtensorMap& b, const AuxParams& p, cudaStream_t st) {
   using C = AuxCfg<MODE>;
   static_assert(C::TOTAL <= 232448, "shared memory budget");
   auto kern = aux_tc_kernel<MODE>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::TOTAL); });
-  if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
-  const int grid = p.items < aux_sm_count() ? p.items : aux_sm_count();
+  static PerDeviceOnce smem_limit;      // this instantiation's shared-memory limit, raised once on every device it runs on
+  if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::TOTAL); }) != QALORA_OK)
+    return QALORA_ERR_CUDA;
+  const int grid = p.items < device_sm_count() ? p.items : device_sm_count();
   kern<<<grid, AUX_THREADS, C::TOTAL, st>>>(a, b, p);
   count_launch();
   return cuda_status(cudaGetLastError());
@@ -302,7 +291,7 @@ int launch_tc_dT(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const __nv
 // Number of token splits (and bytes of fp32 partials) the dB kernel uses.
 int tc_dB_splits(const Shape& sh, int64_t M) {
   const int n_tiles = (sh.N + 255) / 256;
-  long long splits = (aux_sm_count() + n_tiles - 1) / n_tiles;
+  long long splits = (device_sm_count() + n_tiles - 1) / n_tiles;
   const long long max_by_rows = (M + 511) / 512;
   if (splits > max_by_rows) splits = max_by_rows;
   return (int)(splits < 1 ? 1 : splits);

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "qalora.h"
 
 namespace qalora {
@@ -37,6 +39,16 @@ struct Workspace {
   size_t total;
 };
 Workspace workspace_layout(const Shape& sh, int64_t m, int op);
+
+// The public forward / backward in two halves (api.cu): checks that launch nothing, and the
+// launches with a say on whether the workspace's status word is cleared first.
+int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
+                     const void* A, const void* B, const void* y, const void* workspace, size_t workspace_bytes);
+int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
+                   const void* A, const void* B, void* y, void* workspace, void* cuda_stream, bool reset_status);
+int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void* dy, const void* codes,
+                  const float* qparams, const void* A, const void* B, void* dx, float* dA, float* dB,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status);
 
 // --------------------------------------------------------------- device side --
 __device__ __forceinline__ float bf16_to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -108,10 +120,13 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
                  __nv_bfloat16* dx, int* status, cudaStream_t st);
 
-// Few-token forward (gemv.cu): M <= 32.
+// Few-token forward (gemv.cu): M <= 32.  `reset_status`: the kernel clears *status at its start.
 bool gemv_supported(const Shape& sh, int64_t M);
 int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
-                const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, cudaStream_t st);
+                const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, bool reset_status,
+                cudaStream_t st);
+
+void arm_few_token_wait_expiry(int stages, unsigned long long limit_ns);   // test hook, one-shot
 
 // out[i] = sum over splits of partial[z][i], added in a fixed order.
 int launch_sum_partials(const float* partial, float* out, size_t count, int splits, cudaStream_t st);
@@ -136,6 +151,34 @@ int launch_adamw(const AdamwArgs& a, int64_t n, const float* grad, float* param,
                  __nv_bfloat16* param_bf16, float* parts, float* norm_out, cudaStream_t st);
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? QALORA_OK : QALORA_ERR_CUDA; }
+
+// ---- per-device host state ---------------------------------------------------
+// A process may drive several GPUs.  Everything the library remembers about a device (its
+// SM count, whether a kernel's shared-memory limit has been raised there) is kept per
+// device ordinal of the device that is current at the call.
+constexpr int kMaxDevices = 64;
+int current_device();        // ordinal of the current device, -1 when it cannot be had or is beyond kMaxDevices
+int device_sm_count();       // multiprocessors of the current device (148 when the query fails)
+
+// One-time set-up per device, e.g. cudaFuncSetAttribute of one kernel: `run(fn)` calls
+// fn() -> cudaError_t the first time it is reached with a given device current and returns
+// that first outcome (as a qalora_status) from then on.  One static instance per kernel.
+struct PerDeviceOnce {
+  std::atomic<int> state[kMaxDevices];     // 0: not yet, 1: done, 2: failed
+  PerDeviceOnce() { for (auto& s : state) s.store(0, std::memory_order_relaxed); }
+  template <class Fn>
+  int run(Fn fn) {
+    const int dev = current_device();
+    if (dev < 0) return QALORA_ERR_CUDA;
+    int s = state[dev].load(std::memory_order_acquire);
+    if (s == 0) {
+      // two threads may both get here: the set-up is idempotent, so both just do it
+      s = fn() == cudaSuccess ? 1 : 2;
+      state[dev].store(s, std::memory_order_release);
+    }
+    return s == 1 ? QALORA_OK : QALORA_ERR_CUDA;
+  }
+};
 
 // Instrumentation: launch counter and the one-shot event probe around a main kernel.
 void count_launch(int n = 1);

@@ -40,6 +40,12 @@ extern "C" int qalora_forward_static(const qalora_desc* desc, int64_t m, const v
   int st = qalora_workspace_bytes(desc, m, QALORA_OP_FORWARD, &need);
   if (st != QALORA_OK) return st;
   if (need > (size_t)QALORA_STATIC_SCRATCH_BYTES) return QALORA_ERR_STATIC_SCRATCH_EXCEEDED;
+  // every check of qalora_forward first, against a stand-in for the (256-byte aligned) array:
+  // a rejected call must not have enqueued anything, nor touched the CUDA runtime
+  alignas(16) static const char aligned_stand_in = 0;
+  if ((st = qalora::forward_validate(desc, m, x, codes, qparams, A, B, y, &aligned_stand_in,
+                                     (size_t)QALORA_STATIC_SCRATCH_BYTES)) != QALORA_OK)
+    return st;
   if (m == 0) return QALORA_OK;
   void* scratch = nullptr;
   if ((st = static_scratch_address(&scratch)) != QALORA_OK) return st;

@@ -552,16 +552,6 @@ bool make_act_map(CUtensorMap* map, const void* base, long long rows, int cols, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
-
 // bf16 output [rows][cols] row-major, box = 128 columns x 32 rows, no swizzle (store side)
 bool make_out_map(CUtensorMap* map, void* base, long long rows, int cols) {
   EncodeTiledFn fn = encode_fn();
@@ -628,12 +618,11 @@ int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams&
   if (!make_qp_map(&qmap, p.qparams, p.K / p.g, p.N, S::TILE_NC, p.qp_rows)) return QALORA_ERR_CUDA;
   static_assert(S::TOTAL <= 232448, "shared memory budget");
   auto kern = qalora_tc_kernel<BITS, MODE, PARTS, TT>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
-  if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
+  static PerDeviceOnce smem_limit;      // this instantiation's shared-memory limit, raised once on every device it runs on
+  if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
+    return QALORA_ERR_CUDA;
   const int tiles = p.c_tiles * p.m_tiles * p.ksplit;
-  const int grid = tiles < sm_count() ? tiles : sm_count();
+  const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
   {
     MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
     kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, out, cmap, qmap, p);
@@ -674,7 +663,7 @@ int tc_forward_parts(const Shape& sh, int64_t M) {
   if (M <= TILE_T_FEW && sh.K / TILE_J >= 8) {
     // the 64-token variant always writes partial results; as many parts as fill the SMs evenly
     const long long tiles = sh.N / TILE_C;
-    const int steps = sh.K / TILE_J, sms = sm_count();
+    const int steps = sh.K / TILE_J, sms = device_sm_count();
     int best = 1;
     double best_cost = 1e30;
     for (int ks = 1; ks <= 8; ++ks) {
@@ -685,7 +674,7 @@ int tc_forward_parts(const Shape& sh, int64_t M) {
     return -best;                                              // negative: the 64-token variant
   }
   const long long tiles = (long long)(sh.N / TILE_C) * ((M + TILE_T - 1) / TILE_T);
-  const int steps = sh.K / TILE_J, sms = sm_count();
+  const int steps = sh.K / TILE_J, sms = device_sm_count();
   if (tiles * 4 > sms) return 1;          // enough tiles: the parts' extra epilogues and scratch traffic cost more than they save
   int best = 1;
   double best_cost = (double)((tiles + sms - 1) / sms);          // waves x (share of a tile per wave)

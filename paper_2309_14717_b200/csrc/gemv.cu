@@ -70,6 +70,9 @@ struct GvParams {
   int M, K, N, g, r;
   int total_stages;             // K / 128
   int* status;
+  int reset_status;             // the first block clears *status before any wait can expire
+  int stop_after_stages;        // normally INT_MAX; a test makes every producer stop early, so that waits expire
+  unsigned long long wait_limit_ns;
 };
 
 // (not volatile: a pure function of its operands, so that independent MMAs can be interleaved)
@@ -152,7 +155,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     ptx::prefetch_tensormap(&x_map);
     ptx::prefetch_tensormap(&codes_map);
     ptx::prefetch_tensormap(&qp_map);
-    if (blockIdx.x == 0) *p.status = 0;     // every block is resident from the start; a timeout is seconds away
+    if (blockIdx.x == 0 && p.reset_status) *p.status = 0;     // a wait gives up only after seconds: no block can have raised it yet
   }
   __syncthreads();
 
@@ -160,9 +163,9 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     // ------------------------------------------------------------ producer ----
     if (lane == 0) {
       bool ok = true;
-      for (int st = st_beg, it = 0; st < st_end && ok; ++st, ++it) {
+      for (int st = st_beg, it = 0; st < st_end && ok && it < p.stop_after_stages; ++st, ++it) {
         const int s = it % GV_STAGES;
-        if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / GV_STAGES) & 1) ^ 1, abort_flag))) break;
+        if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / GV_STAGES) & 1) ^ 1, abort_flag, p.wait_limit_ns))) break;
         const uint32_t stage = smem_base + s * S::STAGE_BYTES;
         // three tiled copies per stage: 4 k-block rows of pack units, the rows of
         // (alpha, beta) they need (128 / g of them) and the x slice
@@ -207,7 +210,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     bool ok = true;
     for (int st = st_beg, it = 0; st < st_end && ok; ++st, ++it) {
       const int s = it % GV_STAGES;
-      if (!(ok = ptx::mbar_wait(bar_full(s), (it / GV_STAGES) & 1, abort_flag))) break;
+      if (!(ok = ptx::mbar_wait(bar_full(s), (it / GV_STAGES) & 1, abort_flag, p.wait_limit_ns))) break;
       const uint8_t* stage = smem + s * S::STAGE_BYTES;
       if constexpr (CHAIN) {
         // the set's two k-blocks lie in one quantization group: one accumulator chain over
@@ -406,16 +409,6 @@ EncodeTiledFn gv_encode_fn() {
   return fn;
 }
 
-int gv_sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
-
 template <int BITS, int NTS, bool CHAIN>
 int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
   EncodeTiledFn fn = gv_encode_fn();
@@ -444,10 +437,9 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   }
   using S = GvSmem<BITS, NTS>;
   auto kern = qalora_gemv_kernel<BITS, NTS, CHAIN>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [&] { attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); });
-  if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
+  static PerDeviceOnce smem_limit;      // this instantiation's shared-memory limit, raised once on every device it runs on
+  if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
+    return QALORA_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((p.N / GV_COLS) * splits));
   cfg.blockDim = dim3(GV_THREADS);
@@ -478,6 +470,17 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
 
 }  // namespace
 
+// Test hook (see qalora_debug_expire_next_few_token_wait in api.cu): when armed, the producers
+// of the next few-token launch stop after `stages` stages of their slice and its waits give up
+// after `limit_ns`, so that the consumers' waits run out: the bounded-wait path (status word,
+// orderly exit) can be exercised without a fault and without a kernel that hangs.
+std::atomic<int> g_expire_after_stages{0x7fffffff};
+std::atomic<unsigned long long> g_expire_limit_ns{ptx::WAIT_LIMIT_NS};
+void arm_few_token_wait_expiry(int stages, unsigned long long limit_ns) {
+  g_expire_limit_ns.store(limit_ns);
+  g_expire_after_stages.store(stages < 0 ? 0 : stages);
+}
+
 // Slices per column tile (= cluster size): the count among {1,2,3,4,6,8} that brings the
 // grid closest to two blocks per SM.  Three blocks fit on an SM, so the grid stays one
 // wave with room for imbalance, while a block still streams enough bytes to amortize its
@@ -485,7 +488,7 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
 // than 16 token rows only two blocks fit on an SM: there the grid must not exceed two blocks
 // per SM, or a second wave would follow.
 static int gv_slices(const Shape& sh, int64_t M) {
-  const int tiles = sh.N / GV_COLS, total_stages = sh.K / (GV_KBS * 32), target = 2 * gv_sm_count();
+  const int tiles = sh.N / GV_COLS, total_stages = sh.K / (GV_KBS * 32), target = 2 * device_sm_count();
   const bool capped = M > 16;
   int splits = 1, best = 1 << 30;
   for (int sp : {1, 2, 3, 4, 6, 8}) {
@@ -509,7 +512,7 @@ bool gemv_supported(const Shape& sh, int64_t M) {
     // fill 58 %), and only for a layer without adapter: the tensor-core kernel folds the
     // adapter into its MMA steps, while here T * B is summed per output at the end, which
     // costs more than the streaming saves once there are thousands of outputs per block.
-    const int sms = gv_sm_count();
+    const int sms = device_sm_count();
     const long long blocks = (long long)(sh.N / GV_COLS) * gv_slices(sh, M);
     const long long waves = (blocks + sms - 1) / sms;
     if (blocks > sms && (waves > 2 || blocks * 4 < waves * sms * 3)) return false;
@@ -519,7 +522,8 @@ bool gemv_supported(const Shape& sh, int64_t M) {
 
 // y = x * W~ + T * B for M <= 32 rows; Tb is T = s * pool(x) * A in bf16 [M][r] (null when r == 0).
 int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
-                const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, cudaStream_t st) {
+                const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, bool reset_status,
+                cudaStream_t st) {
   EncodeTiledFn fn = gv_encode_fn();
   CUtensorMap xm;
   cuuint64_t dims[2] = {(cuuint64_t)sh.K, (cuuint64_t)M};
@@ -535,6 +539,9 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;
+  p.reset_status = reset_status ? 1 : 0;
+  p.stop_after_stages = g_expire_after_stages.exchange(0x7fffffff);     // one-shot: the next launch only
+  p.wait_limit_ns = p.stop_after_stages != 0x7fffffff ? g_expire_limit_ns.load() : ptx::WAIT_LIMIT_NS;
   const int splits = gv_slices(sh, M);
   const int nts = M > 16 ? 4 : (M > 8 ? 2 : 1);
   const bool chain = sh.g >= 64;

@@ -113,19 +113,6 @@ adamw_kernel(const float* __restrict__ grad, float* __restrict__ param, float* _
   }
 }
 
-int device_sms() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-      sms = v;
-    else
-      return 148;
-  }
-  return sms;
-}
-
 }  // namespace
 
 size_t adamw_workspace_bytes() { return OPT_MAX_PARTS * sizeof(float); }
@@ -147,7 +134,7 @@ int launch_adamw(const AdamwArgs& a, int64_t n64, const float* grad, float* para
   k.inv_sqrt_bc2 = (float)(1.0 / sqrt(1.0 - pow((double)a.beta2, (double)a.step)));
   k.eps = a.eps; k.max_norm = a.max_grad_norm;
   const size_t want = (n / 4 + OPT_THREADS - 1) / OPT_THREADS;
-  size_t blocks = (size_t)device_sms() * OPT_BLOCKS_PER_SM;
+  size_t blocks = (size_t)device_sm_count() * OPT_BLOCKS_PER_SM;
   if (blocks > want) blocks = want > 0 ? want : 1;
   adamw_kernel<<<(unsigned)blocks, OPT_THREADS, 0, st>>>(grad, param, exp_avg, exp_avg_sq, param_bf16, n, parts, nparts, k,
                                                          norm_out);

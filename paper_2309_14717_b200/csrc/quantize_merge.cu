@@ -15,9 +15,12 @@ constexpr int QCOLS = 128;   // columns (threads) per block
 // floating-point step is a single IEEE fp32 operation (no FMA contraction), so
 // the integer decision is reproducible bit for bit on a CPU.  The division
 // t = (w - beta) / alpha is the expensive one; the code only needs rint(t), so the
-// kernel first takes t' = (w - beta) * (1 / alpha), which is within 2e-6 of t for
+// kernel first takes t' = (w - beta) * (1 / alpha), which is within 4e-6 of t for
 // t in [0, 15], and falls back to the IEEE division only where t' lies within 1e-4
 // of a rounding boundary (a half-integer): everywhere else rint(t') = rint(t).
+// The shortcut is taken only for 1e-30 < alpha < 1e30: outside that range 1 / alpha
+// overflows or is a subnormal with few significant bits (a group of nearly equal tiny
+// weights, or of huge ones), and every element takes the division.
 template <int BITS>
 __global__ void __launch_bounds__(QCOLS)
 quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
@@ -47,7 +50,8 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
   qparams[(size_t)q * N + n] = make_float2(alpha, beta);
   if (bad && dev_status != nullptr) atomicOr(dev_status, 1);
 
-  const float inv_alpha = __frcp_rn(alpha);
+  const bool fast = alpha > 1e-30f && alpha < 1e30f;
+  const float inv_alpha = fast ? __frcp_rn(alpha) : 0.0f;
   const int kb0 = q * (g / 32);
   for (int k0 = 0; k0 < g; k0 += 32) {
     float v[32];
@@ -61,7 +65,7 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
       const float d = __fsub_rn(v[j], beta);
       const float t = __fmul_rn(d, inv_alpha);
       float c = rintf(t);                              // round half to even
-      if (fabsf(t - c) > 0.4999f) c = rintf(__fdiv_rn(d, alpha));   // near a boundary (or a tie): exact
+      if (!fast || !(fabsf(t - c) <= 0.4999f)) c = rintf(__fdiv_rn(d, alpha));   // near a boundary (or a tie): exact
       c = fminf(fmaxf(c, 0.0f), QMAX);
       unit_insert<BITS>(u, j, (uint32_t)(int)c);
     }

@@ -219,13 +219,14 @@ int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv
   const bool rows_path = M >= 64 && (sh.g == 32 || sh.g == 64 || sh.g == 128) && sh.K % 256 == 0 &&
                          sh.r >= 8 && smem <= kPool16MaxSmem;
   if (rows_path) {
-    static const cudaError_t attr_err = [] {             // once: allow more than the default 48 KiB
+    static PerDeviceOnce smem_limit;                     // once per device: allow more than the default 48 KiB
+    const int attr_st = smem_limit.run([] {
       cudaError_t e = cudaFuncSetAttribute(pool_T_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPool16MaxSmem);
       if (e == cudaSuccess) e = cudaFuncSetAttribute(pool_T_rows_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPool16MaxSmem);
       if (e == cudaSuccess) e = cudaFuncSetAttribute(pool_T_rows_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPool16MaxSmem);
       return e;
-    }();
-    if (attr_err != cudaSuccess) return QALORA_ERR_CUDA;
+    });
+    if (attr_st != QALORA_OK) return attr_st;
     const unsigned grid = (unsigned)((M + POOL16_ROWS - 1) / POOL16_ROWS);
     if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
     else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);

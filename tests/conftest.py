@@ -1,3 +1,4 @@
+import json
 import os
 import sys
 
@@ -6,6 +7,18 @@ import pytest
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
+
+# Worst max|err| / max|ref| seen per (parity case, output), filled by the GPU parity tests
+# through `record_margin`, printed at the end of the run and, when the environment
+# variable QALORA_PARITY_MARGINS names a file, written there as JSON.
+PARITY_MARGINS = {}
+
+
+def record_margin(case: str, output: str, err: float, tol: float):
+    """Notes the error of one output of one parity case and asserts it against `tol`."""
+    worst = PARITY_MARGINS.setdefault(case, {})
+    worst[output] = max(float(err), worst.get(output, 0.0))
+    assert err <= tol, f"{case}: {output} max|err|/max|ref| = {err:.3e} > {tol:.1e}"
 
 
 def pytest_configure(config):
@@ -24,3 +37,16 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    if not PARITY_MARGINS:
+        return
+    tr = terminalreporter
+    tr.write_sep("-", "parity margins: worst max|err|/max|ref| per case and output (tolerance 5e-3)")
+    for case in sorted(PARITY_MARGINS):
+        tr.write_line(case + ": " + ", ".join(f"{k}={v:.2e}" for k, v in sorted(PARITY_MARGINS[case].items())))
+    path = os.environ.get("QALORA_PARITY_MARGINS")
+    if path:
+        with open(path, "w") as f:
+            json.dump(PARITY_MARGINS, f, indent=1, sort_keys=True)

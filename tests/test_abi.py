@@ -89,6 +89,24 @@ def test_null_and_misaligned_pointers_are_rejected_without_a_launch():
     assert lib.qalora_forward(r(d), 0, None, None, None, None, None, None, None, 0, None) == 0
 
 
+def test_static_scratch_forward_checks_its_arguments_before_anything_else():
+    """qalora_forward_static must turn a bad argument down before it looks up its scratch
+    array or enqueues the clearing of the status word: on a machine without a GPU a call
+    that reached the CUDA runtime first would come back as a CUDA error (-6) instead."""
+    lib = Q.load()
+    d = Q.desc(512, 512, 32, 4, 16, 1.0)
+    p = ctypes.c_void_p
+    buf = ctypes.create_string_buffer(64)          # host memory: must never be dereferenced
+    a16 = (ctypes.addressof(buf) + 15) // 16 * 16
+    r = ctypes.byref
+    assert lib.qalora_forward_static(r(d), 8, None, p(a16), p(a16), p(a16), p(a16), p(a16), None) == -2
+    assert lib.qalora_forward_static(r(d), 8, p(a16), p(a16), p(a16), None, p(a16), p(a16), None) == -2
+    assert lib.qalora_forward_static(r(d), 8, p(a16 + 2), p(a16), p(a16), p(a16), p(a16), p(a16), None) == -4
+    assert lib.qalora_forward_static(r(d), -3, p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), None) == -1
+    assert lib.qalora_forward_static(r(d), 1 << 20, p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), None) == -7
+    assert lib.qalora_forward_static(r(d), 0, None, None, None, None, None, None, None) == 0
+
+
 def test_adamw_argument_checks_need_no_gpu():
     lib = Q.load()
     p = ctypes.c_void_p

@@ -1,12 +1,22 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py
-times.  Codes, packed words and (alpha, beta) are compared in full; y and dX on
-a seeded sample of token rows (rows are independent, so the oracle evaluates
-exactly those rows); dA, dB and the merged zeros in full (the oracle adds the
-adapter gradients over row blocks)."""
+times: every shape x bit width of the 13B configuration, every shape x group size
+of the 65B configuration, and both 7B MLP shapes.
+
+Codes, packed words and (alpha, beta) are compared in full.  y and dX are compared
+on ALL token rows for the 7B and 13B shapes; for the 65B shapes (where the fp64
+oracle would need tens of seconds per case) on a seeded sample of token rows: rows
+are independent, so the oracle evaluates exactly those rows.  dA, dB and the merged
+zeros are compared in full everywhere (the oracle adds the adapter gradients over
+row blocks).  The few-token forward is checked at full size too: the merged layer
+at one token, and the adapted layer (rank 64) at 1 and 16 tokens.
+
+Every comparison goes through `record_margin`, which keeps the worst
+max|err| / max|ref| per case and output for the summary at the end of the run."""
 import numpy as np
 import pytest
 import torch
 
+from conftest import record_margin
 from oracle import qalora_oracle as O
 from paper_2309_14717_b200 import binding as Q
 from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs, to_f64
@@ -23,22 +33,20 @@ def rel_err(got, ref):
     return float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
 
 
-CASES = [
-    # config, overrides
-    ("cfg3_7b_up", {}),
-    ("cfg3_7b_down", {}),
-    ("cfg4_13b_up", {"bits": 3}),
-    ("cfg4_13b_down", {"bits": 2}),
-    ("cfg4_13b_attn", {"bits": 2}),
-    ("cfg5_65b_attn", {"group_size": 64}),
-    ("cfg5_65b_down", {"group_size": 128}),
-    ("cfg5_65b_up", {}),
-]
+CASES = [("cfg3_7b_up", {}), ("cfg3_7b_down", {})]
+CASES += [(n, {"bits": b}) for n in ("cfg4_13b_up", "cfg4_13b_down", "cfg4_13b_attn") for b in (3, 2)]
+CASES += [(n, {"group_size": g}) for n in ("cfg5_65b_up", "cfg5_65b_down", "cfg5_65b_attn") for g in (32, 64, 128)]
 
 
-@pytest.mark.parametrize("name,over", CASES, ids=[c[0] + "".join(f"_{k[0]}{v}" for k, v in c[1].items()) for c in CASES])
+def case_id(c):
+    return c[0] + "".join(f"_{k[0]}{v}" for k, v in c[1].items())
+
+
+@pytest.mark.parametrize("name,over", CASES, ids=[case_id(c) for c in CASES])
 def test_full_size_layer(name, over):
+    case = case_id((name, over))
     cfg = CONFIGS[name].with_(**over)
+    all_rows = not name.startswith("cfg5")            # the 65B shapes keep the row sample
     cpu = make_inputs(cfg)
     M, K, N, G, r, g, s = cfg.tokens, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank, cfg.group_size, cfg.scale
     d = Q.desc(K, N, g, cfg.bits, r, s)
@@ -66,26 +74,41 @@ def test_full_size_layer(name, over):
     assert np.array_equal(codes_d.cpu().numpy().view(np.uint32), O.pack(codes, cfg.bits))
     qp = qparams.cpu().numpy()
     assert np.array_equal(qp[..., 0], alpha) and np.array_equal(qp[..., 1], beta)
-    del dev["W"]
+    del dev["W"], cpu["W"]
 
     A, B = to_f64(cpu["A"]), to_f64(cpu["B"])
-    rows = np.unique(np.concatenate([[0, M - 1, 255, 256], np.random.default_rng(cfg.seed).integers(0, M, SAMPLE_ROWS)]))
+    if all_rows:
+        rows = np.arange(M)
+    else:
+        rows = np.unique(np.concatenate([[0, M - 1, 255, 256], np.random.default_rng(cfg.seed).integers(0, M, SAMPLE_ROWS)]))
     rows_t = torch.from_numpy(rows)
-    xs, dys = to_f64(cpu["x"][rows_t]), to_f64(cpu["dy"][rows_t])
-    y_ref = O.forward(xs, codes, alpha, beta, g, A, B, s)
-    assert rel_err(y[rows_t.cuda()].float().cpu().numpy(), y_ref) <= TOL
-    dx_ref, _, _ = O.backward(xs, dys, codes, alpha, beta, g, A, B, s)
-    assert rel_err(dx[rows_t.cuda()].float().cpu().numpy(), dx_ref) <= TOL
+    y_got = y[rows_t.cuda()].cpu()
+    dx_got = dx[rows_t.cuda()].cpu()
+    y_err = dx_err = y_max = dx_max = 0.0
+    y_first = None
+    for b0 in range(0, len(rows), 2048):               # row blocks keep the fp64 temporaries small
+        rb = rows_t[b0:b0 + 2048]
+        xs, dys = to_f64(cpu["x"][rb]), to_f64(cpu["dy"][rb])
+        y_ref = O.forward(xs, codes, alpha, beta, g, A, B, s)
+        dx_ref, _, _ = O.backward(xs, dys, codes, alpha, beta, g, A, B, s)
+        if y_first is None:
+            y_first = y_ref[:1].copy()
+        y_err = max(y_err, float(np.max(np.abs(y_got[b0:b0 + 2048].double().numpy() - y_ref))))
+        dx_err = max(dx_err, float(np.max(np.abs(dx_got[b0:b0 + 2048].double().numpy() - dx_ref))))
+        y_max = max(y_max, float(np.max(np.abs(y_ref))))
+        dx_max = max(dx_max, float(np.max(np.abs(dx_ref))))
+    record_margin(case, "y", y_err / y_max, TOL)
+    record_margin(case, "dX", dx_err / dx_max, TOL)
 
     dA_ref = np.zeros((G, r)); dB_ref = np.zeros((r, N))
     for m0 in range(0, M, 1024):                          # sums over token rows: add row blocks
         a, b = O.backward_adapter(to_f64(cpu["x"][m0:m0 + 1024]), to_f64(cpu["dy"][m0:m0 + 1024]), g, A, B, s)
         dA_ref += a; dB_ref += b
-    assert rel_err(dA.cpu().numpy(), dA_ref) <= TOL
-    assert rel_err(dB.cpu().numpy(), dB_ref) <= TOL
+    record_margin(case, "dA", rel_err(dA.cpu().numpy(), dA_ref), TOL)
+    record_margin(case, "dB", rel_err(dB.cpu().numpy(), dB_ref), TOL)
     q2n = q2.cpu().numpy()
     assert np.array_equal(q2n[..., 0], alpha)
-    assert rel_err(q2n[..., 1], O.merge(beta, A, B, s)) <= TOL
+    record_margin(case, "beta_merged", rel_err(q2n[..., 1], O.merge(beta, A, B, s)), TOL)
 
     # the deployed layer at one token (the few-token kernel at full size) reproduces the adapted output
     d0 = Q.desc(K, N, g, cfg.bits, 0, s)
@@ -95,4 +118,16 @@ def test_full_size_layer(name, over):
     Q.qalora_forward(d0, 1, x1, codes_d, q2, None, None, y1, w1)
     torch.cuda.synchronize()
     assert Q.qalora_main_kernel_name() == "qalora_gemv_kernel"
-    assert rel_err(y1.float().cpu().numpy(), y_ref[:1]) <= TOL
+    record_margin(case, "y_merged_m1", rel_err(y1.float().cpu().numpy(), y_first), TOL)
+
+    # the adapted layer (rank r) on the few-token path at full size: 1 and 16 tokens
+    rows16 = rows_t[:16] if len(rows_t) >= 16 else rows_t
+    y16_ref = O.forward(to_f64(cpu["x"][rows16]), codes, alpha, beta, g, A, B, s)
+    for m in (1, 16):
+        xm = dev["x"][rows16[:m].cuda()].contiguous()
+        ym = torch.empty((m, N), dtype=torch.bfloat16, device="cuda")
+        wm = Q.alloc_workspace(d, m, Q.OP_FORWARD)
+        Q.qalora_forward(d, m, xm, codes_d, qparams, dev["A"], dev["B"], ym, wm)
+        torch.cuda.synchronize()
+        assert Q.qalora_main_kernel_name() == "qalora_gemv_kernel" and Q.workspace_status(wm) == 0
+        record_margin(case, f"y_adapted_m{m}", rel_err(ym.float().cpu().numpy(), y16_ref[:m]), TOL)

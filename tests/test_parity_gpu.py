@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+from conftest import record_margin
 from oracle import qalora_oracle as O
 from paper_2309_14717_b200 import binding as Q
 from paper_2309_14717_b200.synthetic import CONFIGS, LayerConfig, make_inputs, to_f64
@@ -22,6 +23,11 @@ def rel_err(got, ref):
         return 0.0
     denom = np.max(np.abs(ref))
     return float(np.max(np.abs(got - ref)) / (denom if denom > 0 else 1.0))
+
+
+def margin(case, output, got, ref):
+    """Compares one output with the oracle's and keeps the error for the end-of-run summary."""
+    record_margin(case, output, rel_err(got, ref), TOL)
 
 
 class GpuLayer:
@@ -116,21 +122,21 @@ def test_small_shapes_all_ops(case):
     codes, alpha, beta = check_quantize(layer)
     x, A, B, dy = (to_f64(layer.cpu[k]) for k in ("x", "A", "B", "dy"))
     y_ref = O.forward(x, codes, alpha, beta, g, A, B, s)
-    assert rel_err(layer.forward().float().cpu().numpy(), y_ref) <= TOL
+    margin(name, "y", layer.forward().float().cpu().numpy(), y_ref)
     dx, dA, dB = layer.backward()
     dx_ref, dA_ref, dB_ref = O.backward(x, dy, codes, alpha, beta, g, A, B, s)
-    assert rel_err(dx.float().cpu().numpy(), dx_ref) <= TOL
-    assert rel_err(dA.cpu().numpy(), dA_ref) <= TOL
-    assert rel_err(dB.cpu().numpy(), dB_ref) <= TOL
+    margin(name, "dX", dx.float().cpu().numpy(), dx_ref)
+    margin(name, "dA", dA.cpu().numpy(), dA_ref)
+    margin(name, "dB", dB.cpu().numpy(), dB_ref)
     # merge, then the plain quantized layer must reproduce the adapted one
     q2 = torch.empty_like(layer.qparams)
     Q.qalora_merge(layer.d, layer.qparams, layer.dev["A"], layer.dev["B"], q2)
     torch.cuda.synchronize()
     q2n = q2.cpu().numpy()
     assert np.array_equal(q2n[..., 0], alpha)
-    assert rel_err(q2n[..., 1], O.merge(beta, A, B, s)) <= TOL
+    margin(name, "beta_merged", q2n[..., 1], O.merge(beta, A, B, s))
     y_merged = layer.forward(qparams=q2, rank=0)
-    assert rel_err(y_merged.float().cpu().numpy(), y_ref) <= TOL
+    margin(name, "y_merged", y_merged.float().cpu().numpy(), y_ref)
     # in-place merge gives the same bytes
     q3 = layer.qparams.clone()
     Q.qalora_merge(layer.d, q3, layer.dev["A"], layer.dev["B"], q3)
@@ -144,12 +150,12 @@ def test_config1_full():
     codes, alpha, beta = check_quantize(layer)
     x, A, B, dy = (to_f64(layer.cpu[k]) for k in ("x", "A", "B", "dy"))
     g, s = cfg.group_size, cfg.scale
-    assert rel_err(layer.forward().float().cpu().numpy(), O.forward(x, codes, alpha, beta, g, A, B, s)) <= TOL
+    margin("cfg1_512", "y", layer.forward().float().cpu().numpy(), O.forward(x, codes, alpha, beta, g, A, B, s))
     dx, dA, dB = layer.backward()
     dx_ref, dA_ref, dB_ref = O.backward(x, dy, codes, alpha, beta, g, A, B, s)
-    assert rel_err(dx.float().cpu().numpy(), dx_ref) <= TOL
-    assert rel_err(dA.cpu().numpy(), dA_ref) <= TOL
-    assert rel_err(dB.cpu().numpy(), dB_ref) <= TOL
+    margin("cfg1_512", "dX", dx.float().cpu().numpy(), dx_ref)
+    margin("cfg1_512", "dA", dA.cpu().numpy(), dA_ref)
+    margin("cfg1_512", "dB", dB.cpu().numpy(), dB_ref)
 
 
 @pytest.mark.parametrize("M", [1, 4, 16])
@@ -160,11 +166,11 @@ def test_config2_small_m_forward_and_merge(M):
     x, A, B = (to_f64(layer.cpu[k]) for k in ("x", "A", "B"))
     g, s = cfg.group_size, cfg.scale
     y_ref = O.forward(x, codes, alpha, beta, g, A, B, s)
-    assert rel_err(layer.forward().float().cpu().numpy(), y_ref) <= TOL
+    margin(f"cfg2_7b_attn_m{M}", "y", layer.forward().float().cpu().numpy(), y_ref)
     q2 = torch.empty_like(layer.qparams)
     Q.qalora_merge(layer.d, layer.qparams, layer.dev["A"], layer.dev["B"], q2)
-    assert rel_err(q2.cpu().numpy()[..., 1], O.merge(beta, A, B, s)) <= TOL
-    assert rel_err(layer.forward(qparams=q2, rank=0).float().cpu().numpy(), y_ref) <= TOL
+    margin(f"cfg2_7b_attn_m{M}", "beta_merged", q2.cpu().numpy()[..., 1], O.merge(beta, A, B, s))
+    margin(f"cfg2_7b_attn_m{M}", "y_merged", layer.forward(qparams=q2, rank=0).float().cpu().numpy(), y_ref)
 
 
 @pytest.mark.parametrize("bits,g,M,r", [(4, 32, 1, 16), (4, 128, 8, 0), (3, 32, 16, 24), (3, 64, 3, 8),
@@ -185,7 +191,7 @@ def test_few_token_forward_all_widths(bits, g, M, r):
         y_ref = O.forward(x, codes, alpha, beta, g, A, B, cfg.scale)
         got = layer.forward()
     assert Q.qalora_main_kernel_name() == "qalora_gemv_kernel"
-    assert rel_err(got.float().cpu().numpy(), y_ref) <= TOL
+    margin(f"few_token_b{bits}_g{g}_m{M}_r{r}", "y", got.float().cpu().numpy(), y_ref)
 
 
 @pytest.mark.parametrize("M", [1, 8])
@@ -276,6 +282,93 @@ def test_edge_cases():
     # m = 0 is a no-op that still succeeds
     empty = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
     assert layer.forward(x=empty).shape == (0, 64)
+
+
+def test_quantize_groups_with_extreme_scales():
+    """Groups whose scale alpha is a subnormal (nearly equal tiny weights) or huge: 1 / alpha
+    overflows or loses its precision there, so the kernel must take Eq. 1's division for them;
+    the codes stay bit-exact."""
+    K, N, g = 64, 128, 32
+    d = Q.desc(K, N, g, 4, 8, 1.0)
+    gen = torch.Generator(device="cpu").manual_seed(3)
+    W = torch.randn((K, N), generator=gen, dtype=torch.float32) * 0.02
+    W[:32, 0:8] = 1.2e-38 + torch.rand((32, 8), generator=gen) * 1.5e-38  # normal weights, alpha about 1e-39 (subnormal)
+    W[:32, 8:16] = torch.rand((32, 8), generator=gen) * 3e-38             # alpha about 2e-39
+    W[32:, 16:24] = 1e37 + torch.rand((32, 8), generator=gen) * 2e37      # alpha above 1e35
+    W[32:, 24:32] = torch.rand((32, 8), generator=gen) * 1e-29            # alpha just below the fast range
+    codes_d, qparams = Q.alloc_packed(d)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Q.qalora_quantize(d, W.cuda(), codes_d, qparams, status)
+    torch.cuda.synchronize()
+    codes, alpha, beta = O.quantize(W.numpy(), g, 4)
+    assert 0 < float(alpha[0, 0]) < 1.1e-38 and 0 < float(alpha[0, 8]) < 1.1e-38 and float(alpha[1, 16]) > 1e35   # the cases are what they claim to be
+    assert np.array_equal(codes_d.cpu().numpy().view(np.uint32), O.pack(codes, 4))
+    qp = qparams.cpu().numpy()
+    assert np.array_equal(qp[..., 0], alpha) and np.array_equal(qp[..., 1], beta)
+    assert int(status.item()) == 0
+
+
+@pytest.mark.parametrize("case", [("simt", 320, 200, 77), ("tensor_core", 256, 256, 300), ("few_token", 1280, 384, 5),
+                                  ("parts", 2048, 256, 40)],
+                         ids=lambda c: c[0])
+def test_status_word_is_cleared_whatever_the_workspace_held(case):
+    """The workspace's content is undefined on entry; after a call that went well its first
+    int32 must read 0 on every dispatch path, also when the workspace was full of 0xFF."""
+    name, K, N, M = case
+    cfg = LayerConfig("status_" + name, K, N, 32, 4, 16, 1.0, M, seed=K + M)
+    layer = GpuLayer(cfg)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.full((max(Q.qalora_workspace_bytes(layer.d, M, Q.OP_FORWARD), 16),), 0xFF, dtype=torch.uint8, device="cuda")
+    Q.qalora_forward(layer.d, M, layer.dev["x"], layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"], y, ws)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(ws) == 0
+    assert torch.equal(y, layer.forward())
+    wb = torch.full((Q.qalora_workspace_bytes(layer.d, M, Q.OP_BACKWARD),), 0xFF, dtype=torch.uint8, device="cuda")
+    dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dA = torch.empty((cfg.groups, cfg.rank), dtype=torch.float32, device="cuda")
+    dB = torch.empty((cfg.rank, N), dtype=torch.float32, device="cuda")
+    Q.qalora_backward(layer.d, M, layer.dev["x"], layer.dev["dy"], layer.codes, layer.qparams, layer.dev["A"],
+                      layer.dev["B"], dx, dA, dB, wb)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(wb) == 0
+    ref = layer.backward()
+    assert torch.equal(dx, ref[0]) and torch.equal(dA, ref[1]) and torch.equal(dB, ref[2])
+
+
+def test_an_expired_wait_raises_the_status_word_and_the_next_call_is_clean():
+    """Failure detection without a fault: a test hook makes the producers of ONE few-token
+    launch stop after two stages and shortens that launch's wait limit to a millisecond.  The
+    consumers' bounded waits then run out; the kernel must come back by itself with the status
+    word at 1 (outputs invalid), the context must stay usable, and the following ordinary
+    call must give the very same bits as before."""
+    import ctypes
+    cfg = LayerConfig("expire", 2048, 512, 32, 4, 16, 1.0, 4, seed=11)
+    layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
+    lib = Q.load()
+    hook = lib.qalora_debug_expire_next_few_token_wait
+    hook.restype = ctypes.c_int
+    hook.argtypes = [ctypes.c_int, ctypes.c_uint64]
+    M = cfg.tokens
+    d0 = Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, 0, cfg.scale)
+    ws = Q.alloc_workspace(d0, M, Q.OP_FORWARD)
+    before = torch.empty((M, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+    Q.qalora_forward(d0, M, layer.dev["x"], layer.codes, layer.qparams, None, None, before, ws)
+    torch.cuda.synchronize()
+    assert Q.qalora_main_kernel_name() == "qalora_gemv_kernel" and Q.workspace_status(ws) == 0
+    assert hook(2, 1_000_000) == 0
+    broken = torch.empty_like(before)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    Q.qalora_forward(d0, M, layer.dev["x"], layer.codes, layer.qparams, None, None, broken, ws)
+    t1.record()
+    torch.cuda.synchronize()                              # returns: the kernel gave up by itself
+    assert Q.workspace_status(ws) == 1
+    assert t0.elapsed_time(t1) < 1000.0                   # ms: far below the ordinary two-second limit
+    after = torch.empty_like(before)
+    Q.qalora_forward(d0, M, layer.dev["x"], layer.codes, layer.qparams, None, None, after, ws)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(ws) == 0                    # the hook was one-shot and the word was cleared
+    assert torch.equal(after, before)
 
 
 def test_results_do_not_depend_on_scheduling():
