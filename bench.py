@@ -36,13 +36,57 @@ SMALL_M = "cfg2_7b_attn"
 
 
 # ----------------------------------------------------------- work accounting --
-# DRAM traffic of ONE launch of the forward contraction kernel at the benchmark size
-# (4096 -> 11008, M = 8192), from a one-pass ncu capture of
-#   python bench.py --only fwd --tokens 8192 --steps 3
-# with --metrics dram__bytes_read.sum,dram__bytes_write.sum (156.8 MB read + 155.6 MB
-# written; algorithmic 282.7 MB).  Counters of the kernel as it stands; set to None when
-# qalora_tc_kernel changes until they have been taken again.
-FWD_KERNEL_DRAM_BYTES = 312.4e6
+# DRAM traffic of ONE launch of the forward contraction kernel at the benchmark size comes
+# from the record kept beside the profile summaries (written by hand from an ncu capture,
+# with the SHA-256 of the kernel's sources at the time): when the sources have changed
+# since, the counters no longer describe the kernel and the bench reports null.
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "qalora_tc_kernel_fwd_cfg3_up_m8192_dram_traffic.txt")
+KERNEL_SOURCES = ("gemm_tc.cu", "ptx.cuh", "common.cuh")
+
+
+def kernel_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2309_14717_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def fwd_kernel_dram_traffic():
+    """(bytes per launch or None, note) from the traffic record, valid only for unchanged sources."""
+    try:
+        rec = dict(line.split(":", 1) for line in open(TRAFFIC_RECORD).read().splitlines() if ":" in line)
+        rec = {k.strip(): v.strip() for k, v in rec.items()}
+        if rec.get("sources_sha256") != kernel_sources_sha256():
+            return None, "kernel sources changed since the counters were taken"
+        return float(rec["dram_bytes_read"]) + float(rec["dram_bytes_write"]), "profiles/" + os.path.basename(TRAFFIC_RECORD)
+    except (OSError, KeyError, ValueError) as e:
+        return None, f"no usable traffic record ({type(e).__name__})"
+
+
+def host_threads():
+    """Threads the CPU oracle can use: the affinity mask of this process and the thread
+    count of the BLAS that numpy calls."""
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    blas = None
+    try:
+        from threadpoolctl import threadpool_info
+        blas = max((int(p.get("num_threads", 0)) for p in threadpool_info() if p.get("user_api") == "blas"), default=None)
+    except Exception:
+        pass
+    return cores, blas
+
+
+def tensor_sha256(t):
+    """SHA-256 of a CPU tensor's bytes (bf16 viewed as int16)."""
+    import hashlib
+
+    import torch
+    t = t.contiguous()
+    if t.dtype == torch.bfloat16:
+        t = t.view(torch.int16)
+    return hashlib.sha256(t.numpy().tobytes()).hexdigest()
 
 
 def fwd_flops(M, K, N, G, r):
@@ -171,7 +215,7 @@ def oracle_sample(rows=32):
         fl_sum += fl
         descs.append(desc)
         del state
-    return fl_sum / dt_sum / 1e12, dt_sum, "; ".join(descs), torch.get_num_threads()
+    return fl_sum / dt_sum / 1e12, dt_sum, "; ".join(descs), host_threads()
 
 
 def run_reference(args):
@@ -188,12 +232,13 @@ def run_reference(args):
             times.append(dt)
     ms = 1e3 * sum(times) / max(1, len(times))
     value = fl / (ms / 1e3) / 1e12
-    cores = torch.get_num_threads()
+    cores, blas = host_threads()
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": WORKLOAD, "sample": desc},
-            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "blas_threads": blas, "kind": "oracle",
+                             "sample": desc},
             "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -207,6 +252,8 @@ class ShapeState:
         shared = make_inputs(cfg, need=("W", "A", "B"))
         batch = make_inputs(cfg.with_(seed=cfg.seed + 1000 * (rank + 1)), need=("x", "dy"))
         self.host = {"x": batch["x"].pin_memory(), "dy": batch["dy"].pin_memory()}
+        self.sha256 = {k: tensor_sha256(v) for k, v in (("W", shared["W"]), ("A", shared["A"]), ("B", shared["B"]),
+                                                      ("x", batch["x"]), ("dy", batch["dy"]))}
         self.W = shared["W"].cuda()
         self.A = shared["A"].cuda()
         self.B = shared["B"].cuda()
@@ -344,15 +391,32 @@ def run_gpu(args):
     kms = sum(a.elapsed_time(b) for a, b in probe_pairs) / len(probe_pairs)
     pk = peaks()
     achieved = s0.main_flops / (kms / 1e3) / 1e12
-    roofline = {"bound": "tensor", "kernel": kernel_name, "achieved": achieved, "peak": pk["tensor"],
-                "unit": "TFLOP/s", "frac": achieved / pk["tensor"], "peak_source": pk["source"] + " (sustained bf16)",
-                "kernel_ms": kms, "launches_timed": len(probe_pairs), "traffic": FWD_KERNEL_DRAM_BYTES,
+    # Which measured cuBLAS figure fits this run: the sustained one (a seconds-long loop under
+    # the power cap) only when the timed region was itself seconds long AND the power cap was
+    # seen active in it; a short region at full clocks is compared with the burst figure.
+    sustained = (ms_total >= 2000.0) and clocks is not None and "sw_power_cap" in (clocks.get("reasons") or [])
+    peak = pk["tensor"] if sustained else pk["tensor_burst"]
+    traffic, traffic_note = fwd_kernel_dram_traffic()
+    roofline = {"bound": "tensor", "kernel": kernel_name, "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_source": pk["source"] + (" (sustained bf16)" if sustained else " (burst bf16)"),
+                "frac_burst": achieved / pk["tensor_burst"], "frac_sustained": achieved / pk["tensor"],
+                "peak_burst": pk["tensor_burst"], "peak_sustained": pk["tensor"],
+                "step_frac_burst": value / world / pk["tensor_burst"], "step_frac_sustained": value / world / pk["tensor"],
+                "kernel_ms": kms, "launches_timed": len(probe_pairs), "traffic": traffic, "traffic_source": traffic_note,
                 "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum)",
                 "flops_per_launch": s0.main_flops}
 
     # single-token forward of the merged layer: HBM-bound leg of the metric
     small = small_m_bandwidth(Q, torch, pk)
-    small_65b = small_m_bandwidth(Q, torch, pk, shape="cfg5_65b_up", ms=(1,)) if rank == 0 else None
+    small_65b = mid = None
+    if rank == 0:
+        from paper_2309_14717_b200.synthetic import CONFIGS
+        small_65b = small_m_bandwidth(Q, torch, pk, shape="cfg5_65b_up", ms=(1, 16))
+        for g in (64, 128):          # the group-size sweep of the 65B configuration, one token
+            r_ = small_m_bandwidth(Q, torch, pk, ms=(1,), cfg=CONFIGS["cfg5_65b_up"].with_(group_size=g))
+            small_65b[f"g{g}"] = {k: r_[k] for k in ("M1", "M1_merged")}
+        mid = {name: mid_m_roofline(Q, torch, pk, name) for name in (SMALL_M, "cfg5_65b_up")}
 
     adamw = adapter_update_bandwidth(Q, torch, pk) if rank == 0 else None
 
@@ -365,8 +429,9 @@ def run_gpu(args):
         # the CPU oracle is timed at N = 1 only (the other GPUs would be held idle meanwhile)
         cpu = None
         if world == 1:
-            v, dt, desc, cores = oracle_sample(rows=8192)
-            cpu = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc, "seconds": dt}
+            v, dt, desc, (cores, blas) = oracle_sample(rows=8192)
+            cpu = {"value": v, "unit": "TFLOP/s", "cores": cores, "blas_threads": blas, "kind": "oracle", "sample": desc,
+                   "seconds": dt}
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -379,12 +444,29 @@ def run_gpu(args):
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": flops_step / (e2e_ms / 1e3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "roofline": roofline, "small_m": small, "small_m_65b": small_65b,
+            "roofline": roofline, "small_m": small, "small_m_65b": small_65b, "mid_m": mid,
             "adapter_update": adamw, "cpu_baseline": cpu,
+            "inputs_sha256": {s.cfg.name: s.sha256 for s in shapes}, "inputs_match_record": inputs_match_record(shapes),
         }
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def inputs_match_record(shapes):
+    """Compares the hashes of this run's synthetic inputs (rank 0's batch) with the record kept
+    in tests/golden/bench_inputs_sha256.txt, written by tests/golden/make_bench_inputs_sha256.py
+    from the generator alone: a torch version that drew other numbers would show here."""
+    path = os.path.join(ROOT, "tests", "golden", "bench_inputs_sha256.txt")
+    try:
+        want = {}
+        for line in open(path):
+            if line.strip() and not line.startswith("#"):
+                name, tensor, digest = line.split()
+                want[(name, tensor)] = digest
+    except OSError:
+        return None
+    return all(want.get((s.cfg.name, k)) == v for s in shapes for k, v in s.sha256.items())
 
 
 def adapter_update_bandwidth(Q, torch, pk, reps=10):
@@ -470,6 +552,64 @@ def small_m_bandwidth(Q, torch, pk, shape=SMALL_M, ms=(1, 4, 16), cfg=None):
     out["peak_source"] = pk["source"]
     out["l2"] = (f"CUDA-graph replay rotating over {ncopies} weight copies ({ncopies * layer_bytes / 1e6:.0f} MB) "
                  "so codes stream from HBM")
+    return out
+
+
+def mid_m_roofline(Q, torch, pk, shape, ms=(64, 128, 256, 512)):
+    """Forward of one layer shape at a few hundred tokens, adapted and merged, rotating over
+    weight copies like small_m_bandwidth.  Both rooflines are given: the bytes of one call at
+    the measured copy bandwidth and 2 M K N flops at the measured burst bf16 rate; `frac` is
+    against the slower (larger) of the two bounds."""
+    from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
+    cfg = CONFIGS[shape]
+    t = make_inputs(cfg.with_(tokens=max(ms)), need=("W", "x", "A", "B"))
+    K, N, G, r = cfg.d_in, cfg.d_out, cfg.groups, cfg.rank
+    d = Q.desc(K, N, cfg.group_size, cfg.bits, r, cfg.scale)
+    d0 = Q.desc(K, N, cfg.group_size, cfg.bits, 0, cfg.scale)
+    W = t["W"].cuda()
+    A, B = t["A"].cuda(), t["B"].cuda()
+    codes, qparams = Q.alloc_packed(d)
+    Q.qalora_quantize(d, W, codes, qparams)
+    del W
+    layer_bytes = codes.numel() * 4 + qparams.numel() * 4
+    ncopies = max(4, -(-5 * 126 * 2 ** 20 // layer_bytes))
+    copies = [(codes.clone(), qparams.clone()) for _ in range(ncopies)]
+    out = {}
+    side = torch.cuda.Stream()
+    for M in ms:
+        x = t["x"][:M].contiguous().cuda()
+        y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        for name, dd, a_, b_ in (("", d, A, B), ("_merged", d0, None, None)):
+            ws = Q.alloc_workspace(dd, M, Q.OP_FORWARD)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                for c, q in copies[:3]:
+                    Q.qalora_forward(dd, M, x, c, q, a_, b_, y, ws)
+            side.synchronize()
+            kernel = Q.qalora_main_kernel_name()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for c, q in copies:
+                    Q.qalora_forward(dd, M, x, c, q, a_, b_, y, ws)
+            graph.replay()
+            torch.cuda.synchronize()
+            reps = 3
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / (reps * ncopies)
+            nbytes = fwd_bytes(M, K, N, G, dd.rank, cfg.bits)
+            flops = 2 * M * K * N
+            t_hbm, t_tc = nbytes / (pk["hbm"] * 1e9) * 1e6, flops / (pk["tensor_burst"] * 1e12) * 1e6
+            out[f"M{M}{name}"] = {"us_per_call": us, "kernel": kernel, "bytes": nbytes, "flops": flops,
+                                  "hbm_bound_us": t_hbm, "tensor_bound_us": t_tc, "frac": max(t_hbm, t_tc) / us,
+                                  "bound": "hbm" if t_hbm >= t_tc else "tensor"}
+            del graph
+    out["shape"] = shape
+    out["peaks"] = {"hbm_GB/s": pk["hbm"], "bf16_burst_TFLOP/s": pk["tensor_burst"], "source": pk["source"]}
     return out
 
 

@@ -153,6 +153,7 @@ def alloc_packed(d: QaloraDesc, device="cuda"):
 
 
 def alloc_workspace(d: QaloraDesc, m: int, op: int, device="cuda") -> torch.Tensor:
+    """Zeroed scratch of qalora_workspace_bytes() bytes (at least 16) for `m` rows."""
     return torch.zeros(max(qalora_workspace_bytes(d, m, op), 16), dtype=torch.uint8, device=device)
 
 

@@ -91,3 +91,45 @@ class AdapterBucket:
         h = Q.adamw_hyper(self.step_count, lr, beta1, beta2, eps, weight_decay, max_grad_norm)
         Q.qalora_adamw_step(h, self.n, self.grad, self.master, self.exp_avg, self.exp_avg_sq, self.bf16, self.norm,
                             self._workspace, stream)
+
+
+class AdaptedLayer:
+    """One quantized layer of a data-parallel fine-tuning step: its descriptor, packed codes and
+    (alpha, beta) (frozen, replicated on every rank) and the workspaces of its two passes for
+    `tokens` rows per rank.  The trained factors are not here: they live in the AdapterBucket."""
+
+    def __init__(self, d, codes, qparams, tokens: int):
+        from . import binding as Q
+        self.d, self.codes, self.qparams, self.tokens = d, codes, qparams, tokens
+        self.ws_forward = Q.alloc_workspace(d, tokens, Q.OP_FORWARD, device=codes.device)
+        self.ws_backward = Q.alloc_workspace(d, tokens, Q.OP_BACKWARD, device=codes.device)
+
+    @property
+    def shape(self):
+        """(G, r, N): the entry AdapterBucket wants for this layer."""
+        return self.d.d_in // self.d.group_size, self.d.rank, self.d.d_out
+
+
+def finetune_step(layers, bucket: AdapterBucket, xs, dys, ys, dxs, lr, group=None, stream=None, **adamw):
+    """One data-parallel fine-tuning step over `layers` (Section 4.1: only A and B are trained,
+    AdamW with a maximum gradient norm), every piece of it a call into the CUDA library:
+
+      forward of layer i from the bucket's bf16 factors  -> ys[i]
+      backward of layer i, dA and dB written STRAIGHT into the bucket's gradient views, dX -> dxs[i]
+      ONE all-reduce of the whole gradient array over the ranks (the step's only exchange)
+      ONE clipped AdamW update of every factor; it also refreshes the bf16 copies the next
+      step's forward reads.
+
+    xs[i] / dys[i] are this rank's rows of layer i's input and output gradient (each layer has its
+    own here: the layers are independent linear layers, not a chain).  Everything is enqueued on
+    `stream` (torch's current stream by default) without synchronizing."""
+    from . import binding as Q
+    for i, L in enumerate(layers):
+        A, B = bucket.factors(i)
+        Q.qalora_forward(L.d, L.tokens, xs[i], L.codes, L.qparams, A, B, ys[i], L.ws_forward, stream)
+    for i, L in enumerate(layers):
+        A, B = bucket.factors(i)
+        dA, dB = bucket.grads(i)
+        Q.qalora_backward(L.d, L.tokens, xs[i], dys[i], L.codes, L.qparams, A, B, dxs[i], dA, dB, L.ws_backward, stream)
+    bucket.reduce(group)
+    bucket.update(lr, stream=stream, **adamw)

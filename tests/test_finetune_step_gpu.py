@@ -1,0 +1,94 @@
+"""The composed data-parallel fine-tuning step (world size 1 here): forward from the bucket's
+bf16 factors, backward writing dA and dB straight into the bucket's gradient views, the (no-op)
+all-reduce, and the clipped AdamW update that refreshes the factors the next forward reads.
+Two consecutive steps are checked against the CPU oracles: qalora_oracle for the layer,
+optimizer_oracle for the update (Section 4.1).  The oracle side never sees a GPU value: it
+carries its own fp64 state from the same seeded start."""
+import numpy as np
+import pytest
+import torch
+
+from conftest import record_margin
+from oracle import optimizer_oracle as P
+from oracle import qalora_oracle as O
+from paper_2309_14717_b200 import binding as Q
+from paper_2309_14717_b200 import dp
+from paper_2309_14717_b200.synthetic import LayerConfig, make_inputs, to_f64
+
+pytestmark = pytest.mark.gpu
+TOL = 5e-3
+
+CFGS = [LayerConfig("step_a", 256, 256, 32, 4, 16, 8.0, 300, seed=41),
+        LayerConfig("step_b", 384, 256, 64, 3, 24, 8.0, 300, seed=42),
+        LayerConfig("step_c", 320, 200, 32, 2, 8, 8.0, 300, seed=43)]     # the last one runs on the CUDA-core kernels
+
+
+def rel(got, ref):
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    return float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
+
+
+def bf16_round(a64):
+    return torch.from_numpy(np.asarray(a64, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def test_two_consecutive_steps_match_the_oracles():
+    lr, max_norm = 4e-3, 0.3
+    cpu = [make_inputs(c) for c in CFGS]
+    layers, quant = [], []
+    for c, t in zip(CFGS, cpu):
+        d = Q.desc(c.d_in, c.d_out, c.group_size, c.bits, c.rank, c.scale)
+        codes, qparams = Q.alloc_packed(d)
+        Q.qalora_quantize(d, t["W"].cuda(), codes, qparams)
+        layers.append(dp.AdaptedLayer(d, codes, qparams, c.tokens))
+        quant.append(O.quantize(t["W"].numpy(), c.group_size, c.bits))
+    bucket = dp.AdapterBucket([L.shape for L in layers], device="cuda")
+    for i, t in enumerate(cpu):
+        bucket.load(i, t["A"].cuda(), t["B"].cuda())
+    xs = [t["x"].cuda() for t in cpu]
+    dys = [t["dy"].cuda() for t in cpu]
+    ys = [torch.empty((c.tokens, c.d_out), dtype=torch.bfloat16, device="cuda") for c in CFGS]
+    dxs = [torch.empty((c.tokens, c.d_in), dtype=torch.bfloat16, device="cuda") for c in CFGS]
+
+    # oracle state: fp64 masters from the same bf16 start, zero moments
+    master = [np.concatenate([to_f64(t["A"]).ravel(), to_f64(t["B"]).ravel()]) for t in cpu]
+    master = [np.concatenate(master)]
+    m1, m2 = [np.zeros_like(master[0])], [np.zeros_like(master[0])]
+    first_y = None
+    for step in (1, 2):
+        dp.finetune_step(layers, bucket, xs, dys, ys, dxs, lr, max_grad_norm=max_norm)
+        torch.cuda.synchronize()
+        for L in layers:
+            assert Q.workspace_status(L.ws_forward) == 0 and Q.workspace_status(L.ws_backward) == 0
+        grads, off = [], 0
+        for i, (c, t, (codes, alpha, beta)) in enumerate(zip(CFGS, cpu, quant)):
+            G, r, N = layers[i].shape
+            A = bf16_round(master[0][off:off + G * r].reshape(G, r)); off += G * r
+            B = bf16_round(master[0][off:off + r * N].reshape(r, N)); off += r * N
+            x, dy = to_f64(t["x"]), to_f64(t["dy"])
+            y_ref = O.forward(x, codes, alpha, beta, c.group_size, A, B, c.scale)
+            dx_ref, dA_ref, dB_ref = O.backward(x, dy, codes, alpha, beta, c.group_size, A, B, c.scale)
+            case = f"finetune_step{step}_{c.name}"
+            record_margin(case, "y", rel(ys[i].float().cpu().numpy(), y_ref), TOL)
+            record_margin(case, "dX", rel(dxs[i].float().cpu().numpy(), dx_ref), TOL)
+            grads += [dA_ref.ravel(), dB_ref.ravel()]
+            if i == 0:
+                if first_y is None:
+                    first_y = y_ref
+                else:   # the update is visible in the second step's output (the test would not pass on stale factors)
+                    assert rel(first_y, y_ref) > 2 * TOL
+        g_ref = np.concatenate(grads)
+        # the gradient array the update consumed is still in the bucket (the update does not touch it)
+        record_margin(f"finetune_step{step}", "grad_bucket", rel(bucket.grad.cpu().numpy(), g_ref), TOL)
+        master, m1, m2, norm, coef = P.adamw_step(master, [g_ref], m1, m2, step, np.float32(lr).item(), 0.9, 0.999,
+                                                   np.float32(1e-8).item(), 0.0, np.float32(max_norm).item())
+        assert coef < 1.0                                   # these gradients are clipped
+        gn, gc = bucket.norm.cpu().tolist()
+        assert gn == pytest.approx(norm, rel=TOL) and gc == pytest.approx(coef, rel=TOL)
+        # parameters: against the accumulated movement (AdamW moves every value by about lr per
+        # step, in the direction of its gradient's sign: the few values whose gradient is within
+        # the bf16 intermediates' error of zero may move the other way, by up to 2 lr per step)
+        diff = np.abs(bucket.master.cpu().double().numpy() - master[0])
+        assert float(np.mean(diff > 0.05 * step * lr)) < 0.01 and float(diff.max()) <= 2.1 * step * lr
+        assert torch.equal(bucket.bf16, bucket.master.to(torch.bfloat16))
+    assert bucket.step_count == 2

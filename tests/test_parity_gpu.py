@@ -342,7 +342,7 @@ def test_an_expired_wait_raises_the_status_word_and_the_next_call_is_clean():
     word at 1 (outputs invalid), the context must stay usable, and the following ordinary
     call must give the very same bits as before."""
     import ctypes
-    cfg = LayerConfig("expire", 2048, 512, 32, 4, 16, 1.0, 4, seed=11)
+    cfg = LayerConfig("expire", 8192, 512, 32, 4, 16, 1.0, 4, seed=11)    # 64 stages over at most 8 slices: 8 or more per block
     layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
     lib = Q.load()
     hook = lib.qalora_debug_expire_next_few_token_wait
