@@ -10,9 +10,10 @@ by the time of the whole step).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
-runs the same step on its own batch (data parallel over tokens) and the
-adapter gradients are all-reduced over NCCL.  `--impl reference` times the CPU
+The adapter gradients of both shapes land in one flat bucket that one clipped
+AdamW call (Section 4.1) consumes inside the step.  With N > 1 (launched by
+torch.distributed.run, one rank per GPU) every rank runs the same step on its own
+batch (data parallel over tokens) and the bucket is all-reduced once over NCCL.  `--impl reference` times the CPU
 oracle on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
@@ -266,8 +267,6 @@ class ShapeState:
         self.qmerged = torch.empty_like(self.qparams)
         self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
         self.dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
-        self.dA = torch.empty((G, r), dtype=torch.float32, device="cuda")
-        self.dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
         self.ws_f = Q.alloc_workspace(self.d, M, Q.OP_FORWARD)
         self.ws_b = Q.alloc_workspace(self.d, M, Q.OP_BACKWARD)
         self.x1 = self.x[:1].contiguous()
@@ -306,34 +305,48 @@ def run_gpu(args):
 
     shapes = [ShapeState(n, rank, Q, torch) for n in SHAPES]
     stream = torch.cuda.current_stream()
+    # All trained factors of the step live in one bucket: the backward passes write dA and dB into
+    # its gradient views, ONE all-reduce sums it over the ranks and ONE clipped AdamW call
+    # (Section 4.1) updates every factor and the bf16 copies the next forward reads.
+    bucket = dp.AdapterBucket([(s.cfg.groups, s.cfg.rank, s.cfg.d_out) for s in shapes], device="cuda")
+    for i, s in enumerate(shapes):
+        bucket.load(i, s.A, s.B)
+    LR = 2e-5                                          # the paper's learning rate for the 7B model
 
-    def device_step(s, probe=None):
+    def device_step(i, s, probe=None):
+        A, B = bucket.factors(i)
+        dA, dB = bucket.grads(i)
         Q.qalora_quantize(s.d, s.W, s.codes, s.qparams)
         if probe is not None:                      # events around the forward contraction kernel of this call
             Q.qalora_profile_next_main_kernel(*probe)
-        Q.qalora_forward(s.d, s.cfg.tokens, s.x, s.codes, s.qparams, s.A, s.B, s.y, s.ws_f)
-        Q.qalora_backward(s.d, s.cfg.tokens, s.x, s.dy, s.codes, s.qparams, s.A, s.B, s.dx, s.dA, s.dB, s.ws_b)
-        if world > 1:
-            dp.allreduce_adapter_grads(s.dA, s.dB)
-        Q.qalora_merge(s.d, s.qparams, s.A, s.B, s.qmerged)
+        Q.qalora_forward(s.d, s.cfg.tokens, s.x, s.codes, s.qparams, A, B, s.y, s.ws_f)
+        Q.qalora_backward(s.d, s.cfg.tokens, s.x, s.dy, s.codes, s.qparams, A, B, s.dx, dA, dB, s.ws_b)
+
+    def deploy_step(i, s):
+        A, B = bucket.factors(i)
+        Q.qalora_merge(s.d, s.qparams, A, B, s.qmerged)
         Q.qalora_forward(s.d0, 1, s.x1, s.codes, s.qmerged, None, None, s.y1, s.ws1)
 
     probes = []                                     # one event pair per timed step (first shape's forward kernel)
 
     def step():
         for j, s in enumerate(shapes):
-            device_step(s, probes.pop() if (j == 0 and probes) else None)
+            device_step(j, s, probes.pop() if (j == 0 and probes) else None)
+        bucket.reduce()                             # the step's only exchange (a no-op on one GPU)
+        bucket.update(LR)
+        for j, s in enumerate(shapes):
+            deploy_step(j, s)
 
     def e2e_step():
         # the same step through the C ABI with HOST buffers: x, dy go up and y, dx, dA, dB
         # come back inside qalora_step_host; quantize, merge and the merged one-token
         # forward work on resident weights as in the device-resident step
-        for s in shapes:
+        for j, s in enumerate(shapes):
+            A, B = bucket.factors(j)
             Q.qalora_quantize(s.d, s.W, s.codes, s.qparams)
-            Q.qalora_step_host(s.d, s.cfg.tokens, s.host["x"], s.host["dy"], s.codes, s.qparams, s.A, s.B,
+            Q.qalora_step_host(s.d, s.cfg.tokens, s.host["x"], s.host["dy"], s.codes, s.qparams, A, B,
                                s.host_out["y"], s.host_out["dx"], s.host_out["dA"], s.host_out["dB"], s.staging)
-            Q.qalora_merge(s.d, s.qparams, s.A, s.B, s.qmerged)
-            Q.qalora_forward(s.d0, 1, s.x1, s.codes, s.qmerged, None, None, s.y1, s.ws1)
+            deploy_step(j, s)
 
     def timed(fn, steps, sampler=None):
         if world > 1:
@@ -377,7 +390,7 @@ def run_gpu(args):
     launches0 = Q.qalora_kernel_launches()
     ms_total, clocks = timed(step, args.steps, sampler)
     s0_ = shapes[0]
-    Q.qalora_forward(s0_.d, s0_.cfg.tokens, s0_.x, s0_.codes, s0_.qparams, s0_.A, s0_.B, s0_.y, s0_.ws_f)
+    Q.qalora_forward(s0_.d, s0_.cfg.tokens, s0_.x, s0_.codes, s0_.qparams, *bucket.factors(0), s0_.y, s0_.ws_f)
     kernel_name = Q.qalora_main_kernel_name()       # which kernel the library picks for this shape
     torch.cuda.synchronize()
     launches = (Q.qalora_kernel_launches() - launches0) // max(1, args.steps)
@@ -438,7 +451,9 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "shapes": list(SHAPES), "tokens_per_gpu": 8192, "bits": 4,
                        "group_size": 32, "rank": 64,
-                       "step": "quantize+forward+backward+merge+merged M=1 forward, both shapes",
+                       "step": "both shapes: quantize+forward+backward (dA, dB into one gradient bucket); one all-reduce "
+                               "of the bucket (N > 1); one clipped AdamW update of all factors; both shapes: merge + "
+                               "merged M=1 forward",
                        "l2": "inputs exceed L2 (x+dy+y+dx > 470 MB per shape)",
                        "parallelism": f"dp{world}" if world > 1 else "single"},
             "clocks": clocks, "gpu_launches": int(launches),

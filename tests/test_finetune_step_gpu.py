@@ -33,7 +33,10 @@ def bf16_round(a64):
 
 
 def test_two_consecutive_steps_match_the_oracles():
-    lr, max_norm = 4e-3, 0.3
+    # eps is taken of the size of a clipped gradient (0.3 / sqrt(14 K values) = 2.5e-3): with the usual
+    # 1e-8 AdamW's first steps are lr * sign(g), and the few values whose gradient lies within the bf16
+    # intermediates' error of zero would move the other way on the GPU, which the next forward then shows
+    lr, max_norm, eps = 4e-3, 0.3, 1e-3
     cpu = [make_inputs(c) for c in CFGS]
     layers, quant = [], []
     for c, t in zip(CFGS, cpu):
@@ -56,7 +59,7 @@ def test_two_consecutive_steps_match_the_oracles():
     m1, m2 = [np.zeros_like(master[0])], [np.zeros_like(master[0])]
     first_y = None
     for step in (1, 2):
-        dp.finetune_step(layers, bucket, xs, dys, ys, dxs, lr, max_grad_norm=max_norm)
+        dp.finetune_step(layers, bucket, xs, dys, ys, dxs, lr, max_grad_norm=max_norm, eps=eps)
         torch.cuda.synchronize()
         for L in layers:
             assert Q.workspace_status(L.ws_forward) == 0 and Q.workspace_status(L.ws_backward) == 0
@@ -81,14 +84,12 @@ def test_two_consecutive_steps_match_the_oracles():
         # the gradient array the update consumed is still in the bucket (the update does not touch it)
         record_margin(f"finetune_step{step}", "grad_bucket", rel(bucket.grad.cpu().numpy(), g_ref), TOL)
         master, m1, m2, norm, coef = P.adamw_step(master, [g_ref], m1, m2, step, np.float32(lr).item(), 0.9, 0.999,
-                                                   np.float32(1e-8).item(), 0.0, np.float32(max_norm).item())
+                                                   np.float32(eps).item(), 0.0, np.float32(max_norm).item())
         assert coef < 1.0                                   # these gradients are clipped
         gn, gc = bucket.norm.cpu().tolist()
         assert gn == pytest.approx(norm, rel=TOL) and gc == pytest.approx(coef, rel=TOL)
-        # parameters: against the accumulated movement (AdamW moves every value by about lr per
-        # step, in the direction of its gradient's sign: the few values whose gradient is within
-        # the bf16 intermediates' error of zero may move the other way, by up to 2 lr per step)
+        # parameters: against the accumulated movement (at most lr per step and value)
         diff = np.abs(bucket.master.cpu().double().numpy() - master[0])
-        assert float(np.mean(diff > 0.05 * step * lr)) < 0.01 and float(diff.max()) <= 2.1 * step * lr
+        assert float(diff.max()) <= 0.02 * step * lr, float(diff.max())
         assert torch.equal(bucket.bf16, bucket.master.to(torch.bfloat16))
     assert bucket.step_count == 2
