@@ -643,11 +643,19 @@ def run_only(args):
         print(json.dumps({"only": "adamw", **adapter_update_bandwidth(Q, torch, peaks(), reps=max(1, args.steps))}))
         return
     cfg = CONFIGS[args.shape].with_(tokens=args.tokens)
+    if args.group_size:
+        cfg = cfg.with_(group_size=args.group_size)
+    if args.bits:
+        cfg = cfg.with_(bits=args.bits)
     t = {k: v.cuda() for k, v in make_inputs(cfg).items()}
     M, K, N, G, r = cfg.tokens, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank
     d = Q.desc(K, N, cfg.group_size, cfg.bits, r, cfg.scale)
     codes, qparams = Q.alloc_packed(d)
     Q.qalora_quantize(d, t["W"], codes, qparams)
+    if args.merged:                                # the deployed layer: adapter folded into the zeros, rank 0
+        Q.qalora_merge(d, qparams, t["A"], t["B"], qparams)
+        d = Q.desc(K, N, cfg.group_size, cfg.bits, 0, cfg.scale)
+        t["A"] = t["B"] = None
     y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
     dA = torch.empty((G, r), dtype=torch.float32, device="cuda")
@@ -862,6 +870,9 @@ def main():
     ap.add_argument("--only", default=None, choices=("fwd", "bwd", "gemv", "quantize", "merge", "adamw"))
     ap.add_argument("--shape", default="cfg3_7b_up")
     ap.add_argument("--tokens", type=int, default=4096)
+    ap.add_argument("--merged", action="store_true", help="with --only fwd/gemv: the merged (rank 0) layer")
+    ap.add_argument("--group-size", type=int, default=0, help="with --only: override the shape's group size")
+    ap.add_argument("--bits", type=int, default=0, help="with --only: override the shape's bit width")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)

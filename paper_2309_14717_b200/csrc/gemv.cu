@@ -1,4 +1,4 @@
-// Few-token forward (M <= 16): y = x * W~ (+ T * B), bound by streaming the packed
+// Few-token forward (M <= 32): y = x * W~ (+ T * B), bound by streaming the packed
 // codes and the (alpha, beta) pairs from HBM exactly once.
 //
 // Design
@@ -13,17 +13,26 @@
 //  * The products run on mma.sync.m16n8k16 (bf16 in, fp32 accumulate) with 16
 //    columns of W as the rows and 8 tokens as the columns: a lane's 32-bit words
 //    of packed codes ARE its A fragments after one shift and one mask per pair
-//    (the code is OR-ed into the mantissa of bf16 128.0, no conversion), and its
+//    (the code is OR-ed into the mantissa of bf16 128.0, no conversion; with 4-bit
+//    codes one ldmatrix fetches the four words a lane needs for a k-block), and its
 //    16-byte load of x is its B fragments.  The products x * (128 + c) are exact
-//    in fp32; the MMAs of a 32-channel block start from C = -128 xp, so that
-//    D = sum c x, and the block is folded as
-//        acc += alpha * D + beta * xp,
-//    where xp (the group sum of x, which the paper's pooling also needs) comes
-//    from one more MMA with ones as the A operand.  alpha and beta stay fp32.
-//    With group sizes 64 and 128 a set's two k-blocks share (alpha, beta): they go into
-//    one accumulator chain and are folded once.
+//    in fp32; the two MMAs of a 32-channel block give D = sum (128 + c) x, and the
+//    block is folded as
+//        acc += alpha * D + (beta - 128 alpha) * xp,
+//    where xp (the group sum of x, which the paper's pooling also needs) comes from one
+//    more MMA with ones as the A operand (independent of the code MMAs).  alpha and beta
+//    stay fp32.  With group sizes 64 and 128 a set's two k-blocks share (alpha, beta):
+//    they go into one accumulator chain and are folded once.
 //  * The same reduction step adds the adapter term T * B (T = s * pool(x) * A is
 //    computed by the pooling kernel) and rounds to bf16.
+//  * Launches of the layer without adapter carry the programmatic-dependent-launch
+//    attribute: the kernel lets its successor start at once and itself starts as soon
+//    as its predecessor allows, streams the first ring of codes and (alpha, beta) -
+//    weights, which no kernel of a forward pass writes - and waits for the
+//    predecessor's completion (griddepcontrol.wait) only before it fetches x; y is
+//    written after every stage, hence every x slice, has been consumed.
+//    Back-to-back layers of a decoding step thus overlap one layer's tail with the
+//    next one's start.
 #include <cooperative_groups.h>
 
 #include <mutex>
@@ -56,8 +65,13 @@ struct GvSmem {
   static constexpr uint32_t OFF_QP = GV_KBS * CODE_ROW;
   static constexpr uint32_t OFF_X = OFF_QP + GV_KBS * QP_ROW;
   static constexpr uint32_t STAGE_BYTES = ((OFF_X + X_BYTES + 127) / 128) * 128;
-  static constexpr uint32_t OFF_PARTIAL = STAGES * STAGE_BYTES;         // fp32 [sets][rows][128]
-  static constexpr uint32_t OFF_BARS = OFF_PARTIAL + GV_SETS * ROWS * GV_COLS * 4;
+  static constexpr uint32_t RING_BYTES = STAGES * STAGE_BYTES;
+  // fp32 partial sums [sets][rows][128]: written after the last stage has been consumed,
+  // over the ring's memory
+  static constexpr uint32_t PARTIAL_BYTES = GV_SETS * ROWS * GV_COLS * 4;
+  static constexpr uint32_t OFF_PARTIAL = 0;
+  static_assert(PARTIAL_BYTES <= RING_BYTES, "the partial sums reuse the ring");
+  static constexpr uint32_t OFF_BARS = RING_BYTES;
   static constexpr uint32_t TOTAL = OFF_BARS + 128 + 128;               // + alignment slack
 };
 
@@ -71,6 +85,7 @@ struct GvParams {
   int total_stages;             // K / 128
   int* status;
   int reset_status;             // the first block clears *status before any wait can expire
+  int pdl_wait;                 // launched beside its predecessor: the producer waits for it before it fetches x
   int stop_after_stages;        // normally INT_MAX; a test makes every producer stop early, so that waits expire
   unsigned long long wait_limit_ns;
 };
@@ -143,6 +158,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
   const int n0 = (blockIdx.x / splits) * GV_COLS;
   const int st_beg = (int)((long long)p.total_stages * rank / splits);
   const int st_end = (int)((long long)p.total_stages * (rank + 1) / splits);
+  const int n_stages = st_end - st_beg;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 
   if (threadIdx.x == 0) {
@@ -156,82 +172,135 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     ptx::prefetch_tensormap(&codes_map);
     ptx::prefetch_tensormap(&qp_map);
     if (blockIdx.x == 0 && p.reset_status) *p.status = 0;     // a wait gives up only after seconds: no block can have raised it yet
+    // the next kernel in the stream may start (it waits for this one's completion before it
+    // reads or writes anything this one touches)
+    asm volatile("griddepcontrol.launch_dependents;");
   }
   __syncthreads();
 
   if (warp == GV_WARPS) {
     // ------------------------------------------------------------ producer ----
     if (lane == 0) {
+      const int n_issue = n_stages < p.stop_after_stages ? n_stages : p.stop_after_stages;
+      const int qrows = (GV_KBS * 32) / p.g;
+      const uint32_t stage_tx = GV_KBS * S::CODE_ROW + qrows * S::QP_ROW + S::X_BYTES;
+      // three tiled copies per stage: 4 k-block rows of pack units, the rows of
+      // (alpha, beta) they need (128 / g of them) and the x slice.  The first ring of
+      // weights goes out at once; x follows when the predecessor kernel is complete.
+      const int first = n_issue < GV_STAGES ? n_issue : GV_STAGES;
+      if (p.pdl_wait) {
+        for (int it = 0; it < first; ++it) {
+          const int st = st_beg + it;
+          const uint32_t stage = smem_base + it * S::STAGE_BYTES;
+          ptx::mbar_arrive_expect_tx(bar_full(it), stage_tx);
+          ptx::tma_load_2d(stage + S::OFF_CODES, &codes_map, n0 * WORDS / 2, st * GV_KBS, bar_full(it));
+          ptx::tma_load_2d(stage + S::OFF_QP, &qp_map, 2 * n0, st * GV_KBS * 32 / p.g, bar_full(it));
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        for (int it = 0; it < first; ++it)
+          ptx::tma_load_2d(smem_base + it * S::STAGE_BYTES + S::OFF_X, &x_map, (st_beg + it) * GV_KBS * 32, 0, bar_full(it));
+      } else {
+        for (int it = 0; it < first; ++it) {      // no predecessor to wait for: each stage's three copies together
+          const int st = st_beg + it;
+          const uint32_t stage = smem_base + it * S::STAGE_BYTES;
+          ptx::mbar_arrive_expect_tx(bar_full(it), stage_tx);
+          ptx::tma_load_2d(stage + S::OFF_CODES, &codes_map, n0 * WORDS / 2, st * GV_KBS, bar_full(it));
+          ptx::tma_load_2d(stage + S::OFF_QP, &qp_map, 2 * n0, st * GV_KBS * 32 / p.g, bar_full(it));
+          ptx::tma_load_2d(stage + S::OFF_X, &x_map, st * GV_KBS * 32, 0, bar_full(it));
+        }
+      }
       bool ok = true;
-      for (int st = st_beg, it = 0; st < st_end && ok && it < p.stop_after_stages; ++st, ++it) {
-        const int s = it % GV_STAGES;
-        if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / GV_STAGES) & 1) ^ 1, abort_flag, p.wait_limit_ns))) break;
+      int s = 0;
+      uint32_t ph = 0;                              // phase of bar_empty(s) the refill of slot s waits for
+      for (int it = first; it < n_issue && ok; ++it) {
+        const int st = st_beg + it;
+        if (!(ok = ptx::mbar_wait(bar_empty(s), ph, abort_flag, p.wait_limit_ns))) break;
         const uint32_t stage = smem_base + s * S::STAGE_BYTES;
-        // three tiled copies per stage: 4 k-block rows of pack units, the rows of
-        // (alpha, beta) they need (128 / g of them) and the x slice
-        const int qrows = (GV_KBS * 32) / p.g;
-        ptx::mbar_arrive_expect_tx(bar_full(s), GV_KBS * S::CODE_ROW + qrows * S::QP_ROW + S::X_BYTES);
+        ptx::mbar_arrive_expect_tx(bar_full(s), stage_tx);
         ptx::tma_load_2d(stage + S::OFF_CODES, &codes_map, n0 * WORDS / 2, st * GV_KBS, bar_full(s));
         ptx::tma_load_2d(stage + S::OFF_QP, &qp_map, 2 * n0, st * GV_KBS * 32 / p.g, bar_full(s));
         ptx::tma_load_2d(stage + S::OFF_X, &x_map, st * GV_KBS * 32, 0, bar_full(s));
+        if (++s == GV_STAGES) { s = 0; ph ^= 1; }
       }
     }
   } else {
     // ----------------------------------------------------------- consumers ----
     // Warp w of set s owns columns 32 (w % 4) .. + 31 and the k-blocks b of each stage
-    // with b % GV_SETS == s.  The weights are the A operand (16 columns x 16 channels per
+    // with b / 2 == s.  The weights are the A operand (16 columns x 16 channels per
     // MMA) and the tokens the B operand (8 token columns), so that a lane's fragments of x
     // are the register pairs its 16-byte load delivered and the code fragments are built
     // in place.  Every k-block is folded on its own (the fold is linear, so the k-blocks
     // of one quantization group may be folded separately with the same alpha and beta).
-    // The MMAs of a k-block start from C = -128 xp, which takes the offset of the raw
-    // codes out again: D = sum c x, and acc += alpha * D + beta * xp.
     const int set = warp / 4, wcol = (warp % 4) * 32;
     const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block of the stage -> its (alpha, beta) row
     const int gq = lane / 4, t = lane % 4;        // fragment row (column of W, token), quad lane
+
     // per-thread byte offsets inside a stage; everything else is a compile-time constant
     const uint32_t x_off = S::OFF_X + gq * (GV_KBS * 64) + t * 16 + set * (GV_KBS / GV_SETS) * 64;
     const uint32_t lo_word = BITS == 4 ? t : (t >> 1);
     const uint32_t lo_shift = BITS == 4 ? 0 : 8 * (t & 1);
     const uint32_t c_off = S::OFF_CODES + set * (GV_KBS / GV_SETS) * S::CODE_ROW + ((wcol + gq) * WORDS + lo_word) * 4;
     const uint32_t h_off = S::OFF_CODES + set * (GV_KBS / GV_SETS) * S::CODE_ROW + ((wcol + gq) * WORDS + 2) * 4;   // 3-bit codes: third-bit word
+    // 4-bit codes: ldmatrix row address of this lane (matrix lane / 8 = 8-column group, row lane % 8:
+    // the unit of column wcol + lane); thread (gq, t) then holds word t of the units of columns
+    // wcol + gq, + 8, + 16, + 24
+    const uint32_t m_off = S::OFF_CODES + set * (GV_KBS / GV_SETS) * S::CODE_ROW + (wcol + lane) * 16;
     const uint32_t q_off = S::OFF_QP + (wcol + gq) * 8;
     float acc[2][NTS][4];                         // [16-column group][token set][(col gq | gq + 8) x (token 2t | 2t + 1)]
-    const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c = 0; c < 2; ++c)
 #pragma unroll
       for (int ts = 0; ts < NTS; ++ts)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[c][ts][i] = 0.f;
+    const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
     const FragConsts fk = frag_consts<BITS>();
     constexpr uint32_t ONES = 0x3f803f80u;        // bf16x2 (1, 1)
     const uint32_t ones4[4] = {ONES, ONES, ONES, ONES};
     bool ok = true;
-    for (int st = st_beg, it = 0; st < st_end && ok; ++st, ++it) {
-      const int s = it % GV_STAGES;
-      if (!(ok = ptx::mbar_wait(bar_full(s), (it / GV_STAGES) & 1, abort_flag, p.wait_limit_ns))) break;
+    int s = 0;
+    uint32_t ph = 0;
+    for (int it = 0; it < n_stages && ok; ++it) {
+      if (!(ok = ptx::mbar_wait(bar_full(s), ph, abort_flag, p.wait_limit_ns))) break;
       const uint8_t* stage = smem + s * S::STAGE_BYTES;
+      // words of the codes of a k-block: w[2 cg + j] = this lane's word of column wcol + 16 cg + 8 j + gq
+      auto load_words = [&](int bb, uint32_t* w, uint32_t* hi) {
+        if constexpr (BITS == 4) {
+          const uint32_t addr = smem_base + s * S::STAGE_BYTES + m_off + bb * S::CODE_ROW;
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+          hi[0] = hi[1] = hi[2] = hi[3] = 0u;
+        } else {
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            const uint32_t coff = bb * S::CODE_ROW + (m * 8) * WORDS * 4;
+            w[m] = *reinterpret_cast<const uint32_t*>(stage + c_off + coff) >> lo_shift;
+            hi[m] = BITS == 3 ? *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t) : 0u;
+          }
+        }
+      };
       if constexpr (CHAIN) {
         // the set's two k-blocks lie in one quantization group: one accumulator chain over
         // both (four MMAs per 16 columns), one fold, one (alpha, beta) load
         uint4 xs[2][NTS];
-#pragma unroll
-        for (int bb = 0; bb < 2; ++bb) {
-#pragma unroll
-          for (int ts = 0; ts < NTS; ++ts)
-            xs[bb][ts] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + ts * 8 * (GV_KBS * 64));
-        }
-        float cinit[NTS][4], xp[NTS][2];
+        float xp[NTS][2];
 #pragma unroll
         for (int ts = 0; ts < NTS; ++ts) {
-          mma16816(cinit[ts], ones4, xs[0][ts].x, xs[0][ts].y, zero4);
-          mma16816(cinit[ts], ones4, xs[0][ts].z, xs[0][ts].w, cinit[ts]);
-          mma16816(cinit[ts], ones4, xs[1][ts].x, xs[1][ts].y, cinit[ts]);
-          mma16816(cinit[ts], ones4, xs[1][ts].z, xs[1][ts].w, cinit[ts]);
-          xp[ts][0] = cinit[ts][0];
-          xp[ts][1] = cinit[ts][1];
+#pragma unroll
+          for (int bb = 0; bb < 2; ++bb)
+            xs[bb][ts] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + ts * 8 * (GV_KBS * 64));
+          // xp of the tokens over both k-blocks (ones as the A operand: every row of the product holds the sums)
+          float pool[4];
+          mma16816(pool, ones4, xs[0][ts].x, xs[0][ts].y, zero4);
+          mma16816(pool, ones4, xs[0][ts].z, xs[0][ts].w, pool);
+          mma16816(pool, ones4, xs[1][ts].x, xs[1][ts].y, pool);
+          mma16816(pool, ones4, xs[1][ts].z, xs[1][ts].w, pool);
+          xp[ts][0] = pool[0];
+          xp[ts][1] = pool[1];
         }
+        uint32_t w[2][4], hi[2][4];
+        load_words(0, w[0], hi[0]);
+        load_words(1, w[1], hi[1]);
         const uint8_t* qrow = stage + q_off + (((set * (GV_KBS / GV_SETS)) >> qsh) * S::QP_ROW);
 #pragma unroll
         for (int cg = 0; cg < 2; ++cg) {
@@ -240,13 +309,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
           for (int bb = 0; bb < 2; ++bb) {
             uint32_t f[2][4];
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-              const uint32_t coff = bb * S::CODE_ROW + (cg * 16 + j * 8) * WORDS * 4;
-              const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + coff) >> lo_shift;
-              uint32_t hi = 0;
-              if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t);
-              code_fragments<BITS>(lo, hi, fk, f[j]);
-            }
+            for (int j = 0; j < 2; ++j) code_fragments<BITS>(w[bb][2 * cg + j], hi[bb][2 * cg + j], fk, f[j]);
             const uint32_t a0[4] = {f[0][0], f[1][0], f[0][1], f[1][1]};
             const uint32_t a1[4] = {f[0][2], f[1][2], f[0][3], f[1][3]};
 #pragma unroll
@@ -269,56 +332,55 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         }
       } else {
 #pragma unroll
-      for (int bb = 0; bb < GV_KBS / GV_SETS; ++bb) {
-        // this set's k-block b = 2 set + bb; B fragments: x[token gq (+ 8)][32 b + 8 t .. + 7]:
-        // the lane's k slots (2t, 2t+1 | 2t+8, 2t+9) of MMA 0 are channels 8t .. 8t+3, those of MMA 1 8t+4 .. 8t+7
-        uint4 xs[NTS];
-#pragma unroll
-        for (int ts = 0; ts < NTS; ++ts)
-          xs[ts] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + ts * 8 * (GV_KBS * 64));
-        // xp of the tokens (ones as the A operand: every row of the product holds the sums), then C = -128 xp
-        float cinit[NTS][4], xp[NTS][2];
-#pragma unroll
-        for (int ts = 0; ts < NTS; ++ts) {
-          mma16816(cinit[ts], ones4, xs[ts].x, xs[ts].y, zero4);
-          mma16816(cinit[ts], ones4, xs[ts].z, xs[ts].w, cinit[ts]);
-          xp[ts][0] = cinit[ts][0];
-          xp[ts][1] = cinit[ts][1];
-        }
-        const uint8_t* qrow = stage + q_off + (((set * (GV_KBS / GV_SETS) + bb) >> qsh) * S::QP_ROW);
-#pragma unroll
-        for (int cg = 0; cg < 2; ++cg) {
-          // columns wcol + 16 cg + gq (fragment rows 0..7) and + 8 (rows 8..15)
-          uint32_t f[2][4];
-          float2 q[2];
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const uint32_t coff = bb * S::CODE_ROW + (cg * 16 + j * 8) * WORDS * 4;
-            const uint32_t lo = *reinterpret_cast<const uint32_t*>(stage + c_off + coff) >> lo_shift;
-            uint32_t hi = 0;
-            if (BITS == 3) hi = *reinterpret_cast<const uint32_t*>(stage + h_off + coff) >> (4 * t);
-            code_fragments<BITS>(lo, hi, fk, f[j]);
-            q[j] = *reinterpret_cast<const float2*>(qrow + (cg * 16 + j * 8) * 8);
-            q[j].y = fmaf(-128.f, q[j].x, q[j].y);    // D holds sum (128 + c) x: the offset goes into the xp term
-          }
-          const uint32_t a0[4] = {f[0][0], f[1][0], f[0][1], f[1][1]};
-          const uint32_t a1[4] = {f[0][2], f[1][2], f[0][3], f[1][3]};
+        for (int bb = 0; bb < GV_KBS / GV_SETS; ++bb) {
+          // this set's k-block b = 2 set + bb; B fragments: x[token gq (+ 8)][32 b + 8 t .. + 7]:
+          // the lane's k slots (2t, 2t+1 | 2t+8, 2t+9) of MMA 0 are channels 8t .. 8t+3, those of MMA 1 8t+4 .. 8t+7
+          uint4 xs[NTS];
+          float xp[NTS][2];
 #pragma unroll
           for (int ts = 0; ts < NTS; ++ts) {
-            float D[4];
-            mma16816(D, a0, xs[ts].x, xs[ts].y, zero4);
-            mma16816(D, a1, xs[ts].z, xs[ts].w, D);
-            acc[cg][ts][0] = fmaf(q[0].x, D[0], fmaf(q[0].y, xp[ts][0], acc[cg][ts][0]));
-            acc[cg][ts][1] = fmaf(q[0].x, D[1], fmaf(q[0].y, xp[ts][1], acc[cg][ts][1]));
-            acc[cg][ts][2] = fmaf(q[1].x, D[2], fmaf(q[1].y, xp[ts][0], acc[cg][ts][2]));
-            acc[cg][ts][3] = fmaf(q[1].x, D[3], fmaf(q[1].y, xp[ts][1], acc[cg][ts][3]));
+            xs[ts] = *reinterpret_cast<const uint4*>(stage + x_off + bb * 64 + ts * 8 * (GV_KBS * 64));
+            // xp of the tokens (ones as the A operand: every row of the product holds the sums)
+            float pool[4];
+            mma16816(pool, ones4, xs[ts].x, xs[ts].y, zero4);
+            mma16816(pool, ones4, xs[ts].z, xs[ts].w, pool);
+            xp[ts][0] = pool[0];
+            xp[ts][1] = pool[1];
+          }
+          uint32_t w[4], hi[4];
+          load_words(bb, w, hi);
+          const uint8_t* qrow = stage + q_off + (((set * (GV_KBS / GV_SETS) + bb) >> qsh) * S::QP_ROW);
+#pragma unroll
+          for (int cg = 0; cg < 2; ++cg) {
+            // columns wcol + 16 cg + gq (fragment rows 0..7) and + 8 (rows 8..15)
+            uint32_t f[2][4];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) code_fragments<BITS>(w[2 * cg + j], hi[2 * cg + j], fk, f[j]);
+            float2 q0 = *reinterpret_cast<const float2*>(qrow + (cg * 16) * 8);
+            float2 q1 = *reinterpret_cast<const float2*>(qrow + (cg * 16 + 8) * 8);
+            q0.y = fmaf(-128.f, q0.x, q0.y);    // D holds sum (128 + c) x: the offset goes into the xp term
+            q1.y = fmaf(-128.f, q1.x, q1.y);
+            const uint32_t a0[4] = {f[0][0], f[1][0], f[0][1], f[1][1]};
+            const uint32_t a1[4] = {f[0][2], f[1][2], f[0][3], f[1][3]};
+#pragma unroll
+            for (int ts = 0; ts < NTS; ++ts) {
+              float D[4];
+              mma16816(D, a0, xs[ts].x, xs[ts].y, zero4);
+              mma16816(D, a1, xs[ts].z, xs[ts].w, D);
+              acc[cg][ts][0] = fmaf(q0.x, D[0], fmaf(q0.y, xp[ts][0], acc[cg][ts][0]));
+              acc[cg][ts][1] = fmaf(q0.x, D[1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
+              acc[cg][ts][2] = fmaf(q1.x, D[2], fmaf(q1.y, xp[ts][0], acc[cg][ts][2]));
+              acc[cg][ts][3] = fmaf(q1.x, D[3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
+            }
           }
         }
-      }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar_empty(s));
+      if (++s == GV_STAGES) { s = 0; ph ^= 1; }
     }
+    // every consumer warp has left the ring before the partial sums overwrite it
+    ptx::named_barrier(1, GV_WARPS * 32);
     if (p.r > 0 && rank == 0) {
       // Adapter term T * B, once per column tile (by the cluster's first block), as more MMAs
       // into the same accumulators: rows = columns of B (A operand: B transposed, two 2-byte
@@ -450,15 +512,18 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
   attr[0].val.clusterDim.x = (unsigned)splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
-  // With an adapter the kernel before this one in the stream is the pooling kernel that
-  // writes T, which is read only after the last stage: let this kernel start beside it.  With
-  // more than 8 token rows the pooling kernel is larger, and beside a short main loop the
-  // overlap measured slower (4096 x 4096, 16 rows: 15.7 against 14.8 us), beside a long one
-  // faster (8192 x 22016: 56 against 63 us): there it is used from 64 Mi weights on.
+  // Programmatic stream serialization lets this kernel start before its predecessor in the
+  // stream has finished.  Without adapter (p.pdl_wait) that is always wanted: the kernel
+  // streams its first ring of weights at once and waits for the predecessor only before it
+  // touches x or y.  With an adapter the predecessor is the pooling kernel that writes T, which
+  // is read only after the last stage: the kernel starts beside it.  With more than 8 token
+  // rows the pooling kernel is larger, and beside a short main loop the overlap measured
+  // slower (4096 x 4096, 16 rows: 15.7 against 14.8 us), beside a long one faster
+  // (8192 x 22016: 56 against 63 us): there it is used from 64 Mi weights on.
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (p.Tb != nullptr && (NTS == 1 || (long long)p.K * p.N >= (64ll << 20))) ? 2 : 1;
+  cfg.numAttrs = (p.pdl_wait != 0 || (p.Tb != nullptr && (NTS == 1 || (long long)p.K * p.N >= (64ll << 20)))) ? 2 : 1;
   cudaError_t e;
   {
     MainKernelProbe probe("qalora_gemv_kernel", st);
@@ -509,9 +574,8 @@ bool gemv_supported(const Shape& sh, int64_t M) {
     // on an SM, so this kernel beats the 64-token tensor-core tile only where its grid fills
     // the SMs evenly (measured, merged layers: 15 against 20 us for a 4096 x 4096 layer whose
     // 256 blocks fill 86 % of two per SM; 116 against 88 us for 8192 x 22016, whose 172 blocks
-    // fill 58 %), and only for a layer without adapter: the tensor-core kernel folds the
-    // adapter into its MMA steps, while here T * B is summed per output at the end, which
-    // costs more than the streaming saves once there are thousands of outputs per block.
+    // fill 58 %).  Layers with and without adapter alike: the adapter term is a few more MMAs
+    // into the same accumulators.
     const int sms = device_sm_count();
     const long long blocks = (long long)(sh.N / GV_COLS) * gv_slices(sh, M);
     const long long waves = (blocks + sms - 1) / sms;
@@ -536,6 +600,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
     return QALORA_ERR_CUDA;
   GvParams p{};
   p.codes = codes; p.qparams = qparams; p.Tb = Tb; p.B = B; p.y = y;
+  p.pdl_wait = Tb == nullptr ? 1 : 0;
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;
