@@ -422,7 +422,7 @@ def run_gpu(args):
 
     # single-token forward of the merged layer: HBM-bound leg of the metric
     small = small_m_bandwidth(Q, torch, pk)
-    small_65b = mid = None
+    small_65b = mid = grouped = None
     if rank == 0:
         from paper_2309_14717_b200.synthetic import CONFIGS
         small_65b = small_m_bandwidth(Q, torch, pk, shape="cfg5_65b_up", ms=(1, 16))
@@ -430,6 +430,7 @@ def run_gpu(args):
             r_ = small_m_bandwidth(Q, torch, pk, ms=(1,), cfg=CONFIGS["cfg5_65b_up"].with_(group_size=g))
             small_65b[f"g{g}"] = {k: r_[k] for k in ("M1", "M1_merged")}
         mid = {name: mid_m_roofline(Q, torch, pk, name) for name in (SMALL_M, "cfg5_65b_up")}
+        grouped = {f"M{m}": grouped_block_bandwidth(Q, torch, pk, m) for m in (1, 16)}
 
     adamw = adapter_update_bandwidth(Q, torch, pk) if rank == 0 else None
 
@@ -460,7 +461,7 @@ def run_gpu(args):
             "e2e": {"value": flops_step / (e2e_ms / 1e3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "roofline": roofline, "small_m": small, "small_m_65b": small_65b, "mid_m": mid,
-            "adapter_update": adamw, "cpu_baseline": cpu,
+            "grouped_block": grouped, "adapter_update": adamw, "cpu_baseline": cpu,
             "inputs_sha256": {s.cfg.name: s.sha256 for s in shapes}, "inputs_match_record": inputs_match_record(shapes),
         }
         print(json.dumps(line))
@@ -625,6 +626,69 @@ def mid_m_roofline(Q, torch, pk, shape, ms=(64, 128, 256, 512)):
             del graph
     out["shape"] = shape
     out["peaks"] = {"hbm_GB/s": pk["hbm"], "bf16_burst_TFLOP/s": pk["tensor_burst"], "source": pk["source"]}
+    return out
+
+
+def grouped_block_bandwidth(Q, torch, pk, M=1):
+    """The five projections of a LLaMA-7B block that read the block's input (q, k, v: 4096 -> 4096;
+    gate, up: 4096 -> 11008; merged INT4 layers, group size 32) on M tokens: five qalora_forward
+    calls against ONE qalora_forward_group call.  CUDA-graph replay over rotating weight copies
+    (> 4 x L2 in total) as in small_m_bandwidth."""
+    from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs
+    shapes = [CONFIGS["cfg2_7b_attn"]] * 3 + [CONFIGS["cfg3_7b_up"]] * 2
+    base = {}
+    for cfg in {c.name: c for c in shapes}.values():
+        t = make_inputs(cfg.with_(tokens=M), need=("W", "x"))
+        d = Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, 0, cfg.scale)
+        codes, qparams = Q.alloc_packed(d)
+        Q.qalora_quantize(d, t["W"].cuda(), codes, qparams)
+        base[cfg.name] = (d, codes, qparams)
+    x = t["x"][:M].contiguous().cuda()                      # every projection reads the same input
+    set_bytes = sum(base[c.name][1].numel() * 4 + base[c.name][2].numel() * 4 for c in shapes)
+    ncopies = max(4, -(-5 * 126 * 2 ** 20 // set_bytes))
+    sets = []
+    for _ in range(ncopies):
+        layers = []
+        for c in shapes:
+            d, codes, qparams = base[c.name]
+            y = torch.empty((M, c.d_out), dtype=torch.bfloat16, device="cuda")
+            layers.append((d, x, codes.clone(), qparams.clone(), None, None, y))
+        sets.append(layers)
+    ws = torch.zeros(max(Q.qalora_forward_group_workspace_bytes(sets[0], M), 16), dtype=torch.uint8, device="cuda")
+    arrays = [Q.group_layers(layers) for layers in sets]
+
+    def separate(i):
+        for d, x_, c, q, _, _, y in sets[i]:
+            Q.qalora_forward(d, M, x_, c, q, None, None, y, ws)
+
+    def grouped(i):
+        Q.qalora_forward_group(arrays[i], M, ws)
+
+    nbytes = sum(fwd_bytes(M, c.d_in, c.d_out, c.groups, 0, c.bits) for c in shapes)
+    out = {"layers": [f"{c.d_in}x{c.d_out}" for c in shapes], "M": M, "bytes": nbytes}
+    side = torch.cuda.Stream()
+    for name, fn in (("separate", separate), ("grouped", grouped)):
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn(0); fn(1)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(ncopies):
+                fn(i)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 5
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (reps * ncopies)
+        out[name] = {"us_per_block": us, "GB/s": nbytes / (us * 1e-6) / 1e9, "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / pk["hbm"],
+                     "launches": 5 if name == "separate" else 1}
+        del graph
     return out
 
 

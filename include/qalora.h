@@ -114,10 +114,46 @@ int qalora_quantize(const qalora_desc* desc, const float* W, void* codes, float*
  *   x bf16 [m][K];  A bf16 [G][r];  B bf16 [r][N];  y out bf16 [m][N].
  * Products are bf16 x bf16 accumulated in float32.  Any m >= 0 is accepted; the
  * kernel is chosen from m (a bandwidth-bound path for a few rows, a
- * tensor-core path otherwise). */
+ * tensor-core path otherwise).  The few-token kernel of a layer without adapter may
+ * start while the kernel before it in the stream is still running (programmatic dependent
+ * launch): it then reads only codes and qparams early and waits for that kernel's
+ * completion before it reads x or writes y.  Codes and qparams must therefore not be
+ * outputs of a kernel that itself lets its successors start early; no kernel of this
+ * library that writes them (quantize, merge, the format conversions) does. */
 int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
                    const float* qparams, const void* A, const void* B, void* y,
                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The forward pass of SEVERAL layers in one call, for serving a merged model a few tokens at
+ * a time (Section 3.2 states efficient deployment as the method's second goal; Section 4.2:
+ * the merged model stays quantized and is therefore faster at inference).  The layers are
+ * independent: each has its own input x, e.g. the q, k and v projections or the gate and up
+ * projections of a transformer block (which read the same x), or any layers whose inputs are
+ * ready.  Layer l computes what qalora_forward computes,
+ *     y_l = x_l * W~_l  (+ s_l * (pool(x_l) * A_l) * B_l  when its rank is not 0),
+ * on the same number m of token rows.  When every layer is a plain quantized layer (rank 0),
+ * m <= 16, there are at most 8 layers, all with the same bit width, all with group size 32 or
+ * all with group size 64/128, and every shape has d_out and d_in multiples of 128, the whole
+ * group runs as ONE kernel launch (launch, cluster set-up and first-byte latency are paid once,
+ * and the layers' blocks fill the GPU together); otherwise the layers run one after the other
+ * exactly as qalora_forward would run them.  Results do not depend on which way was taken
+ * beyond the summation order of the reduction slices.
+ *   layers   : HOST array of n descriptors with DEVICE pointers (A, B ignored when rank == 0)
+ *   workspace: DEVICE scratch of qalora_forward_group_workspace_bytes() bytes; its first int32
+ *              is the status word described at qalora_workspace_bytes, for the whole group
+ * Errors are those of qalora_forward; every layer is checked before anything is launched. */
+typedef struct qalora_group_layer {
+  qalora_desc desc;
+  const void* x;          /* bf16 [m][d_in]  */
+  const void* codes;
+  const float* qparams;
+  const void* A;          /* bf16 [G][r], or NULL when rank == 0 */
+  const void* B;          /* bf16 [r][d_out], or NULL when rank == 0 */
+  void* y;                /* bf16 [m][d_out], out */
+} qalora_group_layer;
+int qalora_forward_group_workspace_bytes(const qalora_group_layer* layers, int n, int64_t m, size_t* bytes);
+int qalora_forward_group(const qalora_group_layer* layers, int n, int64_t m,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Backward pass with the base weights frozen (Section 3.1: only A and B are
  * adjusted).  With l the loss and dy = dl/dy:

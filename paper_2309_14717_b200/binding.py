@@ -23,6 +23,7 @@ EXPORTS = (
     "qalora_forward_static", "qalora_step_host_bytes", "qalora_step_host",
     "qalora_adamw_workspace_bytes", "qalora_adamw_step",
     "qalora_dequantize", "qalora_qparams_from_zero_point", "qalora_qparams_to_zero_point",
+    "qalora_forward_group_workspace_bytes", "qalora_forward_group",
 )
 
 STATIC_SCRATCH_BYTES = 1 << 20
@@ -31,6 +32,11 @@ STATIC_SCRATCH_BYTES = 1 << 20
 class QaloraDesc(Structure):
     _fields_ = [("d_in", c_int32), ("d_out", c_int32), ("group_size", c_int32), ("bits", c_int32),
                 ("rank", c_int32), ("scale", c_float)]
+
+
+class GroupLayer(Structure):
+    _fields_ = [("desc", QaloraDesc), ("x", c_void_p), ("codes", c_void_p), ("qparams", c_void_p),
+                ("A", c_void_p), ("B", c_void_p), ("y", c_void_p)]
 
 
 class AdamwHyper(Structure):
@@ -89,6 +95,10 @@ def load() -> ctypes.CDLL:
     lib.qalora_adamw_workspace_bytes.argtypes = [POINTER(c_size_t)]
     lib.qalora_adamw_step.restype = c_int
     lib.qalora_adamw_step.argtypes = [POINTER(AdamwHyper), c_int64] + [c_void_p] * 6 + [c_void_p, c_size_t, c_void_p]
+    lib.qalora_forward_group_workspace_bytes.restype = c_int
+    lib.qalora_forward_group_workspace_bytes.argtypes = [POINTER(GroupLayer), c_int, c_int64, POINTER(c_size_t)]
+    lib.qalora_forward_group.restype = c_int
+    lib.qalora_forward_group.argtypes = [POINTER(GroupLayer), c_int, c_int64, c_void_p, c_size_t, c_void_p]
     lib.qalora_kernel_launches.restype = ctypes.c_uint64
     lib.qalora_kernel_launches.argtypes = []
     lib.qalora_profile_next_main_kernel.restype = c_int
@@ -182,6 +192,30 @@ def qalora_forward_static(d: QaloraDesc, m: int, x, codes, qparams, A, B, y, str
     Calls that overlap on the GPU share the array and must be serialized."""
     _check("qalora_forward_static", load().qalora_forward_static(byref(d), m, _ptr(x), _ptr(codes), _ptr(qparams),
                                                                  _ptr(A), _ptr(B), _ptr(y), _stream(stream)))
+
+
+def group_layers(layers):
+    """ctypes array for qalora_forward_group from (desc, x, codes, qparams, A, B, y) tuples of tensors."""
+    arr = (GroupLayer * len(layers))()
+    for i, (d, x, codes, qparams, A, B, y) in enumerate(layers):
+        ptr = lambda t: _ptr(t).value if t is not None else None
+        arr[i] = GroupLayer(d, ptr(x), ptr(codes), ptr(qparams), ptr(A), ptr(B), ptr(y))
+    return arr
+
+
+def qalora_forward_group_workspace_bytes(layers, m: int) -> int:
+    arr = layers if isinstance(layers, ctypes.Array) else group_layers(layers)
+    b = c_size_t()
+    _check("qalora_forward_group_workspace_bytes", load().qalora_forward_group_workspace_bytes(arr, len(arr), m, byref(b)))
+    return b.value
+
+
+def qalora_forward_group(layers, m: int, workspace, stream=None):
+    """Forward of several independent layers ((desc, x, codes, qparams, A, B, y) tuples, or the
+    array group_layers() made of them) on m rows each; one launch when the layers allow it."""
+    arr = layers if isinstance(layers, ctypes.Array) else group_layers(layers)
+    _check("qalora_forward_group", load().qalora_forward_group(arr, len(arr), m, _ptr(workspace), workspace.numel(),
+                                                               _stream(stream)))
 
 
 def qalora_step_host_bytes(d: QaloraDesc, m: int) -> int:

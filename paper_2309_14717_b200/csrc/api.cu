@@ -316,6 +316,62 @@ int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void
   return forward_launch(desc, m, x, codes, qparams, A, B, y, workspace, cuda_stream, /*reset_status=*/true);
 }
 
+int qalora_forward_group_workspace_bytes(const qalora_group_layer* layers, int n, int64_t m, size_t* bytes) {
+  if (layers == nullptr || bytes == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (n < 0 || m < 0) return QALORA_ERR_INVALID_ARG;
+  size_t need = 256;                                 // the status word
+  for (int i = 0; i < n; ++i) {
+    Shape sh;
+    int st = check_desc(&layers[i].desc, &sh);
+    if (st != QALORA_OK) return st;
+    const size_t w = workspace_layout(sh, m, QALORA_OP_FORWARD).total;
+    need = w > need ? w : need;
+  }
+  *bytes = need;
+  return QALORA_OK;
+}
+
+int qalora_forward_group(const qalora_group_layer* layers, int n, int64_t m,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (layers == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (n < 0 || m < 0) return QALORA_ERR_INVALID_ARG;
+  size_t need = 0;
+  int st = qalora_forward_group_workspace_bytes(layers, n, m, &need);
+  if (st != QALORA_OK) return st;
+  // every layer's arguments are checked before anything is launched
+  for (int i = 0; i < n; ++i) {
+    const qalora_group_layer& L = layers[i];
+    st = forward_validate(&L.desc, m, L.x, L.codes, L.qparams, L.A, L.B, L.y, workspace, workspace_bytes);
+    if (st != QALORA_OK) return st;
+  }
+  if (n == 0 || m == 0) return QALORA_OK;
+  if (workspace == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (workspace_bytes < need) return QALORA_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  constexpr int kMaxGroup = 8;
+  GemvGroupItem items[kMaxGroup];
+  bool one_launch = n <= kMaxGroup;
+  for (int i = 0; i < n && one_launch; ++i) {
+    check_desc(&layers[i].desc, &items[i].sh);
+    items[i].x = static_cast<const __nv_bfloat16*>(layers[i].x);
+    items[i].codes = static_cast<const uint32_t*>(layers[i].codes);
+    items[i].qparams = reinterpret_cast<const float2*>(layers[i].qparams);
+    items[i].y = static_cast<__nv_bfloat16*>(layers[i].y);
+  }
+  one_launch = one_launch && gemv_group_supported(items, n, m);
+  if (one_launch) return launch_gemv_group(items, n, m, static_cast<int*>(workspace), /*reset_status=*/true, stream);
+  // Otherwise (adapters, more than 16 rows, mixed bit widths, shapes the few-token kernel does
+  // not tile, more than 8 layers): one forward pass per layer, sharing the workspace; the status
+  // word is cleared once and only ever raised.
+  if ((st = cuda_status(cudaMemsetAsync(workspace, 0, sizeof(int), stream))) != QALORA_OK) return st;
+  for (int i = 0; i < n; ++i) {
+    const qalora_group_layer& L = layers[i];
+    st = forward_launch(&L.desc, m, L.x, L.codes, L.qparams, L.A, L.B, L.y, workspace, cuda_stream, /*reset_status=*/false);
+    if (st != QALORA_OK) return st;
+  }
+  return QALORA_OK;
+}
+
 int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
                     const void* codes, const float* qparams, const void* A, const void* B,
                     void* dx, float* dA, float* dB,

@@ -128,6 +128,17 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
 
 void arm_few_token_wait_expiry(int stages, unsigned long long limit_ns);   // test hook, one-shot
 
+// Several layers without adapter, the same M <= 16 rows each, in ONE few-token launch.
+struct GemvGroupItem {
+  Shape sh;
+  const __nv_bfloat16* x;
+  const uint32_t* codes;
+  const float2* qparams;
+  __nv_bfloat16* y;
+};
+bool gemv_group_supported(const GemvGroupItem* items, int n, int64_t M);
+int launch_gemv_group(const GemvGroupItem* items, int n, int64_t M, int* status, bool reset_status, cudaStream_t st);
+
 // out[i] = sum over splits of partial[z][i], added in a fixed order.
 int launch_sum_partials(const float* partial, float* out, size_t count, int splits, cudaStream_t st);
 

@@ -136,10 +136,11 @@ __device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, const F
 
 // NTS: sets of 8 token rows in use (M <= 8 NTS).  CHAIN: the group size is 64 or 128, so the two
 // k-blocks a warp set takes from a stage share (alpha, beta) and are folded together.
+// The work of one block: `block` is its index among the blocks of the layer described by p
+// (a layer's blocks are consecutive in the grid, a whole number of clusters).
 template <int BITS, int NTS, bool CHAIN>
-__global__ void __launch_bounds__(GV_THREADS, NTS == 4 ? 2 : 3)
-qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
-                   const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
+__device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUtensorMap& codes_map,
+                                           const CUtensorMap& qp_map, const GvParams& p, const int block) {
   using S = GvSmem<BITS, NTS>;
   constexpr int WORDS = S::WORDS;
   constexpr int GV_STAGES = S::STAGES;
@@ -155,7 +156,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
   cg::cluster_group cluster = cg::this_cluster();
   const int splits = (int)cluster.num_blocks();
   const int rank = (int)cluster.block_rank();
-  const int n0 = (blockIdx.x / splits) * GV_COLS;
+  const int n0 = (block / splits) * GV_COLS;
   const int st_beg = (int)((long long)p.total_stages * rank / splits);
   const int st_end = (int)((long long)p.total_stages * (rank + 1) / splits);
   const int n_stages = st_end - st_beg;
@@ -171,7 +172,7 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     ptx::prefetch_tensormap(&x_map);
     ptx::prefetch_tensormap(&codes_map);
     ptx::prefetch_tensormap(&qp_map);
-    if (blockIdx.x == 0 && p.reset_status) *p.status = 0;     // a wait gives up only after seconds: no block can have raised it yet
+    if (block == 0 && p.reset_status) *p.status = 0;     // a wait gives up only after seconds: no block can have raised it yet
     // the next kernel in the stream may start (it waits for this one's completion before it
     // reads or writes anything this one touches)
     asm volatile("griddepcontrol.launch_dependents;");
@@ -454,6 +455,33 @@ qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
   if (threadIdx.x == 0 && *abort_flag != 0) atomicExch(p.status, 1);
 }
 
+template <int BITS, int NTS, bool CHAIN>
+__global__ void __launch_bounds__(GV_THREADS, NTS == 4 ? 2 : 3)
+qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
+                   const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
+  gemv_block<BITS, NTS, CHAIN>(x_map, codes_map, qp_map, p, (int)blockIdx.x);
+}
+
+// Several layers in ONE launch (the projections of a transformer block that read finished
+// inputs: q, k, v; gate, up; or any set of independent layers): block b works for the layer l
+// with first_block[l] <= b < first_block[l + 1].  Launch, cluster set-up and the first bytes'
+// latency are paid once for all of them.
+constexpr int GV_GROUP_MAX = 8;
+struct GvGroup {
+  CUtensorMap x_map[GV_GROUP_MAX], codes_map[GV_GROUP_MAX], qp_map[GV_GROUP_MAX];
+  GvParams p[GV_GROUP_MAX];
+  int first_block[GV_GROUP_MAX + 1];
+  int n;
+};
+
+template <int BITS, int NTS, bool CHAIN>
+__global__ void __launch_bounds__(GV_THREADS, NTS == 4 ? 2 : 3)
+qalora_gemv_group_kernel(const __grid_constant__ GvGroup grp) {
+  int l = 0;
+  while (l + 1 < grp.n && (int)blockIdx.x >= grp.first_block[l + 1]) ++l;      // the same for every thread of a cluster
+  gemv_block<BITS, NTS, CHAIN>(grp.x_map[l], grp.codes_map[l], grp.qp_map[l], grp.p[l], (int)blockIdx.x - grp.first_block[l]);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -471,66 +499,101 @@ EncodeTiledFn gv_encode_fn() {
   return fn;
 }
 
-template <int BITS, int NTS, bool CHAIN>
-int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
+// Tensor maps of a layer's weights: packed codes [K/32][N][words] uint32 seen as a 2-D matrix of
+// 8-byte elements, so that one box row is the whole contiguous run of 128 pack units (2 KiB at
+// 4 bits), and (alpha, beta) float32 [G][2N] with a box of 256 floats x (128 / g) rows.
+bool make_weight_maps(const GvParams& p, int words, CUtensorMap* cm, CUtensorMap* qm) {
   EncodeTiledFn fn = gv_encode_fn();
-  CUtensorMap cm, qm;
-  {
-    // packed codes [K/32][N][words] uint32 seen as a 2-D matrix of 8-byte elements, so that
-    // one box row is the whole contiguous run of 128 pack units (2 KiB at 4 bits)
-    constexpr int W = GvSmem<BITS, NTS>::WORDS;
-    cuuint64_t dims[2] = {(cuuint64_t)p.N * W / 2, (cuuint64_t)(p.K / 32)};
-    cuuint64_t strides[1] = {(cuuint64_t)p.N * W * 4};
-    cuuint32_t box[2] = {(cuuint32_t)(GV_COLS * W / 2), GV_KBS};
-    cuuint32_t estr[2] = {1, 1};
-    if (fn(&cm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<uint32_t*>(p.codes), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return QALORA_ERR_CUDA;
-    // (alpha, beta) float32 [G][2N]; box = 256 floats x (128 / g) rows
-    cuuint64_t qdims[2] = {(cuuint64_t)p.N * 2, (cuuint64_t)(p.K / p.g)};
-    cuuint64_t qstrides[1] = {(cuuint64_t)p.N * 8};
-    cuuint32_t qbox[2] = {2 * GV_COLS, (cuuint32_t)((GV_KBS * 32) / p.g)};
-    cuuint32_t qestr[2] = {1, 1};
-    if (fn(&qm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float2*>(p.qparams), qdims, qstrides, qbox, qestr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return QALORA_ERR_CUDA;
-  }
-  using S = GvSmem<BITS, NTS>;
-  auto kern = qalora_gemv_kernel<BITS, NTS, CHAIN>;
-  static PerDeviceOnce smem_limit;      // this instantiation's shared-memory limit, raised once on every device it runs on
-  if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
-    return QALORA_ERR_CUDA;
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)p.N * words / 2, (cuuint64_t)(p.K / 32)};
+  cuuint64_t strides[1] = {(cuuint64_t)p.N * words * 4};
+  cuuint32_t box[2] = {(cuuint32_t)(GV_COLS * words / 2), GV_KBS};
+  cuuint32_t estr[2] = {1, 1};
+  if (fn(cm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<uint32_t*>(p.codes), dims, strides, box, estr,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  cuuint64_t qdims[2] = {(cuuint64_t)p.N * 2, (cuuint64_t)(p.K / p.g)};
+  cuuint64_t qstrides[1] = {(cuuint64_t)p.N * 8};
+  cuuint32_t qbox[2] = {2 * GV_COLS, (cuuint32_t)((GV_KBS * 32) / p.g)};
+  cuuint32_t qestr[2] = {1, 1};
+  return fn(qm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float2*>(p.qparams), qdims, qstrides, qbox, qestr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// x bf16 [M][K]; box = 128 channels x the token rows the kernel keeps (8, 16 or 32; rows beyond M read as zero)
+bool make_x_map(const __nv_bfloat16* x, int K, int64_t M, CUtensorMap* xm) {
+  EncodeTiledFn fn = gv_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {GV_KBS * 32, (cuuint32_t)(M > 16 ? 32 : (M > 8 ? 16 : 8))};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(xm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Launch configuration shared by the single-layer and the grouped kernel: `blocks` blocks in
+// clusters of `splits`; with `programmatic` the launch carries programmatic stream serialization.
+template <class Kernel, class... Args>
+cudaError_t launch_clustered(Kernel kern, unsigned blocks, int splits, size_t smem, bool programmatic, cudaStream_t st,
+                             const char* probe_name, const Args&... args) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((p.N / GV_COLS) * splits));
+  cfg.gridDim = dim3(blocks);
   cfg.blockDim = dim3(GV_THREADS);
-  cfg.dynamicSmemBytes = S::TOTAL;
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = programmatic ? 2 : 1;
+  cudaError_t e;
+  {
+    MainKernelProbe probe(probe_name, st);
+    e = cudaLaunchKernelEx(&cfg, kern, args...);
+  }
+  count_launch();
+  return e;
+}
+
+template <int BITS, int NTS, bool CHAIN>
+int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
+  using S = GvSmem<BITS, NTS>;
+  CUtensorMap cm, qm;
+  if (!make_weight_maps(p, S::WORDS, &cm, &qm)) return QALORA_ERR_CUDA;
+  auto kern = qalora_gemv_kernel<BITS, NTS, CHAIN>;
+  static PerDeviceOnce smem_limit;      // this instantiation's shared-memory limit, raised once on every device it runs on
+  if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
+    return QALORA_ERR_CUDA;
   // Programmatic stream serialization lets this kernel start before its predecessor in the
   // stream has finished.  Without adapter (p.pdl_wait) that is always wanted: the kernel
   // streams its first ring of weights at once and waits for the predecessor only before it
-  // touches x or y.  With an adapter the predecessor is the pooling kernel that writes T, which
+  // fetches x.  With an adapter the predecessor is the pooling kernel that writes T, which
   // is read only after the last stage: the kernel starts beside it.  With more than 8 token
   // rows the pooling kernel is larger, and beside a short main loop the overlap measured
   // slower (4096 x 4096, 16 rows: 15.7 against 14.8 us), beside a long one faster
   // (8192 x 22016: 56 against 63 us): there it is used from 64 Mi weights on.
-  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = (p.pdl_wait != 0 || (p.Tb != nullptr && (NTS == 1 || (long long)p.K * p.N >= (64ll << 20)))) ? 2 : 1;
-  cudaError_t e;
-  {
-    MainKernelProbe probe("qalora_gemv_kernel", st);
-    e = cudaLaunchKernelEx(&cfg, kern, xm, cm, qm, p);
-  }
-  count_launch();
-  return cuda_status(e);
+  const bool programmatic = p.pdl_wait != 0 || (p.Tb != nullptr && (NTS == 1 || (long long)p.K * p.N >= (64ll << 20)));
+  return cuda_status(launch_clustered(kern, (unsigned)((p.N / GV_COLS) * splits), splits, S::TOTAL, programmatic, st,
+                                      "qalora_gemv_kernel", xm, cm, qm, p));
+}
+
+template <int BITS, int NTS, bool CHAIN>
+int launch_gemv_group_t(const GvGroup& grp, int splits, cudaStream_t st) {
+  using S = GvSmem<BITS, NTS>;
+  auto kern = qalora_gemv_group_kernel<BITS, NTS, CHAIN>;
+  static PerDeviceOnce smem_limit;
+  if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
+    return QALORA_ERR_CUDA;
+  return cuda_status(launch_clustered(kern, (unsigned)grp.first_block[grp.n], splits, S::TOTAL, true, st,
+                                      "qalora_gemv_group_kernel", grp));
 }
 
 }  // namespace
@@ -588,16 +651,8 @@ bool gemv_supported(const Shape& sh, int64_t M) {
 int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
                 const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, bool reset_status,
                 cudaStream_t st) {
-  EncodeTiledFn fn = gv_encode_fn();
   CUtensorMap xm;
-  cuuint64_t dims[2] = {(cuuint64_t)sh.K, (cuuint64_t)M};
-  cuuint64_t strides[1] = {(cuuint64_t)sh.K * 2};
-  cuuint32_t box[2] = {GV_KBS * 32, (cuuint32_t)(M > 16 ? 32 : (M > 8 ? 16 : 8))};   // the token rows the kernel keeps
-  cuuint32_t estr[2] = {1, 1};
-  if (fn(&xm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(x), dims, strides, box, estr,
-         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return QALORA_ERR_CUDA;
+  if (!make_x_map(x, sh.K, M, &xm)) return QALORA_ERR_CUDA;
   GvParams p{};
   p.codes = codes; p.qparams = qparams; p.Tb = Tb; p.B = B; p.y = y;
   p.pdl_wait = Tb == nullptr ? 1 : 0;
@@ -618,6 +673,70 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   return QALORA_GV(2);
 #undef QALORA_GV
 #undef QALORA_GV_N
+}
+
+
+// Slices per column tile for a group of layers (one cluster size for the whole launch): the
+// count that brings the grid closest to two blocks per SM and that every layer can be cut into.
+static int gv_group_slices(const GemvGroupItem* items, int n) {
+  long long tiles = 0;
+  int min_stages = 1 << 30;
+  for (int i = 0; i < n; ++i) {
+    tiles += items[i].sh.N / GV_COLS;
+    const int stages = items[i].sh.K / (GV_KBS * 32);
+    min_stages = stages < min_stages ? stages : min_stages;
+  }
+  const long long target = 2ll * device_sm_count();
+  int splits = 1;
+  long long best = 1ll << 60;
+  for (int sp : {1, 2, 3, 4, 6, 8}) {
+    if (sp > min_stages) break;
+    const long long miss = tiles * sp > target ? tiles * sp - target : target - tiles * sp;
+    if (miss < best) { best = miss; splits = sp; }
+  }
+  return splits;
+}
+
+bool gemv_group_supported(const GemvGroupItem* items, int n, int64_t M) {
+  if (n < 1 || n > GV_GROUP_MAX || M < 1 || M > 16) return false;
+  for (int i = 0; i < n; ++i) {
+    const Shape& sh = items[i].sh;
+    if (sh.r != 0 || sh.bits != items[0].sh.bits || (sh.g >= 64) != (items[0].sh.g >= 64) || !gemv_supported(sh, M)) return false;
+  }
+  return true;
+}
+
+// y_l = x_l * W~_l for the layers of a group (no adapters), M <= 16 rows each, in one launch.
+int launch_gemv_group(const GemvGroupItem* items, int n, int64_t M, int* status, bool reset_status, cudaStream_t st) {
+  GvGroup grp{};
+  grp.n = n;
+  const int splits = gv_group_slices(items, n);
+  const int words = words_per_unit(items[0].sh.bits);
+  int blocks = 0;
+  for (int i = 0; i < n; ++i) {
+    const Shape& sh = items[i].sh;
+    GvParams& p = grp.p[i];
+    p.codes = items[i].codes; p.qparams = items[i].qparams; p.Tb = nullptr; p.B = nullptr; p.y = items[i].y;
+    p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = 0;
+    p.total_stages = sh.K / (GV_KBS * 32);
+    p.status = status;
+    p.reset_status = (reset_status && i == 0) ? 1 : 0;
+    p.pdl_wait = 1;
+    p.stop_after_stages = 0x7fffffff;
+    p.wait_limit_ns = ptx::WAIT_LIMIT_NS;
+    if (!make_x_map(items[i].x, sh.K, M, &grp.x_map[i]) || !make_weight_maps(p, words, &grp.codes_map[i], &grp.qp_map[i]))
+      return QALORA_ERR_CUDA;
+    grp.first_block[i] = blocks;
+    blocks += (sh.N / GV_COLS) * splits;
+  }
+  grp.first_block[n] = blocks;
+  const bool two_sets = M > 8, chain = items[0].sh.g >= 64;
+#define QALORA_GVG(BITS) (two_sets ? (chain ? launch_gemv_group_t<BITS, 2, true>(grp, splits, st) : launch_gemv_group_t<BITS, 2, false>(grp, splits, st)) \
+                                   : (chain ? launch_gemv_group_t<BITS, 1, true>(grp, splits, st) : launch_gemv_group_t<BITS, 1, false>(grp, splits, st)))
+  if (items[0].sh.bits == 4) return QALORA_GVG(4);
+  if (items[0].sh.bits == 3) return QALORA_GVG(3);
+  return QALORA_GVG(2);
+#undef QALORA_GVG
 }
 
 }  // namespace qalora

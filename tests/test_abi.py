@@ -107,6 +107,31 @@ def test_static_scratch_forward_checks_its_arguments_before_anything_else():
     assert lib.qalora_forward_static(r(d), 0, None, None, None, None, None, None, None) == 0
 
 
+def test_forward_group_argument_checks_need_no_gpu():
+    lib = Q.load()
+    buf = ctypes.create_string_buffer(64)          # host memory: must never be dereferenced
+    a16 = (ctypes.addressof(buf) + 15) // 16 * 16
+    good = Q.GroupLayer(Q.desc(512, 512, 32, 4, 0, 1.0), a16, a16, a16, None, None, a16)
+    bad_desc = Q.GroupLayer(Q.desc(512, 512, 48, 4, 0, 1.0), a16, a16, a16, None, None, a16)
+    no_x = Q.GroupLayer(Q.desc(512, 512, 32, 4, 0, 1.0), None, a16, a16, None, None, a16)
+    need_ab = Q.GroupLayer(Q.desc(512, 512, 32, 4, 16, 1.0), a16, a16, a16, None, None, a16)
+    arr = lambda *ls: (Q.GroupLayer * len(ls))(*ls)
+    size = ctypes.c_size_t()
+    assert lib.qalora_forward_group_workspace_bytes(arr(good, good), 2, 4, ctypes.byref(size)) == 0 and size.value >= 256
+    assert lib.qalora_forward_group_workspace_bytes(arr(good, bad_desc), 2, 4, ctypes.byref(size)) == -3
+    assert lib.qalora_forward_group_workspace_bytes(None, 2, 4, ctypes.byref(size)) == -2
+    ws = ctypes.c_void_p(a16)
+    assert lib.qalora_forward_group(None, 1, 4, ws, 1 << 20, None) == -2
+    assert lib.qalora_forward_group(arr(good), -1, 4, ws, 1 << 20, None) == -1
+    assert lib.qalora_forward_group(arr(good, bad_desc), 2, 4, ws, 1 << 20, None) == -3
+    assert lib.qalora_forward_group(arr(good, no_x), 2, 4, ws, 1 << 20, None) == -2       # the second layer spoils the call
+    assert lib.qalora_forward_group(arr(good, need_ab), 2, 4, ws, 1 << 20, None) == -2
+    assert lib.qalora_forward_group(arr(good), 1, 4, ws, 8, None) == -5
+    assert lib.qalora_forward_group(arr(good), 1, 4, ctypes.c_void_p(a16 + 4), 1 << 20, None) == -4
+    assert lib.qalora_forward_group(arr(good), 0, 4, ws, 1 << 20, None) == 0
+    assert lib.qalora_forward_group(arr(good), 1, 0, ws, 1 << 20, None) == 0
+
+
 def test_adamw_argument_checks_need_no_gpu():
     lib = Q.load()
     p = ctypes.c_void_p
