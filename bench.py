@@ -268,7 +268,7 @@ class ShapeState:
         self.y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
         self.dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
         self.ws_f = Q.alloc_workspace(self.d, M, Q.OP_FORWARD)
-        self.ws_b = Q.alloc_workspace(self.d, M, Q.OP_BACKWARD)
+        self.ws_t = Q.alloc_workspace(self.d, M, Q.OP_TRAIN)          # forward + backward of a step share it
         self.x1 = self.x[:1].contiguous()
         self.y1 = torch.empty((1, N), dtype=torch.bfloat16, device="cuda")
         self.ws1 = Q.alloc_workspace(self.d0, 1, Q.OP_FORWARD)
@@ -319,8 +319,8 @@ def run_gpu(args):
         Q.qalora_quantize(s.d, s.W, s.codes, s.qparams)
         if probe is not None:                      # events around the forward contraction kernel of this call
             Q.qalora_profile_next_main_kernel(*probe)
-        Q.qalora_forward(s.d, s.cfg.tokens, s.x, s.codes, s.qparams, A, B, s.y, s.ws_f)
-        Q.qalora_backward(s.d, s.cfg.tokens, s.x, s.dy, s.codes, s.qparams, A, B, s.dx, dA, dB, s.ws_b)
+        Q.qalora_forward_train(s.d, s.cfg.tokens, s.x, s.codes, s.qparams, A, B, s.y, s.ws_t)
+        Q.qalora_backward_train(s.d, s.cfg.tokens, s.x, s.dy, s.codes, s.qparams, A, B, s.dx, dA, dB, s.ws_t)
 
     def deploy_step(i, s):
         A, B = bucket.factors(i)

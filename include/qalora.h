@@ -75,7 +75,8 @@ typedef struct qalora_desc {
   float   scale;       /* s */
 } qalora_desc;
 
-typedef enum qalora_op { QALORA_OP_FORWARD = 0, QALORA_OP_BACKWARD = 1 } qalora_op;
+/* QALORA_OP_TRAIN: one workspace shared by qalora_forward_train and qalora_backward_train. */
+typedef enum qalora_op { QALORA_OP_FORWARD = 0, QALORA_OP_BACKWARD = 1, QALORA_OP_TRAIN = 2 } qalora_op;
 
 /* Library version * 100 + QALORA_LAYOUT_VERSION. */
 int qalora_version(void);
@@ -166,6 +167,23 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
                     const void* codes, const float* qparams, const void* A, const void* B,
                     void* dx, float* dA, float* dB,
                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The same two passes for a fine-tuning step, sharing one workspace of
+ * qalora_workspace_bytes(desc, m, QALORA_OP_TRAIN) bytes (Algorithm 1's forward and its
+ * gradients; Section 3.1).  The pooled input pool(x) and T = s * pool(x) * A are needed by
+ * both passes: qalora_forward_train computes them once and leaves them in the workspace,
+ * qalora_backward_train takes them from there instead of streaming x a second time.  The
+ * caller must pass the SAME workspace, desc, m, x and A to both and must not write to the
+ * workspace in between.  Results are identical to qalora_forward / qalora_backward.  The
+ * status word is cleared by qalora_forward_train only, so that after the pair it tells
+ * whether either pass gave up a wait.  rank must be > 0. */
+int qalora_forward_train(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
+                         const float* qparams, const void* A, const void* B, void* y,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+int qalora_backward_train(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
+                          const void* codes, const float* qparams, const void* A, const void* B,
+                          void* dx, float* dA, float* dB,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Merge for deployment (Algorithm 1, merge_with_quantization; Appendix B
  * Eq. 7): folds s*A*B into the zero factors, after which the plain quantized
@@ -267,9 +285,14 @@ int qalora_adamw_step(const qalora_adamw_hyper* hyper, int64_t n, const float* g
  * library's device image.  It calls no cudaMalloc/cudaFree and no allocating
  * routine.
  *   - Limit: qalora_workspace_bytes(desc, m, QALORA_OP_FORWARD) must not exceed
- *     QALORA_STATIC_SCRATCH_BYTES (about m * rank * 6 bytes + 1 KiB; e.g. 2048
- *     tokens at rank 64).  Larger requests return
- *     QALORA_ERR_STATIC_SCRATCH_EXCEEDED and launch nothing.
+ *     QALORA_STATIC_SCRATCH_BYTES.  That is about m * rank * 6 bytes + 1 KiB where the
+ *     few-token kernel runs (m <= 16; m <= 32 on layers whose grid fills the GPU evenly)
+ *     and for m > 512, e.g. 2048 tokens at rank 64.  For 17 <= m <= 512 on the tensor-core
+ *     path the forward pass also keeps float32 partial results of its reduction, several
+ *     times m * d_out * 4 bytes, which is beyond 1 MiB on LLaMA-sized layers (d_out = 4096:
+ *     m = 64 needs 4 MiB).  Larger requests return QALORA_ERR_STATIC_SCRATCH_EXCEEDED;
+ *     a call that is rejected, for this or any reason qalora_forward would reject it for,
+ *     launches nothing and does not touch the CUDA runtime.
  *   - Cost: every GPU on which the library's device code is loaded holds the
  *     array until the process exits, whether or not this function is used.
  *   - The first call on each device looks up the array's device address (with

@@ -14,7 +14,7 @@ import torch
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqalora.so")
 
-OP_FORWARD, OP_BACKWARD = 0, 1
+OP_FORWARD, OP_BACKWARD, OP_TRAIN = 0, 1, 2
 
 EXPORTS = (
     "qalora_version", "qalora_status_string", "qalora_packed_bytes", "qalora_workspace_bytes",
@@ -24,6 +24,7 @@ EXPORTS = (
     "qalora_adamw_workspace_bytes", "qalora_adamw_step",
     "qalora_dequantize", "qalora_qparams_from_zero_point", "qalora_qparams_to_zero_point",
     "qalora_forward_group_workspace_bytes", "qalora_forward_group",
+    "qalora_forward_train", "qalora_backward_train",
 )
 
 STATIC_SCRATCH_BYTES = 1 << 20
@@ -77,6 +78,10 @@ def load() -> ctypes.CDLL:
     lib.qalora_forward.argtypes = [D, c_int64] + [c_void_p] * 6 + [c_void_p, c_size_t, c_void_p]
     lib.qalora_backward.restype = c_int
     lib.qalora_backward.argtypes = [D, c_int64] + [c_void_p] * 9 + [c_void_p, c_size_t, c_void_p]
+    lib.qalora_forward_train.restype = c_int
+    lib.qalora_forward_train.argtypes = lib.qalora_forward.argtypes
+    lib.qalora_backward_train.restype = c_int
+    lib.qalora_backward_train.argtypes = lib.qalora_backward.argtypes
     lib.qalora_merge.restype = c_int
     lib.qalora_merge.argtypes = [D, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.qalora_forward_static.restype = c_int
@@ -246,6 +251,23 @@ def qalora_backward(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, 
                                                      _ptr(workspace),
                                                      workspace.numel() if workspace is not None else 0,
                                                      _stream(stream)))
+
+
+def qalora_forward_train(d: QaloraDesc, m: int, x, codes, qparams, A, B, y, workspace, stream=None):
+    """qalora_forward that leaves pool(x) and T in a workspace of OP_TRAIN size for qalora_backward_train."""
+    _check("qalora_forward_train", load().qalora_forward_train(byref(d), m, _ptr(x), _ptr(codes), _ptr(qparams), _ptr(A),
+                                                               _ptr(B), _ptr(y), _ptr(workspace),
+                                                               workspace.numel() if workspace is not None else 0,
+                                                               _stream(stream)))
+
+
+def qalora_backward_train(d: QaloraDesc, m: int, x, dy, codes, qparams, A, B, dx, dA, dB, workspace, stream=None):
+    """qalora_backward on the workspace the preceding qalora_forward_train of the same step filled."""
+    _check("qalora_backward_train", load().qalora_backward_train(byref(d), m, _ptr(x), _ptr(dy), _ptr(codes),
+                                                                 _ptr(qparams), _ptr(A), _ptr(B), _ptr(dx), _ptr(dA),
+                                                                 _ptr(dB), _ptr(workspace),
+                                                                 workspace.numel() if workspace is not None else 0,
+                                                                 _stream(stream)))
 
 
 def qalora_merge(d: QaloraDesc, qparams_in, A, B, qparams_out, stream=None):

@@ -65,7 +65,8 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t at = off; off += round_up(bytes, 256); return at; };
   const size_t M = (size_t)(m > 0 ? m : 0);
-  const bool bwd = op == QALORA_OP_BACKWARD;
+  const bool train = op == QALORA_OP_TRAIN;           // one workspace for a forward + backward pair
+  const bool bwd = op == QALORA_OP_BACKWARD || train;
   w.status = take(256);
   w.xp = take(bwd ? M * sh.G * sizeof(float) : 0);
   w.T = take(M * sh.r * sizeof(float));
@@ -86,7 +87,7 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   // partial results of the tensor-core forward whose reduction is cut into parts; none where the
   // dispatcher takes the few-token kernel (same predicate as in forward_launch)
   const bool few = m <= kFewTokenM && gemv_supported(sh, m);
-  w.fwd_parts = take(!bwd && !few && m > kSmallM && tc_forward_supported(sh, m) ? tc_forward_partial_bytes(sh, m) : 0);
+  w.fwd_parts = take((!bwd || train) && !few && m > kSmallM && tc_forward_supported(sh, m) ? tc_forward_partial_bytes(sh, m) : 0);
   w.total = off;
   return w;
 }
@@ -94,7 +95,7 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
 
 // Argument checks of the forward pass: everything qalora_forward rejects, nothing launched.
 int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
-                     const void* A, const void* B, const void* y, const void* workspace, size_t workspace_bytes) {
+                     const void* A, const void* B, const void* y, const void* workspace, size_t workspace_bytes, int layout_op) {
   Shape sh;
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
@@ -102,7 +103,8 @@ int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const vo
   if (m == 0) return QALORA_OK;
   if (x == nullptr || codes == nullptr || qparams == nullptr || y == nullptr) return QALORA_ERR_NULL_POINTER;
   if (sh.r > 0 && (A == nullptr || B == nullptr)) return QALORA_ERR_NULL_POINTER;
-  const Workspace ws = workspace_layout(sh, m, QALORA_OP_FORWARD);
+  if (layout_op == QALORA_OP_TRAIN && sh.r == 0) return QALORA_ERR_INVALID_ARG;
+  const Workspace ws = workspace_layout(sh, m, layout_op);
   if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
   if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
   if (!aligned16(x) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) || !aligned16(B) ||
@@ -116,11 +118,12 @@ int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const vo
 // `reset_status` is set (a public call); qalora_step_host zeroes it once for all its chunks
 // and passes false, so that a time-out raised by an earlier chunk survives to the end.
 int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
-                   const void* A, const void* B, void* y, void* workspace, void* cuda_stream, bool reset_status) {
+                   const void* A, const void* B, void* y, void* workspace, void* cuda_stream, bool reset_status,
+                   int layout_op) {
   Shape sh;
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
-  const Workspace ws = workspace_layout(sh, m, QALORA_OP_FORWARD);
+  const Workspace ws = workspace_layout(sh, m, layout_op);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   char* wsp = static_cast<char*>(workspace);
   float* T = reinterpret_cast<float*>(wsp + ws.T);
@@ -131,8 +134,10 @@ int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void
   // expire): a memset node between the pooling kernel and it would undo their overlap.
   if (reset_status && !few && (st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
   if (sh.r > 0) {
+    // a forward + backward pair keeps the pooled input too: the backward pass reads it for dA
+    float* xp = layout_op == QALORA_OP_TRAIN ? reinterpret_cast<float*>(wsp + ws.xp) : nullptr;
     st = launch_pool_T(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(A),
-                       nullptr, T, Tb, stream);
+                       xp, T, Tb, stream);
     if (st != QALORA_OK) return st;
   }
   if (few) {
@@ -153,14 +158,16 @@ int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void
 int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
                   const void* codes, const float* qparams, const void* A, const void* B,
                   void* dx, float* dA, float* dB,
-                  void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status) {
+                  void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status, bool pooled) {
   Shape sh;
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
   if (m < 0 || sh.r == 0) return QALORA_ERR_INVALID_ARG;
   if (x == nullptr || dy == nullptr || codes == nullptr || qparams == nullptr || A == nullptr || B == nullptr)
     return QALORA_ERR_NULL_POINTER;
-  const Workspace ws = workspace_layout(sh, m, QALORA_OP_BACKWARD);
+  // `pooled`: the workspace is the one qalora_forward_train filled for the same x, A and m; its
+  // pooled input, T and bf16(T) are taken as they are
+  const Workspace ws = workspace_layout(sh, m, pooled ? QALORA_OP_TRAIN : QALORA_OP_BACKWARD);
   if (ws.total > 0 && workspace == nullptr) return QALORA_ERR_NULL_POINTER;
   if (workspace_bytes < ws.total) return QALORA_ERR_WORKSPACE_TOO_SMALL;
   if (!aligned16(x) || !aligned16(dy) || !aligned16(codes) || !aligned16(qparams) || !aligned16(A) ||
@@ -190,7 +197,7 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
   if (aux_tc) st = launch_tc_dT(sh, m, dyb, Bb, dT, dTb, status, stream);
   else st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream);
   if (st != QALORA_OK) return st;
-  if (dA != nullptr || dB != nullptr) {
+  if (!pooled && (dA != nullptr || dB != nullptr)) {
     if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
   }
   if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
@@ -278,7 +285,7 @@ int qalora_workspace_bytes(const qalora_desc* desc, int64_t m, int op, size_t* b
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
   if (bytes == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (m < 0 || (op != QALORA_OP_FORWARD && op != QALORA_OP_BACKWARD)) return QALORA_ERR_INVALID_ARG;
+  if (m < 0 || (op != QALORA_OP_FORWARD && op != QALORA_OP_BACKWARD && op != QALORA_OP_TRAIN)) return QALORA_ERR_INVALID_ARG;
   *bytes = workspace_layout(sh, m, op).total;
   return QALORA_OK;
 }
@@ -311,9 +318,25 @@ int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A
 int qalora_forward(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
                    const float* qparams, const void* A, const void* B, void* y,
                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  int st = forward_validate(desc, m, x, codes, qparams, A, B, y, workspace, workspace_bytes);
+  int st = forward_validate(desc, m, x, codes, qparams, A, B, y, workspace, workspace_bytes, QALORA_OP_FORWARD);
   if (st != QALORA_OK || m == 0) return st;
-  return forward_launch(desc, m, x, codes, qparams, A, B, y, workspace, cuda_stream, /*reset_status=*/true);
+  return forward_launch(desc, m, x, codes, qparams, A, B, y, workspace, cuda_stream, /*reset_status=*/true, QALORA_OP_FORWARD);
+}
+
+int qalora_forward_train(const qalora_desc* desc, int64_t m, const void* x, const void* codes,
+                         const float* qparams, const void* A, const void* B, void* y,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int st = forward_validate(desc, m, x, codes, qparams, A, B, y, workspace, workspace_bytes, QALORA_OP_TRAIN);
+  if (st != QALORA_OK || m == 0) return st;
+  return forward_launch(desc, m, x, codes, qparams, A, B, y, workspace, cuda_stream, /*reset_status=*/true, QALORA_OP_TRAIN);
+}
+
+int qalora_backward_train(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
+                          const void* codes, const float* qparams, const void* A, const void* B,
+                          void* dx, float* dA, float* dB,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return backward_impl(desc, m, x, dy, codes, qparams, A, B, dx, dA, dB, workspace, workspace_bytes, cuda_stream,
+                       /*reset_status=*/false, /*pooled=*/true);
 }
 
 int qalora_forward_group_workspace_bytes(const qalora_group_layer* layers, int n, int64_t m, size_t* bytes) {
@@ -341,7 +364,7 @@ int qalora_forward_group(const qalora_group_layer* layers, int n, int64_t m,
   // every layer's arguments are checked before anything is launched
   for (int i = 0; i < n; ++i) {
     const qalora_group_layer& L = layers[i];
-    st = forward_validate(&L.desc, m, L.x, L.codes, L.qparams, L.A, L.B, L.y, workspace, workspace_bytes);
+    st = forward_validate(&L.desc, m, L.x, L.codes, L.qparams, L.A, L.B, L.y, workspace, workspace_bytes, QALORA_OP_FORWARD);
     if (st != QALORA_OK) return st;
   }
   if (n == 0 || m == 0) return QALORA_OK;
@@ -366,7 +389,8 @@ int qalora_forward_group(const qalora_group_layer* layers, int n, int64_t m,
   if ((st = cuda_status(cudaMemsetAsync(workspace, 0, sizeof(int), stream))) != QALORA_OK) return st;
   for (int i = 0; i < n; ++i) {
     const qalora_group_layer& L = layers[i];
-    st = forward_launch(&L.desc, m, L.x, L.codes, L.qparams, L.A, L.B, L.y, workspace, cuda_stream, /*reset_status=*/false);
+    st = forward_launch(&L.desc, m, L.x, L.codes, L.qparams, L.A, L.B, L.y, workspace, cuda_stream, /*reset_status=*/false,
+                        QALORA_OP_FORWARD);
     if (st != QALORA_OK) return st;
   }
   return QALORA_OK;
@@ -377,7 +401,7 @@ int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const voi
                     void* dx, float* dA, float* dB,
                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
   return backward_impl(desc, m, x, dy, codes, qparams, A, B, dx, dA, dB, workspace, workspace_bytes, cuda_stream,
-                       /*reset_status=*/true);
+                       /*reset_status=*/true, /*pooled=*/false);
 }
 
 
@@ -403,9 +427,7 @@ StepLayout step_layout(const Shape& sh, int64_t m) {
   const size_t M = (size_t)m;
   L.rows = step_chunk_rows(m);
   L.chunks = m > 0 ? (int)((m + L.rows - 1) / L.rows) : 1;
-  const size_t wf = workspace_layout(sh, L.rows, QALORA_OP_FORWARD).total,
-               wb = workspace_layout(sh, L.rows, QALORA_OP_BACKWARD).total;
-  L.ws_bytes = wf > wb ? wf : wb;
+  L.ws_bytes = workspace_layout(sh, L.rows, QALORA_OP_TRAIN).total;
   L.ws = take(L.ws_bytes);                         // first: the status word sits at the head of the staging area
   L.x = take(M * sh.K * 2); L.dy = take(M * sh.N * 2); L.y = take(M * sh.N * 2); L.dx = take(M * sh.K * 2);
   L.dA = take((size_t)sh.G * sh.r * 4); L.dB = take((size_t)sh.r * sh.N * 4);
@@ -494,14 +516,16 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
         !ok(cudaMemcpyAsync(base + L.dy + yo, static_cast<const char*>(dy_host) + yo, yb, cudaMemcpyHostToDevice, P->in)) ||
         !ok(cudaEventRecord(P->dy[c], P->in)) || !ok(cudaStreamWaitEvent(stream, P->x[c], 0)))
       return QALORA_ERR_CUDA;
-    st = forward_validate(desc, rows, base + L.x + xo, codes, qparams, A, B, base + L.y + yo, base + L.ws, L.ws_bytes);
+    // (forward and backward of a chunk share the workspace: the pooled input is computed once)
+    st = forward_validate(desc, rows, base + L.x + xo, codes, qparams, A, B, base + L.y + yo, base + L.ws, L.ws_bytes,
+                          QALORA_OP_TRAIN);
     if (st == QALORA_OK)
       st = forward_launch(desc, rows, base + L.x + xo, codes, qparams, A, B, base + L.y + yo, base + L.ws, cuda_stream,
-                          /*reset_status=*/false);
+                          /*reset_status=*/false, QALORA_OP_TRAIN);
     if (st != QALORA_OK) return st;
     if (!ok(cudaEventRecord(P->fwd[c], stream)) || !ok(cudaStreamWaitEvent(stream, P->dy[c], 0))) return QALORA_ERR_CUDA;
     st = backward_impl(desc, rows, base + L.x + xo, base + L.dy + yo, codes, qparams, A, B, base + L.dx + xo, dA_c, dB_c,
-                       base + L.ws, L.ws_bytes, cuda_stream, /*reset_status=*/false);
+                       base + L.ws, L.ws_bytes, cuda_stream, /*reset_status=*/false, /*pooled=*/true);
     if (st != QALORA_OK) return st;
     if (!ok(cudaEventRecord(P->bwd[c], stream)) || !ok(cudaStreamWaitEvent(P->out, P->fwd[c], 0)) ||
         !ok(cudaMemcpyAsync(static_cast<char*>(y_host) + yo, base + L.y + yo, yb, cudaMemcpyDeviceToHost, P->out)) ||

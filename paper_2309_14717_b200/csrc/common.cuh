@@ -42,13 +42,17 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op);
 
 // The public forward / backward in two halves (api.cu): checks that launch nothing, and the
 // launches with a say on whether the workspace's status word is cleared first.
+// `layout_op`: which qalora_op layout the workspace has (FORWARD, or TRAIN for a forward whose
+// pooled input the backward pass of the same step reuses: `pooled`).
 int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
-                     const void* A, const void* B, const void* y, const void* workspace, size_t workspace_bytes);
+                     const void* A, const void* B, const void* y, const void* workspace, size_t workspace_bytes,
+                     int layout_op);
 int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
-                   const void* A, const void* B, void* y, void* workspace, void* cuda_stream, bool reset_status);
+                   const void* A, const void* B, void* y, void* workspace, void* cuda_stream, bool reset_status,
+                   int layout_op);
 int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void* dy, const void* codes,
                   const float* qparams, const void* A, const void* B, void* dx, float* dA, float* dB,
-                  void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status);
+                  void* workspace, size_t workspace_bytes, void* cuda_stream, bool reset_status, bool pooled);
 
 // --------------------------------------------------------------- device side --
 __device__ __forceinline__ float bf16_to_float(__nv_bfloat16 v) { return __bfloat162float(v); }

@@ -44,7 +44,7 @@ extern "C" int qalora_forward_static(const qalora_desc* desc, int64_t m, const v
   // a rejected call must not have enqueued anything, nor touched the CUDA runtime
   alignas(16) static const char aligned_stand_in = 0;
   if ((st = qalora::forward_validate(desc, m, x, codes, qparams, A, B, y, &aligned_stand_in,
-                                     (size_t)QALORA_STATIC_SCRATCH_BYTES)) != QALORA_OK)
+                                     (size_t)QALORA_STATIC_SCRATCH_BYTES, QALORA_OP_FORWARD)) != QALORA_OK)
     return st;
   if (m == 0) return QALORA_OK;
   void* scratch = nullptr;

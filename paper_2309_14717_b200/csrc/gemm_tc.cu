@@ -19,7 +19,8 @@
 //
 // Warp roles (768 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
 // owner, warps 4-19 = four dequantizing warpgroups (each owns every fourth
-// reduction step), warps 20-23 = epilogue.  Stages are handed
+// reduction step), warps 20-23 = epilogue (dx: two accumulators, so that a tile is
+// drained while the next one is multiplied).  Stages are handed
 // over with mbarriers; every wait is bounded and a timeout raises a status word
 // instead of hanging.
 #include <mutex>
@@ -38,7 +39,7 @@ constexpr int TILE_J = 64;       // reduction step per stage
 constexpr int DQ_GROUPS = 4;     // dequantizing warpgroups
 constexpr int THREADS = 128 + 128 * DQ_GROUPS + 128;
 constexpr int TMEM_COLS = 512;
-constexpr int ACC_COL = 0;       // accumulator: columns [0, 256)
+constexpr int ACC_COL = 0;       // accumulator: columns [0, 256); dx keeps a second one at [256, 512)
 constexpr int A_COL = 256;       // forward operand ring: 8 slots of 32 columns
 constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx)
 
@@ -113,6 +114,12 @@ struct Smem {
   static constexpr int IPS = MODE == FWD ? 2 : 1;                                // reduction steps per code stage
   static constexpr int TILE_NC = MODE == FWD ? TILE_C : TILE_J;                  // columns of a code stage
   static constexpr int NOUT = MODE == FWD ? 2 : 1;                               // epilogue staging buffers
+  // Accumulators in tensor memory.  The forward product keeps its operand ring in the upper 256
+  // columns, so it has one; dx takes its operand from shared memory and alternates between two,
+  // so that the epilogue drains one tile while the next one is being multiplied.  (A forward
+  // kernel with the operand in shared memory and two accumulators was built too: 5-8 % slower
+  // than the operand in tensor memory, 0.665 against 0.615 ms for 4096 -> 11008 at 8192 tokens.)
+  static constexpr int NACC = MODE == DX ? 2 : 1;
   // a code stage = 4 k-block rows x TILE_NC columns of pack units + up to 4 rows of (alpha, beta)
   static constexpr uint32_t CODE_BYTES = 4 * TILE_NC * WORDS * 4;
   static constexpr uint32_t QP_ROW_BYTES = TILE_NC * 8;
@@ -124,7 +131,7 @@ struct Smem {
   static constexpr uint32_t OFF_C = OFF_A + (MODE == DX ? NX * ATILE_BYTES : 0);
   static constexpr uint32_t OFF_OUT = OFF_C + NC * CSTAGE_BYTES;
   static constexpr uint32_t OFF_BARS = OFF_OUT + NOUT * OUT_BYTES;
-  static constexpr int NBARS = 2 * NB + 2 * NC + 2;
+  static constexpr int NBARS = 2 * NB + 2 * NC + 2 * NACC;
   static constexpr uint32_t TOTAL = OFF_BARS + 8 * NBARS + 64 + 1024;            // + alignment slack
 };
 
@@ -234,8 +241,9 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   auto bar_empty_x = [&](int s) { return bar_base + 8u * (NB + s); };
   auto bar_full_c = [&](int s) { return bar_base + 8u * (2 * NB + s); };
   auto bar_empty_c = [&](int s) { return bar_base + 8u * (2 * NB + NC + s); };
-  const uint32_t bar_acc_full = bar_base + 8u * (2 * NB + 2 * NC);
-  const uint32_t bar_acc_empty = bar_acc_full + 8u;
+  constexpr int NACC = S::NACC;
+  auto bar_acc_full = [&](int b) { return bar_base + 8u * (2 * NB + 2 * NC + b); };
+  auto bar_acc_empty = [&](int b) { return bar_base + 8u * (2 * NB + 2 * NC + NACC + b); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + S::OFF_BARS + 8 * S::NBARS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_BARS + 8 * S::NBARS + 8);
 
@@ -246,8 +254,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     // dequantizer warps have written the operand slot: one wait per step for the MMA issuer
     for (int s = 0; s < NB; ++s) { ptx::mbar_init(bar_full_x(s), 1 + 4); ptx::mbar_init(bar_empty_x(s), 1); }
     for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4 * S::IPS); }
-    ptx::mbar_init(bar_acc_full, 1);
-    ptx::mbar_init(bar_acc_empty, 4);
+    for (int b = 0; b < NACC; ++b) { ptx::mbar_init(bar_acc_full(b), 1); ptx::mbar_init(bar_acc_empty(b), 4); }
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&act_map);
@@ -327,7 +334,9 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       bool ready = false;
       for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x, ++tcount) {
         const TcSegment sg = tc_segment<PARTS>(p, vt);
-        if (!(ok = ptx::mbar_wait(bar_acc_empty, (tcount & 1) ^ 1, abort_flag))) break;
+        const int ab = tcount % NACC;                 // accumulator of this tile
+        const uint32_t acc_tmem = tmem_base + ACC_COL + ab * TILE_T;
+        if (!(ok = ptx::mbar_wait(bar_acc_empty(ab), ((tcount / NACC) & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int j = 0; j < sg.n_steps; ++j, ++it) {
           const int sx = it % NX, sb = it % NB;
@@ -341,18 +350,18 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           const uint32_t acc = j > 0 ? 1u : 0u;
           // the commit frees the activation tile AND the operand slot
           if (MODE == FWD) {
-            ready = ptx::mma4_ts_commit_probe<2>(tmem_base + ACC_COL, tmem_base + A_COL + sb * 32, bdesc, IDESC_MAIN, acc,
+            ready = ptx::mma4_ts_commit_probe<2>(acc_tmem, tmem_base + A_COL + sb * 32, bdesc, IDESC_MAIN, acc,
                                                  bar_empty_x(sb), next_bar, next_par) != 0;
           } else if (j < sg.n_main) {
             // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO); 2 KiB per step
-            ready = ptx::mma4_ss_commit_probe<128, 2>(tmem_base + ACC_COL, ptx::smem_desc(as, 8192, 1024), bdesc, IDESC_MAIN,
+            ready = ptx::mma4_ss_commit_probe<128, 2>(acc_tmem, ptx::smem_desc(as, 8192, 1024), bdesc, IDESC_MAIN,
                                                       acc, bar_empty_x(sb), next_bar, next_par) != 0;
           } else {
-            ready = ptx::mma4_ss_commit_probe<2, 2>(tmem_base + ACC_COL, ptx::smem_desc(as, 16, 1024), bdesc, IDESC_LORA, acc,
+            ready = ptx::mma4_ss_commit_probe<2, 2>(acc_tmem, ptx::smem_desc(as, 16, 1024), bdesc, IDESC_LORA, acc,
                                                     bar_empty_x(sb), next_bar, next_par) != 0;
           }
         }
-        if (ok) ptx::mma_commit(bar_acc_full);
+        if (ok) ptx::mma_commit(bar_acc_full(ab));
       }
     }
   } else if (warp >= 4 && warp < 4 + 4 * DQ_GROUPS) {
@@ -472,17 +481,18 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x, ++tcount) {
       const int tile = PARTS ? vt / p.ksplit : vt, sp = PARTS ? vt % p.ksplit : 0;
       const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
-      if (!(ok = ptx::mbar_wait(bar_acc_full, tcount & 1, abort_flag))) break;
+      const int ab = tcount % NACC;
+      if (!(ok = ptx::mbar_wait(bar_acc_full(ab), (tcount / NACC) & 1, abort_flag))) break;
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int col = 0; col < TT; col += 32, ++chunk) {
         uint32_t v[32];
-        ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ACC_COL + col, v);
+        ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ACC_COL + ab * TILE_T + col, v);
         ptx::tmem_wait_ld();
         if (col == TT - 32) {                     // all columns read: hand the accumulator back
           ptx::tc_fence_before();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(bar_acc_empty);
+          if (lane == 0) ptx::mbar_arrive(bar_acc_empty(ab));
         }
         if constexpr (PARTS) {
           // a part of the reduction: fp32 partial results [part][token][channel], added up by

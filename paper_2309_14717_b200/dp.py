@@ -95,14 +95,14 @@ class AdapterBucket:
 
 class AdaptedLayer:
     """One quantized layer of a data-parallel fine-tuning step: its descriptor, packed codes and
-    (alpha, beta) (frozen, replicated on every rank) and the workspaces of its two passes for
-    `tokens` rows per rank.  The trained factors are not here: they live in the AdapterBucket."""
+    (alpha, beta) (frozen, replicated on every rank) and the workspace its forward and backward
+    pass share for `tokens` rows per rank (the pooled input is computed once per step).  The
+    trained factors are not here: they live in the AdapterBucket."""
 
     def __init__(self, d, codes, qparams, tokens: int):
         from . import binding as Q
         self.d, self.codes, self.qparams, self.tokens = d, codes, qparams, tokens
-        self.ws_forward = Q.alloc_workspace(d, tokens, Q.OP_FORWARD, device=codes.device)
-        self.ws_backward = Q.alloc_workspace(d, tokens, Q.OP_BACKWARD, device=codes.device)
+        self.workspace = Q.alloc_workspace(d, tokens, Q.OP_TRAIN, device=codes.device)
 
     @property
     def shape(self):
@@ -114,7 +114,7 @@ def finetune_step(layers, bucket: AdapterBucket, xs, dys, ys, dxs, lr, group=Non
     """One data-parallel fine-tuning step over `layers` (Section 4.1: only A and B are trained,
     AdamW with a maximum gradient norm), every piece of it a call into the CUDA library:
 
-      forward of layer i from the bucket's bf16 factors  -> ys[i]
+      forward of layer i from the bucket's bf16 factors  -> ys[i]  (keeps pool(x) and T for the backward pass)
       backward of layer i, dA and dB written STRAIGHT into the bucket's gradient views, dX -> dxs[i]
       ONE all-reduce of the whole gradient array over the ranks (the step's only exchange)
       ONE clipped AdamW update of every factor; it also refreshes the bf16 copies the next
@@ -126,10 +126,10 @@ def finetune_step(layers, bucket: AdapterBucket, xs, dys, ys, dxs, lr, group=Non
     from . import binding as Q
     for i, L in enumerate(layers):
         A, B = bucket.factors(i)
-        Q.qalora_forward(L.d, L.tokens, xs[i], L.codes, L.qparams, A, B, ys[i], L.ws_forward, stream)
+        Q.qalora_forward_train(L.d, L.tokens, xs[i], L.codes, L.qparams, A, B, ys[i], L.workspace, stream)
     for i, L in enumerate(layers):
         A, B = bucket.factors(i)
         dA, dB = bucket.grads(i)
-        Q.qalora_backward(L.d, L.tokens, xs[i], dys[i], L.codes, L.qparams, A, B, dxs[i], dA, dB, L.ws_backward, stream)
+        Q.qalora_backward_train(L.d, L.tokens, xs[i], dys[i], L.codes, L.qparams, A, B, dxs[i], dA, dB, L.workspace, stream)
     bucket.reduce(group)
     bucket.update(lr, stream=stream, **adamw)

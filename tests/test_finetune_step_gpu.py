@@ -32,6 +32,33 @@ def bf16_round(a64):
     return torch.from_numpy(np.asarray(a64, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
 
 
+@pytest.mark.parametrize("cfg", CFGS + [LayerConfig("step_few", 1280, 384, 32, 4, 16, 1.0, 12, seed=44)], ids=lambda c: c.name)
+def test_training_pair_gives_the_bits_of_the_separate_passes(cfg):
+    """qalora_forward_train + qalora_backward_train (pooled input computed once, one workspace)
+    against qalora_forward + qalora_backward: the same kernels on the same values."""
+    t = {k: v.cuda() for k, v in make_inputs(cfg).items()}
+    d = Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, cfg.rank, cfg.scale)
+    codes, qparams = Q.alloc_packed(d)
+    Q.qalora_quantize(d, t["W"], codes, qparams)
+    M = cfg.tokens
+    mk = lambda *shape, dt=torch.bfloat16: torch.full(shape, float("nan"), dtype=dt, device="cuda")
+    y0, dx0 = mk(M, cfg.d_out), mk(M, cfg.d_in)
+    dA0, dB0 = mk(cfg.groups, cfg.rank, dt=torch.float32), mk(cfg.rank, cfg.d_out, dt=torch.float32)
+    Q.qalora_forward(d, M, t["x"], codes, qparams, t["A"], t["B"], y0, Q.alloc_workspace(d, M, Q.OP_FORWARD))
+    Q.qalora_backward(d, M, t["x"], t["dy"], codes, qparams, t["A"], t["B"], dx0, dA0, dB0, Q.alloc_workspace(d, M, Q.OP_BACKWARD))
+    y1, dx1 = mk(M, cfg.d_out), mk(M, cfg.d_in)
+    dA1, dB1 = mk(cfg.groups, cfg.rank, dt=torch.float32), mk(cfg.rank, cfg.d_out, dt=torch.float32)
+    ws = torch.full((Q.qalora_workspace_bytes(d, M, Q.OP_TRAIN),), 0xFF, dtype=torch.uint8, device="cuda")
+    Q.qalora_forward_train(d, M, t["x"], codes, qparams, t["A"], t["B"], y1, ws)
+    Q.qalora_backward_train(d, M, t["x"], t["dy"], codes, qparams, t["A"], t["B"], dx1, dA1, dB1, ws)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(ws) == 0
+    assert torch.equal(y0, y1) and torch.equal(dx0, dx1) and torch.equal(dA0, dA1) and torch.equal(dB0, dB1)
+    with pytest.raises(Q.QaloraError):                    # the pair is for layers with an adapter
+        Q.qalora_forward_train(Q.desc(cfg.d_in, cfg.d_out, cfg.group_size, cfg.bits, 0, 1.0), M, t["x"], codes, qparams,
+                               None, None, y1, ws)
+
+
 def test_two_consecutive_steps_match_the_oracles():
     # eps is taken of the size of a clipped gradient (0.3 / sqrt(14 K values) = 2.5e-3): with the usual
     # 1e-8 AdamW's first steps are lr * sign(g), and the few values whose gradient lies within the bf16
@@ -62,7 +89,7 @@ def test_two_consecutive_steps_match_the_oracles():
         dp.finetune_step(layers, bucket, xs, dys, ys, dxs, lr, max_grad_norm=max_norm, eps=eps)
         torch.cuda.synchronize()
         for L in layers:
-            assert Q.workspace_status(L.ws_forward) == 0 and Q.workspace_status(L.ws_backward) == 0
+            assert Q.workspace_status(L.workspace) == 0
         grads, off = [], 0
         for i, (c, t, (codes, alpha, beta)) in enumerate(zip(CFGS, cpu, quant)):
             G, r, N = layers[i].shape
