@@ -59,6 +59,10 @@ int check_desc(const qalora_desc* d, Shape* sh) {
 static constexpr int64_t kSmallM = 16;
 // The forward pass alone keeps the few-token kernel up to this many tokens (where its shapes allow).
 static constexpr int64_t kFewTokenM = 32;
+// Above the few-token range and up to this many tokens the forward pass takes the kernel with
+// the tokens as the MMA rows (where its shapes allow): one 128-token tile.
+static constexpr int64_t kMidM = 128;
+static bool takes_midm(const Shape& sh, int64_t m) { return m > kSmallM && m <= kMidM && midm_supported(sh, m); }
 
 Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   Workspace w{};
@@ -87,7 +91,12 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   // partial results of the tensor-core forward whose reduction is cut into parts; none where the
   // dispatcher takes the few-token kernel (same predicate as in forward_launch)
   const bool few = m <= kFewTokenM && gemv_supported(sh, m);
-  w.fwd_parts = take((!bwd || train) && !few && m > kSmallM && tc_forward_supported(sh, m) ? tc_forward_partial_bytes(sh, m) : 0);
+  size_t parts_bytes = 0;
+  if ((!bwd || train) && !few && m > kSmallM) {
+    if (takes_midm(sh, m)) parts_bytes = midm_partial_bytes(sh, m);
+    else if (tc_forward_supported(sh, m)) parts_bytes = tc_forward_partial_bytes(sh, m);
+  }
+  w.fwd_parts = take(parts_bytes);
   w.total = off;
   return w;
 }
@@ -144,6 +153,11 @@ int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void
     return launch_gemv(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
                        reinterpret_cast<const float2*>(qparams), sh.r > 0 ? Tb : nullptr,
                        static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(y), status, reset_status, stream);
+  }
+  if (takes_midm(sh, m)) {
+    return launch_midm(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),
+                       reinterpret_cast<const float2*>(qparams), Tb, static_cast<const __nv_bfloat16*>(B),
+                       static_cast<__nv_bfloat16*>(y), reinterpret_cast<float*>(wsp + ws.fwd_parts), status, stream);
   }
   if (m > kSmallM && tc_forward_supported(sh, m)) {
     return launch_tc_forward(sh, m, static_cast<const __nv_bfloat16*>(x), static_cast<const uint32_t*>(codes),

@@ -124,6 +124,14 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
                  __nv_bfloat16* dx, int* status, cudaStream_t st);
 
+// Forward for a few dozen to a few hundred tokens (midm_tc.cu): tokens as the MMA rows, 256
+// channels per instruction.  Tb is the bf16 rank-r intermediate (ignored when r == 0).
+bool midm_supported(const Shape& sh, int64_t M);
+size_t midm_partial_bytes(const Shape& sh, int64_t M);
+int launch_midm(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
+                const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, float* partial, int* status,
+                cudaStream_t st);
+
 // Few-token forward (gemv.cu): M <= 32.  `reset_status`: the kernel clears *status at its start.
 bool gemv_supported(const Shape& sh, int64_t M);
 int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,

@@ -26,7 +26,9 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "dequant.cuh"
 #include "ptx.cuh"
+#include "tc_host.cuh"
 
 namespace qalora {
 
@@ -134,93 +136,6 @@ struct Smem {
   static constexpr int NBARS = 2 * NB + 2 * NC + 2 * NACC;
   static constexpr uint32_t TOTAL = OFF_BARS + 8 * NBARS + 64 + 1024;            // + alignment slack
 };
-
-// ---- dequantization of one pack unit to 16 bf16x2 registers ------------------
-// The two codes of a pair sit at the same bit offset of the two half-words, so one shift
-// and one LOP3 turn them into the bf16 pair (128 + c0, 128 + c1): the code is OR-ed into
-// the mantissa of bf16 128.0, no int-to-float conversion.  Widening each half to fp32 is
-// one more logic op, then W~ = alpha * (128 + c) + (beta - 128 alpha) is ONE fp32 FMA per
-// element, and the pair is rounded once to bf16x2.  alpha and beta stay in fp32, so the
-// only rounding that matters is that of the final weight (rounding alpha or beta
-// themselves would put a common error on all channels of a group, which the pooled input
-// amplifies).
-// The logic/shift pipe is the busiest one in these kernels.  A LOP3 takes at most one
-// immediate, so the masks live in registers (DqConsts, made opaque to the compiler):
-// "(a & mask) | magic" then is one instruction instead of two.
-struct DqConsts {
-  uint32_t mask, magic, himask, third;
-};
-template <int BITS>
-__device__ __forceinline__ DqConsts dq_consts() {
-  DqConsts c;
-  asm volatile("mov.b32 %0, %1;" : "=r"(c.mask) : "n"(BITS == 4 ? 0x000f000f : 0x00030003));
-  asm volatile("mov.b32 %0, 0x43004300;" : "=r"(c.magic));
-  asm volatile("mov.b32 %0, 0xffff0000;" : "=r"(c.himask));
-  asm volatile("mov.b32 %0, 0x00040004;" : "=r"(c.third));
-  return c;
-}
-__device__ __forceinline__ uint32_t lop_and_or(uint32_t a, uint32_t b, uint32_t c) {   // (a & b) | c
-  uint32_t d;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ uint32_t lop_and(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("and.b32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-template <int SHIFT>   // positive: shift left
-__device__ __forceinline__ uint32_t shift_to(uint32_t w) {
-  if constexpr (SHIFT >= 0) return w << SHIFT; else return w >> (-SHIFT);
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&t);
-}
-
-template <int WORDS>
-__device__ __forceinline__ void load_unit(const uint32_t* cw, uint32_t* w) {
-  if constexpr (WORDS == 4) {
-    const uint4 t = *reinterpret_cast<const uint4*>(cw);
-    w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
-  } else if constexpr (WORDS == 2) {
-    const uint2 t = *reinterpret_cast<const uint2*>(cw);
-    w[0] = t.x; w[1] = t.y;
-  } else {
-#pragma unroll
-    for (int q = 0; q < WORDS; ++q) w[q] = cw[q];
-  }
-}
-
-// pair P of word I: positions (2P, 2P+1) of that word's codes
-template <int BITS, int I, int P>
-__device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, float a, float b, const DqConsts& k) {
-  constexpr int W = BITS == 4 ? 4 : 2;             // width of the (low) code bits
-  uint32_t pr = lop_and_or(w[I] >> (W * P), k.mask, k.magic);
-  if constexpr (BITS == 3) {
-    // third bits of the pair: bits PH and 16 + PH of word 2, PH = 8 I + P; they go to bit 2 of each half
-    constexpr int PH = 8 * I + P;
-    pr = lop_and_or(shift_to<2 - PH>(w[2]), k.third, pr);
-  }
-  const float v0 = __uint_as_float(pr << 16), v1 = __uint_as_float(lop_and(pr, k.himask));   // 128 + c, exactly
-  return pack_bf16x2(fmaf(a, v0, b), fmaf(a, v1, b));
-}
-
-template <int BITS, int I, int P>
-__device__ __forceinline__ void dq_all(const uint32_t* w, float a, float b, const DqConsts& k, uint32_t* out) {
-  constexpr int PAIRS = BITS == 4 ? 4 : 8;          // pairs per word
-  constexpr int NWORDS = BITS == 4 ? 4 : 2;         // words that carry the (low) code bits
-  out[I * PAIRS + P] = dq_pair<BITS, I, P>(w, a, b, k);
-  if constexpr (P + 1 < PAIRS) dq_all<BITS, I, P + 1>(w, a, b, k, out);
-  else if constexpr (I + 1 < NWORDS) dq_all<BITS, I + 1, 0>(w, a, b, k, out);
-}
-
-// out[q] = bf16x2 of positions (2q, 2q+1) of the unit, q = 0..15
-template <int BITS>
-__device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, const DqConsts& k, uint32_t* out) {
-  const float b = fmaf(-128.f, ab.x, ab.y);
-  dq_all<BITS, 0, 0>(w, ab.x, b, k, out);
-}
 
 // PARTS: every tile's reduction is cut into p.ksplit parts.  TT: tokens per tile.
 template <int BITS, int MODE, bool PARTS, int TT>
@@ -530,11 +445,10 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   }
 }
 
-// ------------------------------------------------------------------ host side --
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+}  // namespace
 
+// ------------------------------------------------------------------ host side --
+// (tensor-map builders and the sum of parts are shared with midm_tc.cu: tc_host.cuh)
 EncodeTiledFn encode_fn() {
   static EncodeTiledFn fn = nullptr;
   static std::once_flag once;
@@ -550,7 +464,7 @@ EncodeTiledFn encode_fn() {
 
 // bf16 matrix [rows][cols] row-major, box = 64 columns x `box_rows` rows, 128-byte swizzle;
 // out-of-range rows and columns read as zero.
-bool make_act_map(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows = TILE_T) {
+bool make_act_map(CUtensorMap* map, const void* base, long long rows, int cols, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -575,14 +489,14 @@ bool make_out_map(CUtensorMap* map, void* base, long long rows, int cols) {
 }
 
 // packed codes [K/32][N][words] uint32 seen as a 2-D matrix of 8-byte elements, so that one
-// box row is the whole contiguous run of tile_cols pack units; box = 4 k-block rows
-bool make_codes_map(CUtensorMap* map, const uint32_t* codes, int K, int N, int bits, int tile_cols) {
+// box row is the whole contiguous run of tile_cols pack units; box = kb_rows k-block rows
+bool make_codes_map(CUtensorMap* map, const uint32_t* codes, int K, int N, int bits, int tile_cols, int kb_rows) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   const int words = words_per_unit(bits);
   cuuint64_t dims[2] = {(cuuint64_t)N * words / 2, (cuuint64_t)(K / 32)};
   cuuint64_t strides[1] = {(cuuint64_t)N * words * 4};
-  cuuint32_t box[2] = {(cuuint32_t)(tile_cols * words / 2), 4};
+  cuuint32_t box[2] = {(cuuint32_t)(tile_cols * words / 2), (cuuint32_t)kb_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<uint32_t*>(codes), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -602,7 +516,7 @@ bool make_qp_map(CUtensorMap* map, const float2* qp, int G, int N, int tile_cols
 }
 
 // out[i] = bf16(sum over parts of partial[part][i]), added in part order; 8 elements per thread
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 sum_parts_kernel(const float* __restrict__ partial, __nv_bfloat16* __restrict__ out, size_t count, int parts) {
   const size_t i0 = ((size_t)blockIdx.x * 256 + threadIdx.x) * 8;
   if (i0 >= count) return;                                   // count is a multiple of 8
@@ -619,12 +533,20 @@ sum_parts_kernel(const float* __restrict__ partial, __nv_bfloat16* __restrict__ 
   *reinterpret_cast<uint4*>(out + i0) = o;
 }
 
+int launch_sum_parts_bf16(const float* partial, __nv_bfloat16* out, size_t count, int parts, cudaStream_t st) {
+  sum_parts_kernel<<<(unsigned)((count / 8 + 255) / 256), 256, 0, st>>>(partial, out, count, parts);
+  count_launch();
+  return cuda_status(cudaGetLastError());
+}
+
+namespace {
+
 template <int BITS, int MODE, bool PARTS, int TT>
 int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
   using S = Smem<BITS, MODE, TT>;
   CUtensorMap out, cmap, qmap;
   if (!make_out_map(&out, p.out, p.M, p.ld_out)) return QALORA_ERR_CUDA;
-  if (!make_codes_map(&cmap, p.codes, p.K, p.N, BITS, S::TILE_NC)) return QALORA_ERR_CUDA;
+  if (!make_codes_map(&cmap, p.codes, p.K, p.N, BITS, S::TILE_NC, 4)) return QALORA_ERR_CUDA;
   if (!make_qp_map(&qmap, p.qparams, p.K / p.g, p.N, S::TILE_NC, p.qp_rows)) return QALORA_ERR_CUDA;
   static_assert(S::TOTAL <= 232448, "shared memory budget");
   auto kern = qalora_tc_kernel<BITS, MODE, PARTS, TT>;
@@ -639,12 +561,8 @@ int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams&
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
-  if (PARTS) {
-    const size_t count = (size_t)p.M * p.ld_out;
-    sum_parts_kernel<<<(unsigned)((count / 8 + 255) / 256), 256, 0, st>>>(p.partial, p.out, count, p.ksplit);
-    count_launch();
-  }
-  return cuda_status(cudaGetLastError());
+  if (PARTS) return launch_sum_parts_bf16(p.partial, p.out, (size_t)p.M * p.ld_out, p.ksplit, st);
+  return QALORA_OK;
 }
 
 template <int BITS, int MODE>
@@ -730,9 +648,9 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
                  __nv_bfloat16* dx, int* status, cudaStream_t st) {
   CUtensorMap act, lora;
-  if (!make_act_map(&act, dy, M, sh.N)) return QALORA_ERR_CUDA;
+  if (!make_act_map(&act, dy, M, sh.N, TILE_T)) return QALORA_ERR_CUDA;
   lora = act;
-  if (sh.r > 0 && !make_act_map(&lora, dTb, M, sh.r)) return QALORA_ERR_CUDA;
+  if (sh.r > 0 && !make_act_map(&lora, dTb, M, sh.r, TILE_T)) return QALORA_ERR_CUDA;
   TcParams p{};
   p.codes = codes; p.qparams = qparams; p.lora = A; p.out = dx;
   p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.K;

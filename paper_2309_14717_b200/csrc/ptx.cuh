@@ -246,6 +246,35 @@ __device__ __forceinline__ uint32_t mma4_ss_commit_probe(uint32_t d_tmem, uint64
       : "memory");
   return ready;
 }
+// The same with two commits and two probes (a step that frees two resources with their own
+// barriers and whose successor waits on two): returns bit 0 for `next_bar0`, bit 1 for `next_bar1`.
+template <int A_STEP, int B_STEP>
+__device__ __forceinline__ uint32_t mma4_ss_commit2_probe2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                           uint32_t accumulate_first, uint32_t commit_bar0, uint32_t commit_bar1,
+                                                           uint32_t next_bar0, uint32_t next_parity0, uint32_t next_bar1,
+                                                           uint32_t next_parity1) {
+  uint32_t ready;
+  asm volatile(
+      "{\n\t.reg .pred p, q0, q1, t;\n\t.reg .b32 r0, r1;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 q0, [%8], %9;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 q1, [%10], %11;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "setp.eq.b32 t, 0, 0;\n\t"
+      "add.u64 a1, %2, %12;\n\tadd.u64 a2, a1, %12;\n\tadd.u64 a3, a2, %12;\n\t"
+      "add.u64 b1, %3, %13;\n\tadd.u64 b2, b1, %13;\n\tadd.u64 b3, b2, %13;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], a1, b1, %4, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], a2, b2, %4, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%1], a3, b3, %4, t;\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];\n\t"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%7];\n\t"
+      "selp.b32 r0, 1, 0, q0;\n\tselp.b32 r1, 2, 0, q1;\n\tor.b32 %0, r0, r1;\n\t}"
+      : "=r"(ready)
+      : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate_first), "r"(commit_bar0), "r"(commit_bar1),
+        "r"(next_bar0), "r"(next_parity0), "r"(next_bar1), "r"(next_parity1), "n"(A_STEP), "n"(B_STEP)
+      : "memory");
+  return ready;
+}
 // Arrives on `bar` once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

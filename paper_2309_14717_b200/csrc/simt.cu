@@ -9,51 +9,85 @@ namespace qalora {
 // One token row per blockIdx.x: xp[q] = sum of the g channels of group q
 // (Appendix B Eq. 3), then T[i] = s * sum_q xp[q] * A[q][i] for the 32 adapter
 // columns of blockIdx.y (every block pools the row again: it is a few KiB).
+// The kernel is short and bound by the latency of its loads, so they are issued in
+// batches: the block's 32-column slice of A goes to shared memory first (its loads are
+// independent of everything else), the row of x is read four 16-byte pieces per lane at a
+// time before any of them is reduced.
 constexpr int POOL_THREADS = 256;
+constexpr size_t kPoolASliceMax = 40 * 1024;          // the slice of A is kept in shared memory up to this size
 
 __global__ void __launch_bounds__(POOL_THREADS)
 pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
               float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
-              int K, int g, int G, int r, float s) {
-  extern __shared__ float xp[];                       // [G]
+              int K, int g, int G, int r, float s, int a_in_smem) {
+  extern __shared__ __align__(16) uint8_t pool1_smem[];
+  float* xp = reinterpret_cast<float*>(pool1_smem);                                        // [G]
+  __nv_bfloat16* As = reinterpret_cast<__nv_bfloat16*>(pool1_smem + ((size_t)G * 4 + 15) / 16 * 16);   // [G][32] when a_in_smem
   // The few-token forward kernel that follows needs T only at its very end: let it start now
   // (it waits for this grid before it reads T).  Without such a dependent launch this does nothing.
   asm volatile("griddepcontrol.launch_dependents;");
   const size_t m = blockIdx.x;
+  const int i0 = blockIdx.y * 32;
+  if (a_in_smem) {
+    // rows of 32 columns = 4 pieces of 8 (r is a multiple of 8: a piece lies inside the rank or beyond it)
+    for (int idx = threadIdx.x; idx < G * 4; idx += POOL_THREADS) {
+      const int q = idx / 4, c = idx % 4;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (i0 + c * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(A + (size_t)q * r + i0 + c * 8));
+      *reinterpret_cast<uint4*>(As + (size_t)q * 32 + c * 8) = v;
+    }
+  }
   const __nv_bfloat16* xr = x + m * (size_t)K;
-  // four lanes per group, 8 channels (16 bytes) per lane and step; g is a multiple of 32
-  for (int q0 = 0; q0 < G; q0 += POOL_THREADS / 4) {   // uniform trip count: the shuffles see whole warps
-    const int q = q0 + threadIdx.x / 4;
-    const int lane4 = threadIdx.x & 3;
-    float acc = 0.0f;
-    if (q < G) {
-      for (int k = lane4 * 8; k < g; k += 32) {
-        const uint4 v = *reinterpret_cast<const uint4*>(xr + (size_t)q * g + k);
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+  // four lanes per group, 8 channels (16 bytes) per lane and step; g is a multiple of 32.
+  // Groups q0 + 64 u + tid / 4, u = 0..3, are handled together: their loads first, then the sums.
+  const int lane4 = threadIdx.x & 3;
+  for (int q0 = 0; q0 < G; q0 += POOL_THREADS) {       // uniform trip count: the shuffles see whole warps
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k = lane4 * 8; k < g; k += 32) {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int q = q0 + u * (POOL_THREADS / 4) + threadIdx.x / 4;
+        v[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (q < G) v[u] = __ldg(reinterpret_cast<const uint4*>(xr + (size_t)q * g + k));
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v[u]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 f = __bfloat1622float2(h[i]);
-          acc += f.x + f.y;
+          acc[u] += f.x + f.y;
         }
       }
     }
-    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-    if (lane4 == 0 && q < G) {
-      xp[q] = acc;
-      if (xp_out != nullptr && blockIdx.y == 0) xp_out[m * (size_t)G + q] = acc;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int q = q0 + u * (POOL_THREADS / 4) + threadIdx.x / 4;
+      float a = acc[u];
+      a += __shfl_xor_sync(0xffffffffu, a, 1);
+      a += __shfl_xor_sync(0xffffffffu, a, 2);
+      if (lane4 == 0 && q < G) {
+        xp[q] = a;
+        if (xp_out != nullptr && blockIdx.y == 0) xp_out[m * (size_t)G + q] = a;
+      }
     }
   }
   __syncthreads();
   // this block's 32 adapter columns (blockIdx.y); 8 threads share a column, each taking
-  // every eighth group, so that the loads of A of one column are spread over 8 lanes
+  // every eighth group
   __shared__ float part[8][33];
   const int il = threadIdx.x % 32, pr = threadIdx.x / 32;
-  const int i = blockIdx.y * 32 + il;
+  const int i = i0 + il;
   float acc = 0.0f;
   if (i < r) {
+    if (a_in_smem) {
 #pragma unroll 4
-    for (int q = pr; q < G; q += 8) acc = fmaf(xp[q], bf16_to_float(A[(size_t)q * r + i]), acc);
+      for (int q = pr; q < G; q += 8) acc = fmaf(xp[q], bf16_to_float(As[(size_t)q * 32 + il]), acc);
+    } else {
+#pragma unroll 4
+      for (int q = pr; q < G; q += 8) acc = fmaf(xp[q], bf16_to_float(A[(size_t)q * r + i]), acc);
+    }
   }
   part[pr][il] = acc;
   __syncthreads();
@@ -216,7 +250,7 @@ int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv
                   float* xp, float* T, __nv_bfloat16* Tb, cudaStream_t st) {
   if (M == 0) return QALORA_OK;
   const size_t smem = sh.r >= 8 ? pool16_smem_bytes(sh.G, sh.r) : 0;
-  const bool rows_path = M >= 64 && (sh.g == 32 || sh.g == 64 || sh.g == 128) && sh.K % 256 == 0 &&
+  const bool rows_path = M >= 512 && (sh.g == 32 || sh.g == 64 || sh.g == 128) && sh.K % 256 == 0 &&
                          sh.r >= 8 && smem <= kPool16MaxSmem;
   if (rows_path) {
     static PerDeviceOnce smem_limit;                     // once per device: allow more than the default 48 KiB
@@ -233,7 +267,10 @@ int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv
     else pool_T_rows_kernel<16><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
   } else {
     dim3 grid((unsigned)M, (unsigned)((sh.r + 31) / 32 > 0 ? (sh.r + 31) / 32 : 1));
-    pool_T_kernel<<<grid, POOL_THREADS, sh.G * sizeof(float), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G, sh.r, sh.s);
+    const size_t xp_bytes = ((size_t)sh.G * sizeof(float) + 15) / 16 * 16, a_bytes = (size_t)sh.G * 32 * sizeof(__nv_bfloat16);
+    const int a_in_smem = (sh.r > 0 && a_bytes <= kPoolASliceMax) ? 1 : 0;
+    pool_T_kernel<<<grid, POOL_THREADS, xp_bytes + (a_in_smem ? a_bytes : 0), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G, sh.r, sh.s,
+                                                                                    a_in_smem);
   }
   count_launch();
   return cuda_status(cudaGetLastError());

@@ -107,6 +107,14 @@ SMALL = [
     ("parts4", 2048, 256, 32, 4, 16, 1.0, 40),
     ("parts3", 1536, 384, 64, 3, 24, 0.75, 300),
     ("parts2", 4096, 128, 128, 2, 8, 1.5, 33),
+    # 17 to 128 tokens on shapes with N % 256 == 0: the kernel with the tokens as the MMA rows (64- and
+    # 128-row activation tiles, ragged counts, every bit width and group size, adapter ranks that are
+    # not a multiple of the 64-wide adapter step)
+    ("midm2", 512, 512, 128, 2, 8, 2.0, 100),
+    ("midm3", 640, 256, 32, 3, 40, 1.0, 64),
+    ("midm4_128", 256, 512, 64, 4, 16, 1.0, 128),
+    ("midm4_33", 4096, 256, 32, 4, 72, 0.5, 33),
+    ("midm4_r64_65", 1024, 768, 32, 4, 64, 1.0, 65),
     # many tokens, several channel tiles, ragged token count
     ("pair4", 512, 256, 32, 4, 16, 1.0, 700),
     ("pair3", 384, 512, 64, 3, 24, 0.75, 530),
@@ -401,8 +409,10 @@ def test_step_from_host_buffers_matches_device_calls():
 
 def test_chunked_step_from_host_buffers():
     # 2348 rows: three pipelined chunks (1024, 1024 and a ragged 300).  Rows are independent in y
-    # and dx, so those match the whole-batch device calls bit for bit; dA and dB are sums over the
-    # chunks and are held to the oracle's tolerance.
+    # and dx, so dx and the full chunks of y match the whole-batch device calls bit for bit; the
+    # 300-row chunk pools its input with the few-row kernel (another summation order of the rank-r
+    # intermediate), so its y is held to the oracle's tolerance and to a few bf16 steps of the
+    # whole-batch result.  dA and dB are sums over the chunks and are held to the oracle's tolerance.
     cfg = LayerConfig("hostchunks", 512, 384, 64, 4, 64, 1.0, 2348, seed=22)
     layer = GpuLayer(cfg)
     y = layer.forward()
@@ -415,12 +425,16 @@ def test_chunked_step_from_host_buffers():
     codes, alpha, beta = check_quantize(layer)
     xf, Af, Bf, dyf = (to_f64(layer.cpu[k]) for k in ("x", "A", "B", "dy"))
     _, dA_ref, dB_ref = O.backward(xf, dyf, codes, alpha, beta, cfg.group_size, Af, Bf, cfg.scale)
+    y_ref = O.forward(xf, codes, alpha, beta, cfg.group_size, Af, Bf, cfg.scale)
     for _ in range(2):  # the second call reuses the library's streams and events
         hy.zero_(); hdx.zero_(); hdA.zero_(); hdB.zero_()
         Q.qalora_step_host(layer.d, cfg.tokens, hx, hdy, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"],
                            hy, hdx, hdA, hdB, staging)
         torch.cuda.synchronize()
         assert Q.workspace_status(staging) == 0
-        assert torch.equal(hy, y.cpu()) and torch.equal(hdx, dx.cpu())
+        assert torch.equal(hy[:2048], y[:2048].cpu()) and torch.equal(hdx, dx.cpu())
+        assert rel_err(hy[2048:].float().numpy(), y_ref[2048:]) <= TOL
+        assert rel_err(hy[2048:].float().numpy(), y[2048:].float().cpu().numpy()) <= 2e-3
         assert rel_err(hdA.numpy(), dA_ref) <= TOL and rel_err(hdB.numpy(), dB_ref) <= TOL
-        assert rel_err(hdA.numpy(), dA.cpu().numpy()) <= 1e-5 and rel_err(hdB.numpy(), dB.cpu().numpy()) <= 1e-5
+        # dB contracts the bf16 copy of the rank-r intermediate: a few of the tail chunk's entries round the other way
+        assert rel_err(hdA.numpy(), dA.cpu().numpy()) <= 1e-5 and rel_err(hdB.numpy(), dB.cpu().numpy()) <= 5e-4
