@@ -14,8 +14,9 @@
 //             MN-major operand: it goes to shared memory in the 128-byte
 //             swizzled MN-major layout and the MMA takes A from smem.
 // The same packed bytes serve both products.  The adapter is folded in as extra
-// reduction steps of width r: forward appends T = s*pool(x)*A against B, dx
-// appends dT = s*dy*B^T against the group-expanded A.
+// reduction steps of width r: forward appends T = s*pool(x)*A against B (a tile of
+// B[r][n] as it lies in memory IS an MN-major operand: one TMA copy, no thread
+// touches it), dx appends dT = s*dy*B^T against the group-expanded A.
 //
 // Warp roles (768 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
 // owner, warps 4-19 = four dequantizing warpgroups (each owns every fourth
@@ -43,7 +44,7 @@ constexpr int THREADS = 128 + 128 * DQ_GROUPS + 128;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_COL = 0;       // accumulator: columns [0, 256); dx keeps a second one at [256, 512)
 constexpr int A_COL = 256;       // forward operand ring: 8 slots of 32 columns
-constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx)
+constexpr uint32_t ATILE_BYTES = TILE_C * TILE_J * 2;    // 16 KiB dequantized tile (dx); tile of B (forward)
 
 enum Mode { FWD = 0, DX = 1 };
 
@@ -129,11 +130,11 @@ struct Smem {
   static constexpr uint32_t CSTAGE_BYTES = ((CODE_BYTES + QP_BYTES + 127) / 128) * 128;
   static constexpr uint32_t OUT_BYTES = 32 * TILE_C * 2;                         // 32 tokens x 128 channels bf16
   static constexpr uint32_t OFF_X = 0;
-  static constexpr uint32_t OFF_A = NX * ACT_BYTES;                              // dx only
-  static constexpr uint32_t OFF_C = OFF_A + (MODE == DX ? NX * ATILE_BYTES : 0);
+  static constexpr uint32_t OFF_A = NX * ACT_BYTES;                              // dx: operand ring; forward: the adapter's tile of B
+  static constexpr uint32_t OFF_C = OFF_A + (MODE == DX ? NX * ATILE_BYTES : ATILE_BYTES);
   static constexpr uint32_t OFF_OUT = OFF_C + NC * CSTAGE_BYTES;
   static constexpr uint32_t OFF_BARS = OFF_OUT + NOUT * OUT_BYTES;
-  static constexpr int NBARS = 2 * NB + 2 * NC + 2 * NACC;
+  static constexpr int NBARS = 2 * NB + 2 * NC + 2 * NACC + 1;                   // + "tile of B free" (forward)
   static constexpr uint32_t TOTAL = OFF_BARS + 8 * NBARS + 64 + 1024;            // + alignment slack
 };
 
@@ -141,8 +142,9 @@ struct Smem {
 template <int BITS, int MODE, bool PARTS, int TT>
 __global__ void __launch_bounds__(THREADS, 1)
 qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_constant__ CUtensorMap lora_map,
-                 const __grid_constant__ CUtensorMap out_map, const __grid_constant__ CUtensorMap codes_map,
-                 const __grid_constant__ CUtensorMap qp_map, const TcParams p) {
+                 const __grid_constant__ CUtensorMap lb_map, const __grid_constant__ CUtensorMap out_map,
+                 const __grid_constant__ CUtensorMap codes_map, const __grid_constant__ CUtensorMap qp_map,
+                 const TcParams p) {
   using S = Smem<BITS, MODE, TT>;
   constexpr int WORDS = S::WORDS;
   constexpr int NX = S::NX, NB = S::NB, NC = S::NC;
@@ -159,6 +161,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   constexpr int NACC = S::NACC;
   auto bar_acc_full = [&](int b) { return bar_base + 8u * (2 * NB + 2 * NC + b); };
   auto bar_acc_empty = [&](int b) { return bar_base + 8u * (2 * NB + 2 * NC + NACC + b); };
+  const uint32_t bar_lb_empty = bar_base + 8u * (2 * NB + 2 * NC + 2 * NACC);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + S::OFF_BARS + 8 * S::NBARS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_BARS + 8 * S::NBARS + 8);
 
@@ -170,10 +173,12 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     for (int s = 0; s < NB; ++s) { ptx::mbar_init(bar_full_x(s), 1 + 4); ptx::mbar_init(bar_empty_x(s), 1); }
     for (int s = 0; s < NC; ++s) { ptx::mbar_init(bar_full_c(s), 1); ptx::mbar_init(bar_empty_c(s), 4 * S::IPS); }
     for (int b = 0; b < NACC; ++b) { ptx::mbar_init(bar_acc_full(b), 1); ptx::mbar_init(bar_acc_empty(b), 4); }
+    ptx::mbar_init(bar_lb_empty, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&act_map);
     if (p.lora_iters > 0) ptx::prefetch_tensormap(&lora_map);
+    if (MODE == FWD && p.lora_iters > 0) ptx::prefetch_tensormap(&lb_map);
     ptx::prefetch_tensormap(&out_map);
     ptx::prefetch_tensormap(&codes_map);
     ptx::prefetch_tensormap(&qp_map);
@@ -193,21 +198,35 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   if (warp == 0) {
     // ------------------------------------------------- activation producer ----
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0, nlb = 0;                      // steps / adapter steps so far
       bool ok = true;
       for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x) {
         const TcSegment sg = tc_segment<PARTS>(p, vt);
         const int m0 = (sg.tile / p.c_tiles) * TT;
+        const int c0 = (sg.tile % p.c_tiles) * TILE_C;
         for (int j = 0; j < sg.n_steps; ++j, ++it) {
           const int i = tc_step<PARTS>(p, sg, j);
           const int s = it % NX, sb = it % NB;
           // the tile slot was last used by step it - NX: wait until that step has been multiplied
           if (it >= (uint32_t)NX && !(ok = ptx::mbar_wait(bar_empty_x((it - NX) % NB), ((it - NX) / NB) & 1, abort_flag))) break;
-          ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES);
-          if (i < p.red_iters)
+          if (i < p.red_iters) {
+            ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES);
             ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &act_map, i * TILE_J, m0, bar_full_x(sb));
-          else
+          } else if (MODE == FWD) {
+            // adapter step: the tile of T and, as the other operand, rows r0 .. r0 + 63 of B for the
+            // tile's 128 channels (two boxes of 64 channels; rows beyond r arrive as zeros).  The one
+            // buffer is free once the adapter step before this one has been multiplied.
+            const int r0 = (i - p.red_iters) * TILE_J;
+            if (!(ok = ptx::mbar_wait(bar_lb_empty, (nlb & 1) ^ 1, abort_flag))) break;
+            ++nlb;
+            ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES + ATILE_BYTES);
+            ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &lora_map, r0, m0, bar_full_x(sb));
+            ptx::tma_load_2d(smem_base + S::OFF_A, &lb_map, c0, r0, bar_full_x(sb));
+            ptx::tma_load_2d(smem_base + S::OFF_A + ATILE_BYTES / 2, &lb_map, c0 + 64, r0, bar_full_x(sb));
+          } else {
+            ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES);
             ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &lora_map, (i - p.red_iters) * TILE_J, m0, bar_full_x(sb));
+          }
         }
       }
     }
@@ -237,7 +256,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     // ---------------------------------------------------------- MMA issuer ----
     if (lane == 0) {
       constexpr uint32_t IDESC_MAIN = ptx::idesc_bf16(TILE_C, TT, MODE == DX, false);
-      constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(TILE_C, TT, false, false);
+      constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(TILE_C, TT, MODE == FWD, false);   // forward: the tile of B is MN-major
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       // Issuing one tcgen05.mma costs this thread about 110 cycles and the four MMAs of a step
@@ -264,9 +283,14 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           const uint32_t next_bar = bar_full_x((it + 1) % NB), next_par = ((it + 1) / NB) & 1;
           const uint32_t acc = j > 0 ? 1u : 0u;
           // the commit frees the activation tile AND the operand slot
-          if (MODE == FWD) {
+          if (MODE == FWD && j < sg.n_main) {
             ready = ptx::mma4_ts_commit_probe<2>(acc_tmem, tmem_base + A_COL + sb * 32, bdesc, IDESC_MAIN, acc,
                                                  bar_empty_x(sb), next_bar, next_par) != 0;
+          } else if (MODE == FWD) {
+            // adapter step: 64-channel blocks of B 8 KiB apart (LBO), 8-row groups 1 KiB apart (SBO); 2 KiB per K = 16
+            ready = ptx::mma4_ss_commit_probe<128, 2>(acc_tmem, ptx::smem_desc(smem_base + S::OFF_A, 8192, 1024), bdesc,
+                                                      IDESC_LORA, acc, bar_empty_x(sb), next_bar, next_par) != 0;
+            ptx::mma_commit(bar_lb_empty);
           } else if (j < sg.n_main) {
             // MN-major A: 64-channel blocks 8 KiB apart (LBO), 8-column groups 1 KiB apart (SBO); 2 KiB per step
             ready = ptx::mma4_ss_commit_probe<128, 2>(acc_tmem, ptx::smem_desc(as, 8192, 1024), bdesc, IDESC_MAIN,
@@ -307,34 +331,25 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         if (i < p.red_iters && !(ok = ptx::mbar_wait(bar_full_c(sc), (cst / NC) & 1, abort_flag))) break;
         const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         if (MODE == FWD) {
-          ptx::tc_fence_after();
-          const int row = quarter * 32 + lane;   // out channel within the tile = TMEM lane
+          // (an adapter step needs nothing from this group: its operands both come by TMA; the
+          // group still owns the step's slot of the ring and signs it off below)
+          if (i < p.red_iters) {
+            ptx::tc_fence_after();
+            const int row = quarter * 32 + lane;   // out channel within the tile = TMEM lane
 #pragma unroll
-          for (int half = 0; half < 2; ++half) { // the two 32-channel blocks of the step
-            uint32_t v[16];
-            if (i < p.red_iters) {
+            for (int half = 0; half < 2; ++half) { // the two 32-channel blocks of the step
+              uint32_t v[16];
               const int kbl = kb_base + half;
               const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (kbl * TILE_C + row) * WORDS;
               uint32_t w[WORDS];
               load_unit<WORDS>(cw, w);
               const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[(kbl >> qsh) * TILE_C + row];
               dequant_unit<BITS>(w, ab, dk, v);
-            } else {
-              // adapter step: row c of the operand is B[r0 + 0..63][c]; this thread packs 32 of them
-              const int r0 = (i - p.red_iters) * TILE_J + half * 32;
-              const __nv_bfloat16* bp = p.lora + (size_t)r0 * p.N + c0 + row;
-#pragma unroll
-              for (int q = 0; q < 16; ++q) {
-                const int ra = r0 + 2 * q;
-                const uint32_t lo = ra < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q) * p.N) : 0u;
-                const uint32_t hi = ra + 1 < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q + 1) * p.N) : 0u;
-                v[q] = lo | (hi << 16);
-              }
+              ptx::tmem_st16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL + sa * 32 + half * 16, v);
             }
-            ptx::tmem_st16(tmem_base + ((uint32_t)(quarter * 32) << 16) + A_COL + sa * 32 + half * 16, v);
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before();
           }
-          ptx::tmem_wait_st();
-          ptx::tc_fence_before();
         } else {
           uint8_t* atile = smem + S::OFF_A + sa * ATILE_BYTES;
 #pragma unroll
@@ -544,7 +559,9 @@ namespace {
 template <int BITS, int MODE, bool PARTS, int TT>
 int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
   using S = Smem<BITS, MODE, TT>;
-  CUtensorMap out, cmap, qmap;
+  CUtensorMap out, cmap, qmap, lb = act;
+  // forward with adapter: B [r][N] in boxes of 64 channels x 64 rows (rows beyond r read as zero)
+  if (MODE == FWD && p.r > 0 && !make_act_map(&lb, p.lora, p.r, p.N, TILE_J)) return QALORA_ERR_CUDA;
   if (!make_out_map(&out, p.out, p.M, p.ld_out)) return QALORA_ERR_CUDA;
   if (!make_codes_map(&cmap, p.codes, p.K, p.N, BITS, S::TILE_NC, 4)) return QALORA_ERR_CUDA;
   if (!make_qp_map(&qmap, p.qparams, p.K / p.g, p.N, S::TILE_NC, p.qp_rows)) return QALORA_ERR_CUDA;
@@ -557,7 +574,7 @@ int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams&
   const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
   {
     MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
-    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, out, cmap, qmap, p);
+    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, lb, out, cmap, qmap, p);
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
