@@ -325,6 +325,24 @@ int qalora_profile_next_main_kernel(void* start_event, void* stop_event);
  * string. */
 const char* qalora_main_kernel_name(void);
 
+/* Bounds-check build.  The same sources compiled with -DQALORA_DEBUG (libqalora_debug.so)
+ * test every index, offset, tensor-memory column and copy coordinate a kernel computes
+ * against its limit before the access, skip an access that would fall outside, and put a
+ * 256-byte guard behind every region of a workspace (qalora_workspace_bytes and the other
+ * size queries grow accordingly), written before a pass and verified after it.  Nothing
+ * faults: failures are recorded.  qalora_debug_checks() returns 1 in that build and 0 in the
+ * ordinary one.  qalora_debug_report() waits for the current device's work, copies the
+ * record to `words8` (HOST array of 8 int32) and clears it:
+ *   [0] flags: 2 = an index check failed, 4 = a guard word was overwritten;
+ *   [1] first failed check, source file ordinal * 100000 + line;  [2], [3] its index (low,
+ *   high word);  [4], [5] its limit;  [6] failed checks in all;  [7] first overwritten guard,
+ *   region ordinal * 65536 + word + 1.
+ * In the ordinary build it writes zeros.  Both are host functions; the report is the one
+ * call of this library that synchronizes the device, and the bounds-check build the one
+ * that allocates device memory (the 32-byte record, once per device). */
+int qalora_debug_checks(void);
+int qalora_debug_report(int32_t* words8);
+
 #ifdef __cplusplus
 }
 #endif

@@ -12,7 +12,11 @@ from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32,
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libqalora.so")
+# QALORA_LIBRARY=debug selects the bounds-check build (libqalora_debug.so, made by
+# `python -m paper_2309_14717_b200.build --debug`); anything else the ordinary library.
+DEBUG_LIBRARY = os.environ.get("QALORA_LIBRARY", "") == "debug"
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                         "libqalora_debug.so" if DEBUG_LIBRARY else "libqalora.so")
 
 OP_FORWARD, OP_BACKWARD, OP_TRAIN = 0, 1, 2
 
@@ -25,6 +29,7 @@ EXPORTS = (
     "qalora_dequantize", "qalora_qparams_from_zero_point", "qalora_qparams_to_zero_point",
     "qalora_forward_group_workspace_bytes", "qalora_forward_group",
     "qalora_forward_train", "qalora_backward_train",
+    "qalora_debug_checks", "qalora_debug_report",
 )
 
 STATIC_SCRATCH_BYTES = 1 << 20
@@ -66,6 +71,10 @@ def load() -> ctypes.CDLL:
     D = POINTER(QaloraDesc)
     lib.qalora_version.restype = c_int
     lib.qalora_version.argtypes = []
+    lib.qalora_debug_checks.restype = c_int
+    lib.qalora_debug_checks.argtypes = []
+    lib.qalora_debug_report.restype = c_int
+    lib.qalora_debug_report.argtypes = [POINTER(c_int32)]
     lib.qalora_status_string.restype = c_char_p
     lib.qalora_status_string.argtypes = [c_int]
     lib.qalora_packed_bytes.restype = c_int
@@ -317,6 +326,19 @@ def qalora_adamw_step(hyper: AdamwHyper, n: int, grad, param, exp_avg, exp_avg_s
 
 def qalora_kernel_launches() -> int:
     return int(load().qalora_kernel_launches())
+
+
+def qalora_debug_checks() -> bool:
+    """True when the loaded library is the bounds-check build."""
+    return bool(load().qalora_debug_checks())
+
+
+def qalora_debug_report() -> list:
+    """Waits for the device, returns the bounds-check build's eight record words and clears them
+    (all zero when no check failed and no guard word was overwritten; always zero in the ordinary build)."""
+    words = (c_int32 * 8)()
+    _check("qalora_debug_report", load().qalora_debug_report(words))
+    return list(words)
 
 
 def qalora_profile_next_main_kernel(start_event, stop_event):

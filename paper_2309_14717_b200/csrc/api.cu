@@ -1,4 +1,5 @@
 // C-ABI entry points: argument checks, scratch layout and kernel dispatch.
+#define QALORA_TU 1
 #include <atomic>
 #include <mutex>
 
@@ -42,6 +43,66 @@ int device_sm_count() {
   return n;
 }
 
+// ---- bounds-check build: record words and workspace guards ---------------------------
+#ifdef QALORA_DEBUG
+int* debug_words() {
+  static std::atomic<int*> words[kMaxDevices];        // zero-initialized
+  static std::mutex mu;
+  const int dev = current_device();
+  if (dev < 0) return nullptr;
+  int* p = words[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
+    std::lock_guard<std::mutex> lock(mu);
+    p = words[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
+      if (cudaMalloc(&p, kDebugWords * sizeof(int)) != cudaSuccess) return nullptr;
+      if (cudaMemset(p, 0, kDebugWords * sizeof(int)) != cudaSuccess) { cudaFree(p); return nullptr; }
+      words[dev].store(p, std::memory_order_release);
+    }
+  }
+  return p;
+}
+
+struct GuardList { unsigned long long at[12]; int n; };
+
+// one warp per guard, two words per lane
+static __global__ void guard_fill_kernel(unsigned char* ws, GuardList gl) {
+  const int gi = blockIdx.x;
+  unsigned* g = reinterpret_cast<unsigned*>(ws + gl.at[gi]);
+  for (unsigned w = threadIdx.x; w < kGuardBytes / 4; w += blockDim.x) g[w] = kGuardPattern;
+}
+static __global__ void guard_verify_kernel(const unsigned char* ws, GuardList gl, int* dbg) {
+  const int gi = blockIdx.x;
+  const unsigned* g = reinterpret_cast<const unsigned*>(ws + gl.at[gi]);
+  for (unsigned w = threadIdx.x; w < kGuardBytes / 4; w += blockDim.x) {
+    if (g[w] != kGuardPattern) {
+      atomicCAS(dbg + DBG_GUARD, 0, gi * 65536 + (int)w + 1);
+      atomicOr(dbg + DBG_FLAGS, kDebugGuardFlag);
+    }
+  }
+}
+static GuardList guard_list(const Workspace& ws) {
+  GuardList gl{};
+  gl.n = ws.n_guard;
+  for (int i = 0; i < ws.n_guard; ++i) gl.at[i] = ws.guard[i];
+  return gl;
+}
+int debug_fill_guards(const Workspace& ws, void* workspace, cudaStream_t st) {
+  if (ws.n_guard == 0) return QALORA_OK;
+  guard_fill_kernel<<<ws.n_guard, 32, 0, st>>>(static_cast<unsigned char*>(workspace), guard_list(ws));
+  return cuda_status(cudaGetLastError());
+}
+int debug_verify_guards(const Workspace& ws, const void* workspace, cudaStream_t st) {
+  int* dbg = debug_words();
+  if (ws.n_guard == 0 || dbg == nullptr) return dbg == nullptr ? QALORA_ERR_CUDA : QALORA_OK;
+  guard_verify_kernel<<<ws.n_guard, 32, 0, st>>>(static_cast<const unsigned char*>(workspace), guard_list(ws), dbg);
+  return cuda_status(cudaGetLastError());
+}
+#else
+int debug_fill_guards(const Workspace&, void*, cudaStream_t) { return QALORA_OK; }
+int debug_verify_guards(const Workspace&, const void*, cudaStream_t) { return QALORA_OK; }
+#endif
+
 int check_desc(const qalora_desc* d, Shape* sh) {
   if (d == nullptr) return QALORA_ERR_NULL_POINTER;
   if (d->d_in <= 0 || d->d_out <= 0 || d->group_size <= 0 || d->rank < 0) return QALORA_ERR_INVALID_ARG;
@@ -67,7 +128,12 @@ static bool takes_midm(const Shape& sh, int64_t m) { return m > kSmallM && m <= 
 Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   Workspace w{};
   size_t off = 0;
-  auto take = [&](size_t bytes) { size_t at = off; off += round_up(bytes, 256); return at; };
+  auto take = [&](size_t bytes) {
+    size_t at = off;
+    off += round_up(bytes, 256);
+    if (kDebugBuild) { w.guard[w.n_guard++] = off; off += kGuardBytes; }
+    return at;
+  };
   const size_t M = (size_t)(m > 0 ? m : 0);
   const bool train = op == QALORA_OP_TRAIN;           // one workspace for a forward + backward pair
   const bool bwd = op == QALORA_OP_BACKWARD || train;
@@ -126,6 +192,10 @@ int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const vo
 // word at the head of the workspace is zeroed before the first kernel that can raise it when
 // `reset_status` is set (a public call); qalora_step_host zeroes it once for all its chunks
 // and passes false, so that a time-out raised by an earlier chunk survives to the end.
+static int forward_dispatch(const Shape& sh, const Workspace& ws, int64_t m, const void* x, const void* codes,
+                            const float* qparams, const void* A, const void* B, void* y, void* workspace,
+                            cudaStream_t stream, bool reset_status, int layout_op);
+
 int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void* codes, const float* qparams,
                    const void* A, const void* B, void* y, void* workspace, void* cuda_stream, bool reset_status,
                    int layout_op) {
@@ -134,6 +204,18 @@ int forward_launch(const qalora_desc* desc, int64_t m, const void* x, const void
   if (st != QALORA_OK) return st;
   const Workspace ws = workspace_layout(sh, m, layout_op);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // (bounds-check build: the guards behind the workspace's regions are set before the pass and
+  // looked at after its last kernel; both calls are empty otherwise)
+  if ((st = debug_fill_guards(ws, workspace, stream)) != QALORA_OK) return st;
+  st = forward_dispatch(sh, ws, m, x, codes, qparams, A, B, y, workspace, stream, reset_status, layout_op);
+  if (st == QALORA_OK) st = debug_verify_guards(ws, workspace, stream);
+  return st;
+}
+
+static int forward_dispatch(const Shape& sh, const Workspace& ws, int64_t m, const void* x, const void* codes,
+                            const float* qparams, const void* A, const void* B, void* y, void* workspace,
+                            cudaStream_t stream, bool reset_status, int layout_op) {
+  int st = QALORA_OK;
   char* wsp = static_cast<char*>(workspace);
   float* T = reinterpret_cast<float*>(wsp + ws.T);
   __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
@@ -207,6 +289,8 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
   }
   int* status = reinterpret_cast<int*>(wsp + ws.status);
   if (reset_status && (st = cuda_status(cudaMemsetAsync(status, 0, sizeof(int), stream))) != QALORA_OK) return st;
+  // (bounds-check build: a pass on its own sets the guards; after qalora_forward_train they are already set)
+  if (!pooled && (st = debug_fill_guards(ws, workspace, stream)) != QALORA_OK) return st;
   const bool aux_tc = m > kSmallM && tc_aux_supported(sh, m);
   if (aux_tc) st = launch_tc_dT(sh, m, dyb, Bb, dT, dTb, status, stream);
   else st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream);
@@ -237,7 +321,7 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
     }
     if (st != QALORA_OK) return st;
   }
-  return QALORA_OK;
+  return debug_verify_guards(ws, workspace, stream);
 }
 
 }  // namespace qalora
@@ -268,6 +352,52 @@ int qalora_debug_expire_next_few_token_wait(int stages, uint64_t limit_ns) {
   if (limit_ns == 0 || limit_ns > 2000000000ull) return QALORA_ERR_INVALID_ARG;
   arm_few_token_wait_expiry(stages, limit_ns);
   return QALORA_OK;
+}
+
+int qalora_debug_checks(void) { return kDebugBuild ? 1 : 0; }
+
+// Test hook, not declared in the public header: shows that the bounds-check build's record
+// works, without any access outside a buffer.  `buf512` is 512 bytes of device memory used as
+// a one-region workspace (region [0, 256), guard [256, 512)).  The guard is filled, one kernel
+// then (a) asks for index 5 of an array of 4, which the check refuses and records, and (b)
+// overwrites word 3 of the guard, which lies inside the buffer; the verification finds it.
+// Afterwards qalora_debug_report() reads flags 6, index 5, limit 4, one failed check, guard 4.
+#ifdef QALORA_DEBUG
+static __global__ void debug_selftest_kernel(unsigned* buf, int* dbg) {
+  if (QALORA_CHECK(dbg, 5, 4)) buf[5] = 0u;          // never taken
+  buf[kGuardBytes / 4 + 3] = 0u;                      // inside the buffer: the guard's word 3
+}
+#endif
+int qalora_debug_selftest(void* buf512, void* cuda_stream) {
+#ifdef QALORA_DEBUG
+  if (buf512 == nullptr) return QALORA_ERR_NULL_POINTER;
+  if (!aligned16(buf512)) return QALORA_ERR_MISALIGNED;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Workspace ws{};
+  ws.guard[0] = kGuardBytes;
+  ws.n_guard = 1;
+  int* dbg = debug_words();
+  if (dbg == nullptr) return QALORA_ERR_CUDA;
+  int rc = debug_fill_guards(ws, buf512, st);
+  if (rc != QALORA_OK) return rc;
+  debug_selftest_kernel<<<1, 1, 0, st>>>(static_cast<unsigned*>(buf512), dbg);
+  if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
+  return debug_verify_guards(ws, buf512, st);
+#else
+  (void)buf512; (void)cuda_stream;
+  return QALORA_ERR_INVALID_ARG;
+#endif
+}
+
+int qalora_debug_report(int32_t* words8) {
+  if (words8 == nullptr) return QALORA_ERR_NULL_POINTER;
+  for (int i = 0; i < kDebugWords; ++i) words8[i] = 0;
+  if (!kDebugBuild) return QALORA_OK;
+  int* dbg = debug_words();
+  if (dbg == nullptr) return QALORA_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return QALORA_ERR_CUDA;
+  if (cudaMemcpy(words8, dbg, kDebugWords * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return QALORA_ERR_CUDA;
+  return cuda_status(cudaMemset(dbg, 0, kDebugWords * sizeof(int)));
 }
 
 const char* qalora_status_string(int status) {

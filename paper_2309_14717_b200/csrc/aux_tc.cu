@@ -11,6 +11,7 @@
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
 // owner, warps 2-5 = epilogue (TMEM lane quarter = warp % 4).  Waits are bounded.
+#define QALORA_TU 5
 #include <mutex>
 
 #include "common.cuh"
@@ -49,6 +50,7 @@ struct AuxParams {
   float* out_f32;         // dT: dT [M][r] (may be null);  dB: partial [splits][r][N]
   __nv_bfloat16* out_bf16;// dT: dTb [M][r]
   int* status;
+  int* dbg;               // record words of the bounds-check build (null otherwise)
 };
 
 template <int MODE>
@@ -123,13 +125,19 @@ aux_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__
           const int s = it % STAGES;
           if (!(ok = ptx::mbar_wait(bar_empty(s), ((it / STAGES) & 1) ^ 1, abort_flag))) break;
           const uint32_t stage = smem_base + s * C::STAGE_BYTES;
+          // (bounds-check build: the stage lies inside the ring, the copies start inside their matrices)
+          QALORA_CHECK(p.dbg, (s + 1) * C::STAGE_BYTES - 1, STAGES * C::STAGE_BYTES);
           if (MODE == AUX_DT) {
+            QALORA_CHECK(p.dbg, i * STEP, p.N);
+            QALORA_CHECK(p.dbg, (long long)item * C::TILE_N, p.M);
             ptx::mbar_arrive_expect_tx(bar_full(s), C::STAGE_BYTES);
             ptx::tma_load_2d(stage, &a_map, i * STEP, 0, bar_full(s));                       // B[0..127][n..n+63]
             ptx::tma_load_2d(stage + C::A_BYTES, &b_map, i * STEP, item * C::TILE_N, bar_full(s));  // dy[m..][n..]
           } else {
             const int nt = item % p.n_tiles, split = item / p.n_tiles;
             const int m = (int)((long long)split * p.rows_per_split) + i * STEP;
+            QALORA_CHECK(p.dbg, m, p.M);
+            QALORA_CHECK(p.dbg, nt * C::TILE_N, p.N);
             ptx::mbar_arrive_expect_tx(bar_full(s), (second_block ? 16384u : 8192u) + C::B_BYTES);
             ptx::tma_load_2d(stage, &a_map, 0, m, bar_full(s));                              // T[m..m+63][0..63]
             if (second_block) ptx::tma_load_2d(stage + 8192, &a_map, 64, m, bar_full(s));
@@ -182,6 +190,7 @@ aux_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__
 #pragma unroll 1
       for (int col = 0; col < C::TILE_N; col += 32) {
         uint32_t v[32];
+        if (!QALORA_CHECK(p.dbg, col + 31, C::TMEM_COLS)) continue;
         ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + col, v);
         ptx::tmem_wait_ld();
         if (row >= p.r) continue;
@@ -191,6 +200,7 @@ aux_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__
           for (int t = 0; t < 32; ++t) {
             if (m0 + t >= p.M) break;
             const float val = iters > 0 ? p.s * __uint_as_float(v[t]) : 0.0f;
+            if (!QALORA_CHECK(p.dbg, (size_t)(m0 + t) * p.r + row, (size_t)p.M * p.r)) continue;
             if (p.out_f32 != nullptr) p.out_f32[(size_t)(m0 + t) * p.r + row] = val;
             p.out_bf16[(size_t)(m0 + t) * p.r + row] = __float2bfloat16_rn(val);
           }
@@ -201,6 +211,7 @@ aux_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__
 #pragma unroll
           for (int t = 0; t < 32; t += 4) {
             if (n0 + t >= p.N) break;                   // N is a multiple of 8
+            if (!QALORA_CHECK(p.dbg, ((size_t)split * p.r + row) * p.N + n0 + t + 3, (size_t)p.splits * p.r * p.N)) break;
             float4 o;
             o.x = iters > 0 ? __uint_as_float(v[t]) : 0.0f;
             o.y = iters > 0 ? __uint_as_float(v[t + 1]) : 0.0f;
@@ -284,7 +295,7 @@ int launch_tc_dT(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const __nv
   p.M = M; p.N = sh.N; p.r = sh.r; p.s = sh.s;
   p.items = (int)((M + AuxCfg<AUX_DT>::TILE_N - 1) / AuxCfg<AUX_DT>::TILE_N);
   p.red_iters = sh.N / STEP;
-  p.out_f32 = dT; p.out_bf16 = dTb; p.status = status;
+  p.out_f32 = dT; p.out_bf16 = dTb; p.status = status; p.dbg = debug_words();
   return launch_aux<AUX_DT>(a, b, p, st);
 }
 
@@ -314,7 +325,7 @@ int launch_tc_dB_partials(const Shape& sh, int64_t M, const __nv_bfloat16* Tb, c
   p.rows_per_split = rows;
   p.splits = (int)((M + rows - 1) / rows);
   p.items = p.n_tiles * p.splits;
-  p.out_f32 = partial; p.status = status;
+  p.out_f32 = partial; p.status = status; p.dbg = debug_words();
   *splits_out = p.splits;
   return launch_aux<AUX_DB>(a, b, p, st);
 }

@@ -7,6 +7,7 @@
 
 #include <atomic>
 
+#include "debug.cuh"
 #include "qalora.h"
 
 namespace qalora {
@@ -37,8 +38,15 @@ struct Workspace {
   size_t partial_bytes;
   size_t fwd_parts; // float  [parts][M][N] partial results of a forward reduction cut into parts (forward)
   size_t total;
+  // bounds-check build only: a guard of kGuardBytes follows every region (guard[i] = its offset)
+  size_t guard[12];
+  int n_guard;
 };
 Workspace workspace_layout(const Shape& sh, int64_t m, int op);
+// Bounds-check build: fill the workspace's guards / verify them (into the record words) on `st`.
+// Both do nothing and return QALORA_OK in the ordinary build.
+int debug_fill_guards(const Workspace& ws, void* workspace, cudaStream_t st);
+int debug_verify_guards(const Workspace& ws, const void* workspace, cudaStream_t st);
 
 // The public forward / backward in two halves (api.cu): checks that launch nothing, and the
 // launches with a say on whether the workspace's status word is cleared first.

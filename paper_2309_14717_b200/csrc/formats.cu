@@ -1,6 +1,7 @@
 // Format conversions around the packed layer: dequantization of the whole weight matrix
 // (Eq. 1) and the zero-point form of Algorithm 1 (W~ = alpha * (c - z)) in both directions.
 // All three are element-wise and bound by HBM.
+#define QALORA_TU 9
 #include "common.cuh"
 
 namespace qalora {
@@ -19,11 +20,16 @@ template <> __device__ __forceinline__ void store_weight<__nv_bfloat16>(__nv_bfl
 template <int BITS, typename TO>
 __global__ void __launch_bounds__(FMT_THREADS)
 dequantize_kernel(const uint32_t* __restrict__ codes, const float2* __restrict__ qparams, TO* __restrict__ W,
-                  int N, int g) {
+                  int N, int g, int* dbg) {
   constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   const int n = blockIdx.x * FMT_THREADS + threadIdx.x;
   const int kb = blockIdx.y;
   if (n >= N) return;
+  // gridDim.y = K / 32 k-block rows: the unit read, the (alpha, beta) pair and the last of the 32 rows written
+  if (!QALORA_CHECK(dbg, ((size_t)kb * N + n) * WORDS + WORDS - 1, (size_t)gridDim.y * N * WORDS) ||
+      !QALORA_CHECK(dbg, (size_t)(kb * 32 / g) * N + n, (size_t)(gridDim.y * 32 / g) * N) ||
+      !QALORA_CHECK(dbg, ((size_t)kb * 32 + 31) * N + n, (size_t)gridDim.y * 32 * N))
+    return;
   uint32_t u[WORDS];
   const uint32_t* src = codes + ((size_t)kb * N + n) * WORDS;
   if (BITS == 4) {
@@ -67,7 +73,7 @@ to_zero_point_kernel(const float2* __restrict__ qparams, float* __restrict__ alp
 template <int BITS, typename TO>
 void launch_dequantize_t(const Shape& sh, const uint32_t* codes, const float2* qparams, TO* W, cudaStream_t st) {
   const dim3 grid((unsigned)((sh.N + FMT_THREADS - 1) / FMT_THREADS), (unsigned)(sh.K / 32));
-  dequantize_kernel<BITS, TO><<<grid, FMT_THREADS, 0, st>>>(codes, qparams, W, sh.N, sh.g);
+  dequantize_kernel<BITS, TO><<<grid, FMT_THREADS, 0, st>>>(codes, qparams, W, sh.N, sh.g, debug_words());
 }
 
 }  // namespace

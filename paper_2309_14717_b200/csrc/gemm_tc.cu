@@ -24,6 +24,7 @@
 // drained while the next one is multiplied).  Stages are handed
 // over with mbarriers; every wait is bounded and a timeout raises a status word
 // instead of hanging.
+#define QALORA_TU 3
 #include <mutex>
 
 #include "common.cuh"
@@ -63,6 +64,7 @@ struct TcParams {
   int tile_t;                  // tokens per tile: TILE_T, or TILE_T_FEW (forward, M <= 64; always with parts)
   float* partial;              // ksplit > 1: fp32 [ksplit][M][ld_out] partial results
   int* status;                 // device word: set to 1 when a wait timed out
+  int* dbg;                    // record words of the bounds-check build (null otherwise)
 };
 
 // Work item of a block: part `sp` of tile `tile`, i.e. the main steps mb .. mb + n_main - 1
@@ -209,7 +211,11 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           const int s = it % NX, sb = it % NB;
           // the tile slot was last used by step it - NX: wait until that step has been multiplied
           if (it >= (uint32_t)NX && !(ok = ptx::mbar_wait(bar_empty_x((it - NX) % NB), ((it - NX) / NB) & 1, abort_flag))) break;
+          // (bounds-check build: the tile lies inside its ring and the copy starts inside the matrix)
+          QALORA_CHECK(p.dbg, S::OFF_X + (s + 1) * ACT_BYTES - 1, S::OFF_A);
+          QALORA_CHECK(p.dbg, m0, p.M);
           if (i < p.red_iters) {
+            QALORA_CHECK(p.dbg, i * TILE_J, MODE == FWD ? p.K : p.N);
             ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES);
             ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &act_map, i * TILE_J, m0, bar_full_x(sb));
           } else if (MODE == FWD) {
@@ -217,6 +223,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
             // tile's 128 channels (two boxes of 64 channels; rows beyond r arrive as zeros).  The one
             // buffer is free once the adapter step before this one has been multiplied.
             const int r0 = (i - p.red_iters) * TILE_J;
+            QALORA_CHECK(p.dbg, r0, p.r);
+            QALORA_CHECK(p.dbg, c0 + TILE_C - 1, p.N);
             if (!(ok = ptx::mbar_wait(bar_lb_empty, (nlb & 1) ^ 1, abort_flag))) break;
             ++nlb;
             ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES + ATILE_BYTES);
@@ -246,6 +254,9 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           // forward: k-blocks 4 cs .. 4 cs + 3 of columns c0 ..; dx: the tile's 4 k-blocks, columns 64 cs ..
           const int kb0 = MODE == FWD ? cs * 4 : c0 / 32;
           const int col0 = MODE == FWD ? c0 : cs * TILE_J;
+          QALORA_CHECK(p.dbg, S::OFF_C + (s + 1) * S::CSTAGE_BYTES - 1, S::OFF_OUT);
+          QALORA_CHECK(p.dbg, kb0 + 3, p.K / 32);
+          QALORA_CHECK(p.dbg, col0 + S::TILE_NC - 1, p.N);
           ptx::mbar_arrive_expect_tx(bar_full_c(s), S::CODE_BYTES + p.qp_rows * S::QP_ROW_BYTES);
           ptx::tma_load_2d(stage, &codes_map, col0 * WORDS / 2, kb0, bar_full_c(s));
           ptx::tma_load_2d(stage + S::CODE_BYTES, &qp_map, 2 * col0, kb0 * 32 / p.g, bar_full_c(s));
@@ -270,6 +281,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         const TcSegment sg = tc_segment<PARTS>(p, vt);
         const int ab = tcount % NACC;                 // accumulator of this tile
         const uint32_t acc_tmem = tmem_base + ACC_COL + ab * TILE_T;
+        QALORA_CHECK(p.dbg, ACC_COL + ab * TILE_T + TT - 1, MODE == FWD ? A_COL : TMEM_COLS);
         if (!(ok = ptx::mbar_wait(bar_acc_empty(ab), ((tcount / NACC) & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int j = 0; j < sg.n_steps; ++j, ++it) {
@@ -341,6 +353,10 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               uint32_t v[16];
               const int kbl = kb_base + half;
               const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (kbl * TILE_C + row) * WORDS;
+              if (!QALORA_CHECK(p.dbg, (kbl * TILE_C + row) * WORDS + WORDS - 1, S::CODE_BYTES / 4) ||
+                  !QALORA_CHECK(p.dbg, (kbl >> qsh) * TILE_C + row, p.qp_rows * TILE_C) ||
+                  !QALORA_CHECK(p.dbg, A_COL + sa * 32 + half * 16 + 15, TMEM_COLS))
+                continue;
               uint32_t w[WORDS];
               load_unit<WORDS>(cw, w);
               const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[(kbl >> qsh) * TILE_C + row];
@@ -359,6 +375,10 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               uint32_t v[16];
               const int kbl = dq / TILE_J, nl = dq % TILE_J;       // 32-channel block, column
               const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage) + (kbl * TILE_J + nl) * WORDS;
+              if (!QALORA_CHECK(p.dbg, (kbl * TILE_J + nl) * WORDS + WORDS - 1, S::CODE_BYTES / 4) ||
+                  !QALORA_CHECK(p.dbg, (kbl >> qsh) * TILE_J + nl, p.qp_rows * TILE_J) ||
+                  !QALORA_CHECK(p.dbg, S::OFF_A + sa * ATILE_BYTES + (kbl / 2) * 8192 + (nl / 8) * 1024 + (nl % 8) * 128 + 127, S::OFF_C))
+                continue;
               uint32_t w[WORDS];
               load_unit<WORDS>(cw, w);
               const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES)[(kbl >> qsh) * TILE_J + nl];
@@ -377,6 +397,9 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
               const int r0 = (i - p.red_iters) * TILE_J + halfrow * 32;
               const __nv_bfloat16* ap = p.lora + (size_t)((c0 + row) / p.g) * p.r + r0;
               uint8_t* rowp = atile + (row / 8) * 1024 + (row % 8) * 128;
+              if (!QALORA_CHECK(p.dbg, (c0 + row) / p.g, p.K / p.g) ||
+                  !QALORA_CHECK(p.dbg, S::OFF_A + sa * ATILE_BYTES + (row / 8) * 1024 + (row % 8) * 128 + 127, S::OFF_C))
+                continue;
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
                 uint4 t = make_uint4(0u, 0u, 0u, 0u);
@@ -417,7 +440,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
 #pragma unroll 1
       for (int col = 0; col < TT; col += 32, ++chunk) {
         uint32_t v[32];
-        ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ACC_COL + ab * TILE_T + col, v);
+        if (QALORA_CHECK(p.dbg, ACC_COL + ab * TILE_T + col + 31, MODE == FWD ? A_COL : TMEM_COLS))
+          ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ACC_COL + ab * TILE_T + col, v);
         ptx::tmem_wait_ld();
         if (col == TT - 32) {                     // all columns read: hand the accumulator back
           ptx::tc_fence_before();
@@ -430,7 +454,9 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           float* dst = p.partial + ((size_t)sp * p.M + (size_t)mt * TT + col) * p.ld_out + ct * TILE_C + ch;
 #pragma unroll
           for (int t = 0; t < 32; ++t)
-            if ((long long)mt * TT + col + t < p.M) dst[(size_t)t * p.ld_out] = __uint_as_float(v[t]);
+            if ((long long)mt * TT + col + t < p.M &&
+                QALORA_CHECK(p.dbg, ((size_t)sp * p.M + (size_t)mt * TT + col + t) * p.ld_out + ct * TILE_C + ch, (size_t)p.ksplit * p.M * p.ld_out))
+              dst[(size_t)t * p.ld_out] = __uint_as_float(v[t]);
           continue;
         }
         uint8_t* stg = smem + S::OFF_OUT + (chunk % S::NOUT) * S::OUT_BYTES;
@@ -440,7 +466,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
           reinterpret_cast<__nv_bfloat16*>(stg)[t * TILE_C + ch] = __float2bfloat16_rn(__uint_as_float(v[t]));
         ptx::fence_proxy_async();
         ptx::named_barrier(2, 128);
-        if (et == 0 && (long long)mt * TT + col < p.M) {
+        if (et == 0 && (long long)mt * TT + col < p.M && QALORA_CHECK(p.dbg, ct * TILE_C + TILE_C - 1, p.ld_out) &&
+            QALORA_CHECK(p.dbg, S::OFF_OUT + (chunk % S::NOUT + 1) * S::OUT_BYTES - 1, S::OFF_BARS)) {
           ptx::tma_store_2d(&out_map, ct * TILE_C, mt * TT + col, ptx::smem_u32(stg));
           ptx::bulk_commit_group();
           ptx::bulk_wait_group_read<S::NOUT - 1>();
@@ -653,7 +680,7 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
   p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.N;
   p.c_tiles = sh.N / TILE_C; p.m_tiles = (int)((M + tile_t - 1) / tile_t);
   p.red_iters = sh.K / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
-  p.status = status; p.qp_rows = 128 / sh.g;
+  p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
   p.ksplit = parts < 0 ? -parts : parts; p.tile_t = tile_t; p.partial = partial;
   if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, p, st);
@@ -673,7 +700,7 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
   p.M = M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r; p.ld_out = sh.K;
   p.c_tiles = sh.K / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
   p.red_iters = sh.N / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
-  p.status = status; p.qp_rows = 128 / sh.g;
+  p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
   p.ksplit = 1; p.tile_t = TILE_T; p.partial = nullptr;
   if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);

@@ -33,6 +33,7 @@
 //    written after every stage, hence every x slice, has been consumed.
 //    Back-to-back layers of a decoding step thus overlap one layer's tail with the
 //    next one's start.
+#define QALORA_TU 2
 #include <cooperative_groups.h>
 
 #include <mutex>
@@ -88,6 +89,7 @@ struct GvParams {
   int pdl_wait;                 // launched beside its predecessor: the producer waits for it before it fetches x
   int stop_after_stages;        // normally INT_MAX; a test makes every producer stop early, so that waits expire
   unsigned long long wait_limit_ns;
+  int* dbg;                     // record words of the bounds-check build (null otherwise)
 };
 
 // (not volatile: a pure function of its operands, so that independent MMAs can be interleaved)
@@ -189,6 +191,10 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
       // (alpha, beta) they need (128 / g of them) and the x slice.  The first ring of
       // weights goes out at once; x follows when the predecessor kernel is complete.
       const int first = n_issue < GV_STAGES ? n_issue : GV_STAGES;
+      // (bounds-check build: the block's last stage and its columns lie inside the matrices)
+      QALORA_CHECK(p.dbg, (long long)st_end * GV_KBS - 1, p.K / 32);
+      QALORA_CHECK(p.dbg, n0 + GV_COLS - 1, p.N);
+      QALORA_CHECK(p.dbg, st_end * GV_KBS * 32 / p.g - 1, p.K / p.g);
       if (p.pdl_wait) {
         for (int it = 0; it < first; ++it) {
           const int st = st_beg + it;
@@ -259,6 +265,11 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
     constexpr uint32_t ONES = 0x3f803f80u;        // bf16x2 (1, 1)
     const uint32_t ones4[4] = {ONES, ONES, ONES, ONES};
     bool ok = true;
+    // (bounds-check build: the last byte this thread reads of a stage's x slice, code rows and (alpha, beta) rows)
+    ok = QALORA_CHECK(p.dbg, x_off + (GV_KBS / GV_SETS - 1) * 64 + (NTS - 1) * 8 * (GV_KBS * 64) + 15, S::OFF_X + S::X_BYTES) &&
+         QALORA_CHECK(p.dbg, (BITS == 4 ? m_off + 15 : (BITS == 3 ? h_off : c_off) + 24 * WORDS * 4 + 3) + (GV_KBS / GV_SETS - 1) * S::CODE_ROW,
+                      S::OFF_CODES + GV_KBS * S::CODE_ROW) &&
+         QALORA_CHECK(p.dbg, q_off + ((GV_KBS - 1) >> qsh) * S::QP_ROW + 24 * 8 + 7, S::OFF_QP + ((GV_KBS * 32) / p.g) * S::QP_ROW);
     int s = 0;
     uint32_t ph = 0;
     for (int it = 0; it < n_stages && ok; ++it) {
@@ -407,12 +418,14 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
           const int token = ts * 8 + gq;
           const bool live = token < p.M;
           const unsigned short* Tr = Tu + (size_t)(live ? token : 0) * p.r;
+          QALORA_CHECK(p.dbg, (size_t)(live ? token : 0) * p.r, (size_t)p.M * p.r);
           tb[ts][0] = live ? pair(Tr, 1, i0, p.r) : 0u;
           tb[ts][1] = live ? pair(Tr, 1, i0 + 8, p.r) : 0u;
         }
 #pragma unroll
         for (int cg = 0; cg < 2; ++cg) {
           const unsigned short* c0 = Bu + n0 + wcol + cg * 16 + gq;
+          if (!QALORA_CHECK(p.dbg, n0 + wcol + cg * 16 + gq + 8, p.N)) continue;
           const uint32_t a[4] = {pair(c0, p.N, i0, p.r), pair(c0 + 8, p.N, i0, p.r),
                                  pair(c0, p.N, i0 + 8, p.r), pair(c0 + 8, p.N, i0 + 8, p.r)};
 #pragma unroll
@@ -427,6 +440,7 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
 #pragma unroll
       for (int ts = 0; ts < NTS; ++ts) {
         const int col = wcol + cg * 16 + gq, row = ts * 8 + 2 * t;
+        if (!QALORA_CHECK(p.dbg, (set * S::ROWS + row + 1) * GV_COLS + col + 8, S::PARTIAL_BYTES / 4)) continue;
         mine[row * GV_COLS + col] = acc[cg][ts][0];
         mine[(row + 1) * GV_COLS + col] = acc[cg][ts][1];
         mine[row * GV_COLS + col + 8] = acc[cg][ts][2];
@@ -448,7 +462,7 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
 #pragma unroll
         for (int sset = 0; sset < GV_SETS; ++sset) v += remote[sset * (S::ROWS * GV_COLS) + row * GV_COLS + col];
       }
-      p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v);
+      if (QALORA_CHECK(p.dbg, (size_t)row * p.N + n0 + col, (size_t)p.M * p.N)) p.y[(size_t)row * p.N + n0 + col] = __float2bfloat16_rn(v);
     }
   }
   cluster.sync();
@@ -654,7 +668,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   CUtensorMap xm;
   if (!make_x_map(x, sh.K, M, &xm)) return QALORA_ERR_CUDA;
   GvParams p{};
-  p.codes = codes; p.qparams = qparams; p.Tb = Tb; p.B = B; p.y = y;
+  p.codes = codes; p.qparams = qparams; p.Tb = Tb; p.B = B; p.y = y; p.dbg = debug_words();
   p.pdl_wait = Tb == nullptr ? 1 : 0;
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
@@ -716,7 +730,7 @@ int launch_gemv_group(const GemvGroupItem* items, int n, int64_t M, int* status,
   for (int i = 0; i < n; ++i) {
     const Shape& sh = items[i].sh;
     GvParams& p = grp.p[i];
-    p.codes = items[i].codes; p.qparams = items[i].qparams; p.Tb = nullptr; p.B = nullptr; p.y = items[i].y;
+    p.codes = items[i].codes; p.qparams = items[i].qparams; p.Tb = nullptr; p.B = nullptr; p.y = items[i].y; p.dbg = debug_words();
     p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = 0;
     p.total_stages = sh.K / (GV_KBS * 32);
     p.status = status;

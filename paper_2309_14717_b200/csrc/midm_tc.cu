@@ -30,6 +30,7 @@
 // The adapter is folded in as extra reduction steps of the last part: bf16(s pool(x) A) tiles
 // against rows of B gathered from global memory.
 // Every wait is bounded; a wait that gives up raises the status word and the block unwinds.
+#define QALORA_TU 4
 #include "common.cuh"
 #include "dequant.cuh"
 #include "ptx.cuh"
@@ -58,6 +59,7 @@ struct MmParams {
   int red_iters, lora_iters;    // main / adapter reduction steps of a whole tile
   int qp_rows;                  // rows of (alpha, beta) per code stage: 64 / g, at least one
   int* status;
+  int* dbg;                     // record words of the bounds-check build (null otherwise)
 };
 
 // XROWS: token rows an activation tile brings (64 for M <= 64, else 128).  The MMA always reads
@@ -161,6 +163,10 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         for (int j = 0; j < w.n_steps; ++j, ++it) {
           const int s = it % MM_NX;
           if (!(ok = ptx::mbar_wait(bar_empty_x(s), ((it / MM_NX) & 1) ^ 1, abort_flag))) break;
+          // (bounds-check build: the tile lies inside its ring, the copy starts inside the matrix)
+          QALORA_CHECK(p.dbg, S::OFF_X + (s + 1) * MM_X_BYTES - 1, S::OFF_B);
+          QALORA_CHECK(p.dbg, m0, p.M);
+          QALORA_CHECK(p.dbg, j < w.n_main ? (w.mb + j) * MM_J : (j - w.n_main) * MM_J, j < w.n_main ? p.K : p.r);
           ptx::mbar_arrive_expect_tx(bar_full_x(s), MM_X_BYTES);
           if (j < w.n_main)
             ptx::tma_load_2d(smem_base + S::OFF_X + s * MM_X_BYTES, &x_map, (w.mb + j) * MM_J, m0, bar_full_x(s));
@@ -182,6 +188,10 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
           if (!(ok = ptx::mbar_wait(bar_empty_c(s), ((cit / MM_NC) & 1) ^ 1, abort_flag))) break;
           const uint32_t stage = smem_base + S::OFF_C + s * S::CSTAGE_BYTES;
           const int kb0 = (w.mb + j) * 2, q0 = kb0 * 32 / p.g;
+          QALORA_CHECK(p.dbg, S::OFF_C + (s + 1) * S::CSTAGE_BYTES - 1, S::OFF_BARS);
+          QALORA_CHECK(p.dbg, kb0 + 1, p.K / 32);
+          QALORA_CHECK(p.dbg, q0, p.K / p.g);
+          QALORA_CHECK(p.dbg, c0 + MM_CH - 1, p.N);
           ptx::mbar_arrive_expect_tx(bar_full_c(s), S::CODE_BYTES + 2 * p.qp_rows * S::QP_HALF_ROW);
 #pragma unroll
           for (int h = 0; h < 2; ++h) {          // a tiled copy spans at most 256 elements: 128 columns each
@@ -202,6 +212,7 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         const MmItem w = mm_item(p, vt);
         const int ab = tcount % MM_NACC;
         const uint32_t acc_tmem = tmem_base + ab * MM_CH;
+        QALORA_CHECK(p.dbg, ab * MM_CH + MM_CH - 1, 512);
         if (!(ok = ptx::mbar_wait(bar_acc_empty(ab), ((tcount / MM_NACC) & 1) ^ 1, abort_flag))) break;
         ptx::tc_fence_after();
         for (int j = 0; j < w.n_steps; ++j, ++it) {
@@ -246,11 +257,15 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         if (main_step && !(ok = ptx::mbar_wait(bar_full_c(sc), (cst / MM_NC) & 1, abort_flag))) break;
         const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         uint8_t* rowp = smem + S::OFF_B + sb * MM_B_BYTES + (row / 8) * 1024 + (row % 8) * 128;
+        if (!QALORA_CHECK(p.dbg, S::OFF_B + sb * MM_B_BYTES + (row / 8) * 1024 + (row % 8) * 128 + 127, S::OFF_C)) continue;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {   // the two 32-index blocks of the step
           uint32_t v[16];
           if (main_step) {
             const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage + half_col * S::CODE_HALF) + (half * 128 + col_in_half) * WORDS;
+            if (!QALORA_CHECK(p.dbg, half_col * S::CODE_HALF / 4 + (half * 128 + col_in_half) * WORDS + WORDS - 1, S::CODE_BYTES / 4) ||
+                !QALORA_CHECK(p.dbg, half_col * 2 * 128 + (half >> qsh) * 128 + col_in_half, S::QP_BYTES / 8))
+              continue;
             uint32_t wd[WORDS];
             load_unit<WORDS>(cw, wd);
             const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES + half_col * 2 * S::QP_HALF_ROW)[(half >> qsh) * 128 + col_in_half];
@@ -300,14 +315,16 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
 #pragma unroll 1
       for (int col = 0; col < MM_CH; col += 32) {
         uint32_t v[32];
-        ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * MM_CH + col, v);
+        if (QALORA_CHECK(p.dbg, ab * MM_CH + col + 31, 512))
+          ptx::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * MM_CH + col, v);
         ptx::tmem_wait_ld();
         if (col == MM_CH - 32) {                  // all columns read: hand the accumulator back
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(bar_acc_empty(ab));
         }
-        if (token < p.M) {
+        if (token < p.M && QALORA_CHECK(p.dbg, out_off + col + 31, (size_t)p.M * p.N) &&
+            QALORA_CHECK(p.dbg, w.sp, p.parts)) {
           if (p.parts > 1) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
@@ -404,7 +421,7 @@ int launch_midm(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   p.n_tiles = sh.N / MM_CH; p.m_tiles = (int)((M + MM_TOK - 1) / MM_TOK); p.parts = mm_parts(sh, M);
   p.red_iters = sh.K / MM_J; p.lora_iters = (sh.r + MM_J - 1) / MM_J;
   p.qp_rows = MM_J / sh.g > 0 ? MM_J / sh.g : 1;
-  p.status = status;
+  p.status = status; p.dbg = debug_words();
 #define QALORA_MM(BITS) (xrows == 64 ? launch_midm_t<BITS, 64>(xm, tm, p, codes, qparams, st) : launch_midm_t<BITS, 128>(xm, tm, p, codes, qparams, st))
   if (sh.bits == 4) return QALORA_MM(4);
   if (sh.bits == 3) return QALORA_MM(3);

@@ -2,6 +2,7 @@
 // coefficient and AdamW over one flat array of trained parameters.  Two launches, both
 // bound by HBM: the first reads the gradients once, the second reads gradient, master
 // parameter and both moments and writes parameter, moments and the bf16 copy the layers use.
+#define QALORA_TU 8
 #include "common.cuh"
 
 namespace qalora {
@@ -33,7 +34,8 @@ __device__ __forceinline__ T block_sum(T v, T* scratch /*[OPT_THREADS / 32]*/) {
 // parts[b] = sum of squares of block b's contiguous range of the gradient.  The ranges and the
 // order of additions depend only on n and the grid, so the result is reproducible.
 __global__ void __launch_bounds__(OPT_THREADS)
-grad_sqnorm_kernel(const float* __restrict__ grad, size_t n, size_t per_block /*multiple of 4*/, float* __restrict__ parts) {
+grad_sqnorm_kernel(const float* __restrict__ grad, size_t n, size_t per_block /*multiple of 4*/, float* __restrict__ parts,
+                   int* dbg) {
   __shared__ float scratch[OPT_THREADS / 32];
   const size_t lo = (size_t)blockIdx.x * per_block;
   size_t hi = lo + per_block;
@@ -43,15 +45,17 @@ grad_sqnorm_kernel(const float* __restrict__ grad, size_t n, size_t per_block /*
     const size_t vec_hi = lo + ((hi - lo) & ~(size_t)3);
     size_t i = lo + (size_t)threadIdx.x * 4;
     for (; i + 3 * OPT_THREADS * 4 < vec_hi; i += 4 * OPT_THREADS * 4) {   // four independent loads in flight
+      if (!QALORA_CHECK(dbg, i + 3 * OPT_THREADS * 4 + 3, n)) break;
       const float4 a = ld4(grad + i), b = ld4(grad + i + OPT_THREADS * 4), c = ld4(grad + i + 2 * OPT_THREADS * 4),
                    d = ld4(grad + i + 3 * OPT_THREADS * 4);
       acc[0] += sq4(a); acc[1] += sq4(b); acc[2] += sq4(c); acc[3] += sq4(d);
     }
-    for (; i < vec_hi; i += OPT_THREADS * 4) acc[0] += sq4(ld4(grad + i));
+    for (; i < vec_hi; i += OPT_THREADS * 4)
+      if (QALORA_CHECK(dbg, i + 3, n)) acc[0] += sq4(ld4(grad + i));
     for (size_t j = vec_hi + threadIdx.x; j < hi; j += OPT_THREADS) acc[1] += grad[j] * grad[j];
   }
   const float total = block_sum((acc[0] + acc[1]) + (acc[2] + acc[3]), scratch);
-  if (threadIdx.x == 0) parts[blockIdx.x] = total;
+  if (threadIdx.x == 0 && QALORA_CHECK(dbg, blockIdx.x, OPT_MAX_PARTS)) parts[blockIdx.x] = total;
 }
 
 struct AdamConsts {
@@ -76,7 +80,7 @@ __device__ __forceinline__ void adam_one(float g, float& p, float& m, float& v, 
 __global__ void __launch_bounds__(OPT_THREADS)
 adamw_kernel(const float* __restrict__ grad, float* __restrict__ param, float* __restrict__ exp_avg,
              float* __restrict__ exp_avg_sq, __nv_bfloat16* __restrict__ param_bf16, size_t n,
-             const float* __restrict__ parts, int nparts, AdamConsts k, float* __restrict__ norm_out) {
+             const float* __restrict__ parts, int nparts, AdamConsts k, float* __restrict__ norm_out, int* dbg) {
   __shared__ double scratch[OPT_THREADS / 32];
   double mine = 0.0;
   for (int i = threadIdx.x; i < nparts; i += OPT_THREADS) mine += (double)parts[i];
@@ -89,6 +93,7 @@ adamw_kernel(const float* __restrict__ grad, float* __restrict__ param, float* _
   const size_t nvec = n / 4, stride = (size_t)gridDim.x * OPT_THREADS;
   for (size_t q = (size_t)blockIdx.x * OPT_THREADS + threadIdx.x; q < nvec; q += stride) {
     const size_t i = q * 4;
+    if (!QALORA_CHECK(dbg, i + 3, n)) break;
     const float4 g = ld4(grad + i);
     float4 p = ld4(param + i), m = ld4(exp_avg + i), v = ld4(exp_avg_sq + i);
     adam_one(g.x, p.x, m.x, v.x, coef, k); adam_one(g.y, p.y, m.y, v.y, coef, k);
@@ -125,7 +130,7 @@ int launch_adamw(const AdamwArgs& a, int64_t n64, const float* grad, float* para
   size_t per_block = round_up((n + OPT_MAX_PARTS - 1) / OPT_MAX_PARTS, 4);
   if (per_block < 4096) per_block = 4096;
   const int nparts = (int)((n + per_block - 1) / per_block);
-  grad_sqnorm_kernel<<<nparts, OPT_THREADS, 0, st>>>(grad, n, per_block, parts);
+  grad_sqnorm_kernel<<<nparts, OPT_THREADS, 0, st>>>(grad, n, per_block, parts, debug_words());
   AdamConsts k;
   k.decay = (float)(1.0 - (double)a.lr * a.weight_decay);
   k.beta1 = a.beta1; k.beta2 = a.beta2;
@@ -137,7 +142,7 @@ int launch_adamw(const AdamwArgs& a, int64_t n64, const float* grad, float* para
   size_t blocks = (size_t)device_sm_count() * OPT_BLOCKS_PER_SM;
   if (blocks > want) blocks = want > 0 ? want : 1;
   adamw_kernel<<<(unsigned)blocks, OPT_THREADS, 0, st>>>(grad, param, exp_avg, exp_avg_sq, param_bf16, n, parts, nparts, k,
-                                                         norm_out);
+                                                         norm_out, debug_words());
   count_launch(2);
   return cuda_status(cudaGetLastError());
 }

@@ -2,6 +2,7 @@
 // and the merge of the adapter into the zero factors (Appendix B Eq. 7).
 // Both are streaming, HBM-bound kernels: one thread owns one output column of
 // one quantization group, so a warp reads 128 contiguous bytes of each W row.
+#define QALORA_TU 7
 #include <float.h>
 
 #include "common.cuh"
@@ -24,12 +25,13 @@ constexpr int QCOLS = 128;   // columns (threads) per block
 template <int BITS>
 __global__ void __launch_bounds__(QCOLS)
 quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
-                float2* __restrict__ qparams, int N, int g, int ntiles, int32_t* dev_status) {
+                float2* __restrict__ qparams, int N, int g, int G, int ntiles, int32_t* dev_status, int* dbg) {
   constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   constexpr float QMAX = float((1 << BITS) - 1);
   const int q = blockIdx.x / ntiles;
   const int n = (blockIdx.x % ntiles) * QCOLS + threadIdx.x;
   if (n >= N) return;
+  if (!QALORA_CHECK(dbg, ((size_t)q * g + g - 1) * N + n, (size_t)G * g * N)) return;   // the last weight this thread reads
   const float* w = W + (size_t)q * g * N + n;
 
   float lo = FLT_MAX, hi = -FLT_MAX;
@@ -47,7 +49,7 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
   }
   const float alpha = (hi == lo) ? 1.0f : __fdiv_rn(__fsub_rn(hi, lo), QMAX);
   const float beta = lo;
-  qparams[(size_t)q * N + n] = make_float2(alpha, beta);
+  if (QALORA_CHECK(dbg, (size_t)q * N + n, (size_t)G * N)) qparams[(size_t)q * N + n] = make_float2(alpha, beta);
   if (bad && dev_status != nullptr) atomicOr(dev_status, 1);
 
   const bool fast = alpha > 1e-30f && alpha < 1e30f;
@@ -70,6 +72,7 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
       unit_insert<BITS>(u, j, (uint32_t)(int)c);
     }
     uint32_t* dst = codes + ((size_t)(kb0 + k0 / 32) * N + n) * WORDS;
+    if (!QALORA_CHECK(dbg, ((size_t)(kb0 + k0 / 32) * N + n) * WORDS + WORDS - 1, (size_t)G * (g / 32) * N * WORDS)) continue;
     if (WORDS == 4) {
       *reinterpret_cast<uint4*>(dst) = make_uint4(u[0], u[1], u[2], u[3]);
     } else if (WORDS == 2) {
@@ -87,9 +90,9 @@ int launch_quantize(const Shape& sh, const float* W, uint32_t* codes, float2* qp
   const long long blocks = (long long)sh.G * ntiles;
   if (blocks > 0x7fffffffLL) return QALORA_ERR_UNSUPPORTED_SHAPE;
   dim3 grid((unsigned)blocks), block(QCOLS);
-  if (sh.bits == 4) quantize_kernel<4><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
-  else if (sh.bits == 3) quantize_kernel<3><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
-  else quantize_kernel<2><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, ntiles, dev_status);
+  if (sh.bits == 4) quantize_kernel<4><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, sh.G, ntiles, dev_status, debug_words());
+  else if (sh.bits == 3) quantize_kernel<3><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, sh.G, ntiles, dev_status, debug_words());
+  else quantize_kernel<2><<<grid, block, 0, st>>>(W, codes, qparams, sh.N, sh.g, sh.G, ntiles, dev_status, debug_words());
   count_launch();
   return cuda_status(cudaGetLastError());
 }
@@ -103,7 +106,7 @@ constexpr int MERGE_GROUPS = 8;
 __global__ void __launch_bounds__(QCOLS)
 merge_kernel(const float2* __restrict__ qin, const __nv_bfloat16* __restrict__ A,
              const __nv_bfloat16* __restrict__ B, float2* __restrict__ qout,
-             int G, int N, int r, float s, int ntiles) {
+             int G, int N, int r, float s, int ntiles, int* dbg) {
   extern __shared__ float a_rows[];                 // [MERGE_GROUPS][r]
   const int q0 = (blockIdx.x / ntiles) * MERGE_GROUPS;
   const int n = (blockIdx.x % ntiles) * QCOLS + threadIdx.x;
@@ -125,7 +128,7 @@ merge_kernel(const float2* __restrict__ qin, const __nv_bfloat16* __restrict__ A
 #pragma unroll
   for (int j = 0; j < MERGE_GROUPS; ++j) {
     const int q = q0 + j;
-    if (q < G) {
+    if (q < G && QALORA_CHECK(dbg, (size_t)q * N + n, (size_t)G * N)) {
       float2 p = qin[(size_t)q * N + n];
       p.y = fmaf(s, acc[j], p.y);
       qout[(size_t)q * N + n] = p;
@@ -138,7 +141,7 @@ int launch_merge(const Shape& sh, const float2* qin, const __nv_bfloat16* A, con
   const int ntiles = (sh.N + QCOLS - 1) / QCOLS;
   const long long blocks = (long long)((sh.G + MERGE_GROUPS - 1) / MERGE_GROUPS) * ntiles;
   if (blocks > 0x7fffffffLL) return QALORA_ERR_UNSUPPORTED_SHAPE;
-  merge_kernel<<<(unsigned)blocks, QCOLS, MERGE_GROUPS * sh.r * sizeof(float), st>>>(qin, A, B, qout, sh.G, sh.N, sh.r, sh.s, ntiles);
+  merge_kernel<<<(unsigned)blocks, QCOLS, MERGE_GROUPS * sh.r * sizeof(float), st>>>(qin, A, B, qout, sh.G, sh.N, sh.r, sh.s, ntiles, debug_words());
   count_launch();
   return cuda_status(cudaGetLastError());
 }

@@ -1,6 +1,7 @@
 // General-shape CUDA-core kernels of the QA-LoRA layer.  They accept every
 // supported shape and serve (a) shapes the tensor-core kernels do not tile and
 // (b) the small rank-r side products.  fp32 accumulation throughout.
+#define QALORA_TU 6
 #include "common.cuh"
 
 namespace qalora {
@@ -19,7 +20,7 @@ constexpr size_t kPoolASliceMax = 40 * 1024;          // the slice of A is kept 
 __global__ void __launch_bounds__(POOL_THREADS)
 pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
               float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
-              int K, int g, int G, int r, float s, int a_in_smem) {
+              int K, int g, int G, int r, float s, int a_in_smem, int* dbg) {
   extern __shared__ __align__(16) uint8_t pool1_smem[];
   float* xp = reinterpret_cast<float*>(pool1_smem);                                        // [G]
   __nv_bfloat16* As = reinterpret_cast<__nv_bfloat16*>(pool1_smem + ((size_t)G * 4 + 15) / 16 * 16);   // [G][32] when a_in_smem
@@ -34,7 +35,7 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
       const int q = idx / 4, c = idx % 4;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (i0 + c * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(A + (size_t)q * r + i0 + c * 8));
-      *reinterpret_cast<uint4*>(As + (size_t)q * 32 + c * 8) = v;
+      if (QALORA_CHECK(dbg, q * 32 + c * 8 + 7, G * 32)) *reinterpret_cast<uint4*>(As + (size_t)q * 32 + c * 8) = v;
     }
   }
   const __nv_bfloat16* xr = x + m * (size_t)K;
@@ -49,7 +50,7 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
       for (int u = 0; u < 4; ++u) {
         const int q = q0 + u * (POOL_THREADS / 4) + threadIdx.x / 4;
         v[u] = make_uint4(0u, 0u, 0u, 0u);
-        if (q < G) v[u] = __ldg(reinterpret_cast<const uint4*>(xr + (size_t)q * g + k));
+        if (q < G && QALORA_CHECK(dbg, (long long)q * g + k + 7, K)) v[u] = __ldg(reinterpret_cast<const uint4*>(xr + (size_t)q * g + k));
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -69,7 +70,8 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
       a += __shfl_xor_sync(0xffffffffu, a, 2);
       if (lane4 == 0 && q < G) {
         xp[q] = a;
-        if (xp_out != nullptr && blockIdx.y == 0) xp_out[m * (size_t)G + q] = a;
+        if (xp_out != nullptr && blockIdx.y == 0 && QALORA_CHECK(dbg, m * (size_t)G + q, (size_t)gridDim.x * G))
+          xp_out[m * (size_t)G + q] = a;
       }
     }
   }
@@ -96,8 +98,10 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
 #pragma unroll
     for (int k = 0; k < 8; ++k) t += part[k][il];
     t *= s;
-    T[m * (size_t)r + i] = t;
-    if (Tb != nullptr) Tb[m * (size_t)r + i] = __float2bfloat16_rn(t);
+    if (QALORA_CHECK(dbg, m * (size_t)r + i, (size_t)gridDim.x * r)) {
+      T[m * (size_t)r + i] = t;
+      if (Tb != nullptr) Tb[m * (size_t)r + i] = __float2bfloat16_rn(t);
+    }
   }
 }
 
@@ -130,7 +134,7 @@ template <int LANES_PER_GROUP>   // g / 8: 4, 8 or 16
 __global__ void __launch_bounds__(POOL16_ROWS * 32, 2)
 pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
                    float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
-                   long long M, int K, int G, int r, float s) {
+                   long long M, int K, int G, int r, float s, int smem_words, int* dbg) {
   extern __shared__ __align__(16) uint32_t pool_smem[];
   const int SW = pool16_stride_words(G);                 // row stride of the two bf16 arrays, in words
   __nv_bfloat16* xhi = reinterpret_cast<__nv_bfloat16*>(pool_smem);                 // [16][2 SW]
@@ -174,9 +178,11 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
         if (c < chunks && (lane % LANES_PER_GROUP) == 0) {
           const int q = c / LANES_PER_GROUP;
           const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
-          xhi[warp * 2 * SW + q] = hi;
-          xlo[warp * 2 * SW + q] = __float2bfloat16_rn(acc - __bfloat162float(hi));
-          if (xp_out != nullptr) xp_out[(size_t)m * G + q] = acc;
+          if (QALORA_CHECK(dbg, warp * 2 * SW + q, POOL16_ROWS * 2 * SW)) {
+            xhi[warp * 2 * SW + q] = hi;
+            xlo[warp * 2 * SW + q] = __float2bfloat16_rn(acc - __bfloat162float(hi));
+          }
+          if (xp_out != nullptr && QALORA_CHECK(dbg, (size_t)m * G + q, (size_t)M * G)) xp_out[(size_t)m * G + q] = acc;
         }
       }
     };
@@ -219,10 +225,13 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
     }
     float* pp = part + (size_t)part_i * POOL16_ROWS * r;
     const int col = nt * 8 + 2 * t;
-    pp[gq * r + col] = d[0];
-    pp[gq * r + col + 1] = d[1];
-    pp[(gq + 8) * r + col] = d[2];
-    pp[(gq + 8) * r + col + 1] = d[3];
+    // the last element this lane writes must lie inside the block's shared memory
+    if (QALORA_CHECK(dbg, 2 * POOL16_ROWS * SW + (part_i * POOL16_ROWS + gq + 8) * r + col + 1, smem_words)) {
+      pp[gq * r + col] = d[0];
+      pp[gq * r + col + 1] = d[1];
+      pp[(gq + 8) * r + col] = d[2];
+      pp[(gq + 8) * r + col + 1] = d[3];
+    }
   }
   __syncthreads();
   for (int o = threadIdx.x; o < POOL16_ROWS * r; o += POOL16_ROWS * 32) {
@@ -230,7 +239,7 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
     float v = 0.f;
     for (int pi = 0; pi < ksplit; ++pi) v += part[(size_t)pi * POOL16_ROWS * r + o];
     v *= s;
-    if (mm < M) {
+    if (mm < M && QALORA_CHECK(dbg, (size_t)mm * r + o % r, (size_t)M * r)) {
       T[(size_t)mm * r + o % r] = v;
       if (Tb != nullptr) Tb[(size_t)mm * r + o % r] = __float2bfloat16_rn(v);
     }
@@ -262,15 +271,15 @@ int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv
     });
     if (attr_st != QALORA_OK) return attr_st;
     const unsigned grid = (unsigned)((M + POOL16_ROWS - 1) / POOL16_ROWS);
-    if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
-    else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
-    else pool_T_rows_kernel<16><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s);
+    if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
+    else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
+    else pool_T_rows_kernel<16><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
   } else {
     dim3 grid((unsigned)M, (unsigned)((sh.r + 31) / 32 > 0 ? (sh.r + 31) / 32 : 1));
     const size_t xp_bytes = ((size_t)sh.G * sizeof(float) + 15) / 16 * 16, a_bytes = (size_t)sh.G * 32 * sizeof(__nv_bfloat16);
     const int a_in_smem = (sh.r > 0 && a_bytes <= kPoolASliceMax) ? 1 : 0;
     pool_T_kernel<<<grid, POOL_THREADS, xp_bytes + (a_in_smem ? a_bytes : 0), st>>>(x, A, xp, T, Tb, sh.K, sh.g, sh.G, sh.r, sh.s,
-                                                                                    a_in_smem);
+                                                                                    a_in_smem, debug_words());
   }
   count_launch();
   return cuda_status(cudaGetLastError());
@@ -282,7 +291,7 @@ constexpr int DT_THREADS = 256;
 
 __global__ void __launch_bounds__(DT_THREADS)
 dT_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ B,
-          float* __restrict__ dT, __nv_bfloat16* __restrict__ dTb, int N, int r, float s) {
+          float* __restrict__ dT, __nv_bfloat16* __restrict__ dTb, int N, int r, float s, int* dbg) {
   const size_t m = blockIdx.x;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const __nv_bfloat16* dyr = dy + m * (size_t)N;
@@ -305,8 +314,10 @@ dT_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict_
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) {
       acc *= s;
-      dT[m * (size_t)r + i] = acc;
-      if (dTb != nullptr) dTb[m * (size_t)r + i] = __float2bfloat16_rn(acc);
+      if (QALORA_CHECK(dbg, m * (size_t)r + i, (size_t)gridDim.x * r)) {
+        dT[m * (size_t)r + i] = acc;
+        if (dTb != nullptr) dTb[m * (size_t)r + i] = __float2bfloat16_rn(acc);
+      }
     }
   }
 }
@@ -314,7 +325,7 @@ dT_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict_
 int launch_dT(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const __nv_bfloat16* B,
               float* dT, __nv_bfloat16* dTb, cudaStream_t st) {
   if (M == 0) return QALORA_OK;
-  dT_kernel<<<(unsigned)M, DT_THREADS, 0, st>>>(dy, B, dT, dTb, sh.N, sh.r, sh.s);
+  dT_kernel<<<(unsigned)M, DT_THREADS, 0, st>>>(dy, B, dT, dTb, sh.N, sh.r, sh.s, debug_words());
   count_launch();
   return cuda_status(cudaGetLastError());
 }
@@ -329,7 +340,7 @@ __global__ void __launch_bounds__(SIMT_THREADS)
 simt_forward_kernel(const __nv_bfloat16* __restrict__ x, const uint32_t* __restrict__ codes,
                     const float2* __restrict__ qparams, const float* __restrict__ T,
                     const __nv_bfloat16* __restrict__ B, __nv_bfloat16* __restrict__ y,
-                    long long M, int K, int N, int g, int r) {
+                    long long M, int K, int N, int g, int r, int* dbg) {
   constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   __shared__ __align__(16) float xs[TK][TM + 4];
   __shared__ __align__(16) float ws[TK][TN + 4];
@@ -344,7 +355,7 @@ simt_forward_kernel(const __nv_bfloat16* __restrict__ x, const uint32_t* __restr
   for (int k0 = 0; k0 < K; k0 += TK) {
     {
       float v[8] = {};
-      if (m0 + lrow < M) {
+      if (m0 + lrow < M && QALORA_CHECK(dbg, (size_t)(m0 + lrow) * K + k0 + lseg + 7, (size_t)M * K)) {
         const uint4 raw = *reinterpret_cast<const uint4*>(x + (size_t)(m0 + lrow) * K + k0 + lseg);
         const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
@@ -358,7 +369,8 @@ simt_forward_kernel(const __nv_bfloat16* __restrict__ x, const uint32_t* __restr
     }
     {
       const int n = n0 + un;
-      if (n < N) {
+      if (n < N && QALORA_CHECK(dbg, ((size_t)(k0 / 32) * N + n) * WORDS + WORDS - 1, (size_t)(K / 32) * N * WORDS) &&
+          QALORA_CHECK(dbg, (size_t)(k0 / g) * N + n, (size_t)(K / g) * N)) {
         const uint32_t* u = codes + ((size_t)(k0 / 32) * N + n) * WORDS;
         uint32_t w[WORDS];
 #pragma unroll
@@ -400,7 +412,7 @@ simt_forward_kernel(const __nv_bfloat16* __restrict__ x, const uint32_t* __restr
       acc[i][2] = fmaf(tv, b1.x, acc[i][2]); acc[i][3] = fmaf(tv, b1.y, acc[i][3]);
     }
     __nv_bfloat162 o[2] = {__floats2bfloat162_rn(acc[i][0], acc[i][1]), __floats2bfloat162_rn(acc[i][2], acc[i][3])};
-    *reinterpret_cast<uint2*>(y + (size_t)m * N + nb) = *reinterpret_cast<uint2*>(o);
+    if (QALORA_CHECK(dbg, (size_t)m * N + nb + 3, (size_t)M * N)) *reinterpret_cast<uint2*>(y + (size_t)m * N + nb) = *reinterpret_cast<uint2*>(o);
   }
 }
 
@@ -411,7 +423,7 @@ int launch_simt_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, cons
   const long long mt = (M + TM - 1) / TM;
   if (mt > 65535) return QALORA_ERR_UNSUPPORTED_SHAPE;
   dim3 grid((sh.N + TN - 1) / TN, (unsigned)mt), block(SIMT_THREADS);
-#define QALORA_FWD(BITS) simt_forward_kernel<BITS><<<grid, block, 0, st>>>(x, codes, qparams, T, B, y, M, sh.K, sh.N, sh.g, sh.r)
+#define QALORA_FWD(BITS) simt_forward_kernel<BITS><<<grid, block, 0, st>>>(x, codes, qparams, T, B, y, M, sh.K, sh.N, sh.g, sh.r, debug_words())
   {
     MainKernelProbe probe("simt_forward_kernel", st);
     if (sh.bits == 4) QALORA_FWD(4); else if (sh.bits == 3) QALORA_FWD(3); else QALORA_FWD(2);
@@ -427,7 +439,7 @@ __global__ void __launch_bounds__(SIMT_THREADS)
 simt_dx_kernel(const __nv_bfloat16* __restrict__ dy, const uint32_t* __restrict__ codes,
                const float2* __restrict__ qparams, const float* __restrict__ dT,
                const __nv_bfloat16* __restrict__ A, __nv_bfloat16* __restrict__ dx,
-               long long M, int K, int N, int g, int r) {
+               long long M, int K, int N, int g, int r, int* dbg) {
   constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
   __shared__ __align__(16) float ds[TK][TM + 4];        // [n][m]
   __shared__ __align__(16) float ws[TK][TN + 4];        // [n][k]
@@ -442,7 +454,7 @@ simt_dx_kernel(const __nv_bfloat16* __restrict__ dy, const uint32_t* __restrict_
   for (int n0 = 0; n0 < N; n0 += TK) {
     {
       float v[8] = {};
-      if (m0 + lrow < M && n0 + lseg < N) {
+      if (m0 + lrow < M && n0 + lseg < N && QALORA_CHECK(dbg, (size_t)(m0 + lrow) * N + n0 + lseg + 7, (size_t)M * N)) {
         const uint4 raw = *reinterpret_cast<const uint4*>(dy + (size_t)(m0 + lrow) * N + n0 + lseg);
         const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
@@ -456,7 +468,8 @@ simt_dx_kernel(const __nv_bfloat16* __restrict__ dy, const uint32_t* __restrict_
     }
     {
       const int n = n0 + un, k = k0 + ukb * 32;
-      if (n < N && k < K) {
+      if (n < N && k < K && QALORA_CHECK(dbg, ((size_t)(k / 32) * N + n) * WORDS + WORDS - 1, (size_t)(K / 32) * N * WORDS) &&
+          QALORA_CHECK(dbg, (size_t)(k / g) * N + n, (size_t)(K / g) * N)) {
         const uint32_t* u = codes + ((size_t)(k / 32) * N + n) * WORDS;
         uint32_t w[WORDS];
 #pragma unroll
@@ -495,7 +508,7 @@ simt_dx_kernel(const __nv_bfloat16* __restrict__ dy, const uint32_t* __restrict_
       lora = fmaf(__ldg(dT + (size_t)m * r + t), bf16_to_float(A[(size_t)q * r + t]), lora);
     __nv_bfloat162 o[2] = {__floats2bfloat162_rn(acc[i][0] + lora, acc[i][1] + lora),
                            __floats2bfloat162_rn(acc[i][2] + lora, acc[i][3] + lora)};
-    *reinterpret_cast<uint2*>(dx + (size_t)m * K + kc) = *reinterpret_cast<uint2*>(o);
+    if (QALORA_CHECK(dbg, (size_t)m * K + kc + 3, (size_t)M * K)) *reinterpret_cast<uint2*>(dx + (size_t)m * K + kc) = *reinterpret_cast<uint2*>(o);
   }
 }
 
@@ -506,7 +519,7 @@ int launch_simt_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const ui
   const long long mt = (M + TM - 1) / TM;
   if (mt > 65535) return QALORA_ERR_UNSUPPORTED_SHAPE;
   dim3 grid((sh.K + TN - 1) / TN, (unsigned)mt), block(SIMT_THREADS);
-#define QALORA_DX(BITS) simt_dx_kernel<BITS><<<grid, block, 0, st>>>(dy, codes, qparams, dT, A, dx, M, sh.K, sh.N, sh.g, sh.r)
+#define QALORA_DX(BITS) simt_dx_kernel<BITS><<<grid, block, 0, st>>>(dy, codes, qparams, dT, A, dx, M, sh.K, sh.N, sh.g, sh.r, debug_words())
   {
     MainKernelProbe probe("simt_dx_kernel", st);
     if (sh.bits == 4) QALORA_DX(4); else if (sh.bits == 3) QALORA_DX(3); else QALORA_DX(2);
@@ -527,7 +540,7 @@ template <> __device__ __forceinline__ float load_as_float<__nv_bfloat16>(const 
 template <typename TY>
 __global__ void __launch_bounds__(SIMT_THREADS)
 atb_partial_kernel(const float* __restrict__ X, const TY* __restrict__ Y, float* __restrict__ partial,
-                   long long M, int P, int Q, long long rows_per_split) {
+                   long long M, int P, int Q, long long rows_per_split, int* dbg) {
   __shared__ __align__(16) float xs[TK][TM + 4];
   __shared__ __align__(16) float ys[TK][TN + 4];
   const int tid = threadIdx.x;
@@ -562,7 +575,7 @@ atb_partial_kernel(const float* __restrict__ X, const TY* __restrict__ Y, float*
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int p = p0 + ty * 4 + i, q = q0 + tx * 4 + j;
-      if (p < P && q < Q) dst[(size_t)p * Q + q] = acc[i][j];
+      if (p < P && q < Q && QALORA_CHECK(dbg, ((size_t)blockIdx.z * P + p) * Q + q, (size_t)gridDim.z * P * Q)) dst[(size_t)p * Q + q] = acc[i][j];
     }
 }
 
@@ -603,7 +616,7 @@ static int launch_atb(int64_t M, int P, int Q, const float* X, const TY* Y, floa
   rows = (rows + TK - 1) / TK * TK;
   splits = (M + rows - 1) / rows;
   dim3 grid((Q + TN - 1) / TN, (P + TM - 1) / TM, (unsigned)splits);
-  atb_partial_kernel<TY><<<grid, SIMT_THREADS, 0, st>>>(X, Y, partial, M, P, Q, rows);
+  atb_partial_kernel<TY><<<grid, SIMT_THREADS, 0, st>>>(X, Y, partial, M, P, Q, rows, debug_words());
   sum_partials_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(partial, out, count, (int)splits);
   count_launch(2);
   return cuda_status(cudaGetLastError());

@@ -39,7 +39,24 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
+@pytest.fixture(autouse=True)
+def _bounds_check_record(request):
+    """With QALORA_LIBRARY=debug (the bounds-check build) every GPU test ends by reading the
+    library's record words: a failed index check or an overwritten guard word fails the test."""
+    yield
+    if os.environ.get("QALORA_LIBRARY") != "debug" or "gpu" not in request.keywords:
+        return
+    from paper_2309_14717_b200 import binding as Q
+    assert Q.qalora_debug_checks(), "QALORA_LIBRARY=debug but the loaded library has no checks"
+    words = Q.qalora_debug_report()
+    assert not any(words), ("bounds-check build: flags=%d first site=%d index=%d limit=%d failed checks=%d guard=%d"
+                            % (words[0], words[1], (words[3] << 32) | (words[2] & 0xffffffff),
+                               (words[5] << 32) | (words[4] & 0xffffffff), words[6], words[7]))
+
+
 def pytest_terminal_summary(terminalreporter):
+    if os.environ.get("QALORA_LIBRARY") == "debug":
+        terminalreporter.write_line("bounds-check build: record words read after every GPU test")
     if not PARITY_MARGINS:
         return
     tr = terminalreporter
