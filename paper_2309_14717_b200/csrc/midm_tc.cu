@@ -105,8 +105,8 @@ __device__ __forceinline__ MmItem mm_item(const MmParams& p, int vt) {
 template <int BITS, int XROWS>
 __global__ void __launch_bounds__(MM_THREADS, 1)
 qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap t_map,
-                   const __grid_constant__ CUtensorMap codes_map, const __grid_constant__ CUtensorMap qp_map,
-                   const MmParams p) {
+                   const __grid_constant__ CUtensorMap lb_map, const __grid_constant__ CUtensorMap codes_map,
+                   const __grid_constant__ CUtensorMap qp_map, const MmParams p) {
   using S = MmSmem<BITS, XROWS>;
   constexpr int WORDS = S::WORDS;
   constexpr int MM_NX = S::NX;
@@ -136,7 +136,7 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&x_map);
-    if (p.lora_iters > 0) ptx::prefetch_tensormap(&t_map);
+    if (p.lora_iters > 0) { ptx::prefetch_tensormap(&t_map); ptx::prefetch_tensormap(&lb_map); }
     ptx::prefetch_tensormap(&codes_map);
     ptx::prefetch_tensormap(&qp_map);
   }
@@ -205,6 +205,7 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     // ---------------------------------------------------------- MMA issuer ----
     if (lane == 0) {
       constexpr uint32_t IDESC = ptx::idesc_bf16(MM_TOK, MM_CH, false, false);   // both operands K-major
+      constexpr uint32_t IDESC_LORA = ptx::idesc_bf16(MM_TOK, MM_CH, false, true); // adapter step: the tile of B is MN-major
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       uint32_t ready = 0;                          // bit 0: operand slot of the coming step, bit 1: its activation tile
@@ -229,9 +230,18 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
           const uint64_t bdesc = ptx::smem_desc(smem_base + S::OFF_B + sb * MM_B_BYTES, 16, 1024);
           // one block: the probes for the NEXT step, four MMAs, the two commits (the tile and the
           // operand slot are free once these MMAs are done), then the probes' answers
-          ready = ptx::mma4_ss_commit2_probe2<2, 2>(acc_tmem, adesc, bdesc, IDESC, j > 0 ? 1u : 0u, bar_empty_x(sx),
-                                                    bar_empty_b(sb), bar_full_b((it + 1) % MM_NB), ((it + 1) / MM_NB) & 1,
-                                                    bar_full_x((it + 1) % MM_NX), ((it + 1) / MM_NX) & 1);
+          if (j < w.n_main) {
+            ready = ptx::mma4_ss_commit2_probe2<2, 2>(acc_tmem, adesc, bdesc, IDESC, j > 0 ? 1u : 0u, bar_empty_x(sx),
+                                                      bar_empty_b(sb), bar_full_b((it + 1) % MM_NB), ((it + 1) / MM_NB) & 1,
+                                                      bar_full_x((it + 1) % MM_NX), ((it + 1) / MM_NX) & 1);
+          } else {
+            // adapter step: rows r0 .. r0 + 63 of B as they lie in memory: 64-channel blocks 8 KiB apart
+            // (LBO), 8-row groups 1 KiB apart (SBO), 2 KiB per K = 16
+            const uint64_t lbdesc = ptx::smem_desc(smem_base + S::OFF_B + sb * MM_B_BYTES, 8192, 1024);
+            ready = ptx::mma4_ss_commit2_probe2<2, 128>(acc_tmem, adesc, lbdesc, IDESC_LORA, j > 0 ? 1u : 0u, bar_empty_x(sx),
+                                                        bar_empty_b(sb), bar_full_b((it + 1) % MM_NB), ((it + 1) / MM_NB) & 1,
+                                                        bar_full_x((it + 1) % MM_NX), ((it + 1) / MM_NX) & 1);
+          }
         }
         if (ok) ptx::mma_commit(bar_acc_full(ab));
       }
@@ -255,33 +265,38 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         const int sb = it % MM_NB, sc = cst % MM_NC;
         if (!(ok = ptx::mbar_wait(bar_empty_b(sb), ((it / MM_NB) & 1) ^ 1, abort_flag))) break;
         if (main_step && !(ok = ptx::mbar_wait(bar_full_c(sc), (cst / MM_NC) & 1, abort_flag))) break;
+        if (!main_step) {
+          // adapter step: the operand is a tile of B itself, rows r0 .. r0 + 63 for the tile's 256
+          // channels, brought by four tiled copies (64 channels each; rows beyond r arrive as zeros)
+          // straight into the operand slot.  No thread touches it: the group's first thread asks for
+          // the copies, every warp signs the slot off.
+          if (row == 0) {
+            const int r0 = (j - w.n_main) * MM_J;
+            QALORA_CHECK(p.dbg, r0, p.r);
+            QALORA_CHECK(p.dbg, c0 + MM_CH - 1, p.N);
+            ptx::mbar_arrive_expect_tx(bar_full_b(sb), MM_B_BYTES);
+#pragma unroll
+            for (int h = 0; h < 4; ++h)
+              ptx::tma_load_2d(smem_base + S::OFF_B + sb * MM_B_BYTES + h * 8192, &lb_map, c0 + 64 * h, r0, bar_full_b(sb));
+          } else if (lane == 0) {
+            ptx::mbar_arrive(bar_full_b(sb));
+          }
+          continue;
+        }
         const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         uint8_t* rowp = smem + S::OFF_B + sb * MM_B_BYTES + (row / 8) * 1024 + (row % 8) * 128;
         if (!QALORA_CHECK(p.dbg, S::OFF_B + sb * MM_B_BYTES + (row / 8) * 1024 + (row % 8) * 128 + 127, S::OFF_C)) continue;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {   // the two 32-index blocks of the step
           uint32_t v[16];
-          if (main_step) {
-            const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage + half_col * S::CODE_HALF) + (half * 128 + col_in_half) * WORDS;
-            if (!QALORA_CHECK(p.dbg, half_col * S::CODE_HALF / 4 + (half * 128 + col_in_half) * WORDS + WORDS - 1, S::CODE_BYTES / 4) ||
-                !QALORA_CHECK(p.dbg, half_col * 2 * 128 + (half >> qsh) * 128 + col_in_half, S::QP_BYTES / 8))
-              continue;
-            uint32_t wd[WORDS];
-            load_unit<WORDS>(cw, wd);
-            const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES + half_col * 2 * S::QP_HALF_ROW)[(half >> qsh) * 128 + col_in_half];
-            dequant_unit<BITS>(wd, ab, dk, v);
-          } else {
-            // adapter step: row c of the operand is B[r0 + 0..63][c]; this thread packs 32 of them
-            const int r0 = (j - w.n_main) * MM_J + half * 32;
-            const __nv_bfloat16* bp = p.lora_B + (size_t)r0 * p.N + c0 + row;
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              const int ra = r0 + 2 * q;
-              const uint32_t lo = ra < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q) * p.N) : 0u;
-              const uint32_t hi = ra + 1 < p.r ? *reinterpret_cast<const uint16_t*>(bp + (size_t)(2 * q + 1) * p.N) : 0u;
-              v[q] = lo | (hi << 16);
-            }
-          }
+          const uint32_t* cw = reinterpret_cast<const uint32_t*>(cstage + half_col * S::CODE_HALF) + (half * 128 + col_in_half) * WORDS;
+          if (!QALORA_CHECK(p.dbg, half_col * S::CODE_HALF / 4 + (half * 128 + col_in_half) * WORDS + WORDS - 1, S::CODE_BYTES / 4) ||
+              !QALORA_CHECK(p.dbg, half_col * 2 * 128 + (half >> qsh) * 128 + col_in_half, S::QP_BYTES / 8))
+            continue;
+          uint32_t wd[WORDS];
+          load_unit<WORDS>(cw, wd);
+          const float2 ab = reinterpret_cast<const float2*>(cstage + S::CODE_BYTES + half_col * 2 * S::QP_HALF_ROW)[(half >> qsh) * 128 + col_in_half];
+          dequant_unit<BITS>(wd, ab, dk, v);
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const int chunk = (half * 4 + q) ^ (row % 8);
@@ -374,7 +389,9 @@ int launch_midm_t(const CUtensorMap& xm, const CUtensorMap& tm, const MmParams& 
                   const float2* qparams, cudaStream_t st) {
   using S = MmSmem<BITS, XROWS>;
   static_assert(S::TOTAL <= 232448, "shared memory budget");
-  CUtensorMap cm, qm;
+  CUtensorMap cm, qm, lb = xm;
+  // with adapter: B [r][N] in boxes of 64 channels x 64 rows (rows beyond r read as zero)
+  if (p.r > 0 && !make_act_map(&lb, p.lora_B, p.r, p.N, MM_J)) return QALORA_ERR_CUDA;
   if (!make_codes_map(&cm, codes, p.K, p.N, BITS, 128, 2)) return QALORA_ERR_CUDA;
   if (!make_qp_map(&qm, qparams, p.K / p.g, p.N, 128, p.qp_rows)) return QALORA_ERR_CUDA;
   auto kern = qalora_midm_kernel<BITS, XROWS>;
@@ -385,7 +402,7 @@ int launch_midm_t(const CUtensorMap& xm, const CUtensorMap& tm, const MmParams& 
   const int grid = items < device_sm_count() ? items : device_sm_count();
   {
     MainKernelProbe probe("qalora_midm_kernel", st);
-    kern<<<grid, MM_THREADS, S::TOTAL, st>>>(xm, tm, cm, qm, p);
+    kern<<<grid, MM_THREADS, S::TOTAL, st>>>(xm, tm, lb, cm, qm, p);
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
