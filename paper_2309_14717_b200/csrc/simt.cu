@@ -105,14 +105,24 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
   }
 }
 
-// Streaming version for many rows and a group size of 32, 64 or 128: sixteen rows
-// per block, one warp per row.  A lane reads 16 bytes (8 channels) per step, so
-// g / 8 neighbouring lanes hold one group and a few shuffles finish its sum.
+// Streaming version for many rows and a group size of 32, 64 or 128: sixteen rows per block.
+// The group sums themselves run on the tensor cores: with an all-ones B operand,
+// mma.sync.m16n8k16 adds up the 16 reduction slots of each A row whatever their order, so a
+// lane feeds the 16 bytes it loaded from a row (8 channels) straight in as A registers, two
+// MMAs cover 16 rows x 32 channels, and the fp32 sums of the block's 16 rows come out in the
+// accumulator: four instructions per KiB of x instead of converting and adding element by
+// element, which had left the kernel bound by its instruction stream at half the copy rate.
+// Warp w takes the groups w, w + 16, ...; per load instruction the block reads 64 contiguous
+// bytes of each of its rows.
 // T = xp * A then runs on mma.sync.m16n8k16 with the block's 16 rows as the MMA rows
 // and the groups as the reduction dimension; xp enters as a bf16 pair hi + lo
 // (hi = xp rounded, lo = the remainder rounded: 16 significant bits together), so that
 // T keeps fp32-like accuracy although the operands are bf16.
 constexpr int POOL16_ROWS = 16;
+#ifndef QALORA_POOL16_WARPS
+#define QALORA_POOL16_WARPS 8
+#endif
+constexpr int POOL16_WARPS = QALORA_POOL16_WARPS;     // warps per block; several blocks per SM, so that one block's T phase hides behind the others' streaming
 
 __device__ __forceinline__ void mma_bf16_16816(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -131,7 +141,7 @@ __host__ __device__ inline int pool16_stride_words(int G) {
 }
 
 template <int LANES_PER_GROUP>   // g / 8: 4, 8 or 16
-__global__ void __launch_bounds__(POOL16_ROWS * 32, 2)
+__global__ void __launch_bounds__(POOL16_WARPS * 32, 1024 / (POOL16_WARPS * 32))
 pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ A,
                    float* __restrict__ xp_out, float* __restrict__ T, __nv_bfloat16* __restrict__ Tb,
                    long long M, int K, int G, int r, float s, int smem_words, int* dbg) {
@@ -141,57 +151,61 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
   __nv_bfloat16* xlo = reinterpret_cast<__nv_bfloat16*>(pool_smem + POOL16_ROWS * SW);
   float* part = reinterpret_cast<float*>(pool_smem + 2 * POOL16_ROWS * SW);        // [ksplit][16][r]
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const long long m = (long long)blockIdx.x * POOL16_ROWS + warp;
   const int Gp = (G + 15) / 16 * 16;
-  // the padding groups G .. Gp - 1 and the rows beyond M count as zero
-  for (int q = (m < M ? G : 0) + lane; q < Gp; q += 32) {
-    xhi[warp * 2 * SW + q] = __float2bfloat16_rn(0.f);
-    xlo[warp * 2 * SW + q] = __float2bfloat16_rn(0.f);
+  const long long row0 = (long long)blockIdx.x * POOL16_ROWS;
+  // the padding groups G .. Gp - 1 count as zero (rows beyond M load zeros below)
+  for (int i = threadIdx.x; i < POOL16_ROWS * (Gp - G); i += POOL16_WARPS * 32) {
+    const int row = i / (Gp - G), q = G + i % (Gp - G);
+    xhi[row * 2 * SW + q] = __float2bfloat16_rn(0.f);
+    xlo[row * 2 * SW + q] = __float2bfloat16_rn(0.f);
   }
-  if (m < M) {
-    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)m * K);
-    const int chunks = K / 8;                             // K is a multiple of 32
-    constexpr int BATCH = 4;                              // 16-byte loads per lane and batch
-    // two batches in flight: the loads of batch k + 1 are issued before batch k is summed, so
-    // that the rows keep streaming while the warp computes (chunks is a multiple of 32: K % 256 == 0)
-    uint4 v[2][BATCH];
-    auto load_batch = [&](int c0, uint4* dst) {
+  {
+    constexpr int CPG = LANES_PER_GROUP / 4;              // 32-channel chunks per group
+    constexpr int UNR = 4 / CPG;                          // groups whose loads are in flight together (8 x 16 bytes per lane)
+    constexpr uint32_t ONES = 0x3f803f80u;                // bf16x2 (1, 1)
+    const int fr = lane / 4, t4 = lane % 4;               // fragment rows fr and fr + 8; this lane's 8 channels of a chunk
+    const long long ra = row0 + fr, rb = row0 + fr + 8;
+    const bool la = ra < M, lb = rb < M;
+    const uint4* xa = reinterpret_cast<const uint4*>(x + (size_t)(la ? ra : 0) * K) + t4;   // + 4 per chunk
+    const uint4* xb = reinterpret_cast<const uint4*>(x + (size_t)(lb ? rb : 0) * K) + t4;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    for (int qb = warp; qb < G; qb += POOL16_WARPS * UNR) {
+      uint4 va[UNR][CPG], vb[UNR][CPG];
 #pragma unroll
-      for (int b = 0; b < BATCH; ++b) {
-        const int c = c0 + b * 32 + lane;
-        dst[b] = c < chunks ? xr[c] : make_uint4(0u, 0u, 0u, 0u);
-      }
-    };
-    auto sum_batch = [&](int c0, const uint4* src) {
+      for (int u = 0; u < UNR; ++u) {
+        const int q = qb + u * POOL16_WARPS;
 #pragma unroll
-      for (int b = 0; b < BATCH; ++b) {
-        const int c = c0 + b * 32 + lane;
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&src[b]);
-        float acc = 0.0f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 f = __bfloat1622float2(h[i]);
-          acc += f.x + f.y;
+        for (int c = 0; c < CPG; ++c) {
+          const bool in = q < G && QALORA_CHECK(dbg, ((size_t)q * CPG + c) * 32 + t4 * 8 + 7, K);
+          va[u][c] = in && la ? __ldg(xa + ((size_t)q * CPG + c) * 4) : zero;
+          vb[u][c] = in && lb ? __ldg(xb + ((size_t)q * CPG + c) * 4) : zero;
         }
+      }
 #pragma unroll
-        for (int o = 1; o < LANES_PER_GROUP; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (c < chunks && (lane % LANES_PER_GROUP) == 0) {
-          const int q = c / LANES_PER_GROUP;
-          const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
-          if (QALORA_CHECK(dbg, warp * 2 * SW + q, POOL16_ROWS * 2 * SW)) {
-            xhi[warp * 2 * SW + q] = hi;
-            xlo[warp * 2 * SW + q] = __float2bfloat16_rn(acc - __bfloat162float(hi));
+      for (int u = 0; u < UNR; ++u) {
+        const int q = qb + u * POOL16_WARPS;
+        if (q >= G) break;
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < CPG; ++c) {
+          const uint32_t a0[4] = {va[u][c].x, vb[u][c].x, va[u][c].y, vb[u][c].y};
+          const uint32_t a1[4] = {va[u][c].z, vb[u][c].z, va[u][c].w, vb[u][c].w};
+          mma_bf16_16816(d, a0, ONES, ONES);
+          mma_bf16_16816(d, a1, ONES, ONES);
+        }
+        // every column of the product holds the row's sum: d[0] for row fr, d[2] for row fr + 8
+        if (t4 == 0 && QALORA_CHECK(dbg, (fr + 8) * 2 * SW + q, POOL16_ROWS * 2 * SW)) {
+          const __nv_bfloat16 ha = __float2bfloat16_rn(d[0]), hb = __float2bfloat16_rn(d[2]);
+          xhi[fr * 2 * SW + q] = ha;
+          xlo[fr * 2 * SW + q] = __float2bfloat16_rn(d[0] - __bfloat162float(ha));
+          xhi[(fr + 8) * 2 * SW + q] = hb;
+          xlo[(fr + 8) * 2 * SW + q] = __float2bfloat16_rn(d[2] - __bfloat162float(hb));
+          if (xp_out != nullptr) {
+            if (la && QALORA_CHECK(dbg, (size_t)ra * G + q, (size_t)M * G)) xp_out[(size_t)ra * G + q] = d[0];
+            if (lb && QALORA_CHECK(dbg, (size_t)rb * G + q, (size_t)M * G)) xp_out[(size_t)rb * G + q] = d[2];
           }
-          if (xp_out != nullptr && QALORA_CHECK(dbg, (size_t)m * G + q, (size_t)M * G)) xp_out[(size_t)m * G + q] = acc;
         }
       }
-    };
-    load_batch(0, v[0]);
-    for (int c0 = 0; c0 < chunks; c0 += 2 * 32 * BATCH) {
-      load_batch(c0 + 32 * BATCH, v[1]);
-      sum_batch(c0, v[0]);
-      load_batch(c0 + 2 * 32 * BATCH, v[0]);
-      sum_batch(c0 + 32 * BATCH, v[1]);
     }
   }
   __syncthreads();
@@ -199,12 +213,12 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
   // over several warps (ksplit parts), whose sums meet in shared memory
   const int ntiles = r / 8;                               // r is a multiple of 8
   int ksplit = 1;
-  while (ksplit * 2 * ntiles <= POOL16_ROWS) ksplit *= 2;
+  while (ksplit * 2 * ntiles <= POOL16_WARPS) ksplit *= 2;
   const int gq = lane / 4, t = lane % 4;
   const uint32_t* hi32 = pool_smem;
   const uint32_t* lo32 = pool_smem + POOL16_ROWS * SW;
   const uint16_t* A16 = reinterpret_cast<const uint16_t*>(A);
-  for (int job = warp; job < ntiles * ksplit; job += POOL16_ROWS) {
+  for (int job = warp; job < ntiles * ksplit; job += POOL16_WARPS) {
     const int nt = job % ntiles, part_i = job / ntiles;
     const int n = nt * 8 + gq;                            // this lane's column of A
     float d[4] = {0.f, 0.f, 0.f, 0.f};
@@ -234,7 +248,7 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
     }
   }
   __syncthreads();
-  for (int o = threadIdx.x; o < POOL16_ROWS * r; o += POOL16_ROWS * 32) {
+  for (int o = threadIdx.x; o < POOL16_ROWS * r; o += POOL16_WARPS * 32) {
     const long long mm = (long long)blockIdx.x * POOL16_ROWS + o / r;
     float v = 0.f;
     for (int pi = 0; pi < ksplit; ++pi) v += part[(size_t)pi * POOL16_ROWS * r + o];
@@ -251,7 +265,7 @@ constexpr size_t kPool16MaxSmem = 96 * 1024;
 static size_t pool16_smem_bytes(int G, int r) {
   const int ntiles = r / 8;
   int ksplit = 1;
-  while (ksplit * 2 * ntiles <= POOL16_ROWS) ksplit *= 2;
+  while (ksplit * 2 * ntiles <= POOL16_WARPS) ksplit *= 2;
   return (size_t)2 * POOL16_ROWS * pool16_stride_words(G) * 4 + (size_t)ksplit * POOL16_ROWS * r * 4;
 }
 
@@ -271,9 +285,9 @@ int launch_pool_T(const Shape& sh, int64_t M, const __nv_bfloat16* x, const __nv
     });
     if (attr_st != QALORA_OK) return attr_st;
     const unsigned grid = (unsigned)((M + POOL16_ROWS - 1) / POOL16_ROWS);
-    if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
-    else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
-    else pool_T_rows_kernel<16><<<grid, POOL16_ROWS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
+    if (sh.g == 32) pool_T_rows_kernel<4><<<grid, POOL16_WARPS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
+    else if (sh.g == 64) pool_T_rows_kernel<8><<<grid, POOL16_WARPS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
+    else pool_T_rows_kernel<16><<<grid, POOL16_WARPS * 32, smem, st>>>(x, A, xp, T, Tb, M, sh.K, sh.G, sh.r, sh.s, (int)(smem / 4), debug_words());
   } else {
     dim3 grid((unsigned)M, (unsigned)((sh.r + 31) / 32 > 0 ? (sh.r + 31) / 32 : 1));
     const size_t xp_bytes = ((size_t)sh.G * sizeof(float) + 15) / 16 * 16, a_bytes = (size_t)sh.G * 32 * sizeof(__nv_bfloat16);
