@@ -108,12 +108,11 @@ pool_T_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
 // Streaming version for many rows and a group size of 32, 64 or 128: sixteen rows per block.
 // The group sums themselves run on the tensor cores: with an all-ones B operand,
 // mma.sync.m16n8k16 adds up the 16 reduction slots of each A row whatever their order, so a
-// lane feeds the 16 bytes it loaded from a row (8 channels) straight in as A registers, two
-// MMAs cover 16 rows x 32 channels, and the fp32 sums of the block's 16 rows come out in the
-// accumulator: four instructions per KiB of x instead of converting and adding element by
+// lane feeds the 16 bytes it loaded (8 channels) straight in as A registers, two MMAs cover
+// 16 groups x 32 channels, and the fp32 group sums come out in the accumulator: four instructions per KiB of x instead of converting and adding element by
 // element, which had left the kernel bound by its instruction stream at half the copy rate.
-// Warp w takes the groups w, w + 16, ...; per load instruction the block reads 64 contiguous
-// bytes of each of its rows.
+// A warp takes one row of x at a time and lets 16 consecutive GROUPS of it be the MMA's 16
+// rows, so that (g = 32) each of its load instructions reads 512 contiguous bytes.
 // T = xp * A then runs on mma.sync.m16n8k16 with the block's 16 rows as the MMA rows
 // and the groups as the reduction dimension; xp enters as a bf16 pair hi + lo
 // (hi = xp rounded, lo = the remainder rounded: 16 significant bits together), so that
@@ -160,49 +159,60 @@ pool_T_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __r
     xlo[row * 2 * SW + q] = __float2bfloat16_rn(0.f);
   }
   {
-    constexpr int CPG = LANES_PER_GROUP / 4;              // 32-channel chunks per group
-    constexpr int UNR = 4 / CPG;                          // groups whose loads are in flight together (8 x 16 bytes per lane)
+    constexpr int CPG = LANES_PER_GROUP / 4;              // 32-channel chunks (64 bytes) per group
+    constexpr int UNR = 4 / CPG;                          // sets of 16 groups whose loads are in flight together (8 x 16 bytes per lane)
     constexpr uint32_t ONES = 0x3f803f80u;                // bf16x2 (1, 1)
-    const int fr = lane / 4, t4 = lane % 4;               // fragment rows fr and fr + 8; this lane's 8 channels of a chunk
-    const long long ra = row0 + fr, rb = row0 + fr + 8;
-    const bool la = ra < M, lb = rb < M;
-    const uint4* xa = reinterpret_cast<const uint4*>(x + (size_t)(la ? ra : 0) * K) + t4;   // + 4 per chunk
-    const uint4* xb = reinterpret_cast<const uint4*>(x + (size_t)(lb ? rb : 0) * K) + t4;
+    // The 16 "rows" of the MMA are 16 consecutive GROUPS of one row of x: lanes 4v .. 4v + 3
+    // hold the 64 bytes of a chunk of group v (a0, a2) and of group v + 8 (a1, a3), so with
+    // g = 32 a load instruction of the warp reads 512 contiguous bytes.
+    const int v = lane / 4, t4 = lane % 4;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    for (int qb = warp; qb < G; qb += POOL16_WARPS * UNR) {
-      uint4 va[UNR][CPG], vb[UNR][CPG];
-#pragma unroll
-      for (int u = 0; u < UNR; ++u) {
-        const int q = qb + u * POOL16_WARPS;
-#pragma unroll
-        for (int c = 0; c < CPG; ++c) {
-          const bool in = q < G && QALORA_CHECK(dbg, ((size_t)q * CPG + c) * 32 + t4 * 8 + 7, K);
-          va[u][c] = in && la ? __ldg(xa + ((size_t)q * CPG + c) * 4) : zero;
-          vb[u][c] = in && lb ? __ldg(xb + ((size_t)q * CPG + c) * 4) : zero;
+    for (int rr = warp; rr < POOL16_ROWS; rr += POOL16_WARPS) {
+      const long long m = row0 + rr;
+      if (m >= M) {                                       // rows beyond M count as zero
+        for (int q = lane; q < G; q += 32) {
+          xhi[rr * 2 * SW + q] = __float2bfloat16_rn(0.f);
+          xlo[rr * 2 * SW + q] = __float2bfloat16_rn(0.f);
         }
+        continue;
       }
+      const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)m * K) + t4;   // + 4 per chunk
+      for (int qb = 0; qb < G; qb += 16 * UNR) {
+        uint4 va[UNR][CPG], vb[UNR][CPG];
 #pragma unroll
-      for (int u = 0; u < UNR; ++u) {
-        const int q = qb + u * POOL16_WARPS;
-        if (q >= G) break;
-        float d[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int u = 0; u < UNR; ++u) {
+          const int qa = qb + 16 * u + v, qh = qa + 8;    // this lane's two groups of the set
 #pragma unroll
-        for (int c = 0; c < CPG; ++c) {
-          const uint32_t a0[4] = {va[u][c].x, vb[u][c].x, va[u][c].y, vb[u][c].y};
-          const uint32_t a1[4] = {va[u][c].z, vb[u][c].z, va[u][c].w, vb[u][c].w};
-          mma_bf16_16816(d, a0, ONES, ONES);
-          mma_bf16_16816(d, a1, ONES, ONES);
+          for (int c = 0; c < CPG; ++c) {
+            va[u][c] = qa < G && QALORA_CHECK(dbg, ((size_t)qa * CPG + c) * 32 + t4 * 8 + 7, K) ? __ldg(xr + ((size_t)qa * CPG + c) * 4) : zero;
+            vb[u][c] = qh < G && QALORA_CHECK(dbg, ((size_t)qh * CPG + c) * 32 + t4 * 8 + 7, K) ? __ldg(xr + ((size_t)qh * CPG + c) * 4) : zero;
+          }
         }
-        // every column of the product holds the row's sum: d[0] for row fr, d[2] for row fr + 8
-        if (t4 == 0 && QALORA_CHECK(dbg, (fr + 8) * 2 * SW + q, POOL16_ROWS * 2 * SW)) {
-          const __nv_bfloat16 ha = __float2bfloat16_rn(d[0]), hb = __float2bfloat16_rn(d[2]);
-          xhi[fr * 2 * SW + q] = ha;
-          xlo[fr * 2 * SW + q] = __float2bfloat16_rn(d[0] - __bfloat162float(ha));
-          xhi[(fr + 8) * 2 * SW + q] = hb;
-          xlo[(fr + 8) * 2 * SW + q] = __float2bfloat16_rn(d[2] - __bfloat162float(hb));
-          if (xp_out != nullptr) {
-            if (la && QALORA_CHECK(dbg, (size_t)ra * G + q, (size_t)M * G)) xp_out[(size_t)ra * G + q] = d[0];
-            if (lb && QALORA_CHECK(dbg, (size_t)rb * G + q, (size_t)M * G)) xp_out[(size_t)rb * G + q] = d[2];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+          const int qa = qb + 16 * u + v, qh = qa + 8;
+          float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int c = 0; c < CPG; ++c) {
+            const uint32_t a0[4] = {va[u][c].x, vb[u][c].x, va[u][c].y, vb[u][c].y};
+            const uint32_t a1[4] = {va[u][c].z, vb[u][c].z, va[u][c].w, vb[u][c].w};
+            mma_bf16_16816(d, a0, ONES, ONES);
+            mma_bf16_16816(d, a1, ONES, ONES);
+          }
+          // every column of the product holds the sums: d[0] for group qa, d[2] for group qh
+          if (t4 == 0) {
+            if (qa < G && QALORA_CHECK(dbg, rr * 2 * SW + qa, POOL16_ROWS * 2 * SW)) {
+              const __nv_bfloat16 h = __float2bfloat16_rn(d[0]);
+              xhi[rr * 2 * SW + qa] = h;
+              xlo[rr * 2 * SW + qa] = __float2bfloat16_rn(d[0] - __bfloat162float(h));
+              if (xp_out != nullptr && QALORA_CHECK(dbg, (size_t)m * G + qa, (size_t)M * G)) xp_out[(size_t)m * G + qa] = d[0];
+            }
+            if (qh < G && QALORA_CHECK(dbg, rr * 2 * SW + qh, POOL16_ROWS * 2 * SW)) {
+              const __nv_bfloat16 h = __float2bfloat16_rn(d[2]);
+              xhi[rr * 2 * SW + qh] = h;
+              xlo[rr * 2 * SW + qh] = __float2bfloat16_rn(d[2] - __bfloat162float(h));
+              if (xp_out != nullptr && QALORA_CHECK(dbg, (size_t)m * G + qh, (size_t)M * G)) xp_out[(size_t)m * G + qh] = d[2];
+            }
           }
         }
       }
@@ -563,14 +573,31 @@ atb_partial_kernel(const float* __restrict__ X, const TY* __restrict__ Y, float*
   const long long mbeg = (long long)blockIdx.z * rows_per_split;
   const long long mend = min(M, mbeg + rows_per_split);
   float acc[4][4] = {};
-  for (long long m0 = mbeg; m0 < mend; m0 += TK) {
-    for (int e = tid; e < TK * TM; e += SIMT_THREADS) {
+  // The block's share of rows is short (a few 32-row steps), so the kernel is bound by the
+  // latency of its loads: the next step's elements are fetched into registers while the
+  // current step is multiplied out of shared memory.
+  constexpr int PER = TK * TM / SIMT_THREADS;             // elements of each tile per thread
+  float xr[PER], yr[PER];
+  auto fetch = [&](long long m0) {
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = tid + i * SIMT_THREADS;
       const int mm = e / TM, c = e % TM;
       const long long m = m0 + mm;
-      xs[mm][c] = (m < mend && p0 + c < P) ? __ldg(X + (size_t)m * P + p0 + c) : 0.0f;
-      ys[mm][c] = (m < mend && q0 + c < Q) ? load_as_float<TY>(Y + (size_t)m * Q + q0 + c) : 0.0f;
+      xr[i] = (m < mend && p0 + c < P) ? __ldg(X + (size_t)m * P + p0 + c) : 0.0f;
+      yr[i] = (m < mend && q0 + c < Q) ? load_as_float<TY>(Y + (size_t)m * Q + q0 + c) : 0.0f;
+    }
+  };
+  if (mbeg < mend) fetch(mbeg);
+  for (long long m0 = mbeg; m0 < mend; m0 += TK) {
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = tid + i * SIMT_THREADS;
+      xs[e / TM][e % TM] = xr[i];
+      ys[e / TM][e % TM] = yr[i];
     }
     __syncthreads();
+    if (m0 + TK < mend) fetch(m0 + TK);
 #pragma unroll 8
     for (int mm = 0; mm < TK; ++mm) {
       const float4 a = *reinterpret_cast<const float4*>(&xs[mm][ty * 4]);
