@@ -140,7 +140,7 @@ __device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, const F
 // k-blocks a warp set takes from a stage share (alpha, beta) and are folded together.
 // The work of one block: `block` is its index among the blocks of the layer described by p
 // (a layer's blocks are consecutive in the grid, a whole number of clusters).
-template <int BITS, int NTS, bool CHAIN>
+template <int BITS, int NTS, bool CHAIN, bool ONE = false>   // ONE: a single token row (M == 1; NTS == 1)
 __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUtensorMap& codes_map,
                                            const CUtensorMap& qp_map, const GvParams& p, const int block) {
   using S = GvSmem<BITS, NTS>;
@@ -336,10 +336,11 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
           q1.y = fmaf(-128.f, q1.x, q1.y);
 #pragma unroll
           for (int ts = 0; ts < NTS; ++ts) {
+            // (with one token row the odd token column of the fragment is all padding: not folded)
             acc[cg][ts][0] = fmaf(q0.x, D[ts][0], fmaf(q0.y, xp[ts][0], acc[cg][ts][0]));
-            acc[cg][ts][1] = fmaf(q0.x, D[ts][1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
+            if constexpr (!ONE) acc[cg][ts][1] = fmaf(q0.x, D[ts][1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
             acc[cg][ts][2] = fmaf(q1.x, D[ts][2], fmaf(q1.y, xp[ts][0], acc[cg][ts][2]));
-            acc[cg][ts][3] = fmaf(q1.x, D[ts][3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
+            if constexpr (!ONE) acc[cg][ts][3] = fmaf(q1.x, D[ts][3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
           }
         }
       } else {
@@ -380,9 +381,9 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
               mma16816(D, a0, xs[ts].x, xs[ts].y, zero4);
               mma16816(D, a1, xs[ts].z, xs[ts].w, D);
               acc[cg][ts][0] = fmaf(q0.x, D[0], fmaf(q0.y, xp[ts][0], acc[cg][ts][0]));
-              acc[cg][ts][1] = fmaf(q0.x, D[1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
+              if constexpr (!ONE) acc[cg][ts][1] = fmaf(q0.x, D[1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
               acc[cg][ts][2] = fmaf(q1.x, D[2], fmaf(q1.y, xp[ts][0], acc[cg][ts][2]));
-              acc[cg][ts][3] = fmaf(q1.x, D[3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
+              if constexpr (!ONE) acc[cg][ts][3] = fmaf(q1.x, D[3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
             }
           }
         }
@@ -469,11 +470,11 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
   if (threadIdx.x == 0 && *abort_flag != 0) atomicExch(p.status, 1);
 }
 
-template <int BITS, int NTS, bool CHAIN>
+template <int BITS, int NTS, bool CHAIN, bool ONE = false>
 __global__ void __launch_bounds__(GV_THREADS, NTS == 4 ? 2 : 3)
 qalora_gemv_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap codes_map,
                    const __grid_constant__ CUtensorMap qp_map, const GvParams p) {
-  gemv_block<BITS, NTS, CHAIN>(x_map, codes_map, qp_map, p, (int)blockIdx.x);
+  gemv_block<BITS, NTS, CHAIN, ONE>(x_map, codes_map, qp_map, p, (int)blockIdx.x);
 }
 
 // Several layers in ONE launch (the projections of a transformer block that read finished
@@ -577,12 +578,12 @@ cudaError_t launch_clustered(Kernel kern, unsigned blocks, int splits, size_t sm
   return e;
 }
 
-template <int BITS, int NTS, bool CHAIN>
+template <int BITS, int NTS, bool CHAIN, bool ONE = false>
 int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStream_t st) {
   using S = GvSmem<BITS, NTS>;
   CUtensorMap cm, qm;
   if (!make_weight_maps(p, S::WORDS, &cm, &qm)) return QALORA_ERR_CUDA;
-  auto kern = qalora_gemv_kernel<BITS, NTS, CHAIN>;
+  auto kern = qalora_gemv_kernel<BITS, NTS, CHAIN, ONE>;
   static PerDeviceOnce smem_limit;      // this instantiation's shared-memory limit, raised once on every device it runs on
   if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
     return QALORA_ERR_CUDA;
@@ -681,11 +682,13 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   const bool chain = sh.g >= 64;
 #define QALORA_GV_N(BITS, NTS) (chain ? launch_gemv_t<BITS, NTS, true>(xm, p, splits, st) : launch_gemv_t<BITS, NTS, false>(xm, p, splits, st))
 // (32 rows: the per-k-block fold for every group size; the chained form runs out of registers there)
-#define QALORA_GV(BITS) (nts == 4 ? launch_gemv_t<BITS, 4, false>(xm, p, splits, st) : (nts == 2 ? QALORA_GV_N(BITS, 2) : QALORA_GV_N(BITS, 1)))
+#define QALORA_GV_1(BITS) (chain ? launch_gemv_t<BITS, 1, true, true>(xm, p, splits, st) : launch_gemv_t<BITS, 1, false, true>(xm, p, splits, st))
+#define QALORA_GV(BITS) (nts == 4 ? launch_gemv_t<BITS, 4, false>(xm, p, splits, st) : (nts == 2 ? QALORA_GV_N(BITS, 2) : (M == 1 ? QALORA_GV_1(BITS) : QALORA_GV_N(BITS, 1))))
   if (sh.bits == 4) return QALORA_GV(4);
   if (sh.bits == 3) return QALORA_GV(3);
   return QALORA_GV(2);
 #undef QALORA_GV
+#undef QALORA_GV_1
 #undef QALORA_GV_N
 }
 
