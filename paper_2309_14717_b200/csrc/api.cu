@@ -354,6 +354,15 @@ int qalora_debug_expire_next_few_token_wait(int stages, uint64_t limit_ns) {
   return QALORA_OK;
 }
 
+// The same for the tensor-core forward / dX kernels: the next such launch of this process has
+// its activation producers stop after `steps` reduction steps, and its waits give up after
+// `limit_ns`.  Test hook, not declared in the public header.
+int qalora_debug_expire_next_tc_wait(int steps, uint64_t limit_ns) {
+  if (limit_ns == 0 || limit_ns > 2000000000ull) return QALORA_ERR_INVALID_ARG;
+  arm_tc_wait_expiry(steps, limit_ns);
+  return QALORA_OK;
+}
+
 int qalora_debug_checks(void) { return kDebugBuild ? 1 : 0; }
 
 // Test hook, not declared in the public header: shows that the bounds-check build's record

@@ -147,6 +147,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
                 cudaStream_t st);
 
 void arm_few_token_wait_expiry(int stages, unsigned long long limit_ns);   // test hook, one-shot
+void arm_tc_wait_expiry(int steps, unsigned long long limit_ns);           // the same for the next forward / dX tensor-core launch
 
 // Several layers without adapter, the same M <= 16 rows each, in ONE few-token launch.
 struct GemvGroupItem {

@@ -65,6 +65,8 @@ struct TcParams {
   float* partial;              // ksplit > 1: fp32 [ksplit][M][ld_out] partial results
   int* status;                 // device word: set to 1 when a wait timed out
   int* dbg;                    // record words of the bounds-check build (null otherwise)
+  int stop_after_steps;        // normally INT_MAX; a test makes every activation producer stop early, so that waits expire
+  unsigned long long wait_limit_ns;
 };
 
 // Work item of a block: part `sp` of tile `tile`, i.e. the main steps mb .. mb + n_main - 1
@@ -207,10 +209,11 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         const int m0 = (sg.tile / p.c_tiles) * TT;
         const int c0 = (sg.tile % p.c_tiles) * TILE_C;
         for (int j = 0; j < sg.n_steps; ++j, ++it) {
+          if (it >= (uint32_t)p.stop_after_steps) { ok = false; break; }     // (test hook: the tiles stop coming)
           const int i = tc_step<PARTS>(p, sg, j);
           const int s = it % NX, sb = it % NB;
           // the tile slot was last used by step it - NX: wait until that step has been multiplied
-          if (it >= (uint32_t)NX && !(ok = ptx::mbar_wait(bar_empty_x((it - NX) % NB), ((it - NX) / NB) & 1, abort_flag))) break;
+          if (it >= (uint32_t)NX && !(ok = ptx::mbar_wait(bar_empty_x((it - NX) % NB), ((it - NX) / NB) & 1, abort_flag, p.wait_limit_ns))) break;
           // (bounds-check build: the tile lies inside its ring and the copy starts inside the matrix)
           QALORA_CHECK(p.dbg, S::OFF_X + (s + 1) * ACT_BYTES - 1, S::OFF_A);
           QALORA_CHECK(p.dbg, m0, p.M);
@@ -225,7 +228,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
             const int r0 = (i - p.red_iters) * TILE_J;
             QALORA_CHECK(p.dbg, r0, p.r);
             QALORA_CHECK(p.dbg, c0 + TILE_C - 1, p.N);
-            if (!(ok = ptx::mbar_wait(bar_lb_empty, (nlb & 1) ^ 1, abort_flag))) break;
+            if (!(ok = ptx::mbar_wait(bar_lb_empty, (nlb & 1) ^ 1, abort_flag, p.wait_limit_ns))) break;
             ++nlb;
             ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES + ATILE_BYTES);
             ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &lora_map, r0, m0, bar_full_x(sb));
@@ -249,7 +252,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         const int cs_end = (sg.mb + sg.n_main) / S::IPS;
         for (int cs = sg.mb / S::IPS; cs < cs_end; ++cs, ++cit) {
           const int s = cit % NC;
-          if (!(ok = ptx::mbar_wait(bar_empty_c(s), ((cit / NC) & 1) ^ 1, abort_flag))) break;
+          if (!(ok = ptx::mbar_wait(bar_empty_c(s), ((cit / NC) & 1) ^ 1, abort_flag, p.wait_limit_ns))) break;
           const uint32_t stage = smem_base + S::OFF_C + s * S::CSTAGE_BYTES;
           // forward: k-blocks 4 cs .. 4 cs + 3 of columns c0 ..; dx: the tile's 4 k-blocks, columns 64 cs ..
           const int kb0 = MODE == FWD ? cs * 4 : c0 / 32;
@@ -282,12 +285,12 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         const int ab = tcount % NACC;                 // accumulator of this tile
         const uint32_t acc_tmem = tmem_base + ACC_COL + ab * TILE_T;
         QALORA_CHECK(p.dbg, ACC_COL + ab * TILE_T + TT - 1, MODE == FWD ? A_COL : TMEM_COLS);
-        if (!(ok = ptx::mbar_wait(bar_acc_empty(ab), ((tcount / NACC) & 1) ^ 1, abort_flag))) break;
+        if (!(ok = ptx::mbar_wait(bar_acc_empty(ab), ((tcount / NACC) & 1) ^ 1, abort_flag, p.wait_limit_ns))) break;
         ptx::tc_fence_after();
         for (int j = 0; j < sg.n_steps; ++j, ++it) {
           const int sx = it % NX, sb = it % NB;
           const uint32_t ph = (it / NB) & 1;
-          if (!ready && !(ok = ptx::mbar_wait(bar_full_x(sb), ph, abort_flag))) break;
+          if (!ready && !(ok = ptx::mbar_wait(bar_full_x(sb), ph, abort_flag, p.wait_limit_ns))) break;
           ptx::tc_fence_after();
           const uint32_t xs = smem_base + S::OFF_X + sx * ACT_BYTES;
           const uint32_t as = smem_base + S::OFF_A + sb * ATILE_BYTES;     // dx: NB == NX
@@ -336,11 +339,11 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         const int sa = it % NB;
         // operand slot first: once it is free every earlier step has been multiplied, so
         // the code ring's previous phase has certainly completed
-        if (!(ok = ptx::mbar_wait(bar_empty_x(sa), ((it / NB) & 1) ^ 1, abort_flag))) break;
+        if (!(ok = ptx::mbar_wait(bar_empty_x(sa), ((it / NB) & 1) ^ 1, abort_flag, p.wait_limit_ns))) break;
         const uint32_t cst = (mit0 + j) / S::IPS;  // code stage counter (main steps only; mit0 stays even)
         const int sc = cst % NC;
         const int kb_base = MODE == FWD ? ((mit0 + j) % S::IPS) * 2 : 0;   // first k-block row of this step
-        if (i < p.red_iters && !(ok = ptx::mbar_wait(bar_full_c(sc), (cst / NC) & 1, abort_flag))) break;
+        if (i < p.red_iters && !(ok = ptx::mbar_wait(bar_full_c(sc), (cst / NC) & 1, abort_flag, p.wait_limit_ns))) break;
         const uint8_t* cstage = smem + S::OFF_C + sc * S::CSTAGE_BYTES;
         if (MODE == FWD) {
           // (an adapter step needs nothing from this group: its operands both come by TMA; the
@@ -435,7 +438,11 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       const int tile = PARTS ? vt / p.ksplit : vt, sp = PARTS ? vt % p.ksplit : 0;
       const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
       const int ab = tcount % NACC;
-      if (!(ok = ptx::mbar_wait(bar_acc_full(ab), (tcount / NACC) & 1, abort_flag))) break;
+      // The four warps meet at barriers below, so they must agree on leaving: a thread whose wait
+      // gave up (the abort flag was raised elsewhere) and a thread that saw the phase complete in
+      // the same instant would otherwise part ways.
+      ok = ptx::mbar_wait(bar_acc_full(ab), (tcount / NACC) & 1, abort_flag, p.wait_limit_ns);
+      if (!(ok = ptx::named_barrier_and(3, 128, ok))) break;
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int col = 0; col < TT; col += 32, ++chunk) {
@@ -618,6 +625,21 @@ int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p
 
 }  // namespace
 
+// Test hook (qalora_debug_expire_next_tc_wait in api.cu): when armed, the activation producers
+// of the next forward or dX launch stop after `steps` reduction steps and the launch's waits give
+// up after `limit_ns`: every role's bounded wait runs out, the status word is raised and the
+// blocks leave through their ordinary teardown (tensor memory released).  One-shot.
+static std::atomic<int> g_tc_expire_after_steps{0x7fffffff};
+static std::atomic<unsigned long long> g_tc_expire_limit_ns{ptx::WAIT_LIMIT_NS};
+void arm_tc_wait_expiry(int steps, unsigned long long limit_ns) {
+  g_tc_expire_limit_ns.store(limit_ns);
+  g_tc_expire_after_steps.store(steps < 0 ? 0 : steps);
+}
+static void take_expiry(TcParams* p) {
+  p->stop_after_steps = g_tc_expire_after_steps.exchange(0x7fffffff);
+  p->wait_limit_ns = p->stop_after_steps != 0x7fffffff ? g_tc_expire_limit_ns.load() : ptx::WAIT_LIMIT_NS;
+}
+
 static bool tc_group_ok(int g) { return g == 32 || g == 64 || g == 128; }
 
 bool tc_forward_supported(const Shape& sh, int64_t M) {
@@ -681,6 +703,7 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
   p.c_tiles = sh.N / TILE_C; p.m_tiles = (int)((M + tile_t - 1) / tile_t);
   p.red_iters = sh.K / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
   p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
+  take_expiry(&p);
   p.ksplit = parts < 0 ? -parts : parts; p.tile_t = tile_t; p.partial = partial;
   if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, p, st);
@@ -701,6 +724,7 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
   p.c_tiles = sh.K / TILE_C; p.m_tiles = (int)((M + TILE_T - 1) / TILE_T);
   p.red_iters = sh.N / TILE_J; p.lora_iters = (sh.r + TILE_J - 1) / TILE_J;
   p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
+  take_expiry(&p);
   p.ksplit = 1; p.tile_t = TILE_T; p.partial = nullptr;
   if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);

@@ -379,6 +379,53 @@ def test_an_expired_wait_raises_the_status_word_and_the_next_call_is_clean():
     assert torch.equal(after, before)
 
 
+def test_an_expired_wait_in_the_tensor_core_kernels_unwinds_and_the_next_call_is_clean():
+    """The same for the tensor-core forward and dX kernels: the hook makes the activation producers
+    of ONE launch stop after two reduction steps (every block is then in the middle of its first
+    tile) and shortens that launch's wait limit to a millisecond.  Every role's bounded wait runs
+    out, the blocks leave through their ordinary teardown (tensor memory released), the status word
+    reads 1, and the following ordinary call gives the same bits as the one before."""
+    import ctypes
+    cfg = LayerConfig("expire_tc", 1024, 512, 32, 4, 16, 1.0, 512, seed=12)   # 8 tiles of 16 (+1) steps: one per block
+    layer = GpuLayer(cfg)
+    lib = Q.load()
+    hook = lib.qalora_debug_expire_next_tc_wait
+    hook.restype = ctypes.c_int
+    hook.argtypes = [ctypes.c_int, ctypes.c_uint64]
+    M, d = cfg.tokens, layer.d
+    A, B = layer.dev["A"], layer.dev["B"]
+
+    def fwd(ws):
+        y = torch.empty((M, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+        Q.qalora_forward(d, M, layer.dev["x"], layer.codes, layer.qparams, A, B, y, ws)
+        torch.cuda.synchronize()                          # returns: the kernel gave up by itself
+        return y
+
+    def bwd(ws):
+        dx = torch.empty((M, cfg.d_in), dtype=torch.bfloat16, device="cuda")
+        dA = torch.empty((cfg.groups, cfg.rank), dtype=torch.float32, device="cuda")
+        dB = torch.empty((cfg.rank, cfg.d_out), dtype=torch.float32, device="cuda")
+        Q.qalora_backward(d, M, layer.dev["x"], layer.dev["dy"], layer.codes, layer.qparams, A, B, dx, dA, dB, ws)
+        torch.cuda.synchronize()
+        return dx
+
+    for run, op, kernel in ((fwd, Q.OP_FORWARD, "qalora_tc_kernel<fwd>"), (bwd, Q.OP_BACKWARD, "qalora_tc_kernel<dx>")):
+        ws = Q.alloc_workspace(d, M, op)
+        before = run(ws)
+        assert Q.qalora_main_kernel_name() == kernel and Q.workspace_status(ws) == 0
+        assert hook(2, 1_000_000) == 0
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        run(ws)
+        t1.record()
+        torch.cuda.synchronize()
+        assert Q.workspace_status(ws) == 1
+        assert t0.elapsed_time(t1) < 1000.0               # ms: far below the ordinary two-second limit
+        after = run(ws)
+        assert Q.workspace_status(ws) == 0                # the hook was one-shot and the word was cleared
+        assert torch.equal(after, before)
+
+
 def test_results_do_not_depend_on_scheduling():
     cfg = LayerConfig("det", 256, 256, 32, 4, 16, 1.0, 300, seed=5)
     layer = GpuLayer(cfg)
