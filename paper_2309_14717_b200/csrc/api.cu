@@ -298,19 +298,8 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
   if (!pooled && (dA != nullptr || dB != nullptr)) {
     if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
   }
-  if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
-    st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
-                      dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);
-    if (st != QALORA_OK) return st;
-  } else if (dx != nullptr) {
-    st = launch_simt_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
-                        dT, Ab, static_cast<__nv_bfloat16*>(dx), stream);
-    if (st != QALORA_OK) return st;
-  }
-  if (dA != nullptr) {
-    st = launch_atb_f32(m, sh.G, sh.r, xp, dT, dA, partial, ws.partial_bytes, stream);
-    if (st != QALORA_OK) return st;
-  }
+  // dB and dA first, dx last: dB streams dy right after dT did (a gradient of up to about the
+  // size of L2 is then still there), and dx, the long kernel, starts on a warm dy as well
   if (dB != nullptr) {
     if (aux_tc) {
       int splits = 0;
@@ -319,6 +308,19 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
     } else {
       st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial, ws.partial_bytes, stream);
     }
+    if (st != QALORA_OK) return st;
+  }
+  if (dA != nullptr) {
+    st = launch_atb_f32(m, sh.G, sh.r, xp, dT, dA, partial, ws.partial_bytes, stream);
+    if (st != QALORA_OK) return st;
+  }
+  if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
+    st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
+                      dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);
+    if (st != QALORA_OK) return st;
+  } else if (dx != nullptr) {
+    st = launch_simt_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
+                        dT, Ab, static_cast<__nv_bfloat16*>(dx), stream);
     if (st != QALORA_OK) return st;
   }
   return debug_verify_guards(ws, workspace, stream);

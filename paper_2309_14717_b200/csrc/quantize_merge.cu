@@ -11,10 +11,10 @@ namespace qalora {
 
 constexpr int QCOLS = 128;   // columns (threads) per block
 
-// Each thread: two passes over its g weights.  Pass 1 finds min/max, pass 2
-// re-reads (L1/L2 hits), rounds and packs one 32-channel unit at a time.  Every
-// floating-point step is a single IEEE fp32 operation (no FMA contraction), so
-// the integer decision is reproducible bit for bit on a CPU.  The division
+// Each thread: two passes over its g weights.  Pass 1 finds min/max, pass 2 rounds and packs
+// one 32-channel unit at a time (with g = 32 out of the registers pass 1 filled, otherwise a
+// re-read that hits L1/L2).  Every floating-point step is a single IEEE fp32 operation (no FMA
+// contraction), so the integer decision is reproducible bit for bit on a CPU.  The division
 // t = (w - beta) / alpha is the expensive one; the code only needs rint(t), so the
 // kernel first takes t' = (w - beta) * (1 / alpha), which is within 4e-6 of t for
 // t in [0, 15], and falls back to the IEEE division only where t' lies within 1e-4
@@ -22,8 +22,37 @@ constexpr int QCOLS = 128;   // columns (threads) per block
 // The shortcut is taken only for 1e-30 < alpha < 1e30: outside that range 1 / alpha
 // overflows or is a subnormal with few significant bits (a group of nearly equal tiny
 // weights, or of huge ones), and every element takes the division.
+// The kernel is bound by its instruction stream, and the conversion unit (rint, float to
+// int) runs at a quarter of the rate of the others, so the common path avoids it: adding
+// 1.5 * 2^23 rounds t' to the nearest-even integer in the sum's low mantissa bits (exactly
+// rint for 0 <= t' < 2^22), subtracting it again gives rint(t') as a float for the boundary
+// test, and the code bits are taken from the sum's bit pattern with one shift and one logic
+// operation per weight.  No clamp is needed: beta is the group's minimum and alpha its range
+// over 2^b - 1, so 0 <= t <= (2^b - 1)(1 + 2^-22); the mask keeps a non-finite group (which is
+// reported through dev_status) from spilling into its neighbours' bits.
+constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23
+#ifndef QALORA_Q_MINB
+#define QALORA_Q_MINB 6
+#endif
+
+// ORs the code held in the low bits of `rbits` into position j of the unit's words.
 template <int BITS>
-__global__ void __launch_bounds__(QCOLS)
+__device__ __forceinline__ void unit_insert_bits(uint32_t* u, int j, uint32_t rbits) {
+  if (BITS == 4) {
+    const int e = j & 7, pos = 16 * (e & 1) + 4 * (e >> 1);
+    u[j >> 3] |= (rbits << pos) & (15u << pos);
+  } else if (BITS == 2) {
+    const int e = j & 15, pos = 16 * (e & 1) + 2 * (e >> 1);
+    u[j >> 4] |= (rbits << pos) & (3u << pos);
+  } else {
+    const int e = j & 15, pos = 16 * (e & 1) + 2 * (e >> 1), hpos = 16 * (j & 1) + (j >> 1);
+    u[j >> 4] |= (rbits << pos) & (3u << pos);
+    u[2] |= ((rbits >> 2) << hpos) & (1u << hpos);
+  }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(QCOLS, QALORA_Q_MINB)
 quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
                 float2* __restrict__ qparams, int N, int g, int G, int ntiles, int32_t* dev_status, int* dbg) {
   constexpr int WORDS = BITS == 4 ? 4 : (BITS == 3 ? 3 : 2);
@@ -35,30 +64,32 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
   const float* w = W + (size_t)q * g * N + n;
 
   float lo = FLT_MAX, hi = -FLT_MAX;
-  bool bad = false;
+  float nonfinite = 0.0f;                        // stays 0 unless a weight is NaN or infinite (0 * w is then NaN)
+  float v[32];
   for (int k0 = 0; k0 < g; k0 += 32) {
-    float v[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = __ldg(w + (size_t)(k0 + j) * N);
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-      bad |= !(fabsf(v[j]) <= FLT_MAX);
+      nonfinite = fmaf(v[j], 0.0f, nonfinite);
       lo = fminf(lo, v[j]);
       hi = fmaxf(hi, v[j]);
     }
   }
+  const bool bad = !(nonfinite == 0.0f);
   const float alpha = (hi == lo) ? 1.0f : __fdiv_rn(__fsub_rn(hi, lo), QMAX);
   const float beta = lo;
   if (QALORA_CHECK(dbg, (size_t)q * N + n, (size_t)G * N)) qparams[(size_t)q * N + n] = make_float2(alpha, beta);
   if (bad && dev_status != nullptr) atomicOr(dev_status, 1);
 
-  const bool fast = alpha > 1e-30f && alpha < 1e30f;
+  const bool fast = alpha > 1e-30f && alpha < 1e30f && !bad;
   const float inv_alpha = fast ? __frcp_rn(alpha) : 0.0f;
   const int kb0 = q * (g / 32);
   for (int k0 = 0; k0 < g; k0 += 32) {
-    float v[32];
+    if (g > 32) {                                  // (g == 32: v still holds the group)
 #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = __ldg(w + (size_t)(k0 + j) * N);
+      for (int j = 0; j < 32; ++j) v[j] = __ldg(w + (size_t)(k0 + j) * N);
+    }
     uint32_t u[WORDS];
 #pragma unroll
     for (int i = 0; i < WORDS; ++i) u[i] = 0u;
@@ -66,10 +97,14 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
     for (int j = 0; j < 32; ++j) {
       const float d = __fsub_rn(v[j], beta);
       const float t = __fmul_rn(d, inv_alpha);
-      float c = rintf(t);                              // round half to even
-      if (!fast || !(fabsf(t - c) <= 0.4999f)) c = rintf(__fdiv_rn(d, alpha));   // near a boundary (or a tie): exact
-      c = fminf(fmaxf(c, 0.0f), QMAX);
-      unit_insert<BITS>(u, j, (uint32_t)(int)c);
+      float r = __fadd_rn(t, kRoundMagic);               // low mantissa bits: rint(t), round half to even
+      const float c = __fsub_rn(r, kRoundMagic);
+      if (!fast || !(fabsf(__fsub_rn(t, c)) <= 0.4999f)) {   // near a boundary (or a tie, or no shortcut): exact
+        float ce = rintf(__fdiv_rn(d, alpha));
+        ce = fminf(fmaxf(ce, 0.0f), QMAX);               // (a non-finite group: any code will do, but a valid one)
+        r = __fadd_rn(ce, kRoundMagic);
+      }
+      unit_insert_bits<BITS>(u, j, __float_as_uint(r));
     }
     uint32_t* dst = codes + ((size_t)(kb0 + k0 / 32) * N + n) * WORDS;
     if (!QALORA_CHECK(dbg, ((size_t)(kb0 + k0 / 32) * N + n) * WORDS + WORDS - 1, (size_t)G * (g / 32) * N * WORDS)) continue;
