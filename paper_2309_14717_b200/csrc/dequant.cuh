@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include "ptx.cuh"
+
 namespace qalora {
 
 // ---- dequantization of one pack unit to 16 bf16x2 registers ------------------
@@ -66,6 +68,20 @@ __device__ __forceinline__ void load_unit(const uint32_t* cw, uint32_t* w) {
   }
 }
 
+#ifndef QALORA_DQ_FFMA2
+#define QALORA_DQ_FFMA2 1
+#endif
+// alpha * (v0, v1) + b for a pair of codes: one packed two-lane FMA (fma.rn.f32x2; each lane an
+// ordinary IEEE fused multiply-add), then one conversion of the pair to bf16x2
+__device__ __forceinline__ uint32_t dq_fma_pair(float v0, float v1, float a, float b) {
+#if QALORA_DQ_FFMA2
+  const float2 r = ptx::ffma2(make_float2(a, a), make_float2(v0, v1), make_float2(b, b));
+  return pack_bf16x2(r.x, r.y);
+#else
+  return pack_bf16x2(fmaf(a, v0, b), fmaf(a, v1, b));
+#endif
+}
+
 // pair P of word I: positions (2P, 2P+1) of that word's codes
 template <int BITS, int I, int P>
 __device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, float a, float b, const DqConsts& k) {
@@ -77,7 +93,7 @@ __device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, float a, float b,
     pr = lop_and_or(shift_to<2 - PH>(w[2]), k.third, pr);
   }
   const float v0 = __uint_as_float(pr << 16), v1 = __uint_as_float(lop_and(pr, k.himask));   // 128 + c, exactly
-  return pack_bf16x2(fmaf(a, v0, b), fmaf(a, v1, b));
+  return dq_fma_pair(v0, v1, a, b);
 }
 
 template <int BITS, int I, int P>
@@ -104,10 +120,10 @@ __device__ __forceinline__ float dq4_byte(uint32_t nib, uint32_t magic32) {
 __device__ __forceinline__ void dq4_word(uint32_t w, float a, float b, const DqConsts& k, uint32_t* out4) {
   const uint32_t ev = lop_and(w, k.nibbles), od = lop_and(w >> 4, k.nibbles);
   // pairs (positions 2P, 2P + 1): P = 0 and 2 from the even nibbles, P = 1 and 3 from the odd ones
-  out4[0] = pack_bf16x2(fmaf(a, dq4_byte<0>(ev, k.magic32), b), fmaf(a, dq4_byte<2>(ev, k.magic32), b));
-  out4[1] = pack_bf16x2(fmaf(a, dq4_byte<0>(od, k.magic32), b), fmaf(a, dq4_byte<2>(od, k.magic32), b));
-  out4[2] = pack_bf16x2(fmaf(a, dq4_byte<1>(ev, k.magic32), b), fmaf(a, dq4_byte<3>(ev, k.magic32), b));
-  out4[3] = pack_bf16x2(fmaf(a, dq4_byte<1>(od, k.magic32), b), fmaf(a, dq4_byte<3>(od, k.magic32), b));
+  out4[0] = dq_fma_pair(dq4_byte<0>(ev, k.magic32), dq4_byte<2>(ev, k.magic32), a, b);
+  out4[1] = dq_fma_pair(dq4_byte<0>(od, k.magic32), dq4_byte<2>(od, k.magic32), a, b);
+  out4[2] = dq_fma_pair(dq4_byte<1>(ev, k.magic32), dq4_byte<3>(ev, k.magic32), a, b);
+  out4[3] = dq_fma_pair(dq4_byte<1>(od, k.magic32), dq4_byte<3>(od, k.magic32), a, b);
 }
 
 // out[q] = bf16x2 of positions (2q, 2q+1) of the unit, q = 0..15

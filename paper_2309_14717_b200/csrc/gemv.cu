@@ -136,6 +136,36 @@ __device__ __forceinline__ void code_fragments(uint32_t lo, uint32_t hi, const F
   }
 }
 
+// The fold of one k-block (or chain of two) into the running sums of a 16-column group:
+// acc += alpha * D + (beta - 128 alpha) * xp for the fragment's (column gq | gq + 8) x (token
+// 2t | 2t + 1), as packed two-lane FMAs.  With one token row the odd token column of the
+// fragment is all padding and only the two columns of token 2t are folded (one packed pair).
+#ifndef QALORA_GV_FFMA2
+#define QALORA_GV_FFMA2 1
+#endif
+template <bool ONE>
+__device__ __forceinline__ void fold(float* acc, const float* D, const float* xp, float2 q0, float2 q1) {
+#if QALORA_GV_FFMA2
+  if constexpr (ONE) {
+    const float2 r = ptx::ffma2(make_float2(q0.x, q1.x), make_float2(D[0], D[2]),
+                                ptx::ffma2(make_float2(q0.y, q1.y), make_float2(xp[0], xp[0]), make_float2(acc[0], acc[2])));
+    acc[0] = r.x; acc[2] = r.y;
+  } else {
+    const float2 xp2 = make_float2(xp[0], xp[1]);
+    const float2 r0 = ptx::ffma2(make_float2(q0.x, q0.x), make_float2(D[0], D[1]),
+                                 ptx::ffma2(make_float2(q0.y, q0.y), xp2, make_float2(acc[0], acc[1])));
+    const float2 r1 = ptx::ffma2(make_float2(q1.x, q1.x), make_float2(D[2], D[3]),
+                                 ptx::ffma2(make_float2(q1.y, q1.y), xp2, make_float2(acc[2], acc[3])));
+    acc[0] = r0.x; acc[1] = r0.y; acc[2] = r1.x; acc[3] = r1.y;
+  }
+#else
+  acc[0] = fmaf(q0.x, D[0], fmaf(q0.y, xp[0], acc[0]));
+  if constexpr (!ONE) acc[1] = fmaf(q0.x, D[1], fmaf(q0.y, xp[1], acc[1]));
+  acc[2] = fmaf(q1.x, D[2], fmaf(q1.y, xp[0], acc[2]));
+  if constexpr (!ONE) acc[3] = fmaf(q1.x, D[3], fmaf(q1.y, xp[1], acc[3]));
+#endif
+}
+
 // NTS: sets of 8 token rows in use (M <= 8 NTS).  CHAIN: the group size is 64 or 128, so the two
 // k-blocks a warp set takes from a stage share (alpha, beta) and are folded together.
 // The work of one block: `block` is its index among the blocks of the layer described by p
@@ -336,11 +366,7 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
           q1.y = fmaf(-128.f, q1.x, q1.y);
 #pragma unroll
           for (int ts = 0; ts < NTS; ++ts) {
-            // (with one token row the odd token column of the fragment is all padding: not folded)
-            acc[cg][ts][0] = fmaf(q0.x, D[ts][0], fmaf(q0.y, xp[ts][0], acc[cg][ts][0]));
-            if constexpr (!ONE) acc[cg][ts][1] = fmaf(q0.x, D[ts][1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
-            acc[cg][ts][2] = fmaf(q1.x, D[ts][2], fmaf(q1.y, xp[ts][0], acc[cg][ts][2]));
-            if constexpr (!ONE) acc[cg][ts][3] = fmaf(q1.x, D[ts][3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
+            fold<ONE>(acc[cg][ts], D[ts], xp[ts], q0, q1);
           }
         }
       } else {
@@ -380,10 +406,7 @@ __device__ __forceinline__ void gemv_block(const CUtensorMap& x_map, const CUten
               float D[4];
               mma16816(D, a0, xs[ts].x, xs[ts].y, zero4);
               mma16816(D, a1, xs[ts].z, xs[ts].w, D);
-              acc[cg][ts][0] = fmaf(q0.x, D[0], fmaf(q0.y, xp[ts][0], acc[cg][ts][0]));
-              if constexpr (!ONE) acc[cg][ts][1] = fmaf(q0.x, D[1], fmaf(q0.y, xp[ts][1], acc[cg][ts][1]));
-              acc[cg][ts][2] = fmaf(q1.x, D[2], fmaf(q1.y, xp[ts][0], acc[cg][ts][2]));
-              if constexpr (!ONE) acc[cg][ts][3] = fmaf(q1.x, D[3], fmaf(q1.y, xp[ts][1], acc[cg][ts][3]));
+              fold<ONE>(acc[cg][ts], D, xp[ts], q0, q1);
             }
           }
         }
