@@ -42,7 +42,7 @@ SMALL_M = "cfg2_7b_attn"
 # with the SHA-256 of the kernel's sources at the time): when the sources have changed
 # since, the counters no longer describe the kernel and the bench reports null.
 TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "qalora_tc_kernel_fwd_cfg3_up_m8192_dram_traffic.txt")
-KERNEL_SOURCES = ("gemm_tc.cu", "ptx.cuh", "common.cuh")
+KERNEL_SOURCES = ("gemm_tc.cu", "ptx.cuh", "common.cuh", "dequant.cuh", "debug.cuh")
 
 
 def kernel_sources_sha256():
