@@ -624,13 +624,13 @@ int launch_gemv_t(const CUtensorMap& xm, const GvParams& p, int splits, cudaStre
 }
 
 template <int BITS, int NTS, bool CHAIN>
-int launch_gemv_group_t(const GvGroup& grp, int splits, cudaStream_t st) {
+int launch_gemv_group_t(const GvGroup& grp, int splits, bool programmatic, cudaStream_t st) {
   using S = GvSmem<BITS, NTS>;
   auto kern = qalora_gemv_group_kernel<BITS, NTS, CHAIN>;
   static PerDeviceOnce smem_limit;
   if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
     return QALORA_ERR_CUDA;
-  return cuda_status(launch_clustered(kern, (unsigned)grp.first_block[grp.n], splits, S::TOTAL, true, st,
+  return cuda_status(launch_clustered(kern, (unsigned)grp.first_block[grp.n], splits, S::TOTAL, programmatic, st,
                                       "qalora_gemv_group_kernel", grp));
 }
 
@@ -685,6 +685,17 @@ bool gemv_supported(const Shape& sh, int64_t M) {
   return true;
 }
 
+// Programmatic dependent launch (a merged layer's kernel starts beside its predecessor in the
+// stream and streams its first ring of weights at once) pays only with small clusters: with two
+// blocks per cluster the one-token forward of 8192 -> 22016 gains 2.6 us per call in a replay of
+// back-to-back layers, with clusters of 4 to 8 the same replay LOSES 1.5 to 8 us per call
+// (22016 -> 8192: 29.7 us without, 37.4 us with; 8192 -> 8192: 14.3 / 17.4; 4096 -> 11008: 11.6 / 13.1).
+#ifndef QALORA_GV_PDL_MAX_SPLITS
+#define QALORA_GV_PDL_MAX_SPLITS 2
+#endif
+#ifndef QALORA_GV_GROUP_PDL_MAX_SPLITS
+#define QALORA_GV_GROUP_PDL_MAX_SPLITS 2
+#endif
 // y = x * W~ + T * B for M <= 32 rows; Tb is T = s * pool(x) * A in bf16 [M][r] (null when r == 0).
 int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes, const float2* qparams,
                 const __nv_bfloat16* Tb, const __nv_bfloat16* B, __nv_bfloat16* y, int* status, bool reset_status,
@@ -693,7 +704,6 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   if (!make_x_map(x, sh.K, M, &xm)) return QALORA_ERR_CUDA;
   GvParams p{};
   p.codes = codes; p.qparams = qparams; p.Tb = Tb; p.B = B; p.y = y; p.dbg = debug_words();
-  p.pdl_wait = Tb == nullptr ? 1 : 0;
   p.M = (int)M; p.K = sh.K; p.N = sh.N; p.g = sh.g; p.r = sh.r;
   p.total_stages = sh.K / (GV_KBS * 32);
   p.status = status;
@@ -701,6 +711,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
   p.stop_after_stages = g_expire_after_stages.exchange(0x7fffffff);     // one-shot: the next launch only
   p.wait_limit_ns = p.stop_after_stages != 0x7fffffff ? g_expire_limit_ns.load() : ptx::WAIT_LIMIT_NS;
   const int splits = gv_slices(sh, M);
+  p.pdl_wait = (Tb == nullptr && splits <= QALORA_GV_PDL_MAX_SPLITS) ? 1 : 0;
   const int nts = M > 16 ? 4 : (M > 8 ? 2 : 1);
   const bool chain = sh.g >= 64;
 #define QALORA_GV_N(BITS, NTS) (chain ? launch_gemv_t<BITS, NTS, true>(xm, p, splits, st) : launch_gemv_t<BITS, NTS, false>(xm, p, splits, st))
@@ -751,6 +762,7 @@ int launch_gemv_group(const GemvGroupItem* items, int n, int64_t M, int* status,
   GvGroup grp{};
   grp.n = n;
   const int splits = gv_group_slices(items, n);
+  const bool pdl = splits <= QALORA_GV_GROUP_PDL_MAX_SPLITS;   // see launch_gemv
   const int words = words_per_unit(items[0].sh.bits);
   int blocks = 0;
   for (int i = 0; i < n; ++i) {
@@ -761,7 +773,7 @@ int launch_gemv_group(const GemvGroupItem* items, int n, int64_t M, int* status,
     p.total_stages = sh.K / (GV_KBS * 32);
     p.status = status;
     p.reset_status = (reset_status && i == 0) ? 1 : 0;
-    p.pdl_wait = 1;
+    p.pdl_wait = pdl ? 1 : 0;
     p.stop_after_stages = 0x7fffffff;
     p.wait_limit_ns = ptx::WAIT_LIMIT_NS;
     if (!make_x_map(items[i].x, sh.K, M, &grp.x_map[i]) || !make_weight_maps(p, words, &grp.codes_map[i], &grp.qp_map[i]))
@@ -771,8 +783,8 @@ int launch_gemv_group(const GemvGroupItem* items, int n, int64_t M, int* status,
   }
   grp.first_block[n] = blocks;
   const bool two_sets = M > 8, chain = items[0].sh.g >= 64;
-#define QALORA_GVG(BITS) (two_sets ? (chain ? launch_gemv_group_t<BITS, 2, true>(grp, splits, st) : launch_gemv_group_t<BITS, 2, false>(grp, splits, st)) \
-                                   : (chain ? launch_gemv_group_t<BITS, 1, true>(grp, splits, st) : launch_gemv_group_t<BITS, 1, false>(grp, splits, st)))
+#define QALORA_GVG(BITS) (two_sets ? (chain ? launch_gemv_group_t<BITS, 2, true>(grp, splits, pdl, st) : launch_gemv_group_t<BITS, 2, false>(grp, splits, pdl, st)) \
+                                   : (chain ? launch_gemv_group_t<BITS, 1, true>(grp, splits, pdl, st) : launch_gemv_group_t<BITS, 1, false>(grp, splits, pdl, st)))
   if (items[0].sh.bits == 4) return QALORA_GVG(4);
   if (items[0].sh.bits == 3) return QALORA_GVG(3);
   return QALORA_GVG(2);
