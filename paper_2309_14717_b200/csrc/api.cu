@@ -120,10 +120,20 @@ int check_desc(const qalora_desc* d, Shape* sh) {
 static constexpr int64_t kSmallM = 16;
 // The forward pass alone keeps the few-token kernel up to this many tokens (where its shapes allow).
 static constexpr int64_t kFewTokenM = 32;
-// Above the few-token range and up to this many tokens the forward pass takes the kernel with
-// the tokens as the MMA rows (where its shapes allow): one 128-token tile.
-static constexpr int64_t kMidM = 128;
-static bool takes_midm(const Shape& sh, int64_t m) { return m > kSmallM && m <= kMidM && midm_supported(sh, m); }
+// Above the few-token range the forward pass takes the kernel with the tokens as the MMA rows
+// (where its shapes allow): always up to 64 tokens; from 65 to 128 tokens only for layers with
+// 48 to SMs - 1 channel tiles of 128, where the large-tile kernel would have to cut every tile's
+// reduction into parts (measured at 65 / 96 / 128 tokens, merged, us per call, this kernel against
+// the large-tile one: 22016 -> 8192: 68 / 70 / 71 against 79 / 80 / 81; 8192 -> 22016, 172 tiles:
+// 72 / 79 / 86 against 75 / 76 / 77; 4096 -> 4096, 32 tiles: 20.5 / 22.4 / 23.4 against 20.3 /
+// 20.4 / 20.5).
+static constexpr int64_t kMidMAlways = 64, kMidM = 128;
+static bool takes_midm(const Shape& sh, int64_t m) {
+  if (m <= kSmallM || m > kMidM || !midm_supported(sh, m)) return false;
+  if (m <= kMidMAlways) return true;
+  const int tiles = sh.N / 128;
+  return tiles >= 48 && tiles < device_sm_count();
+}
 
 Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   Workspace w{};

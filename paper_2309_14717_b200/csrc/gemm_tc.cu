@@ -60,9 +60,12 @@ struct TcParams {
   int c_tiles, m_tiles;        // tiles along out channels / tokens
   int red_iters, lora_iters;   // main / adapter reduction steps per tile
   int qp_rows;                 // rows of (alpha, beta) per code stage: 128 / g
+  int tile_begin, tile_count;  // this launch works on the tiles tile_begin .. tile_begin + tile_count - 1
   int ksplit;                  // parts the reduction of a tile is cut into (1: none)
   int tile_t;                  // tokens per tile: TILE_T, or TILE_T_FEW (forward, M <= 64; always with parts)
-  float* partial;              // ksplit > 1: fp32 [ksplit][M][ld_out] partial results
+  float* partial;              // parts: fp32 partial results [ksplit][part_rows][part_ld] of the output rectangle that
+  int part_rows, part_ld;      //        starts at row part_row0, channel part_col0 (the whole output: M, ld_out, 0, 0)
+  int part_row0, part_col0;
   int* status;                 // device word: set to 1 when a wait timed out
   int* dbg;                    // record words of the bounds-check build (null otherwise)
   int stop_after_steps;        // normally INT_MAX; a test makes every activation producer stop early, so that waits expire
@@ -78,7 +81,7 @@ struct TcSegment {
 template <bool PARTS>
 __device__ __forceinline__ TcSegment tc_segment(const TcParams& p, int vt) {
   TcSegment g;
-  g.tile = PARTS ? vt / p.ksplit : vt;
+  g.tile = p.tile_begin + (PARTS ? vt / p.ksplit : vt);
   g.sp = PARTS ? vt % p.ksplit : 0;
   if (!PARTS) {
     g.mb = 0;
@@ -197,7 +200,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int total_tiles = p.c_tiles * p.m_tiles * (PARTS ? p.ksplit : 1);      // work items: (tile, part)
+  const int total_tiles = p.tile_count * (PARTS ? p.ksplit : 1);               // work items: (tile, part)
 
   if (warp == 0) {
     // ------------------------------------------------- activation producer ----
@@ -435,7 +438,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     uint32_t tcount = 0, chunk = 0;
     bool ok = true;
     for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x, ++tcount) {
-      const int tile = PARTS ? vt / p.ksplit : vt, sp = PARTS ? vt % p.ksplit : 0;
+      const int tile = p.tile_begin + (PARTS ? vt / p.ksplit : vt), sp = PARTS ? vt % p.ksplit : 0;
       const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
       const int ab = tcount % NACC;
       // The four warps meet at barriers below, so they must agree on leaving: a thread whose wait
@@ -458,12 +461,15 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
         if constexpr (PARTS) {
           // a part of the reduction: fp32 partial results [part][token][channel], added up by
           // sum_parts_kernel; a warp writes 32 neighbouring channels of one token per store
-          float* dst = p.partial + ((size_t)sp * p.M + (size_t)mt * TT + col) * p.ld_out + ct * TILE_C + ch;
+          const long long prow = (long long)mt * TT + col - p.part_row0;       // row and column inside the rectangle
+          const int pcol = ct * TILE_C + ch - p.part_col0;
+          float* dst = p.partial + ((size_t)sp * p.part_rows + prow) * p.part_ld + pcol;
 #pragma unroll
           for (int t = 0; t < 32; ++t)
             if ((long long)mt * TT + col + t < p.M &&
-                QALORA_CHECK(p.dbg, ((size_t)sp * p.M + (size_t)mt * TT + col + t) * p.ld_out + ct * TILE_C + ch, (size_t)p.ksplit * p.M * p.ld_out))
-              dst[(size_t)t * p.ld_out] = __uint_as_float(v[t]);
+                QALORA_CHECK(p.dbg, ((size_t)sp * p.part_rows + prow + t) * p.part_ld + pcol, (size_t)p.ksplit * p.part_rows * p.part_ld) &&
+                QALORA_CHECK(p.dbg, pcol, p.part_ld) && QALORA_CHECK(p.dbg, prow + t, p.part_rows))
+              dst[(size_t)t * p.part_ld] = __uint_as_float(v[t]);
           continue;
         }
         uint8_t* stg = smem + S::OFF_OUT + (chunk % S::NOUT) * S::OUT_BYTES;
@@ -582,6 +588,28 @@ sum_parts_kernel(const float* __restrict__ partial, __nv_bfloat16* __restrict__ 
   *reinterpret_cast<uint4*>(out + i0) = o;
 }
 
+// The same for a rectangle of the output: out[(row0 + r) * out_ld + col0 + c] = bf16(sum over parts of
+// partial[(part * part_rows + r) * cols + c]), r < rows, c < cols (cols a multiple of 8); 8 elements per thread
+static __global__ void __launch_bounds__(256)
+sum_parts_rect_kernel(const float* __restrict__ partial, __nv_bfloat16* __restrict__ out, int rows, int cols, int parts,
+                      int part_rows, long long out_ld, long long row0, int col0) {
+  const size_t i0 = ((size_t)blockIdx.x * 256 + threadIdx.x) * 8;
+  if (i0 >= (size_t)rows * cols) return;
+  const size_t r = i0 / cols, c = i0 % cols;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int s = 0; s < parts; ++s) {
+    const float* src = partial + ((size_t)s * part_rows + r) * cols + c;
+    const float4 a = *reinterpret_cast<const float4*>(src);
+    const float4 b = *reinterpret_cast<const float4*>(src + 4);
+    acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+    acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+  }
+  uint4 o;
+  o.x = pack_bf16x2(acc[0], acc[1]); o.y = pack_bf16x2(acc[2], acc[3]);
+  o.z = pack_bf16x2(acc[4], acc[5]); o.w = pack_bf16x2(acc[6], acc[7]);
+  *reinterpret_cast<uint4*>(out + (row0 + (long long)r) * out_ld + col0 + c) = o;
+}
+
 int launch_sum_parts_bf16(const float* partial, __nv_bfloat16* out, size_t count, int parts, cudaStream_t st) {
   sum_parts_kernel<<<(unsigned)((count / 8 + 255) / 256), 256, 0, st>>>(partial, out, count, parts);
   count_launch();
@@ -604,7 +632,7 @@ int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams&
   static PerDeviceOnce smem_limit;      // this instantiation's shared-memory limit, raised once on every device it runs on
   if (smem_limit.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::TOTAL); }) != QALORA_OK)
     return QALORA_ERR_CUDA;
-  const int tiles = p.c_tiles * p.m_tiles * p.ksplit;
+  const int tiles = p.tile_count * p.ksplit;
   const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
   {
     MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
@@ -612,7 +640,16 @@ int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams&
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
-  if (PARTS) return launch_sum_parts_bf16(p.partial, p.out, (size_t)p.M * p.ld_out, p.ksplit, st);
+  if (PARTS && p.part_ld == p.ld_out && p.part_rows == p.M) return launch_sum_parts_bf16(p.partial, p.out, (size_t)p.M * p.ld_out, p.ksplit, st);
+  if (PARTS) {   // the parts cover a rectangle of the output (the tiles of a last, short wave)
+    const long long left = p.M - p.part_row0;
+    const int rows = (int)(left < p.part_rows ? left : p.part_rows);
+    const size_t count = (size_t)rows * p.part_ld;
+    sum_parts_rect_kernel<<<(unsigned)((count / 8 + 255) / 256), 256, 0, st>>>(p.partial, p.out, rows, p.part_ld, p.ksplit, p.part_rows,
+                                                                             p.ld_out, p.part_row0, p.part_col0);
+    count_launch();
+    return cuda_status(cudaGetLastError());
+  }
   return QALORA_OK;
 }
 
@@ -669,21 +706,48 @@ int tc_forward_parts(const Shape& sh, int64_t M) {
   }
   const long long tiles = (long long)(sh.N / TILE_C) * ((M + TILE_T - 1) / TILE_T);
   const int steps = sh.K / TILE_J, sms = device_sm_count();
-  if (tiles * 4 > sms) return 1;          // enough tiles: the parts' extra epilogues and scratch traffic cost more than they save
+  if (tiles >= sms) return 1;             // at least one full wave (a short LAST wave is cut into parts on its own, see below)
+  // Fewer tiles than SMs: parts fill the idle SMs.  Cost in units of one tile's time: waves of
+  // work items over the parts, a start-up share per part, and the parts' fp32 partial results
+  // (written and read again: 8 bytes per output and part) at the HBM rate against the tile's
+  // steps x 512 tensor cycles.
+  const double tile_us = steps * 0.27, out_mb = (double)M * sh.N * 8e-6;
   int best = 1;
-  double best_cost = (double)((tiles + sms - 1) / sms);          // waves x (share of a tile per wave)
-  for (int ks = 2; ks <= 6; ++ks) {
+  double best_cost = 1.0;
+  for (int ks = 2; ks <= 8; ++ks) {
     if (steps / ks < 8) break;
     if ((size_t)ks * M * sh.N * sizeof(float) > ((size_t)256 << 20)) break;
-    const double cost = (double)((tiles * ks + sms - 1) / sms) / ks + 0.02 * ks;   // + per-part start-up
+    const double cost = (double)((tiles * ks + sms - 1) / sms) / ks + 0.02 * ks + ks * out_mb / 6.0 / tile_us;
     if (cost < best_cost - 1e-9) { best_cost = cost; best = ks; }
   }
   return best;
 }
+// A layer with a few waves of tiles whose last wave is short: the tiles of that wave alone are
+// cut into parts (a second launch), so that the wave costs 1 / parts of a tile's time instead of
+// a whole one; e.g. 172 tiles on 148 SMs are one wave of 148 whole tiles and one of 24 x 6 parts.
+// The parts' fp32 partial results cover only those tiles: a rectangle of the last token tile.
+struct TcTail { int rem, ks; };
+static TcTail tc_forward_tail(const Shape& sh, int64_t M) {
+  TcTail t{0, 1};
+  if (tc_forward_parts(sh, M) != 1) return t;                     // already cut into parts as a whole
+  const long long c_tiles = sh.N / TILE_C, m_tiles = (M + TILE_T - 1) / TILE_T, tiles = c_tiles * m_tiles;
+  const int sms = device_sm_count(), steps = sh.K / TILE_J;
+  if (tiles <= sms || tiles >= 6LL * sms) return t;               // one wave, or so many that the last one hardly matters
+  const int rem = (int)(tiles % sms);
+  if (rem == 0 || rem * 2 > sms || rem > c_tiles) return t;       // (rem <= c_tiles: the tail lies inside the last token tile)
+  int ks = sms / rem;
+  if (ks > 8) ks = 8;
+  if (ks > steps / 8) ks = steps / 8;
+  if (ks < 2) return t;
+  t.rem = rem; t.ks = ks;
+  return t;
+}
 size_t tc_forward_partial_bytes(const Shape& sh, int64_t M) {
   const int ks = tc_forward_parts(sh, M);
   if (ks < 0) return (size_t)(-ks) * M * sh.N * sizeof(float);
-  return ks > 1 ? (size_t)ks * M * sh.N * sizeof(float) : 0;
+  if (ks > 1) return (size_t)ks * M * sh.N * sizeof(float);
+  const TcTail tail = tc_forward_tail(sh, M);
+  return tail.rem > 0 ? (size_t)tail.ks * TILE_T * tail.rem * TILE_C * sizeof(float) : 0;
 }
 
 // y = x * W~ + Tb * B with Tb = bf16(s * pool(x) * A) precomputed ([M][r]).
@@ -705,6 +769,23 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
   p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
   take_expiry(&p);
   p.ksplit = parts < 0 ? -parts : parts; p.tile_t = tile_t; p.partial = partial;
+  p.tile_begin = 0; p.tile_count = p.c_tiles * p.m_tiles;
+  p.part_rows = (int)M; p.part_ld = sh.N; p.part_row0 = 0; p.part_col0 = 0;
+  const TcTail tail = tc_forward_tail(sh, M);
+  if (tail.rem > 0) {
+    // whole tiles first, then the short last wave cut into parts (same stream: one after the other)
+    TcParams pa = p;
+    pa.tile_count = p.tile_count - tail.rem;
+    int st_a = sh.bits == 4 ? launch_tc<4, FWD>(act, lora, pa, st) : (sh.bits == 3 ? launch_tc<3, FWD>(act, lora, pa, st) : launch_tc<2, FWD>(act, lora, pa, st));
+    if (st_a != QALORA_OK) return st_a;
+    TcParams pb = p;
+    pb.tile_begin = pa.tile_count; pb.tile_count = tail.rem; pb.ksplit = tail.ks;
+    pb.part_rows = TILE_T; pb.part_ld = tail.rem * TILE_C;
+    pb.part_row0 = (p.m_tiles - 1) * TILE_T; pb.part_col0 = (p.c_tiles - tail.rem) * TILE_C;
+    if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, pb, st);
+    if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, pb, st);
+    return launch_tc<2, FWD>(act, lora, pb, st);
+  }
   if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, p, st);
   return launch_tc<2, FWD>(act, lora, p, st);
@@ -726,6 +807,8 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
   p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
   take_expiry(&p);
   p.ksplit = 1; p.tile_t = TILE_T; p.partial = nullptr;
+  p.tile_begin = 0; p.tile_count = p.c_tiles * p.m_tiles;
+  p.part_rows = (int)M; p.part_ld = sh.K; p.part_row0 = 0; p.part_col0 = 0;
   if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);
   return launch_tc<2, DX>(act, lora, p, st);
