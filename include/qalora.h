@@ -162,7 +162,11 @@ int qalora_forward_group(const qalora_group_layer* layers, int n, int64_t m,
  *   dA = pool(x)^T * dT; dB = s * (pool(x) * A)^T * dy.
  *   x bf16 [m][K]; dy bf16 [m][N];
  *   dx out bf16 [m][K]; dA out float32 [G][r]; dB out float32 [r][N].
- * rank must be > 0.  dx, dA or dB may be NULL to skip that output. */
+ * rank must be > 0.  dx, dA or dB may be NULL to skip that output.
+ * With more than 16 rows the dB product runs beside dT and dA on a stream of the library's
+ * own (made on first use by the calling host thread, one per device, never destroyed), forked
+ * from `cuda_stream` and joined to it by events inside the call: to the caller the call is
+ * ordered in `cuda_stream` like any other, also inside a stream capture. */
 int qalora_backward(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
                     const void* codes, const float* qparams, const void* A, const void* B,
                     void* dx, float* dA, float* dB,

@@ -153,17 +153,19 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   w.dT = take(bwd ? M * sh.r * sizeof(float) : 0);
   w.Tb = take(M * sh.r * sizeof(__nv_bfloat16));
   w.dTb = take(bwd ? M * sh.r * sizeof(__nv_bfloat16) : 0);
-  size_t pb = 0;
+  size_t pa = 0, pb = 0;
   if (bwd) {
-    const size_t a = atb_partial_bytes(m, sh.G, sh.r), b = atb_partial_bytes(m, sh.r, sh.N);
-    pb = a > b ? a : b;
+    pa = atb_partial_bytes(m, sh.G, sh.r);
+    pb = atb_partial_bytes(m, sh.r, sh.N);
     if (sh.r >= 8 && sh.r <= 128) {
       const size_t c = tc_dB_partial_bytes(sh, m);
       pb = pb > c ? pb : c;
     }
   }
-  w.partial_bytes = pb;
-  w.partial = take(pb);
+  w.partial_bytes = pa;
+  w.partial = take(pa);
+  w.partial_dB_bytes = pb;
+  w.partial_dB = take(pb);
   // partial results of the tensor-core forward whose reduction is cut into parts; none where the
   // dispatcher takes the few-token kernel (same predicate as in forward_launch)
   const bool few = m <= kFewTokenM && gemv_supported(sh, m);
@@ -261,6 +263,35 @@ static int forward_dispatch(const Shape& sh, const Workspace& ws, int64_t m, con
                              static_cast<__nv_bfloat16*>(y), stream);
 }
 
+// A second stream of the library's own, per host thread and device, for the one place where two
+// HBM-bound kernels of a pass are independent (dB beside dT): forked from and joined to the
+// caller's stream with events, so the caller sees one stream-ordered call.  Created on first use
+// and kept; NULL when it cannot be had (the pass then runs in one stream).  During a stream
+// capture of the caller's the fork/join pattern is captured like any other.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+static SideStream* side_stream() {
+  static thread_local SideStream per_device[kMaxDevices];
+  const int dev = current_device();
+  if (dev < 0) return nullptr;
+  SideStream& s = per_device[dev];
+  if (s.stream == nullptr) {
+    cudaStream_t st = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    if (cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&b, cudaEventDisableTiming) != cudaSuccess) {
+      if (a != nullptr) cudaEventDestroy(a);
+      cudaStreamDestroy(st);
+      return nullptr;
+    }
+    s.stream = st; s.fork = a; s.join = b;
+  }
+  return &s;
+}
+
 int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void* dy,
                   const void* codes, const float* qparams, const void* A, const void* B,
                   void* dx, float* dA, float* dB,
@@ -287,6 +318,7 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
   __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.Tb);
   __nv_bfloat16* dTb = reinterpret_cast<__nv_bfloat16*>(wsp + ws.dTb);
   float* partial = reinterpret_cast<float*>(wsp + ws.partial);
+  float* partial_dB = reinterpret_cast<float*>(wsp + ws.partial_dB);
   const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
   const __nv_bfloat16* dyb = static_cast<const __nv_bfloat16*>(dy);
   const __nv_bfloat16* Ab = static_cast<const __nv_bfloat16*>(A);
@@ -302,28 +334,41 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
   // (bounds-check build: a pass on its own sets the guards; after qalora_forward_train they are already set)
   if (!pooled && (st = debug_fill_guards(ws, workspace, stream)) != QALORA_OK) return st;
   const bool aux_tc = m > kSmallM && tc_aux_supported(sh, m);
-  if (aux_tc) st = launch_tc_dT(sh, m, dyb, Bb, dT, dTb, status, stream);
-  else st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream);
-  if (st != QALORA_OK) return st;
   if (!pooled && (dA != nullptr || dB != nullptr)) {
     if ((st = launch_pool_T(sh, m, xb, Ab, xp, T, Tb, stream)) != QALORA_OK) return st;
   }
-  // dB and dA first, dx last: dB streams dy right after dT did (a gradient of up to about the
-  // size of L2 is then still there), and dx, the long kernel, starts on a warm dy as well
+  // dB = T^T dy needs only T (from the forward pass or the pooling above) and dy; dT = s dy B^T
+  // needs only dy and B.  Both stream dy once at little more than half the copy rate with one
+  // block per SM, so they run side by side: dB (and its fixed-order sum) on the library's second
+  // stream, dT and then dA on the caller's, joined before dx, the long kernel that fills every SM.
+  // A gradient of up to about the size of L2 comes from DRAM once for the two, and dx starts on a
+  // warm dy.  (Few rows, where these are small CUDA-core kernels: one stream.)
+  SideStream* side = (dB != nullptr && aux_tc) ? side_stream() : nullptr;
+  cudaStream_t dB_stream = stream;
+  if (side != nullptr) {
+    if (cudaEventRecord(side->fork, stream) != cudaSuccess || cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess)
+      return QALORA_ERR_CUDA;
+    dB_stream = side->stream;
+  }
   if (dB != nullptr) {
     if (aux_tc) {
       int splits = 0;
-      st = launch_tc_dB_partials(sh, m, Tb, dyb, partial, &splits, status, stream);
-      if (st == QALORA_OK) st = launch_sum_partials(partial, dB, (size_t)sh.r * sh.N, splits, stream);
+      st = launch_tc_dB_partials(sh, m, Tb, dyb, partial_dB, &splits, status, dB_stream);
+      if (st == QALORA_OK) st = launch_sum_partials(partial_dB, dB, (size_t)sh.r * sh.N, splits, dB_stream);
     } else {
-      st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial, ws.partial_bytes, stream);
+      st = launch_atb_bf16(m, sh.r, sh.N, T, dyb, dB, partial_dB, ws.partial_dB_bytes, dB_stream);
     }
-    if (st != QALORA_OK) return st;
+    if (side != nullptr && cudaEventRecord(side->join, side->stream) != cudaSuccess) st = QALORA_ERR_CUDA;
   }
-  if (dA != nullptr) {
-    st = launch_atb_f32(m, sh.G, sh.r, xp, dT, dA, partial, ws.partial_bytes, stream);
-    if (st != QALORA_OK) return st;
+  if (st == QALORA_OK) {
+    if (aux_tc) st = launch_tc_dT(sh, m, dyb, Bb, dT, dTb, status, stream);
+    else st = launch_dT(sh, m, dyb, Bb, dT, dTb, stream);
   }
+  if (st == QALORA_OK && dA != nullptr) st = launch_atb_f32(m, sh.G, sh.r, xp, dT, dA, partial, ws.partial_bytes, stream);
+  // join: everything after this point, in the call and after it, is ordered behind dB as well
+  // (also when a launch above failed, so that no work of this call is left outside the caller's stream)
+  if (side != nullptr && cudaStreamWaitEvent(stream, side->join, 0) != cudaSuccess) return QALORA_ERR_CUDA;
+  if (st != QALORA_OK) return st;
   if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
     st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
                       dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);

@@ -34,8 +34,10 @@ struct Workspace {
   size_t dT;        // float  [M][r]   s * dy * B^T                      (backward)
   size_t Tb;        // bf16   [M][r]   T rounded, operand of the tensor-core path
   size_t dTb;       // bf16   [M][r]   dT rounded
-  size_t partial;   // float  split-K / split-M partial sums
+  size_t partial;   // float  split-M partial sums of dA
   size_t partial_bytes;
+  size_t partial_dB;   // float  split-M partial sums of dB (its own region: dB runs beside dT and dA on a second stream)
+  size_t partial_dB_bytes;
   size_t fwd_parts; // float  [parts][M][N] partial results of a forward reduction cut into parts (forward)
   size_t total;
   // bounds-check build only: a guard of kGuardBytes follows every region (guard[i] = its offset)
