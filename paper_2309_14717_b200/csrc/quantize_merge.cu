@@ -133,40 +133,68 @@ int launch_quantize(const Shape& sh, const float* W, uint32_t* codes, float2* qp
 }
 
 // beta'[q][n] = beta[q][n] + s * sum_i A[q][i] * B[i][n]; alpha is copied.
-// One thread per column and MERGE_GROUPS consecutive groups, whose rows of A sit in shared
-// memory: an element of B is loaded once and used for all of them.  In-place use is safe: a
-// thread reads only the elements it then writes.
+// One thread per column and MERGE_GROUPS consecutive groups: an element of B is used for all
+// of them.  The kernel moves a few MB and is bound by the latency of its loads, so they are
+// issued in three batches: the block's [r x 128] slice of B (16-byte loads) and its rows of A
+// go to shared memory together, the thread's (alpha, beta) pairs are fetched before the sums
+// start.  In-place use is safe: a thread reads only the elements it then writes.
 constexpr int MERGE_GROUPS = 8;
 
 __global__ void __launch_bounds__(QCOLS)
 merge_kernel(const float2* __restrict__ qin, const __nv_bfloat16* __restrict__ A,
              const __nv_bfloat16* __restrict__ B, float2* __restrict__ qout,
              int G, int N, int r, float s, int ntiles, int* dbg) {
-  extern __shared__ float a_rows[];                 // [MERGE_GROUPS][r]
+  extern __shared__ __align__(16) float merge_smem[];
+  float* a_rows = merge_smem;                                                    // [MERGE_GROUPS][r]
+  __nv_bfloat16* b_tile = reinterpret_cast<__nv_bfloat16*>(merge_smem + MERGE_GROUPS * r);   // [r][QCOLS]
   const int q0 = (blockIdx.x / ntiles) * MERGE_GROUPS;
-  const int n = (blockIdx.x % ntiles) * QCOLS + threadIdx.x;
+  const int n0 = (blockIdx.x % ntiles) * QCOLS;
+  const int n = n0 + threadIdx.x;
+  // B slice: r rows of 128 columns = 16 pieces of 8 columns per row (N is a multiple of 8)
+  for (int idx = threadIdx.x; idx < r * (QCOLS / 8); idx += QCOLS) {
+    const int i = idx / (QCOLS / 8), c = (idx % (QCOLS / 8)) * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (n0 + c < N) v = __ldg(reinterpret_cast<const uint4*>(B + (size_t)i * N + n0 + c));
+    *reinterpret_cast<uint4*>(b_tile + i * QCOLS + c) = v;
+  }
   for (int i = threadIdx.x; i < MERGE_GROUPS * r; i += QCOLS) {
     const int q = q0 + i / r;
     a_rows[i] = q < G ? bf16_to_float(A[(size_t)q * r + i % r]) : 0.0f;
+  }
+  float2 p[MERGE_GROUPS];
+#pragma unroll
+  for (int j = 0; j < MERGE_GROUPS; ++j) {
+    const int q = q0 + j;
+    p[j] = make_float2(0.f, 0.f);
+    if (n < N && q < G && QALORA_CHECK(dbg, (size_t)q * N + n, (size_t)G * N)) p[j] = qin[(size_t)q * N + n];
   }
   __syncthreads();
   if (n >= N) return;
   float acc[MERGE_GROUPS];
 #pragma unroll
   for (int j = 0; j < MERGE_GROUPS; ++j) acc[j] = 0.0f;
-#pragma unroll 8                                    // keep 8 loads of B in flight
-  for (int i = 0; i < r; ++i) {
-    const float b = bf16_to_float(B[(size_t)i * N + n]);
+  // four adapter indices per step: the rows of A come as 16-byte shared loads (the same address for
+  // every lane), so that the loop is not bound by its shared-memory loads; the sums run in index order
+#pragma unroll 2
+  for (int i = 0; i < r; i += 4) {                 // r is a multiple of 8
+    float b[4];
 #pragma unroll
-    for (int j = 0; j < MERGE_GROUPS; ++j) acc[j] = fmaf(a_rows[j * r + i], b, acc[j]);
+    for (int k = 0; k < 4; ++k) b[k] = bf16_to_float(b_tile[(i + k) * QCOLS + threadIdx.x]);
+#pragma unroll
+    for (int j = 0; j < MERGE_GROUPS; ++j) {
+      const float4 a = *reinterpret_cast<const float4*>(a_rows + j * r + i);
+      acc[j] = fmaf(a.x, b[0], acc[j]);
+      acc[j] = fmaf(a.y, b[1], acc[j]);
+      acc[j] = fmaf(a.z, b[2], acc[j]);
+      acc[j] = fmaf(a.w, b[3], acc[j]);
+    }
   }
 #pragma unroll
   for (int j = 0; j < MERGE_GROUPS; ++j) {
     const int q = q0 + j;
-    if (q < G && QALORA_CHECK(dbg, (size_t)q * N + n, (size_t)G * N)) {
-      float2 p = qin[(size_t)q * N + n];
-      p.y = fmaf(s, acc[j], p.y);
-      qout[(size_t)q * N + n] = p;
+    if (q < G) {
+      p[j].y = fmaf(s, acc[j], p[j].y);
+      qout[(size_t)q * N + n] = p[j];
     }
   }
 }
@@ -176,7 +204,11 @@ int launch_merge(const Shape& sh, const float2* qin, const __nv_bfloat16* A, con
   const int ntiles = (sh.N + QCOLS - 1) / QCOLS;
   const long long blocks = (long long)((sh.G + MERGE_GROUPS - 1) / MERGE_GROUPS) * ntiles;
   if (blocks > 0x7fffffffLL) return QALORA_ERR_UNSUPPORTED_SHAPE;
-  merge_kernel<<<(unsigned)blocks, QCOLS, MERGE_GROUPS * sh.r * sizeof(float), st>>>(qin, A, B, qout, sh.G, sh.N, sh.r, sh.s, ntiles, debug_words());
+  const size_t smem = MERGE_GROUPS * sh.r * sizeof(float) + (size_t)sh.r * QCOLS * sizeof(__nv_bfloat16);   // up to 72 KiB at rank 256
+  static PerDeviceOnce smem_limit;
+  if (smem_limit.run([] { return cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024); }) != QALORA_OK)
+    return QALORA_ERR_CUDA;
+  merge_kernel<<<(unsigned)blocks, QCOLS, smem, st>>>(qin, A, B, qout, sh.G, sh.N, sh.r, sh.s, ntiles, debug_words());
   count_launch();
   return cuda_status(cudaGetLastError());
 }
