@@ -430,6 +430,35 @@ def test_an_expired_wait_in_the_tensor_core_kernels_unwinds_and_the_next_call_is
         assert torch.equal(after, before)
 
 
+def test_backward_pass_in_a_cuda_graph_gives_the_same_bits():
+    """The backward pass forks dB onto a stream of the library's own and joins it again inside
+    the call.  Captured into a CUDA graph (after one ordinary call, which creates that stream) the
+    fork and the join must become part of the graph: the replay gives the bits of the ordinary call."""
+    cfg = LayerConfig("graph_bwd", 512, 384, 32, 4, 16, 1.0, 700, seed=31)
+    layer = GpuLayer(cfg)
+    M, d = cfg.tokens, layer.d
+    ws = Q.alloc_workspace(d, M, Q.OP_BACKWARD)
+    out = lambda: (torch.zeros((M, cfg.d_in), dtype=torch.bfloat16, device="cuda"),
+                   torch.zeros((cfg.groups, cfg.rank), dtype=torch.float32, device="cuda"),
+                   torch.zeros((cfg.rank, cfg.d_out), dtype=torch.float32, device="cuda"))
+    run = lambda o: Q.qalora_backward(d, M, layer.dev["x"], layer.dev["dy"], layer.codes, layer.qparams,
+                                      layer.dev["A"], layer.dev["B"], o[0], o[1], o[2], ws)
+    ref = out()
+    run(ref)
+    torch.cuda.synchronize()
+    got = out()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run(got)
+    for o in got:
+        o.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert Q.workspace_status(ws) == 0
+    for a, b in zip(got, ref):
+        assert torch.equal(a, b)
+
+
 def test_results_do_not_depend_on_scheduling():
     cfg = LayerConfig("det", 256, 256, 32, 4, 16, 1.0, 300, seed=5)
     layer = GpuLayer(cfg)
