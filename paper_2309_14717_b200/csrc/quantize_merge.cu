@@ -6,6 +6,7 @@
 #include <float.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace qalora {
 
@@ -93,18 +94,27 @@ quantize_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
     uint32_t u[WORDS];
 #pragma unroll
     for (int i = 0; i < WORDS; ++i) u[i] = 0u;
+    // two weights per instruction (packed two-lane add / sub / mul, each lane IEEE round-to-nearest)
+    const float2 beta2 = make_float2(beta, beta), inv2 = make_float2(inv_alpha, inv_alpha), magic2 = make_float2(kRoundMagic, kRoundMagic);
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const float d = __fsub_rn(v[j], beta);
-      const float t = __fmul_rn(d, inv_alpha);
-      float r = __fadd_rn(t, kRoundMagic);               // low mantissa bits: rint(t), round half to even
-      const float c = __fsub_rn(r, kRoundMagic);
-      if (!fast || !(fabsf(__fsub_rn(t, c)) <= 0.4999f)) {   // near a boundary (or a tie, or no shortcut): exact
-        float ce = rintf(__fdiv_rn(d, alpha));
+    for (int j = 0; j < 32; j += 2) {
+      const float2 d = ptx::fsub2(make_float2(v[j], v[j + 1]), beta2);
+      const float2 t = ptx::fmul2(d, inv2);
+      float2 r = ptx::fadd2(t, magic2);                   // low mantissa bits: rint(t), round half to even
+      const float2 c = ptx::fsub2(r, magic2);
+      const float2 e = ptx::fsub2(t, c);
+      if (!fast || !(fabsf(e.x) <= 0.4999f)) {            // near a boundary (or a tie, or no shortcut): exact
+        float ce = rintf(__fdiv_rn(d.x, alpha));
         ce = fminf(fmaxf(ce, 0.0f), QMAX);               // (a non-finite group: any code will do, but a valid one)
-        r = __fadd_rn(ce, kRoundMagic);
+        r.x = __fadd_rn(ce, kRoundMagic);
       }
-      unit_insert_bits<BITS>(u, j, __float_as_uint(r));
+      if (!fast || !(fabsf(e.y) <= 0.4999f)) {
+        float ce = rintf(__fdiv_rn(d.y, alpha));
+        ce = fminf(fmaxf(ce, 0.0f), QMAX);
+        r.y = __fadd_rn(ce, kRoundMagic);
+      }
+      unit_insert_bits<BITS>(u, j, __float_as_uint(r.x));
+      unit_insert_bits<BITS>(u, j + 1, __float_as_uint(r.y));
     }
     uint32_t* dst = codes + ((size_t)(kb0 + k0 / 32) * N + n) * WORDS;
     if (!QALORA_CHECK(dbg, ((size_t)(kb0 + k0 / 32) * N + n) * WORDS + WORDS - 1, (size_t)G * (g / 32) * N * WORDS)) continue;
