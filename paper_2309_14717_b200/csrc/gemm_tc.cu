@@ -57,10 +57,11 @@ struct TcParams {
   long long M;
   int K, N, g, r;
   int ld_out;                  // N (FWD) or K (DX)
-  int c_tiles, m_tiles;        // tiles along out channels / tokens
+  int c_tiles, m_tiles;        // tiles along out channels / tokens that this launch works on
+  int c_tile0;                 // its first channel tile (a launch may cover a strip of the channel tiles)
   int red_iters, lora_iters;   // main / adapter reduction steps per tile
   int qp_rows;                 // rows of (alpha, beta) per code stage: 128 / g
-  int tile_begin, tile_count;  // this launch works on the tiles tile_begin .. tile_begin + tile_count - 1
+  int tile_count;              // c_tiles * m_tiles
   int ksplit;                  // parts the reduction of a tile is cut into (1: none)
   int tile_t;                  // tokens per tile: TILE_T, or TILE_T_FEW (forward, M <= 64; always with parts)
   float* partial;              // parts: fp32 partial results [ksplit][part_rows][part_ld] of the output rectangle that
@@ -81,7 +82,7 @@ struct TcSegment {
 template <bool PARTS>
 __device__ __forceinline__ TcSegment tc_segment(const TcParams& p, int vt) {
   TcSegment g;
-  g.tile = p.tile_begin + (PARTS ? vt / p.ksplit : vt);
+  g.tile = PARTS ? vt / p.ksplit : vt;
   g.sp = PARTS ? vt % p.ksplit : 0;
   if (!PARTS) {
     g.mb = 0;
@@ -210,7 +211,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x) {
         const TcSegment sg = tc_segment<PARTS>(p, vt);
         const int m0 = (sg.tile / p.c_tiles) * TT;
-        const int c0 = (sg.tile % p.c_tiles) * TILE_C;
+        const int c0 = (sg.tile % p.c_tiles + p.c_tile0) * TILE_C;
         for (int j = 0; j < sg.n_steps; ++j, ++it) {
           if (it >= (uint32_t)p.stop_after_steps) { ok = false; break; }     // (test hook: the tiles stop coming)
           const int i = tc_step<PARTS>(p, sg, j);
@@ -251,7 +252,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
       bool ok = true;
       for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x) {
         const TcSegment sg = tc_segment<PARTS>(p, vt);
-        const int c0 = (sg.tile % p.c_tiles) * TILE_C;
+        const int c0 = (sg.tile % p.c_tiles + p.c_tile0) * TILE_C;
         const int cs_end = (sg.mb + sg.n_main) / S::IPS;
         for (int cs = sg.mb / S::IPS; cs < cs_end; ++cs, ++cit) {
           const int s = cit % NC;
@@ -335,7 +336,7 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     const int qsh = p.g == 32 ? 0 : (p.g == 64 ? 1 : 2);   // k-block -> (alpha, beta) row of the stage
     for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x) {
       const TcSegment sg = tc_segment<PARTS>(p, vt);
-      const int c0 = (sg.tile % p.c_tiles) * TILE_C;
+      const int c0 = (sg.tile % p.c_tiles + p.c_tile0) * TILE_C;
       for (int j = 0; j < sg.n_steps; ++j, ++it) {
         if ((int)(it % DQ_GROUPS) != wg) continue;
         const int i = tc_step<PARTS>(p, sg, j);
@@ -438,8 +439,8 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
     uint32_t tcount = 0, chunk = 0;
     bool ok = true;
     for (int vt = blockIdx.x; vt < total_tiles && ok; vt += gridDim.x, ++tcount) {
-      const int tile = p.tile_begin + (PARTS ? vt / p.ksplit : vt), sp = PARTS ? vt % p.ksplit : 0;
-      const int ct = tile % p.c_tiles, mt = tile / p.c_tiles;
+      const int tile = PARTS ? vt / p.ksplit : vt, sp = PARTS ? vt % p.ksplit : 0;
+      const int ct = tile % p.c_tiles + p.c_tile0, mt = tile / p.c_tiles;
       const int ab = tcount % NACC;
       // The four warps meet at barriers below, so they must agree on leaving: a thread whose wait
       // gave up (the abort flag was raised elsewhere) and a thread that saw the phase complete in
@@ -722,11 +723,13 @@ int tc_forward_parts(const Shape& sh, int64_t M) {
   }
   return best;
 }
-// A layer with a few waves of tiles whose last wave is short: the tiles of that wave alone are
-// cut into parts (a second launch), so that the wave costs 1 / parts of a tile's time instead of
-// a whole one; e.g. 172 tiles on 148 SMs are one wave of 148 whole tiles and one of 24 x 6 parts.
-// The parts' fp32 partial results cover only those tiles: a rectangle of the last token tile.
-struct TcTail { int rem, ks; };
+// A layer with a few waves of tiles whose last wave is short: a strip of its channel tiles (all
+// token tiles of the last `strip_c` channel tiles, about as many tiles as that wave holds) is
+// cut into parts, in a second launch, so that it costs 1 / parts of a tile's time instead of a
+// whole wave; e.g. 172 tiles on 148 SMs are one wave of 148 whole tiles and one of 24 x 6 parts,
+// 640 tiles (40 x 16) are four waves of 37 x 16 whole tiles and one of 3 x 16 x 3 parts.  The
+// parts' fp32 partial results cover only that strip of the output.
+struct TcTail { int strip_c, ks; };
 static TcTail tc_forward_tail(const Shape& sh, int64_t M) {
   TcTail t{0, 1};
   if (tc_forward_parts(sh, M) != 1) return t;                     // already cut into parts as a whole
@@ -734,12 +737,14 @@ static TcTail tc_forward_tail(const Shape& sh, int64_t M) {
   const int sms = device_sm_count(), steps = sh.K / TILE_J;
   if (tiles <= sms || tiles >= 6LL * sms) return t;               // one wave, or so many that the last one hardly matters
   const int rem = (int)(tiles % sms);
-  if (rem == 0 || rem * 2 > sms || rem > c_tiles) return t;       // (rem <= c_tiles: the tail lies inside the last token tile)
-  int ks = sms / rem;
+  if (rem == 0 || rem * 2 > sms) return t;
+  const long long strip_c = (rem + m_tiles - 1) / m_tiles, strip = strip_c * m_tiles;
+  if (strip_c >= c_tiles || strip > sms) return t;
+  int ks = (int)(sms / strip);
   if (ks > 8) ks = 8;
   if (ks > steps / 8) ks = steps / 8;
   if (ks < 2) return t;
-  t.rem = rem; t.ks = ks;
+  t.strip_c = (int)strip_c; t.ks = ks;
   return t;
 }
 size_t tc_forward_partial_bytes(const Shape& sh, int64_t M) {
@@ -747,7 +752,7 @@ size_t tc_forward_partial_bytes(const Shape& sh, int64_t M) {
   if (ks < 0) return (size_t)(-ks) * M * sh.N * sizeof(float);
   if (ks > 1) return (size_t)ks * M * sh.N * sizeof(float);
   const TcTail tail = tc_forward_tail(sh, M);
-  return tail.rem > 0 ? (size_t)tail.ks * TILE_T * tail.rem * TILE_C * sizeof(float) : 0;
+  return tail.strip_c > 0 ? (size_t)tail.ks * M * tail.strip_c * TILE_C * sizeof(float) : 0;
 }
 
 // y = x * W~ + Tb * B with Tb = bf16(s * pool(x) * A) precomputed ([M][r]).
@@ -769,19 +774,19 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
   p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
   take_expiry(&p);
   p.ksplit = parts < 0 ? -parts : parts; p.tile_t = tile_t; p.partial = partial;
-  p.tile_begin = 0; p.tile_count = p.c_tiles * p.m_tiles;
+  p.c_tile0 = 0; p.tile_count = p.c_tiles * p.m_tiles;
   p.part_rows = (int)M; p.part_ld = sh.N; p.part_row0 = 0; p.part_col0 = 0;
   const TcTail tail = tc_forward_tail(sh, M);
-  if (tail.rem > 0) {
-    // whole tiles first, then the short last wave cut into parts (same stream: one after the other)
+  if (tail.strip_c > 0) {
+    // whole tiles of the other channel tiles first, then the strip cut into parts (same stream: one after the other)
     TcParams pa = p;
-    pa.tile_count = p.tile_count - tail.rem;
+    pa.c_tiles = p.c_tiles - tail.strip_c;
+    pa.tile_count = pa.c_tiles * p.m_tiles;
     int st_a = sh.bits == 4 ? launch_tc<4, FWD>(act, lora, pa, st) : (sh.bits == 3 ? launch_tc<3, FWD>(act, lora, pa, st) : launch_tc<2, FWD>(act, lora, pa, st));
     if (st_a != QALORA_OK) return st_a;
     TcParams pb = p;
-    pb.tile_begin = pa.tile_count; pb.tile_count = tail.rem; pb.ksplit = tail.ks;
-    pb.part_rows = TILE_T; pb.part_ld = tail.rem * TILE_C;
-    pb.part_row0 = (p.m_tiles - 1) * TILE_T; pb.part_col0 = (p.c_tiles - tail.rem) * TILE_C;
+    pb.c_tiles = tail.strip_c; pb.c_tile0 = pa.c_tiles; pb.tile_count = tail.strip_c * p.m_tiles; pb.ksplit = tail.ks;
+    pb.part_rows = (int)M; pb.part_ld = tail.strip_c * TILE_C; pb.part_row0 = 0; pb.part_col0 = pa.c_tiles * TILE_C;
     if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, pb, st);
     if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, pb, st);
     return launch_tc<2, FWD>(act, lora, pb, st);
@@ -807,7 +812,7 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
   p.status = status; p.qp_rows = 128 / sh.g; p.dbg = debug_words();
   take_expiry(&p);
   p.ksplit = 1; p.tile_t = TILE_T; p.partial = nullptr;
-  p.tile_begin = 0; p.tile_count = p.c_tiles * p.m_tiles;
+  p.c_tile0 = 0; p.tile_count = p.c_tiles * p.m_tiles;
   p.part_rows = (int)M; p.part_ld = sh.K; p.part_row0 = 0; p.part_col0 = 0;
   if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);

@@ -116,9 +116,10 @@ SMALL = [
     ("midm4_33", 4096, 256, 32, 4, 72, 0.5, 33),
     ("midm4_r64_65", 1024, 768, 32, 4, 64, 1.0, 65),
     # more 128 x 256 tiles than SMs with a short last wave: that wave's tiles alone are cut into parts
-    # (160 and 320 tiles: 12 and 24 in the tail; the second case with a ragged last token tile)
+    # (160 and 320 tiles: 12 and 24 in the strip; ragged last token tiles)
     ("tail4", 2048, 20480, 32, 4, 16, 1.0, 256),
     ("tail3", 1024, 20480, 64, 3, 8, 1.0, 300),
+    ("tail2", 1024, 5120, 128, 2, 8, 1.0, 1000),      # 40 x 4 tiles: a strip of 3 channel tiles over all four token tiles
     # many tokens, several channel tiles, ragged token count
     ("pair4", 512, 256, 32, 4, 16, 1.0, 700),
     ("pair3", 384, 512, 64, 3, 24, 0.75, 530),
