@@ -166,6 +166,7 @@ Workspace workspace_layout(const Shape& sh, int64_t m, int op) {
   w.partial = take(pa);
   w.partial_dB_bytes = pb;
   w.partial_dB = take(pb);
+  w.dx_parts = take(bwd && m > kSmallM && tc_dx_supported(sh, m) ? tc_dx_partial_bytes(sh, m) : 0);
   // partial results of the tensor-core forward whose reduction is cut into parts; none where the
   // dispatcher takes the few-token kernel (same predicate as in forward_launch)
   const bool few = m <= kFewTokenM && gemv_supported(sh, m);
@@ -371,7 +372,7 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
   if (st != QALORA_OK) return st;
   if (dx != nullptr && m > kSmallM && tc_dx_supported(sh, m)) {
     st = launch_tc_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),
-                      dTb, Ab, static_cast<__nv_bfloat16*>(dx), status, stream);
+                      dTb, Ab, static_cast<__nv_bfloat16*>(dx), reinterpret_cast<float*>(wsp + ws.dx_parts), status, stream);
     if (st != QALORA_OK) return st;
   } else if (dx != nullptr) {
     st = launch_simt_dx(sh, m, dyb, static_cast<const uint32_t*>(codes), reinterpret_cast<const float2*>(qparams),

@@ -38,6 +38,7 @@ struct Workspace {
   size_t partial_bytes;
   size_t partial_dB;   // float  split-M partial sums of dB (its own region: dB runs beside dT and dA on a second stream)
   size_t partial_dB_bytes;
+  size_t dx_parts;  // float  partial results of a strip of dx tiles whose reduction is cut into parts (backward)
   size_t fwd_parts; // float  [parts][M][N] partial results of a forward reduction cut into parts (forward)
   size_t total;
   // bounds-check build only: a guard of kGuardBytes follows every region (guard[i] = its offset)
@@ -130,9 +131,10 @@ size_t tc_forward_partial_bytes(const Shape& sh, int64_t M);   // scratch for a 
 int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
                       const float2* qparams, const __nv_bfloat16* Tb, const __nv_bfloat16* B,
                       __nv_bfloat16* y, float* partial, int* status, cudaStream_t st);
+size_t tc_dx_partial_bytes(const Shape& sh, int64_t M);         // scratch for a short last wave cut into parts
 int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint32_t* codes,
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
-                 __nv_bfloat16* dx, int* status, cudaStream_t st);
+                 __nv_bfloat16* dx, float* partial, int* status, cudaStream_t st);
 
 // Forward for a few dozen to a few hundred tokens (midm_tc.cu): tokens as the MMA rows, 256
 // channels per instruction.  Tb is the bf16 rank-r intermediate (ignored when r == 0).

@@ -657,7 +657,7 @@ int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams&
 template <int BITS, int MODE>
 int launch_tc(const CUtensorMap& act, const CUtensorMap& lora, const TcParams& p, cudaStream_t st) {
   if (MODE == FWD && p.tile_t == TILE_T_FEW) return launch_tc_t<BITS, FWD, true, TILE_T_FEW>(act, lora, p, st);
-  if (MODE == FWD && p.ksplit > 1) return launch_tc_t<BITS, FWD, true, TILE_T>(act, lora, p, st);
+  if (p.ksplit > 1) return launch_tc_t<BITS, MODE, true, TILE_T>(act, lora, p, st);
   return launch_tc_t<BITS, MODE, false, TILE_T>(act, lora, p, st);
 }
 
@@ -730,11 +730,10 @@ int tc_forward_parts(const Shape& sh, int64_t M) {
 // 640 tiles (40 x 16) are four waves of 37 x 16 whole tiles and one of 3 x 16 x 3 parts.  The
 // parts' fp32 partial results cover only that strip of the output.
 struct TcTail { int strip_c, ks; };
-static TcTail tc_forward_tail(const Shape& sh, int64_t M) {
+static TcTail tc_tail(long long c_tiles, long long m_tiles, int steps) {
   TcTail t{0, 1};
-  if (tc_forward_parts(sh, M) != 1) return t;                     // already cut into parts as a whole
-  const long long c_tiles = sh.N / TILE_C, m_tiles = (M + TILE_T - 1) / TILE_T, tiles = c_tiles * m_tiles;
-  const int sms = device_sm_count(), steps = sh.K / TILE_J;
+  const long long tiles = c_tiles * m_tiles;
+  const int sms = device_sm_count();
   if (tiles <= sms || tiles >= 6LL * sms) return t;               // one wave, or so many that the last one hardly matters
   const int rem = (int)(tiles % sms);
   if (rem == 0 || rem * 2 > sms) return t;
@@ -746,6 +745,22 @@ static TcTail tc_forward_tail(const Shape& sh, int64_t M) {
   if (ks < 2) return t;
   t.strip_c = (int)strip_c; t.ks = ks;
   return t;
+}
+static TcTail tc_forward_tail(const Shape& sh, int64_t M) {
+  if (tc_forward_parts(sh, M) != 1) return TcTail{0, 1};          // already cut into parts as a whole
+  return tc_tail(sh.N / TILE_C, (M + TILE_T - 1) / TILE_T, sh.K / TILE_J);
+}
+// the same for dx (channel tiles along K, reduction over N; parts begin on even steps, so N must be a multiple of 128)
+#ifndef QALORA_TC_DX_TAIL
+#define QALORA_TC_DX_TAIL 1
+#endif
+static TcTail tc_dx_tail(const Shape& sh, int64_t M) {
+  if (!QALORA_TC_DX_TAIL || sh.N % (2 * TILE_J) != 0) return TcTail{0, 1};
+  return tc_tail(sh.K / TILE_C, (M + TILE_T - 1) / TILE_T, sh.N / TILE_J);
+}
+size_t tc_dx_partial_bytes(const Shape& sh, int64_t M) {
+  const TcTail tail = tc_dx_tail(sh, M);
+  return tail.strip_c > 0 ? (size_t)tail.ks * M * tail.strip_c * TILE_C * sizeof(float) : 0;
 }
 size_t tc_forward_partial_bytes(const Shape& sh, int64_t M) {
   const int ks = tc_forward_parts(sh, M);
@@ -799,7 +814,7 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
 // dx = dy * W~^T + dTb * expand(A)^T with dTb = bf16(s * dy * B^T) precomputed ([M][r]).
 int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint32_t* codes,
                  const float2* qparams, const __nv_bfloat16* dTb, const __nv_bfloat16* A,
-                 __nv_bfloat16* dx, int* status, cudaStream_t st) {
+                 __nv_bfloat16* dx, float* partial, int* status, cudaStream_t st) {
   CUtensorMap act, lora;
   if (!make_act_map(&act, dy, M, sh.N, TILE_T)) return QALORA_ERR_CUDA;
   lora = act;
@@ -814,6 +829,22 @@ int launch_tc_dx(const Shape& sh, int64_t M, const __nv_bfloat16* dy, const uint
   p.ksplit = 1; p.tile_t = TILE_T; p.partial = nullptr;
   p.c_tile0 = 0; p.tile_count = p.c_tiles * p.m_tiles;
   p.part_rows = (int)M; p.part_ld = sh.K; p.part_row0 = 0; p.part_col0 = 0;
+  const TcTail tail = tc_dx_tail(sh, M);
+  if (tail.strip_c > 0 && partial != nullptr) {
+    // whole tiles of the other channel tiles first, then the strip of a short last wave cut into parts
+    TcParams pa = p;
+    pa.c_tiles = p.c_tiles - tail.strip_c;
+    pa.tile_count = pa.c_tiles * p.m_tiles;
+    int st_a = sh.bits == 4 ? launch_tc<4, DX>(act, lora, pa, st) : (sh.bits == 3 ? launch_tc<3, DX>(act, lora, pa, st) : launch_tc<2, DX>(act, lora, pa, st));
+    if (st_a != QALORA_OK) return st_a;
+    TcParams pb = p;
+    pb.c_tiles = tail.strip_c; pb.c_tile0 = pa.c_tiles; pb.tile_count = tail.strip_c * p.m_tiles; pb.ksplit = tail.ks;
+    pb.partial = partial;
+    pb.part_rows = (int)M; pb.part_ld = tail.strip_c * TILE_C; pb.part_row0 = 0; pb.part_col0 = pa.c_tiles * TILE_C;
+    if (sh.bits == 4) return launch_tc<4, DX>(act, lora, pb, st);
+    if (sh.bits == 3) return launch_tc<3, DX>(act, lora, pb, st);
+    return launch_tc<2, DX>(act, lora, pb, st);
+  }
   if (sh.bits == 4) return launch_tc<4, DX>(act, lora, p, st);
   if (sh.bits == 3) return launch_tc<3, DX>(act, lora, p, st);
   return launch_tc<2, DX>(act, lora, p, st);

@@ -120,6 +120,8 @@ SMALL = [
     ("tail4", 2048, 20480, 32, 4, 16, 1.0, 256),
     ("tail3", 1024, 20480, 64, 3, 8, 1.0, 300),
     ("tail2", 1024, 5120, 128, 2, 8, 1.0, 1000),      # 40 x 4 tiles: a strip of 3 channel tiles over all four token tiles
+    ("tail_dx4", 5120, 1024, 32, 4, 16, 1.0, 1000),   # the same for the input gradient (40 x 4 tiles along the input channels)
+    ("tail_dx3", 5120, 1152, 64, 3, 24, 1.0, 520),    # 40 x 3 tiles: none in a strip (120 < SMs); 1152 = 9 x 128 reduction
     # many tokens, several channel tiles, ragged token count
     ("pair4", 512, 256, 32, 4, 16, 1.0, 700),
     ("pair3", 384, 512, 64, 3, 24, 0.75, 530),
