@@ -10,29 +10,28 @@
 namespace qalora {
 
 // ---- dequantization of one pack unit to 16 bf16x2 registers ------------------
-// The two codes of a pair sit at the same bit offset of the two half-words, so one shift
-// and one LOP3 turn them into the bf16 pair (128 + c0, 128 + c1): the code is OR-ed into
-// the mantissa of bf16 128.0, no int-to-float conversion.  Widening each half to fp32 is
-// one more logic op, then W~ = alpha * (128 + c) + (beta - 128 alpha) is ONE fp32 FMA per
-// element, and the pair is rounded once to bf16x2.  alpha and beta stay in fp32, so the
-// only rounding that matters is that of the final weight (rounding alpha or beta
+// A code is brought into a byte of its own (masks and shifts on whole words, four codes at a
+// time), a byte permute drops that byte into mantissa bits 16.. of the fp32 number 128.0
+// (0x43000000 | c << 16 = 128 + c exactly: no int-to-float conversion), then
+// W~ = alpha * (128 + c) + (beta - 128 alpha) is one fp32 FMA per element, two elements per
+// packed instruction, and the pair is rounded once to bf16x2.  alpha and beta stay in fp32, so
+// the only rounding that matters is that of the final weight (rounding alpha or beta
 // themselves would put a common error on all channels of a group, which the pooled input
 // amplifies).
 // The logic/shift pipe is the busiest one in these kernels.  A LOP3 takes at most one
 // immediate, so the masks live in registers (DqConsts, made opaque to the compiler):
-// "(a & mask) | magic" then is one instruction instead of two.
+// "(a & mask) | x" then is one instruction instead of two.
 struct DqConsts {
-  uint32_t mask, magic, himask, third, nibbles, magic32;
+  uint32_t nibbles, magic32, twobits, third_a, third_b;
 };
 template <int BITS>
 __device__ __forceinline__ DqConsts dq_consts() {
   DqConsts c;
-  asm volatile("mov.b32 %0, %1;" : "=r"(c.mask) : "n"(BITS == 4 ? 0x000f000f : 0x00030003));
-  asm volatile("mov.b32 %0, 0x43004300;" : "=r"(c.magic));
-  asm volatile("mov.b32 %0, 0xffff0000;" : "=r"(c.himask));
-  asm volatile("mov.b32 %0, 0x00040004;" : "=r"(c.third));
   asm volatile("mov.b32 %0, 0x0f0f0f0f;" : "=r"(c.nibbles));
   asm volatile("mov.b32 %0, 0x43000000;" : "=r"(c.magic32));
+  asm volatile("mov.b32 %0, 0x03030303;" : "=r"(c.twobits));
+  asm volatile("mov.b32 %0, 0x00040004;" : "=r"(c.third_a));
+  asm volatile("mov.b32 %0, 0x04000400;" : "=r"(c.third_b));
   return c;
 }
 __device__ __forceinline__ uint32_t lop_and_or(uint32_t a, uint32_t b, uint32_t c) {   // (a & b) | c
@@ -82,29 +81,6 @@ __device__ __forceinline__ uint32_t dq_fma_pair(float v0, float v1, float a, flo
 #endif
 }
 
-// pair P of word I: positions (2P, 2P+1) of that word's codes
-template <int BITS, int I, int P>
-__device__ __forceinline__ uint32_t dq_pair(const uint32_t* w, float a, float b, const DqConsts& k) {
-  constexpr int W = BITS == 4 ? 4 : 2;             // width of the (low) code bits
-  uint32_t pr = lop_and_or(w[I] >> (W * P), k.mask, k.magic);
-  if constexpr (BITS == 3) {
-    // third bits of the pair: bits PH and 16 + PH of word 2, PH = 8 I + P; they go to bit 2 of each half
-    constexpr int PH = 8 * I + P;
-    pr = lop_and_or(shift_to<2 - PH>(w[2]), k.third, pr);
-  }
-  const float v0 = __uint_as_float(pr << 16), v1 = __uint_as_float(lop_and(pr, k.himask));   // 128 + c, exactly
-  return dq_fma_pair(v0, v1, a, b);
-}
-
-template <int BITS, int I, int P>
-__device__ __forceinline__ void dq_all(const uint32_t* w, float a, float b, const DqConsts& k, uint32_t* out) {
-  constexpr int PAIRS = BITS == 4 ? 4 : 8;          // pairs per word
-  constexpr int NWORDS = BITS == 4 ? 4 : 2;         // words that carry the (low) code bits
-  out[I * PAIRS + P] = dq_pair<BITS, I, P>(w, a, b, k);
-  if constexpr (P + 1 < PAIRS) dq_all<BITS, I, P + 1>(w, a, b, k, out);
-  else if constexpr (I + 1 < NWORDS) dq_all<BITS, I + 1, 0>(w, a, b, k, out);
-}
-
 // 4-bit codes, a cheaper route to the same values.  One AND gives the word's four even nibbles
 // as the low nibbles of its four bytes, one shift and one AND the four odd ones; a byte
 // permute then drops such a byte straight into mantissa bits 16-19 of the fp32 number 128.0
@@ -126,6 +102,27 @@ __device__ __forceinline__ void dq4_word(uint32_t w, float a, float b, const DqC
   out4[3] = dq_fma_pair(dq4_byte<1>(od, k.magic32), dq4_byte<3>(od, k.magic32), a, b);
 }
 
+// 2- and 3-bit codes by the same route.  A word of the low code bits holds 16 codes, two bits
+// each: the even positions e = 2k in its low half-word at bit 2k, the odd ones in the high
+// half-word at the same offset.  Shifted right by 2 ss (ss = 0..3) and masked with 0x03030303 it
+// leaves one code in each byte: positions 2 ss | 8 + 2 ss | 2 ss + 1 | 9 + 2 ss in bytes 0..3, i.e.
+// the pairs k = ss (bytes 0, 2) and k = 4 + ss (bytes 1, 3).  The third bit of position j of the
+// unit sits in word 2 at bit 16 (j & 1) + (j >> 1); for those four positions of word I that is
+// b0, b0 + 4, b0 + 16, b0 + 20 with b0 = 8 I + ss, so two shifts bring them to bit 2 of bytes
+// 0 and 2 and of bytes 1 and 3.  Then one byte permute per code, one packed FMA and one
+// conversion per pair: 2.4 (3.4) instructions per 2-bit (3-bit) code instead of 3 (4).
+template <int BITS, int I, int SS>
+__device__ __forceinline__ void dq23_quad(const uint32_t* w, float a, float b, const DqConsts& k, uint32_t* out) {
+  uint32_t nib = lop_and(SS == 0 ? w[I] : (w[I] >> (2 * SS)), k.twobits);
+  if constexpr (BITS == 3) {
+    constexpr int B0 = 8 * I + SS;
+    nib = lop_and_or(shift_to<2 - B0>(w[2]), k.third_a, nib);
+    nib = lop_and_or(shift_to<6 - B0>(w[2]), k.third_b, nib);
+  }
+  out[8 * I + SS] = dq_fma_pair(dq4_byte<0>(nib, k.magic32), dq4_byte<2>(nib, k.magic32), a, b);
+  out[8 * I + 4 + SS] = dq_fma_pair(dq4_byte<1>(nib, k.magic32), dq4_byte<3>(nib, k.magic32), a, b);
+}
+
 // out[q] = bf16x2 of positions (2q, 2q+1) of the unit, q = 0..15
 template <int BITS>
 __device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, const DqConsts& k, uint32_t* out) {
@@ -133,9 +130,12 @@ __device__ __forceinline__ void dequant_unit(const uint32_t* w, float2 ab, const
   if constexpr (BITS == 4) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) dq4_word(w[i], ab.x, b, k, out + 4 * i);
-    return;
+  } else {
+    dq23_quad<BITS, 0, 0>(w, ab.x, b, k, out); dq23_quad<BITS, 0, 1>(w, ab.x, b, k, out);
+    dq23_quad<BITS, 0, 2>(w, ab.x, b, k, out); dq23_quad<BITS, 0, 3>(w, ab.x, b, k, out);
+    dq23_quad<BITS, 1, 0>(w, ab.x, b, k, out); dq23_quad<BITS, 1, 1>(w, ab.x, b, k, out);
+    dq23_quad<BITS, 1, 2>(w, ab.x, b, k, out); dq23_quad<BITS, 1, 3>(w, ab.x, b, k, out);
   }
-  dq_all<BITS, 0, 0>(w, ab.x, b, k, out);
 }
 
 }  // namespace qalora
