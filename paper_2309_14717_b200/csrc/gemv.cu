@@ -728,7 +728,7 @@ int launch_gemv(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32
 
 
 // Slices per column tile for a group of layers (one cluster size for the whole launch): the
-// count that brings the grid closest to two blocks per SM and that every layer can be cut into.
+// count that brings the grid closest to three blocks per SM and that every layer can be cut into.
 static int gv_group_slices(const GemvGroupItem* items, int n) {
   long long tiles = 0;
   int min_stages = 1 << 30;
@@ -737,7 +737,10 @@ static int gv_group_slices(const GemvGroupItem* items, int n) {
     const int stages = items[i].sh.K / (GV_KBS * 32);
     min_stages = stages < min_stages ? stages : min_stages;
   }
-  const long long target = 2ll * device_sm_count();
+  // (three blocks per SM here, two for a single layer: measured on the five projections of a 7B
+  // block, 268 column tiles: 29.8 us with one slice per tile, 25.5 us with two; single layers were
+  // slower with the higher target, e.g. 8192 -> 22016 32.2 against 30.6 us)
+  const long long target = 3ll * device_sm_count();
   int splits = 1;
   long long best = 1ll << 60;
   for (int sp : {1, 2, 3, 4, 6, 8}) {
