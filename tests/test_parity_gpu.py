@@ -462,6 +462,50 @@ def test_backward_pass_in_a_cuda_graph_gives_the_same_bits():
         assert torch.equal(a, b)
 
 
+def test_two_host_threads_run_forward_and_backward_side_by_side():
+    """Two host threads, each with its own stream, workspace and outputs, run the forward and
+    backward pass of the same layer at the same time (the library keeps its second stream and its
+    probe per host thread, its set-up flags per device): both get the bits of a single-threaded run."""
+    import threading
+    cfg = LayerConfig("threads", 512, 384, 32, 4, 16, 1.0, 700, seed=41)
+    layer = GpuLayer(cfg)
+    M, d = cfg.tokens, layer.d
+    ref_y = layer.forward()
+    ref_b = layer.backward()
+    results, errors = {}, []
+
+    def worker(tag):
+        try:
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                wf = Q.alloc_workspace(d, M, Q.OP_FORWARD)
+                wb = Q.alloc_workspace(d, M, Q.OP_BACKWARD)
+                for _ in range(5):
+                    y = torch.empty((M, cfg.d_out), dtype=torch.bfloat16, device="cuda")
+                    dx = torch.empty((M, cfg.d_in), dtype=torch.bfloat16, device="cuda")
+                    dA = torch.empty((cfg.groups, cfg.rank), dtype=torch.float32, device="cuda")
+                    dB = torch.empty((cfg.rank, cfg.d_out), dtype=torch.float32, device="cuda")
+                    Q.qalora_forward(d, M, layer.dev["x"], layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"], y, wf)
+                    Q.qalora_backward(d, M, layer.dev["x"], layer.dev["dy"], layer.codes, layer.qparams, layer.dev["A"],
+                                      layer.dev["B"], dx, dA, dB, wb)
+                stream.synchronize()
+                results[tag] = (y, dx, dA, dB, Q.workspace_status(wf), Q.workspace_status(wb))
+        except Exception as e:  # noqa: BLE001 - reported by the main thread
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for tag in range(2):
+        y, dx, dA, dB, sf, sb = results[tag]
+        assert sf == 0 and sb == 0
+        assert torch.equal(y, ref_y) and torch.equal(dx, ref_b[0]) and torch.equal(dA, ref_b[1]) and torch.equal(dB, ref_b[2])
+
+
 def test_results_do_not_depend_on_scheduling():
     cfg = LayerConfig("det", 256, 256, 32, 4, 16, 1.0, 300, seed=5)
     layer = GpuLayer(cfg)
