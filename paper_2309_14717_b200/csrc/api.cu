@@ -1,5 +1,6 @@
 // C-ABI entry points: argument checks, scratch layout and kernel dispatch.
 #define QALORA_TU 1
+#include <algorithm>
 #include <atomic>
 #include <mutex>
 
@@ -638,7 +639,10 @@ StepLayout step_layout(const Shape& sh, int64_t m) {
   const size_t M = (size_t)m;
   L.rows = step_chunk_rows(m);
   L.chunks = m > 0 ? (int)((m + L.rows - 1) / L.rows) : 1;
-  L.ws_bytes = workspace_layout(sh, L.rows, QALORA_OP_TRAIN).total;
+  // (a shorter last chunk may take another kernel, whose scratch can be LARGER than a full chunk's:
+  // few rows have their reduction cut into parts with fp32 partial results)
+  const int64_t last_rows = m > 0 ? m - (int64_t)(L.chunks - 1) * L.rows : L.rows;
+  L.ws_bytes = std::max(workspace_layout(sh, L.rows, QALORA_OP_TRAIN).total, workspace_layout(sh, last_rows, QALORA_OP_TRAIN).total);
   L.ws = take(L.ws_bytes);                         // first: the status word sits at the head of the staging area
   L.x = take(M * sh.K * 2); L.dy = take(M * sh.N * 2); L.y = take(M * sh.N * 2); L.dx = take(M * sh.K * 2);
   L.dA = take((size_t)sh.G * sh.r * 4); L.dB = take((size_t)sh.r * sh.N * 4);

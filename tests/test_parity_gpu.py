@@ -565,3 +565,30 @@ def test_chunked_step_from_host_buffers():
         assert rel_err(hdA.numpy(), dA_ref) <= TOL and rel_err(hdB.numpy(), dB_ref) <= TOL
         # dB contracts the bf16 copy of the rank-r intermediate: a few of the tail chunk's entries round the other way
         assert rel_err(hdA.numpy(), dA.cpu().numpy()) <= 1e-5 and rel_err(hdB.numpy(), dB.cpu().numpy()) <= 5e-4
+
+
+@pytest.mark.gpu
+def test_host_step_whose_short_last_chunk_needs_more_scratch_than_a_full_one():
+    # 2560 rows of a 1024 x 768 layer: two chunks of 1024 rows and one of 512, whose kernels cut
+    # their reductions into more parts and keep larger fp32 partial results than a full chunk's.
+    # The staging area must be sized for both; the results are those of the whole-batch device
+    # calls (rows are independent in y and dx: bit for bit on the full chunks' rows).
+    cfg = LayerConfig("hostchunks_tail", 1024, 768, 32, 4, 64, 1.0, 2560, seed=23)
+    layer = GpuLayer(cfg)
+    assert Q.qalora_workspace_bytes(layer.d, 512, Q.OP_TRAIN) > Q.qalora_workspace_bytes(layer.d, 1024, Q.OP_TRAIN)
+    y = layer.forward()
+    dx, dA, dB = layer.backward()
+    pin = lambda t: t.pin_memory()
+    hx, hdy = pin(layer.cpu["x"]), pin(layer.cpu["dy"])
+    hy, hdx = pin(torch.zeros_like(y, device="cpu")), pin(torch.zeros_like(dx, device="cpu"))
+    hdA, hdB = pin(torch.zeros_like(dA, device="cpu")), pin(torch.zeros_like(dB, device="cpu"))
+    staging = torch.zeros(Q.qalora_step_host_bytes(layer.d, cfg.tokens), dtype=torch.uint8, device="cuda")
+    Q.qalora_step_host(layer.d, cfg.tokens, hx, hdy, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"],
+                       hy, hdx, hdA, hdB, staging)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(staging) == 0
+    assert torch.equal(hy[:2048], y[:2048].cpu()) and torch.equal(hdx[:2048], dx[:2048].cpu())
+    # (the short chunk adds its partial results in another order: one bf16 step of the largest output at most)
+    assert rel_err(hy[2048:].float().numpy(), y[2048:].float().cpu().numpy()) <= 4e-3
+    assert rel_err(hdx[2048:].float().numpy(), dx[2048:].float().cpu().numpy()) <= 4e-3
+    assert rel_err(hdA.numpy(), dA.cpu().numpy()) <= 1e-4 and rel_err(hdB.numpy(), dB.cpu().numpy()) <= 1e-3
