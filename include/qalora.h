@@ -93,7 +93,10 @@ int qalora_packed_bytes(const qalora_desc* desc, size_t* code_bytes, size_t* qpa
  * input, the rank-r intermediates and split-K partial sums; its content is
  * undefined on entry.  On exit its first int32 is a device status word: 0, or
  * 1 when a bounded wait inside a tensor-core kernel expired (the outputs of
- * that call are then invalid; nothing hangs or traps). */
+ * that call are then invalid; nothing hangs or traps).  The size is for exactly
+ * `m` rows and does not grow monotonically with m: a smaller batch may take a
+ * kernel that cuts its reduction into more parts and keeps larger partial sums,
+ * so a workspace that serves several batch sizes takes the largest of their sizes. */
 int qalora_workspace_bytes(const qalora_desc* desc, int64_t m, int op, size_t* bytes);
 
 /* Group-wise min-max quantization, Eq. 1 per (group, column) (Section 3.3):
@@ -207,9 +210,12 @@ int qalora_merge(const qalora_desc* desc, const float* qparams_in, const void* A
  * more are cut into up to 8 row chunks (multiples of 256 rows, at least 1024):
  * the copies run on two streams of the library's own (made on first use, one
  * pair per device), so that a chunk's inputs arrive while the previous chunk
- * computes and the one before that returns.  y and dx are the same bits as from
- * one qalora_forward / qalora_backward over all rows; dA and dB are then the sums
- * of the chunks' results in chunk order (a different, fixed, summation order).
+ * computes and the one before that returns.  Rows are independent in y and dx:
+ * the full chunks' rows are the same bits as from one qalora_forward /
+ * qalora_backward over all rows; a shorter last chunk may take another kernel
+ * (another summation order: its rows agree to within one bf16 step).  dA and dB
+ * are then the sums of the chunks' results in chunk order (a different, fixed,
+ * summation order).
  * Calls from several host threads are serialized by the library.
  *   x_host, dy_host   in : HOST memory (pinned for asynchronous copies), bf16 [m][K], [m][N]
  *   codes, qparams, A, B : DEVICE memory, as for qalora_forward
