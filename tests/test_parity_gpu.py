@@ -159,6 +159,56 @@ def test_small_shapes_all_ops(case):
     assert torch.equal(q3, q2)
 
 
+BOUNDARY_M = [1, 2, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 100, 127, 128, 129, 255, 256, 257, 384, 511, 512,
+              513, 767, 1024, 1025]
+
+
+@pytest.mark.parametrize("bits,g,r", [(4, 32, 24), (3, 64, 64)])
+def test_token_counts_around_every_dispatch_boundary(bits, g, r):
+    """One layer (1024 -> 6144: 48 channel tiles, so every kernel family is eligible somewhere),
+    token counts on both sides of every row-count threshold of the dispatch (few-token kernel up
+    to 16 or 32 rows, tokens-as-MMA-rows kernel up to 64 or 128, token-rows pooling from 512,
+    256-token tiles with ragged tails).  y and dX of the first M rows do not depend on the rows
+    behind them, so one oracle pass over all rows serves every M; dA and dB are sums over the rows
+    and are taken from the oracle per M."""
+    K, N, s = 1024, 6144, 0.75
+    name = f"boundary_b{bits}"
+    cfg = LayerConfig(name, K, N, g, bits, r, s, max(BOUNDARY_M), dy_std=1.0, outlier_frac=0.01, seed=31 + bits)
+    layer = GpuLayer(cfg)
+    codes, alpha, beta = check_quantize(layer)
+    x, A, B, dy = (to_f64(layer.cpu[k]) for k in ("x", "A", "B", "dy"))
+    y_ref = O.forward(x, codes, alpha, beta, g, A, B, s)
+    dx_ref, _, _ = O.backward(x, dy, codes, alpha, beta, g, A, B, s)
+    q2 = torch.empty_like(layer.qparams)
+    Q.qalora_merge(layer.d, layer.qparams, layer.dev["A"], layer.dev["B"], q2)
+    for M in BOUNDARY_M:
+        xm, dym = layer.dev["x"][:M].contiguous(), layer.dev["dy"][:M].contiguous()
+        # (scale of a slice's comparison: the slice's own largest reference value, as everywhere)
+        margin(name, "y", layer.forward(x=xm).float().cpu().numpy(), y_ref[:M])
+        margin(name, "y_merged", layer.forward(x=xm, qparams=q2, rank=0).float().cpu().numpy(), y_ref[:M])
+        dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        dA = torch.full((cfg.groups, r), float("nan"), dtype=torch.float32, device="cuda")
+        dB = torch.full((r, N), float("nan"), dtype=torch.float32, device="cuda")
+        ws = torch.full((max(Q.qalora_workspace_bytes(layer.d, M, Q.OP_BACKWARD), 16),), 0xFF, dtype=torch.uint8, device="cuda")
+        Q.qalora_backward(layer.d, M, xm, dym, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"], dx, dA, dB, ws)
+        torch.cuda.synchronize()
+        assert Q.workspace_status(ws) == 0, M
+        _, dA_ref, dB_ref = O.backward(x[:M], dy[:M], codes, alpha, beta, g, A, B, s)
+        margin(name, "dX", dx.float().cpu().numpy(), dx_ref[:M])
+        margin(name, "dA", dA.cpu().numpy(), dA_ref)
+        margin(name, "dB", dB.cpu().numpy(), dB_ref)
+        # the fine-tuning pair (one workspace, the input pooled once) gives the bits of the separate calls
+        wt = torch.full((max(Q.qalora_workspace_bytes(layer.d, M, Q.OP_TRAIN), 16),), 0xFF, dtype=torch.uint8, device="cuda")
+        y_t = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        dx_t, dA_t, dB_t = torch.empty_like(dx), torch.empty_like(dA), torch.empty_like(dB)
+        Q.qalora_forward_train(layer.d, M, xm, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"], y_t, wt)
+        Q.qalora_backward_train(layer.d, M, xm, dym, layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"], dx_t, dA_t, dB_t, wt)
+        torch.cuda.synchronize()
+        assert Q.workspace_status(wt) == 0, M
+        assert torch.equal(y_t, layer.forward(x=xm)) and torch.equal(dx_t, dx), M
+        assert torch.equal(dA_t, dA) and torch.equal(dB_t, dB), M
+
+
 def test_config1_full():
     cfg = CONFIGS["cfg1_512"]
     layer = GpuLayer(cfg)
