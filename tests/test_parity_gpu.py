@@ -122,6 +122,21 @@ SMALL = [
     ("tail2", 1024, 5120, 128, 2, 8, 1.0, 1000),      # 40 x 4 tiles: a strip of 3 channel tiles over all four token tiles
     ("tail_dx4", 5120, 1024, 32, 4, 16, 1.0, 1000),   # the same for the input gradient (40 x 4 tiles along the input channels)
     ("tail_dx3", 5120, 1152, 64, 3, 24, 1.0, 520),    # 40 x 3 tiles: none in a strip (120 < SMs); 1152 = 9 x 128 reduction
+    # tile counts just above one and two full waves of SMs (149, 150, 185, 222, 295, 297 tiles with one token
+    # tile; 150 and 297 with three): the last wave's strip holds 1 to 147 tiles and is cut into parts
+    ("strip_f149", 256, 149 * 128, 32, 4, 16, 1.0, 200),
+    ("strip_f150", 256, 150 * 128, 64, 3, 8, 1.0, 256),
+    ("strip_f185", 512, 185 * 128, 32, 4, 16, 1.0, 130),
+    ("strip_f222", 256, 222 * 128, 128, 2, 8, 1.0, 200),
+    ("strip_f295", 256, 295 * 128, 32, 4, 8, 1.0, 255),
+    ("strip_f297", 384, 297 * 128, 32, 4, 16, 1.0, 200),
+    ("strip_f50x3", 512, 50 * 128, 32, 4, 16, 1.0, 520),
+    ("strip_f99x3", 256, 99 * 128, 64, 4, 16, 1.0, 700),
+    # the same for the input gradient (tiles along the input channels)
+    ("strip_d149", 149 * 128, 256, 32, 4, 16, 1.0, 200),
+    ("strip_d185", 185 * 128, 384, 64, 3, 8, 1.0, 130),
+    ("strip_d297", 297 * 128, 256, 32, 4, 16, 1.0, 256),
+    ("strip_d50x3", 50 * 128, 512, 128, 2, 8, 1.0, 520),
     # many tokens, several channel tiles, ragged token count
     ("pair4", 512, 256, 32, 4, 16, 1.0, 700),
     ("pair3", 384, 512, 64, 3, 24, 0.75, 530),
@@ -236,6 +251,24 @@ def test_config2_small_m_forward_and_merge(M):
     Q.qalora_merge(layer.d, layer.qparams, layer.dev["A"], layer.dev["B"], q2)
     margin(f"cfg2_7b_attn_m{M}", "beta_merged", q2.cpu().numpy()[..., 1], O.merge(beta, A, B, s))
     margin(f"cfg2_7b_attn_m{M}", "y_merged", layer.forward(qparams=q2, rank=0).float().cpu().numpy(), y_ref)
+
+
+@pytest.mark.parametrize("K,N", [(128, 128), (384, 128), (640, 128), (896, 640), (1408, 256), (2176, 1152), (128, 19072)])
+def test_few_token_forward_slice_counts(K, N):
+    """Few-token kernel: reductions of 1, 3, 5, 7, 11 and 17 stages of 128 channels (so the slices of
+    a column tile are unequal, and a layer of one stage cannot be cut at all) on 1 to 149 column
+    tiles, i.e. every slice count the host can pick, with 1, 8, 16 and 32 rows, with and without
+    the adapter, 4-bit g = 32 and 3-bit g = 128."""
+    for bits, g, r in ((4, 32, 24), (3, 128, 0)):
+        name = f"slices_{K}x{N}_b{bits}"
+        cfg = LayerConfig(name, K, N, g, bits, max(r, 8), 1.25, 32, outlier_frac=0.01, seed=K + N + bits)
+        layer = GpuLayer(cfg, need=("W", "x", "A", "B"))
+        codes, alpha, beta = check_quantize(layer)
+        x, A, B = (to_f64(layer.cpu[k]) for k in ("x", "A", "B"))
+        y_ref = O.forward(x, codes, alpha, beta, g, A if r else None, B if r else None, cfg.scale)
+        for M in (1, 8, 16, 32):
+            xm = layer.dev["x"][:M].contiguous()
+            margin(name, "y", layer.forward(x=xm, rank=None if r else 0).float().cpu().numpy(), y_ref[:M])
 
 
 @pytest.mark.parametrize("bits,g,M,r", [(4, 32, 1, 16), (4, 128, 8, 0), (3, 32, 16, 24), (3, 64, 3, 8),
