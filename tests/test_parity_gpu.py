@@ -115,6 +115,13 @@ SMALL = [
     ("midm4_128", 256, 512, 64, 4, 16, 1.0, 128),
     ("midm4_33", 4096, 256, 32, 4, 72, 0.5, 33),
     ("midm4_r64_65", 1024, 768, 32, 4, 64, 1.0, 65),
+    # the same kernel with the shortest reduction it takes (4 steps of 64 channels), odd step counts (5, 17, 19,
+    # 65: the parts of a cut reduction are unequal) and reductions that are not a multiple of 128 channels
+    ("midm_4st", 256, 2560, 128, 2, 8, 1.0, 50),
+    ("midm_5st", 320, 256, 32, 4, 16, 1.0, 33),
+    ("midm_17st", 1088, 256, 32, 4, 16, 1.0, 40),
+    ("midm_19st", 1216, 768, 64, 3, 8, 1.0, 17),
+    ("midm_65st", 4160, 512, 32, 4, 64, 1.0, 64),
     # more 128 x 256 tiles than SMs with a short last wave: that wave's tiles alone are cut into parts
     # (160 and 320 tiles: 12 and 24 in the strip; ragged last token tiles)
     ("tail4", 2048, 20480, 32, 4, 16, 1.0, 256),
