@@ -71,6 +71,18 @@ def test_merged_layers_of_different_shapes_run_in_one_launch(bits, g, M):
     check_against_oracle(layers, M, f"group_b{bits}_g{g}_m{M}", 0)
 
 
+def test_eight_layers_take_one_launch_and_nine_run_one_by_one():
+    # the work list holds up to eight layers; one of them has a single 128-channel stage, so the
+    # whole group runs with one slice per column tile
+    shapes = [(512, 384), (1280, 256), (128, 128), (2048, 640), (384, 1152), (896, 128), (640, 512), (256, 256)]
+    layers = build_layers(shapes, 4, 32, 3, rank=0)
+    assert run_group(layers, 3) == 1 and Q.qalora_main_kernel_name() == "qalora_gemv_group_kernel"
+    check_against_oracle(layers, 3, "group_of_8", 0)
+    layers = build_layers(shapes + [(512, 128)], 4, 32, 3, rank=0)
+    assert run_group(layers, 3) == 9
+    check_against_oracle(layers, 3, "group_of_9", 0)
+
+
 def test_groups_outside_the_one_launch_path_fall_back_layer_by_layer():
     # adapters: pooling kernel + few-token kernel per layer
     layers = build_layers([(512, 384), (1280, 256)], 4, 32, 4, rank=16)
