@@ -50,6 +50,9 @@ extern "C" {
 
 #define QALORA_LAYOUT_VERSION 1
 
+/* Most token rows a call takes (2^22): beyond it QALORA_ERR_INVALID_ARG. */
+#define QALORA_MAX_ROWS 4194304
+
 typedef enum qalora_status {
   QALORA_OK = 0,
   QALORA_ERR_INVALID_ARG = -1,      /* a size or enum outside its domain        */
@@ -116,7 +119,10 @@ int qalora_quantize(const qalora_desc* desc, const float* W, void* codes, float*
 /* Forward pass, Algorithm 1 / Appendix B Eq. 4:
  *   y = x * W~ + s * (pool(x) * A) * B.
  *   x bf16 [m][K];  A bf16 [G][r];  B bf16 [r][N];  y out bf16 [m][N].
- * Products are bf16 x bf16 accumulated in float32.  Any m >= 0 is accepted; the
+ * Products are bf16 x bf16 accumulated in float32.  Any m with 0 <= m <= QALORA_MAX_ROWS
+ * is accepted by every call that takes a row count, more is QALORA_ERR_INVALID_ARG
+ * (element and byte offsets are 64-bit: tensors of more than 2^31 elements are fine, a
+ * test runs 200 000 rows of an 11008-wide layer; tile counts are 32-bit); the
  * kernel is chosen from m (a bandwidth-bound path for a few rows, a
  * tensor-core path otherwise).  The few-token kernel of a layer without adapter may
  * start while the kernel before it in the stream is still running (programmatic dependent

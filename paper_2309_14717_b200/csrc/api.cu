@@ -188,7 +188,7 @@ int forward_validate(const qalora_desc* desc, int64_t m, const void* x, const vo
   Shape sh;
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
-  if (m < 0) return QALORA_ERR_INVALID_ARG;
+  if (m < 0 || m > QALORA_MAX_ROWS) return QALORA_ERR_INVALID_ARG;
   if (m == 0) return QALORA_OK;
   if (x == nullptr || codes == nullptr || qparams == nullptr || y == nullptr) return QALORA_ERR_NULL_POINTER;
   if (sh.r > 0 && (A == nullptr || B == nullptr)) return QALORA_ERR_NULL_POINTER;
@@ -301,7 +301,7 @@ int backward_impl(const qalora_desc* desc, int64_t m, const void* x, const void*
   Shape sh;
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
-  if (m < 0 || sh.r == 0) return QALORA_ERR_INVALID_ARG;
+  if (m < 0 || m > QALORA_MAX_ROWS || sh.r == 0) return QALORA_ERR_INVALID_ARG;
   if (x == nullptr || dy == nullptr || codes == nullptr || qparams == nullptr || A == nullptr || B == nullptr)
     return QALORA_ERR_NULL_POINTER;
   // `pooled`: the workspace is the one qalora_forward_train filled for the same x, A and m; its
@@ -497,7 +497,7 @@ int qalora_workspace_bytes(const qalora_desc* desc, int64_t m, int op, size_t* b
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
   if (bytes == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (m < 0 || (op != QALORA_OP_FORWARD && op != QALORA_OP_BACKWARD && op != QALORA_OP_TRAIN)) return QALORA_ERR_INVALID_ARG;
+  if (m < 0 || m > QALORA_MAX_ROWS || (op != QALORA_OP_FORWARD && op != QALORA_OP_BACKWARD && op != QALORA_OP_TRAIN)) return QALORA_ERR_INVALID_ARG;
   *bytes = workspace_layout(sh, m, op).total;
   return QALORA_OK;
 }
@@ -553,7 +553,7 @@ int qalora_backward_train(const qalora_desc* desc, int64_t m, const void* x, con
 
 int qalora_forward_group_workspace_bytes(const qalora_group_layer* layers, int n, int64_t m, size_t* bytes) {
   if (layers == nullptr || bytes == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (n < 0 || m < 0) return QALORA_ERR_INVALID_ARG;
+  if (n < 0 || m < 0 || m > QALORA_MAX_ROWS) return QALORA_ERR_INVALID_ARG;
   size_t need = 256;                                 // the status word
   for (int i = 0; i < n; ++i) {
     Shape sh;
@@ -569,7 +569,7 @@ int qalora_forward_group_workspace_bytes(const qalora_group_layer* layers, int n
 int qalora_forward_group(const qalora_group_layer* layers, int n, int64_t m,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (layers == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (n < 0 || m < 0) return QALORA_ERR_INVALID_ARG;
+  if (n < 0 || m < 0 || m > QALORA_MAX_ROWS) return QALORA_ERR_INVALID_ARG;
   size_t need = 0;
   int st = qalora_forward_group_workspace_bytes(layers, n, m, &need);
   if (st != QALORA_OK) return st;
@@ -687,7 +687,7 @@ int qalora_step_host_bytes(const qalora_desc* desc, int64_t m, size_t* bytes) {
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
   if (bytes == nullptr) return QALORA_ERR_NULL_POINTER;
-  if (m < 0) return QALORA_ERR_INVALID_ARG;
+  if (m < 0 || m > QALORA_MAX_ROWS) return QALORA_ERR_INVALID_ARG;
   *bytes = step_layout(sh, m).total;
   return QALORA_OK;
 }
@@ -699,7 +699,7 @@ int qalora_step_host(const qalora_desc* desc, int64_t m, const void* x_host, con
   Shape sh;
   int st = check_desc(desc, &sh);
   if (st != QALORA_OK) return st;
-  if (m < 0 || sh.r == 0) return QALORA_ERR_INVALID_ARG;
+  if (m < 0 || m > QALORA_MAX_ROWS || sh.r == 0) return QALORA_ERR_INVALID_ARG;
   if (x_host == nullptr || dy_host == nullptr || y_host == nullptr || dx_host == nullptr || dA_host == nullptr ||
       dB_host == nullptr || staging == nullptr)
     return QALORA_ERR_NULL_POINTER;

@@ -80,6 +80,10 @@ def test_null_and_misaligned_pointers_are_rejected_without_a_launch():
     assert lib.qalora_quantize(r(d), p(a16 + 4), p(a16), p(a16), None, None) == -4
     assert lib.qalora_merge(r(d), p(a16), None, p(a16), p(a16), None) == -2
     assert lib.qalora_forward(r(d), -1, p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), 1 << 30, None) == -1
+    assert lib.qalora_forward(r(d), (1 << 22) + 1, p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), 1 << 30, None) == -1
+    size = ctypes.c_size_t(0)
+    assert lib.qalora_workspace_bytes(r(d), 1 << 22, Q.OP_TRAIN, r(size)) == 0 and size.value > 0
+    assert lib.qalora_workspace_bytes(r(d), (1 << 22) + 1, Q.OP_TRAIN, r(size)) == -1
     assert lib.qalora_forward(r(d), 8, None, p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), 1 << 30, None) == -2
     assert lib.qalora_forward(r(d), 8, p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), 0, None) == -5
     assert lib.qalora_forward(r(d), 8, p(a16 + 2), p(a16), p(a16), p(a16), p(a16), p(a16), p(a16), 1 << 30, None) == -4

@@ -131,3 +131,56 @@ def test_full_size_layer(name, over):
         torch.cuda.synchronize()
         assert Q.qalora_main_kernel_name() == "qalora_gemv_kernel" and Q.workspace_status(wm) == 0
         record_margin(case, f"y_adapted_m{m}", rel_err(ym.float().cpu().numpy(), y16_ref[:m]), TOL)
+
+
+@pytest.mark.parametrize("name", ["cfg3_7b_up", "cfg3_7b_down"])
+def test_two_hundred_thousand_rows_index_past_2_to_the_31(name):
+    """200 000 token rows on the 7B MLP shapes: y (4096 -> 11008) resp. x and dX (11008 -> 4096)
+    hold 2.2e9 elements, so every element offset of their last rows lies beyond 2^31 (and the
+    byte offsets beyond 2^32).  The fp64 oracle cannot take this size, so the check is by
+    properties that hold at any size: rows are independent in y and dX, hence the first and the
+    last 256 rows must agree with a 256-row call on those rows alone (the paths checked against
+    the oracle above); dA and dB are sums over the rows, hence equal to the sum of the results
+    of eight 25 000-row calls.  x and dy are drawn on the device from a seeded generator."""
+    cfg = CONFIGS[name]
+    M, K, N, G, r, g, s = 200_000, cfg.d_in, cfg.d_out, cfg.groups, cfg.rank, cfg.group_size, cfg.scale
+    assert M * max(K, N) > 2 ** 31
+    cpu = make_inputs(cfg, need=("W", "A", "B"))
+    d = Q.desc(K, N, g, cfg.bits, r, s)
+    W, A, B = cpu["W"].cuda(), cpu["A"].cuda(), cpu["B"].cuda()
+    codes, qparams = Q.alloc_packed(d)
+    Q.qalora_quantize(d, W, codes, qparams)
+    del W
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234 + K)
+    x = torch.empty((M, K), dtype=torch.bfloat16, device="cuda").normal_(0.0, 1.0, generator=gen)
+    dy = torch.empty((M, N), dtype=torch.bfloat16, device="cuda").normal_(0.0, cfg.dy_std, generator=gen)
+
+    def run(xs, dys):
+        m = xs.shape[0]
+        y = torch.empty((m, N), dtype=torch.bfloat16, device="cuda")
+        dx = torch.empty((m, K), dtype=torch.bfloat16, device="cuda")
+        dA = torch.empty((G, r), dtype=torch.float32, device="cuda")
+        dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
+        ws = Q.alloc_workspace(d, m, Q.OP_TRAIN)
+        Q.qalora_forward_train(d, m, xs, codes, qparams, A, B, y, ws)
+        Q.qalora_backward_train(d, m, xs, dys, codes, qparams, A, B, dx, dA, dB, ws)
+        torch.cuda.synchronize()
+        assert Q.workspace_status(ws) == 0
+        return y, dx, dA, dB
+
+    y, dx, dA, dB = run(x, dy)
+    case = f"{name}_m200000"
+    for lo in (0, M - 256):
+        ys, dxs, _, _ = run(x[lo:lo + 256].contiguous(), dy[lo:lo + 256].contiguous())
+        # (the 256-row call cuts its reduction into parts: another summation order, within one bf16 step)
+        record_margin(case, f"y_rows_{lo}", rel_err(y[lo:lo + 256].float().cpu().numpy(), ys.float().cpu().numpy()), 4e-3)
+        record_margin(case, f"dX_rows_{lo}", rel_err(dx[lo:lo + 256].float().cpu().numpy(), dxs.float().cpu().numpy()), 4e-3)
+    dA_sum = torch.zeros((G, r), dtype=torch.float64, device="cuda")
+    dB_sum = torch.zeros((r, N), dtype=torch.float64, device="cuda")
+    for lo in range(0, M, 25_000):
+        _, _, dA_c, dB_c = run(x[lo:lo + 25_000], dy[lo:lo + 25_000])
+        dA_sum += dA_c.double()
+        dB_sum += dB_c.double()
+    record_margin(case, "dA_additive", rel_err(dA.cpu().numpy(), dA_sum.cpu().numpy()), 1e-4)
+    record_margin(case, "dB_additive", rel_err(dB.cpu().numpy(), dB_sum.cpu().numpy()), 1e-3)
