@@ -19,7 +19,7 @@ import torch
 from conftest import record_margin
 from oracle import qalora_oracle as O
 from paper_2309_14717_b200 import binding as Q
-from paper_2309_14717_b200.synthetic import CONFIGS, make_inputs, to_f64
+from paper_2309_14717_b200.synthetic import CONFIGS, LayerConfig, make_inputs, to_f64
 
 pytestmark = pytest.mark.gpu
 TOL = 5e-3
@@ -184,3 +184,70 @@ def test_two_hundred_thousand_rows_index_past_2_to_the_31(name):
         dB_sum += dB_c.double()
     record_margin(case, "dA_additive", rel_err(dA.cpu().numpy(), dA_sum.cpu().numpy()), 1e-4)
     record_margin(case, "dB_additive", rel_err(dB.cpu().numpy(), dB_sum.cpu().numpy()), 1e-3)
+
+
+VOCAB = 128256     # 1002 channel tiles of 128
+
+
+@pytest.mark.parametrize("K,N", [(4096, VOCAB), (VOCAB, 4096)], ids=["to_vocabulary", "from_vocabulary"])
+def test_vocabulary_sized_dimension(K, N):
+    """A layer with 128256 output resp. input channels (an output head, an embedding-sized input):
+    a thousand channel tiles, 525 M weights.  The oracle quantizes and contracts what it is
+    asked for, so it is asked for samples that are exact by themselves: y on three ranges of
+    output columns (a column of y needs that column of W alone), dX on three quantization groups
+    of input channels (a channel of dX needs that row group of W alone), codes and (alpha, beta)
+    on both samples, dA and dB in full (they do not involve W)."""
+    g, bits, r, s, M = 32, 4, 64, 1.0, 300
+    case = f"vocab_{K}x{N}"
+    cfg = LayerConfig(case, K, N, g, bits, r, s, M, seed=91)
+    cpu = make_inputs(cfg)
+    d = Q.desc(K, N, g, bits, r, s)
+    dev = {k: v.cuda() for k, v in cpu.items() if k != "W"}
+    codes_d, qparams = Q.alloc_packed(d)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    W_dev = cpu["W"].cuda()
+    Q.qalora_quantize(d, W_dev, codes_d, qparams, status)
+    del W_dev
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    words = codes_d.cpu().numpy().view(np.uint32).reshape(K // 32, N, -1)
+    qp = qparams.cpu().numpy().reshape(K // g, N, 2)
+    Wn = cpu["W"].numpy()
+    x, A, B, dy = (to_f64(cpu[k]) for k in ("x", "A", "B", "dy"))
+
+    # ---- output-column sample: quantization, forward (300, 16 and 1 rows), merge + merged forward
+    cols = np.r_[0:256, N // 2 + 37:N // 2 + 237, N - 256:N]
+    codes, alpha, beta = O.quantize(np.ascontiguousarray(Wn[:, cols]), g, bits)
+    assert np.array_equal(words[:, cols, :], O.pack(codes, bits).reshape(K // 32, len(cols), -1))
+    assert np.array_equal(qp[:, cols, 0], alpha) and np.array_equal(qp[:, cols, 1], beta)
+    y_ref = O.forward(x, codes, alpha, beta, g, A, B[:, cols], s)
+    q2 = torch.empty_like(qparams)
+    Q.qalora_merge(d, qparams, dev["A"], dev["B"], q2)
+    record_margin(case, "beta_merged", rel_err(q2.cpu().numpy().reshape(K // g, N, 2)[:, cols, 1], O.merge(beta, A, B[:, cols], s)), TOL)
+    d0 = Q.desc(K, N, g, bits, 0, s)
+    for m in (300, 16, 1):
+        xm = dev["x"][:m].contiguous()
+        y = torch.empty((m, N), dtype=torch.bfloat16, device="cuda")
+        Q.qalora_forward(d, m, xm, codes_d, qparams, dev["A"], dev["B"], y, Q.alloc_workspace(d, m, Q.OP_FORWARD))
+        record_margin(case, f"y_m{m}", rel_err(y.float().cpu().numpy()[:, cols], y_ref[:m]), TOL)
+        Q.qalora_forward(d0, m, xm, codes_d, q2, None, None, y, Q.alloc_workspace(d0, m, Q.OP_FORWARD))
+        record_margin(case, f"y_merged_m{m}", rel_err(y.float().cpu().numpy()[:, cols], y_ref[:m]), TOL)
+
+    # ---- input-channel sample (whole quantization groups): quantization and dX; dA, dB in full
+    groups = np.array([0, (K // g) // 2 + 3, K // g - 1])
+    rows = (groups[:, None] * g + np.arange(g)[None, :]).reshape(-1)
+    codes_k, alpha_k, beta_k = O.quantize(np.ascontiguousarray(Wn[rows, :]), g, bits)
+    assert np.array_equal(words[groups * (g // 32)], O.pack(codes_k, bits).reshape(len(groups), N, -1))
+    assert np.array_equal(qp[groups, :, 0], alpha_k) and np.array_equal(qp[groups, :, 1], beta_k)
+    dx = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dA = torch.empty((K // g, r), dtype=torch.float32, device="cuda")
+    dB = torch.empty((r, N), dtype=torch.float32, device="cuda")
+    wb = Q.alloc_workspace(d, M, Q.OP_BACKWARD)
+    Q.qalora_backward(d, M, dev["x"], dev["dy"], codes_d, qparams, dev["A"], dev["B"], dx, dA, dB, wb)
+    torch.cuda.synchronize()
+    assert Q.workspace_status(wb) == 0
+    dx_ref, _, _ = O.backward(x[:, rows], dy, codes_k, alpha_k, beta_k, g, A[groups], B, s)
+    record_margin(case, "dX", rel_err(dx.float().cpu().numpy()[:, rows], dx_ref), TOL)
+    dA_ref, dB_ref = O.backward_adapter(x, dy, g, A, B, s)
+    record_margin(case, "dA", rel_err(dA.cpu().numpy(), dA_ref), TOL)
+    record_margin(case, "dB", rel_err(dB.cpu().numpy(), dB_ref), TOL)
