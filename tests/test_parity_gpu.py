@@ -94,6 +94,10 @@ SMALL = [
     ("ragged2", 256, 72, 128, 2, 8, 2.0, 33),
     ("g64_4", 512, 384, 64, 4, 64, 1.0, 200),
     ("colwise", 128, 64, 128, 4, 8, 1.0, 16),
+    # group sizes other than 32, 64, 128 (multiples of 32): CUDA-core kernels whatever the other sizes are
+    ("g96", 384, 136, 96, 4, 8, 1.0, 50),
+    ("g256", 512, 256, 256, 3, 16, 1.0, 300),
+    ("g1024", 1024, 128, 1024, 2, 8, 1.0, 20),
     # shapes the tensor-core kernels tile (N % 128 == 0, K % 128 == 0), ragged in M
     ("tc4", 256, 256, 32, 4, 16, 1.0, 300),
     ("tc3", 384, 256, 64, 3, 24, 0.75, 270),
