@@ -67,6 +67,7 @@ struct TcParams {
   float* partial;              // parts: fp32 partial results [ksplit][part_rows][part_ld] of the output rectangle that
   int part_rows, part_ld;      //        starts at row part_row0, channel part_col0 (the whole output: M, ld_out, 0, 0)
   int part_row0, part_col0;
+  int beside_pool;             // host side: launch beside the few-row pooling kernel before this one (forward with adapter)
   int* status;                 // device word: set to 1 when a wait timed out
   int* dbg;                    // record words of the bounds-check build (null otherwise)
   int stop_after_steps;        // normally INT_MAX; a test makes every activation producer stop early, so that waits expire
@@ -235,6 +236,10 @@ qalora_tc_kernel(const __grid_constant__ CUtensorMap act_map, const __grid_const
             if (!(ok = ptx::mbar_wait(bar_lb_empty, (nlb & 1) ^ 1, abort_flag, p.wait_limit_ns))) break;
             ++nlb;
             ptx::mbar_arrive_expect_tx(bar_full_x(sb), ACT_BYTES + ATILE_BYTES);
+            // T is written by the pooling kernel, beside which this kernel may have started
+            // (programmatic dependent launch): wait for it only here, before T is fetched (a
+            // no-op without such a launch, or once that kernel has finished)
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             ptx::tma_load_2d(smem_base + S::OFF_X + s * ACT_BYTES, &lora_map, r0, m0, bar_full_x(sb));
             ptx::tma_load_2d(smem_base + S::OFF_A, &lb_map, c0, r0, bar_full_x(sb));
             ptx::tma_load_2d(smem_base + S::OFF_A + ATILE_BYTES / 2, &lb_map, c0 + 64, r0, bar_full_x(sb));
@@ -637,7 +642,21 @@ int launch_tc_t(const CUtensorMap& act, const CUtensorMap& lora, const TcParams&
   const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
   {
     MainKernelProbe probe(MODE == FWD ? "qalora_tc_kernel<fwd>" : "qalora_tc_kernel<dx>", st);
-    kern<<<grid, THREADS, S::TOTAL, st>>>(act, lora, lb, out, cmap, qmap, p);
+    // p.beside_pool: the kernel before this one in the stream is the few-row pooling kernel that
+    // writes T and lets its successor start at once; this kernel then starts beside it and waits
+    // for it only before an adapter step fetches T (x, the weights and the status word are final:
+    // the pooling kernel itself started after them).
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = S::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (MODE == FWD && p.beside_pool != 0) ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kern, act, lora, lb, out, cmap, qmap, p) != cudaSuccess) return QALORA_ERR_CUDA;
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
@@ -770,6 +789,9 @@ size_t tc_forward_partial_bytes(const Shape& sh, int64_t M) {
   return tail.strip_c > 0 ? (size_t)tail.ks * M * tail.strip_c * TILE_C * sizeof(float) : 0;
 }
 
+#ifndef QALORA_TC_BESIDE_POOL_ROWS
+#define QALORA_TC_BESIDE_POOL_ROWS 512
+#endif
 // y = x * W~ + Tb * B with Tb = bf16(s * pool(x) * A) precomputed ([M][r]).
 // `partial`: tc_forward_partial_bytes() of scratch.
 int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const uint32_t* codes,
@@ -791,6 +813,8 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
   p.ksplit = parts < 0 ? -parts : parts; p.tile_t = tile_t; p.partial = partial;
   p.c_tile0 = 0; p.tile_count = p.c_tiles * p.m_tiles;
   p.part_rows = (int)M; p.part_ld = sh.N; p.part_row0 = 0; p.part_col0 = 0;
+  // (below 512 rows the pooling kernel is the few-row one, which releases its successor at its start)
+  p.beside_pool = (sh.r > 0 && M < QALORA_TC_BESIDE_POOL_ROWS) ? 1 : 0;
   const TcTail tail = tc_forward_tail(sh, M);
   if (tail.strip_c > 0) {
     // whole tiles of the other channel tiles first, then the strip cut into parts (same stream: one after the other)
@@ -802,6 +826,7 @@ int launch_tc_forward(const Shape& sh, int64_t M, const __nv_bfloat16* x, const 
     TcParams pb = p;
     pb.c_tiles = tail.strip_c; pb.c_tile0 = pa.c_tiles; pb.tile_count = tail.strip_c * p.m_tiles; pb.ksplit = tail.ks;
     pb.part_rows = (int)M; pb.part_ld = tail.strip_c * TILE_C; pb.part_row0 = 0; pb.part_col0 = pa.c_tiles * TILE_C;
+    pb.beside_pool = 0;                              // its predecessor is the kernel above
     if (sh.bits == 4) return launch_tc<4, FWD>(act, lora, pb, st);
     if (sh.bits == 3) return launch_tc<3, FWD>(act, lora, pb, st);
     return launch_tc<2, FWD>(act, lora, pb, st);

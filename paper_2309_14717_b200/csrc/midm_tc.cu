@@ -170,8 +170,13 @@ qalora_midm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
           ptx::mbar_arrive_expect_tx(bar_full_x(s), MM_X_BYTES);
           if (j < w.n_main)
             ptx::tma_load_2d(smem_base + S::OFF_X + s * MM_X_BYTES, &x_map, (w.mb + j) * MM_J, m0, bar_full_x(s));
-          else
+          else {
+            // T is written by the pooling kernel, beside which this kernel may have started
+            // (programmatic dependent launch): wait for it only here, before T is fetched (a
+            // no-op when the launch carried no such attribute or the kernel has long finished)
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             ptx::tma_load_2d(smem_base + S::OFF_X + s * MM_X_BYTES, &t_map, (j - w.n_main) * MM_J, m0, bar_full_x(s));
+          }
         }
       }
     }
@@ -384,6 +389,9 @@ int mm_parts(const Shape& sh, int64_t M) {
   return best;
 }
 
+#ifndef QALORA_MM_PDL
+#define QALORA_MM_PDL 1
+#endif
 template <int BITS, int XROWS>
 int launch_midm_t(const CUtensorMap& xm, const CUtensorMap& tm, const MmParams& p, const uint32_t* codes,
                   const float2* qparams, cudaStream_t st) {
@@ -402,7 +410,21 @@ int launch_midm_t(const CUtensorMap& xm, const CUtensorMap& tm, const MmParams& 
   const int grid = items < device_sm_count() ? items : device_sm_count();
   {
     MainKernelProbe probe("qalora_midm_kernel", st);
-    kern<<<grid, MM_THREADS, S::TOTAL, st>>>(xm, tm, lb, cm, qm, p);
+    // With an adapter the kernel before this one in the stream is the few-row pooling kernel that
+    // writes T (it lets its successor start at once): this kernel starts beside it, streams and
+    // multiplies the weights, and waits for it only before the adapter step fetches T.  x, the
+    // weights and the status word are final by then: the pooling kernel itself started after them.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(MM_THREADS);
+    cfg.dynamicSmemBytes = S::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (QALORA_MM_PDL && p.r > 0) ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kern, xm, tm, lb, cm, qm, p) != cudaSuccess) return QALORA_ERR_CUDA;
   }
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return QALORA_ERR_CUDA;
