@@ -23,7 +23,7 @@ def _oracle_layer(cfg):
 
 
 @pytest.mark.parametrize("K,N,g,bits", [(64, 64, 32, 4), (320, 200, 32, 4), (192, 136, 64, 3), (256, 72, 128, 2),
-                                        (1024, 1000, 32, 3), (2048, 264, 64, 2)])
+                                        (1024, 1000, 32, 3), (2048, 264, 64, 2), (4096, 4096, 32, 4), (5120, 2048, 128, 3)])
 def test_dequantize_is_the_rounded_oracle_value(K, N, g, bits):
     cfg = LayerConfig("deq", K, N, g, bits, 8, 1.0, 4, outlier_frac=0.01, seed=K + bits)
     _, codes, alpha, beta, packed, qparams = _oracle_layer(cfg)
