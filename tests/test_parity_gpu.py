@@ -235,6 +235,25 @@ def test_token_counts_around_every_dispatch_boundary(bits, g, r):
         assert torch.equal(dA_t, dA) and torch.equal(dB_t, dB), M
 
 
+@pytest.mark.parametrize("M", [5, 100, 600])
+def test_backward_outputs_can_be_skipped_one_by_one(M):
+    """dx, dA or dB may be NULL: the other outputs are then the bits of the full call, and nothing
+    else is written (few rows, the CUDA-core side kernels; 100 and 600 rows, the tensor-core ones
+    with dB on the library's second stream)."""
+    cfg = LayerConfig("skip_outputs", 512, 384, 32, 4, 16, 1.0, M, dy_std=1.0, seed=5 + M)
+    layer = GpuLayer(cfg)
+    dx, dA, dB = layer.backward()
+    args = (layer.d, M, layer.dev["x"], layer.dev["dy"], layer.codes, layer.qparams, layer.dev["A"], layer.dev["B"])
+    for keep in ((1, 0, 0), (0, 1, 0), (0, 0, 1), (1, 1, 0), (0, 1, 1), (0, 0, 0)):
+        outs = [torch.full_like(t, float("nan")) for t in (dx, dA, dB)]
+        ws = torch.full((max(Q.qalora_workspace_bytes(layer.d, M, Q.OP_BACKWARD), 16),), 0xFF, dtype=torch.uint8, device="cuda")
+        Q.qalora_backward(*args, *[o if k else None for o, k in zip(outs, keep)], ws)
+        torch.cuda.synchronize()
+        assert Q.workspace_status(ws) == 0
+        for o, k, full in zip(outs, keep, (dx, dA, dB)):
+            assert torch.equal(o, full) if k else bool(torch.isnan(o).all()), (M, keep)
+
+
 def test_config1_full():
     cfg = CONFIGS["cfg1_512"]
     layer = GpuLayer(cfg)
