@@ -647,7 +647,8 @@ def test_step_from_host_buffers_matches_device_calls():
     assert torch.equal(hdA, dA.cpu()) and torch.equal(hdB, dB.cpu())
 
 
-def test_chunked_step_from_host_buffers():
+@pytest.mark.parametrize("pinned", [True, False], ids=["pinned", "pageable"])
+def test_chunked_step_from_host_buffers(pinned):
     # 2348 rows: three pipelined chunks (1024, 1024 and a ragged 300).  Rows are independent in y
     # and dx, so dx and the full chunks of y match the whole-batch device calls bit for bit; the
     # 300-row chunk pools its input with the few-row kernel (another summation order of the rank-r
@@ -657,7 +658,7 @@ def test_chunked_step_from_host_buffers():
     layer = GpuLayer(cfg)
     y = layer.forward()
     dx, dA, dB = layer.backward()
-    pin = lambda t: t.pin_memory()
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t.clone())   # pageable buffers: the copies are staged by the driver
     hx, hdy = pin(layer.cpu["x"]), pin(layer.cpu["dy"])
     hy, hdx = pin(torch.empty_like(y, device="cpu")), pin(torch.empty_like(dx, device="cpu"))
     hdA, hdB = pin(torch.empty_like(dA, device="cpu")), pin(torch.empty_like(dB, device="cpu"))
