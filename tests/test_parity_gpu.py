@@ -94,6 +94,11 @@ SMALL = [
     ("ragged2", 256, 72, 128, 2, 8, 2.0, 33),
     ("g64_4", 512, 384, 64, 4, 64, 1.0, 200),
     ("colwise", 128, 64, 128, 4, 8, 1.0, 16),
+    # adapter coefficient zero and negative (few rows, the tokens-as-MMA-rows kernel, the large-tile kernels)
+    ("s_zero_few", 512, 384, 32, 4, 16, 0.0, 6),
+    ("s_zero_tc", 512, 512, 64, 3, 16, 0.0, 300),
+    ("s_negative_mid", 512, 512, 32, 4, 24, -1.5, 50),
+    ("s_negative_tc", 512, 384, 128, 2, 8, -0.5, 700),
     # group sizes other than 32, 64, 128 (multiples of 32): CUDA-core kernels whatever the other sizes are
     ("g96", 384, 136, 96, 4, 8, 1.0, 50),
     ("g256", 512, 256, 256, 3, 16, 1.0, 300),
